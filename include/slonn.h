@@ -1,0 +1,205 @@
+/*
+ * slonn.h -- C ABI of the SLO-NN inference library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-query inference path of an SLO-Aware Neural
+ * Network ("Dynamic Network Adaptation at Inference", arxiv 2204.08400):
+ *   build : Node-Activator training -- Algorithm 1 with FreeHash hash functions
+ *           (Def. 2, Eq. 5) sampled in proportion to activation variance (Sec. 3.4);
+ *   run   : the SLO-aware forward pass (Fig. 2 steps 1, 3, 4; Sec. 3.3): hash the
+ *           layer input, fetch one ranked node list per table, keep the top k% of
+ *           the lists, compute only those nodes, pass the sparse activation on.
+ * The percentage k is chosen elsewhere (the paper's ACLO / LCAO policies) and
+ * arrives here as a per-query budget.
+ *
+ * Conventions
+ *   - Every function returns SLONN_OK (0) or a negative SLONN_ERR_* code.  Nothing
+ *     throws, aborts or traps; device-side problems are reported through the
+ *     batch's status words.
+ *   - Pointers are DEVICE pointers unless the comment says "host".
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - Ownership: the caller owns every buffer it passes in.  Weights and biases
+ *     given to slonn_build are referenced, not copied: they must stay valid and
+ *     unchanged until slonn_free.  The library owns what it allocates inside
+ *     slonn_model (tables, hash-node ids, a transposed first-layer copy).
+ *   - A model is read-only after slonn_build; slonn_run may be called
+ *     concurrently on different streams with different workspaces.
+ *   - Arithmetic: every dot product is summed in fp32 in one fixed order (32
+ *     partial sums; input element j goes to partial (j / V) mod 32 by fused
+ *     multiply-add in ascending j, V = 16 bytes / weight element size; a fixed
+ *     pairwise tree with strides 16, 8, 4, 2, 1; bias added last).  For a
+ *     first layer fed by CSR input, j is the position in the row's id-ascending
+ *     nonzero list and V = 1.  Hash bits are signs of such sums, so the order is
+ *     part of the interface: it does not depend on batch size, budget or launch
+ *     shape.  bf16 weights are widened exactly; activations and biases are fp32.
+ */
+#ifndef SLONN_H
+#define SLONN_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SLONN_VERSION 1
+
+/* weight storage types */
+#define SLONN_F32 0
+#define SLONN_BF16 1
+
+/* error codes */
+#define SLONN_OK 0
+#define SLONN_ERR_ARG (-1)       /* null pointer, bad handle, bad flag combination        */
+#define SLONN_ERR_DIM (-2)       /* a width is 0 / too large, K*L exceeds a layer's width   */
+#define SLONN_ERR_DTYPE (-3)     /* unknown weight type                                    */
+#define SLONN_ERR_ALIGN (-4)     /* a weight row or buffer is not 16-byte aligned          */
+#define SLONN_ERR_BUDGET (-5)    /* budget outside 1..10000 bp, above the batch's stated   */
+                                 /* maximum, or above list_cap without being 100 %         */
+#define SLONN_ERR_NOMEM (-6)     /* host or device allocation failed (build only)          */
+#define SLONN_ERR_CUDA (-7)      /* a CUDA runtime call failed                             */
+#define SLONN_ERR_TIMEOUT (-8)   /* a bounded device-side wait ran out                     */
+#define SLONN_ERR_WORKSPACE (-9) /* workspace missing, misaligned or too small             */
+
+#define SLONN_MAX_LAYERS 16
+
+typedef struct slonn_model slonn_model;
+
+int slonn_version(void);
+/* Static, NUL-terminated description of an error code. */
+const char *slonn_strerror(int code);
+
+/* ---------------------------------------------------------------------------
+ * Build (Algorithm 1; hash-function sampling of Sec. 3.4)
+ * ------------------------------------------------------------------------- */
+typedef struct {
+    uint32_t n_layers;             /* weight layers (hidden + output), 1..SLONN_MAX_LAYERS   */
+    const uint32_t *dims;          /* host: n_layers+1 widths D0, N1, ..., N_out             */
+    const uint8_t *has_activator;  /* host: per layer, 1 = the layer carries a Node Activator */
+    int32_t dtype;                 /* SLONN_F32 | SLONN_BF16: storage type of every W         */
+    uint32_t K, L;                 /* key bits per table (1..16), tables (1..8); paper: 10, 2 */
+    uint32_t list_cap;             /* entries kept per bucket list; 0 = the whole layer       */
+    uint64_t seed;                 /* seed of the hash-node sampling                          */
+    uint32_t first_layer_sparse;   /* 1: layer 0 is fed CSR rows (sparse operand); it must    */
+                                   /*    then carry no activator; calibration is CSR as well  */
+    const uint32_t *const *hash_nodes_override; /* host, nullable; per layer nullable: L*K    */
+                                   /* distinct node ids to use instead of sampling            */
+} slonn_build_desc;
+
+typedef struct {
+    uint32_t n_rows;
+    const float *dense;            /* [n_rows][D0] fp32 row-major, or NULL when CSR           */
+    const uint64_t *indptr;        /* CSR: [n_rows+1]                                         */
+    const uint32_t *ids;           /* CSR: column ids, ascending and distinct within a row    */
+    const float *vals;             /* CSR: values                                             */
+} slonn_rows;
+
+/*
+ * Trains the Node-Importance tables of every activator layer on the calibration
+ * rows (the paper's LSH training set): complete forward pass of the calibration
+ * rows, per-node activation variance, K*L hash nodes per layer drawn with
+ * probability proportional to variance, per table and bucket the sum of the
+ * activations of the rows that hash there, and the node ids sorted by that sum
+ * (highest first, equal sums by lower id).  A bucket no row reached holds the
+ * ranking of the sums over all rows.
+ *   W[l]    : row-major [N_l][D_l], rows 16-byte aligned (D_l * element size
+ *             must be a multiple of 16), fp32 or bf16 bit patterns per desc->dtype
+ *   bias[l] : [N_l] fp32
+ * W and bias are host arrays of device pointers.  Hidden layers use ReLU, the
+ * last layer the identity.  Synchronises `stream` before returning (the build
+ * allocates, reads variances back and samples on the host).  *out is set only
+ * on success.
+ */
+int slonn_build(const slonn_build_desc *desc, const void *const *W, const float *const *bias,
+                const slonn_rows *calib, void *stream, slonn_model **out);
+
+/*
+ * Layer facts for parity checks.  hash_nodes: host buffer of L*K ids (nullable);
+ * the other outputs are nullable too.  tables_dev points at the layer's lists,
+ * laid out [L][2^K][cap] with ids of id_bytes (2 when N_l <= 65536, else 4).
+ * Layers without activator report cap 0 and a NULL table.
+ */
+int slonn_model_info(const slonn_model *m, uint32_t layer, uint32_t *hash_nodes,
+                     const void **tables_dev, uint64_t *table_bytes, uint32_t *id_bytes,
+                     uint32_t *cap);
+
+/*
+ * Copies a layer's tables ([L][2^K][cap] ids of id_bytes each) into a HOST
+ * buffer of at least table_bytes; synchronous.  For parity checks and for
+ * persisting a trained activator.
+ */
+int slonn_model_tables_to_host(const slonn_model *m, uint32_t layer, void *dst_host, uint64_t dst_bytes);
+
+/* Frees the model and everything it owns.  NULL is accepted. */
+void slonn_free(slonn_model *m);
+
+/* ---------------------------------------------------------------------------
+ * Run (Fig. 2 steps 1, 3, 4; Sec. 3.3)
+ * ------------------------------------------------------------------------- */
+typedef struct {
+    uint32_t n_queries;
+    /* inputs */
+    const float *x_dense;          /* [n][D0], or NULL when the model takes CSR rows          */
+    const uint64_t *x_indptr;      /* CSR alternative (first_layer_sparse models)            */
+    const uint32_t *x_ids;
+    const float *x_vals;
+    const uint16_t *budget_bp;     /* [n] per-query budget k in basis points, 1..10000;       */
+                                   /* node count per activator layer = max(1, round half up   */
+                                   /* of bp * N_l / 10000)                                    */
+    uint32_t max_budget_bp;        /* HOST value: upper bound of budget_bp[] (0 = 10000);     */
+                                   /* sizes the launch grids, the workspace and logit_stride  */
+    /* outputs (nullable unless stated) */
+    float *logits;                 /* required. [n][logit_stride]: the last layer's           */
+                                   /* pre-activations.  logit_stride = N_out, or, when the    */
+                                   /* last layer is budgeted, the node count of max_budget_bp */
+                                   /* (entries past a query's own count are left untouched)   */
+    uint32_t *logit_ids;           /* [n][logit_stride] node id of each logit; required when  */
+                                   /* the last layer is budgeted, ignored otherwise           */
+    uint32_t *pred;                /* [n] argmax node id over the computed logits, lowest id  */
+                                   /* on ties                                                 */
+    uint16_t *codes;               /* [n][n_act_layers][L] hash keys                          */
+    uint64_t *active_indptr;       /* [n*n_act_layers + 1] offsets into active_ids/vals,      */
+                                   /* entry q*n_act_layers + a                                */
+    uint32_t *active_ids;          /* active node ids, ascending within (query, layer);       */
+                                   /* capacity = slonn_active_capacity()                      */
+    float *active_vals;            /* their activations (zeros kept), same layout             */
+    uint32_t *status;              /* required. [4] words: [0] first error code seen on the   */
+                                   /* device (0 = ok, else -SLONN_ERR_*), [1] query index,    */
+                                   /* [2] layer index, [3] reserved.  Cleared by slonn_run    */
+} slonn_batch;
+
+/* Number of entries active_ids / active_vals need for n queries at max_budget_bp. */
+int slonn_active_capacity(const slonn_model *m, uint32_t n_queries, uint32_t max_budget_bp,
+                          uint64_t *entries);
+/* logit_stride for this model at max_budget_bp (see slonn_batch.logits). */
+int slonn_logit_stride(const slonn_model *m, uint32_t max_budget_bp, uint32_t *stride);
+/* Bytes of device workspace slonn_run needs (256-byte aligned buffer). */
+int slonn_workspace_bytes(const slonn_model *m, uint32_t n_queries, uint32_t max_budget_bp,
+                          uint64_t *bytes);
+
+/*
+ * Runs the batch on `stream`: asynchronous, no allocation, no host
+ * synchronisation.  The caller synchronises the stream and reads status[0].
+ * A query whose budget is invalid gets a clamped, in-range active set and the
+ * error is recorded in status; other queries are unaffected.
+ */
+int slonn_run(const slonn_model *m, const slonn_batch *batch, void *workspace,
+              uint64_t workspace_bytes, void *stream);
+
+/*
+ * Same computation for callers that keep queries and results in HOST memory:
+ * every pointer of `host_batch` (inputs, outputs, status) is a host pointer,
+ * pinned memory recommended.  Copies the inputs to the device, runs, copies
+ * every non-NULL output back and synchronises `stream` before returning.
+ * `workspace` is device memory of at least slonn_host_workspace_bytes().
+ * h2d_bytes / d2h_bytes (host, nullable) receive the bytes copied each way.
+ */
+int slonn_host_workspace_bytes(const slonn_model *m, uint32_t n_queries, uint32_t max_budget_bp,
+                               uint64_t x_nnz, uint64_t *bytes);
+int slonn_run_host(const slonn_model *m, const slonn_batch *host_batch, void *workspace,
+                   uint64_t workspace_bytes, void *stream, uint64_t *h2d_bytes,
+                   uint64_t *d2h_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLONN_H */

@@ -1,0 +1,277 @@
+"""Python binding of libslonn.so: the same calls as include/slonn.h, with torch
+tensors (device memory) or numpy arrays (host memory) marshalled to raw
+pointers.  No arithmetic happens here; without the compiled CUDA library every
+call raises.
+"""
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+SLONN_F32, SLONN_BF16 = 0, 1
+SLONN_OK = 0
+ERR = {"ARG": -1, "DIM": -2, "DTYPE": -3, "ALIGN": -4, "BUDGET": -5, "NOMEM": -6, "CUDA": -7,
+       "TIMEOUT": -8, "WORKSPACE": -9}
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libslonn.so")
+
+EXPORTS = [
+    "slonn_version", "slonn_strerror", "slonn_build", "slonn_model_info", "slonn_model_tables_to_host",
+    "slonn_free", "slonn_active_capacity", "slonn_logit_stride", "slonn_workspace_bytes", "slonn_run",
+    "slonn_host_workspace_bytes", "slonn_run_host",
+]
+
+
+class SlonnError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class _BuildDesc(C.Structure):
+    _fields_ = [("n_layers", C.c_uint32), ("dims", C.c_void_p), ("has_activator", C.c_void_p),
+                ("dtype", C.c_int32), ("K", C.c_uint32), ("L", C.c_uint32), ("list_cap", C.c_uint32),
+                ("seed", C.c_uint64), ("first_layer_sparse", C.c_uint32),
+                ("hash_nodes_override", C.c_void_p)]
+
+
+class _Rows(C.Structure):
+    _fields_ = [("n_rows", C.c_uint32), ("dense", C.c_void_p), ("indptr", C.c_void_p),
+                ("ids", C.c_void_p), ("vals", C.c_void_p)]
+
+
+class _Batch(C.Structure):
+    _fields_ = [("n_queries", C.c_uint32), ("x_dense", C.c_void_p), ("x_indptr", C.c_void_p),
+                ("x_ids", C.c_void_p), ("x_vals", C.c_void_p), ("budget_bp", C.c_void_p),
+                ("max_budget_bp", C.c_uint32), ("logits", C.c_void_p), ("logit_ids", C.c_void_p),
+                ("pred", C.c_void_p), ("codes", C.c_void_p), ("active_indptr", C.c_void_p),
+                ("active_ids", C.c_void_p), ("active_vals", C.c_void_p), ("status", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               "`python -m paper_2204_08400_b200.build_ext` (there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        L.slonn_version.restype = C.c_int
+        L.slonn_strerror.restype = C.c_char_p
+        L.slonn_strerror.argtypes = [C.c_int]
+        L.slonn_build.restype = C.c_int
+        L.slonn_build.argtypes = [C.POINTER(_BuildDesc), C.c_void_p, C.c_void_p, C.POINTER(_Rows),
+                                  C.c_void_p, C.POINTER(C.c_void_p)]
+        L.slonn_model_info.restype = C.c_int
+        L.slonn_model_info.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.POINTER(C.c_void_p),
+                                       C.POINTER(C.c_uint64), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
+        L.slonn_model_tables_to_host.restype = C.c_int
+        L.slonn_model_tables_to_host.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64]
+        L.slonn_free.restype = None
+        L.slonn_free.argtypes = [C.c_void_p]
+        L.slonn_active_capacity.restype = C.c_int
+        L.slonn_active_capacity.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint64)]
+        L.slonn_logit_stride.restype = C.c_int
+        L.slonn_logit_stride.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
+        L.slonn_workspace_bytes.restype = C.c_int
+        L.slonn_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint64)]
+        L.slonn_run.restype = C.c_int
+        L.slonn_run.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p]
+        L.slonn_host_workspace_bytes.restype = C.c_int
+        L.slonn_host_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64,
+                                                 C.POINTER(C.c_uint64)]
+        L.slonn_run_host.restype = C.c_int
+        L.slonn_run_host.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p,
+                                     C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+        _lib = L
+    return _lib
+
+
+def _ptr(t) -> Optional[int]:
+    """Raw address of a torch tensor, numpy array, int or None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        return None
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def version() -> int:
+    return lib().slonn_version()
+
+
+def strerror(code: int) -> str:
+    return lib().slonn_strerror(code).decode()
+
+
+class Model:
+    """Handle of a built model; keeps the referenced weight tensors alive."""
+
+    def __init__(self, handle, keep, dims, has_activator, dtype, K, L, first_layer_sparse):
+        self.handle = handle
+        self._keep = keep
+        self.dims = list(dims)
+        self.has_activator = list(has_activator)
+        self.n_act = sum(1 for h in has_activator if h)
+        self.dtype, self.K, self.L = dtype, K, L
+        self.first_layer_sparse = first_layer_sparse
+
+    def free(self):
+        if self.handle:
+            lib().slonn_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def slonn_build(dims: Sequence[int], has_activator: Sequence[int], dtype: int, W: List, bias: List,
+                calib_dense=None, calib_csr=None, K: int = 10, L: int = 2, list_cap: int = 0, seed: int = 0,
+                first_layer_sparse: bool = False, hash_nodes_override=None, stream=None) -> Model:
+    """W[l], bias[l], calib_*: device tensors (W as float32 or as uint16/bfloat16 bit patterns)."""
+    n_layers = len(dims) - 1
+    d = np.asarray(dims, dtype=np.uint32)
+    h = np.asarray(has_activator, dtype=np.uint8)
+    Wp = (C.c_void_p * n_layers)(*[_ptr(w) for w in W])
+    bp = (C.c_void_p * n_layers)(*[_ptr(b) for b in bias])
+    keep = [list(W), list(bias), d, h]
+    desc = _BuildDesc()
+    desc.n_layers = n_layers
+    desc.dims = d.ctypes.data
+    desc.has_activator = h.ctypes.data
+    desc.dtype = dtype
+    desc.K, desc.L, desc.list_cap, desc.seed = K, L, list_cap, seed
+    desc.first_layer_sparse = int(bool(first_layer_sparse))
+    ov_keep = []
+    if hash_nodes_override is not None:
+        ov = (C.c_void_p * n_layers)()
+        for l in range(n_layers):
+            if hash_nodes_override[l] is not None:
+                a = np.ascontiguousarray(hash_nodes_override[l], dtype=np.uint32).reshape(-1)
+                ov_keep.append(a)
+                ov[l] = a.ctypes.data
+        desc.hash_nodes_override = C.cast(ov, C.c_void_p)
+        ov_keep.append(ov)
+    rows = _Rows()
+    if calib_csr is not None:
+        indptr, ids, vals = calib_csr
+        rows.n_rows = indptr.numel() - 1
+        rows.indptr, rows.ids, rows.vals = _ptr(indptr), _ptr(ids), _ptr(vals)
+    elif calib_dense is not None:
+        rows.n_rows = calib_dense.shape[0]
+        rows.dense = _ptr(calib_dense)
+    out = C.c_void_p()
+    rc = lib().slonn_build(C.byref(desc), C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p), C.byref(rows),
+                           _stream_ptr(stream), C.byref(out))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_build")
+    return Model(out.value, keep, dims, has_activator, dtype, K, L, bool(first_layer_sparse))
+
+
+def slonn_free(model: Model) -> None:
+    model.free()
+
+
+def slonn_model_info(model: Model, layer: int) -> dict:
+    hn = np.zeros(model.K * model.L, dtype=np.uint32)
+    tables = C.c_void_p()
+    tb = C.c_uint64()
+    ib = C.c_uint32()
+    cap = C.c_uint32()
+    rc = lib().slonn_model_info(model.handle, layer, hn.ctypes.data, C.byref(tables), C.byref(tb),
+                                C.byref(ib), C.byref(cap))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_model_info")
+    return {"hash_nodes": hn.reshape(model.L, model.K), "tables_dev": tables.value, "table_bytes": tb.value,
+            "id_bytes": ib.value, "cap": cap.value}
+
+
+def slonn_model_tables_to_host(model: Model, layer: int) -> np.ndarray:
+    info = slonn_model_info(model, layer)
+    dt = np.uint16 if info["id_bytes"] == 2 else np.uint32
+    out = np.empty((model.L, 1 << model.K, info["cap"]), dtype=dt)
+    rc = lib().slonn_model_tables_to_host(model.handle, layer, out.ctypes.data, out.nbytes)
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_model_tables_to_host")
+    return out
+
+
+def slonn_active_capacity(model: Model, n_queries: int, max_budget_bp: int = 0) -> int:
+    v = C.c_uint64()
+    rc = lib().slonn_active_capacity(model.handle, n_queries, max_budget_bp, C.byref(v))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_active_capacity")
+    return v.value
+
+
+def slonn_logit_stride(model: Model, max_budget_bp: int = 0) -> int:
+    v = C.c_uint32()
+    rc = lib().slonn_logit_stride(model.handle, max_budget_bp, C.byref(v))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_logit_stride")
+    return v.value
+
+
+def slonn_workspace_bytes(model: Model, n_queries: int, max_budget_bp: int = 0) -> int:
+    v = C.c_uint64()
+    rc = lib().slonn_workspace_bytes(model.handle, n_queries, max_budget_bp, C.byref(v))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_workspace_bytes")
+    return v.value
+
+
+def slonn_host_workspace_bytes(model: Model, n_queries: int, max_budget_bp: int = 0, x_nnz: int = 0) -> int:
+    v = C.c_uint64()
+    rc = lib().slonn_host_workspace_bytes(model.handle, n_queries, max_budget_bp, x_nnz, C.byref(v))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_host_workspace_bytes")
+    return v.value
+
+
+def make_batch(n_queries: int, budget_bp, logits, status, x_dense=None, x_csr=None, max_budget_bp: int = 0,
+               logit_ids=None, pred=None, codes=None, active_indptr=None, active_ids=None,
+               active_vals=None) -> _Batch:
+    """Fills a slonn_batch from tensors/arrays (device for slonn_run, host for slonn_run_host)."""
+    b = _Batch()
+    b.n_queries = n_queries
+    b.x_dense = _ptr(x_dense)
+    if x_csr is not None:
+        b.x_indptr, b.x_ids, b.x_vals = _ptr(x_csr[0]), _ptr(x_csr[1]), _ptr(x_csr[2])
+    b.budget_bp = _ptr(budget_bp)
+    b.max_budget_bp = max_budget_bp
+    b.logits, b.logit_ids, b.pred, b.codes = _ptr(logits), _ptr(logit_ids), _ptr(pred), _ptr(codes)
+    b.active_indptr, b.active_ids, b.active_vals = _ptr(active_indptr), _ptr(active_ids), _ptr(active_vals)
+    b.status = _ptr(status)
+    return b
+
+
+def slonn_run(model: Model, batch: _Batch, workspace, workspace_bytes: int, stream=None) -> None:
+    rc = lib().slonn_run(model.handle, C.byref(batch), _ptr(workspace), workspace_bytes, _stream_ptr(stream))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_run")
+
+
+def slonn_run_host(model: Model, host_batch: _Batch, workspace, workspace_bytes: int, stream=None):
+    """Returns (h2d_bytes, d2h_bytes)."""
+    up, down = C.c_uint64(), C.c_uint64()
+    rc = lib().slonn_run_host(model.handle, C.byref(host_batch), _ptr(workspace), workspace_bytes,
+                              _stream_ptr(stream), C.byref(up), C.byref(down))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_run_host")
+    return up.value, down.value

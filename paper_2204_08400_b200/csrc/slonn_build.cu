@@ -1,0 +1,569 @@
+// Node-Activator training on the device (Algorithm 1 of the paper, with the
+// variance-proportional FreeHash sampling of Sec. 3.4), plus model lifetime.
+//
+// Per activator layer l, with A = the layer's complete activations on the
+// calibration rows ([n_cal][N] fp32):
+//   column_stats_kernel   per node: sum and population variance over the rows (fp64, row order)
+//   (host)                K*L distinct hash nodes drawn in proportion to variance
+//   row_keys_kernel       per row and table: key from the signs of the hash nodes' activations
+//   bucket_*_kernel       rows grouped by key, row order kept inside a bucket
+//   bucket_score_kernel   NodeScore[b][key][node] = sum of A over the bucket's rows (fp64, row order)
+//   segment_sort_kernel   node ids ordered by score, highest first, equal scores by lower id
+//   fill_tables_kernel    lists copied into the table; buckets no row reached get the global ranking
+// fp64 sums use explicit add/multiply intrinsics so that no multiply-add is fused.
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "slonn_common.cuh"
+
+namespace {
+
+#define CK(call)                                         \
+    do {                                                 \
+        if ((call) != cudaSuccess) { rc = SLONN_ERR_CUDA; goto fail; } \
+    } while (0)
+
+// ---------------------------------------------------------------------------
+__global__ void transpose_kernel(const void *W, void *WT, uint32_t N, uint32_t D, uint32_t esz)
+{
+    // WT[d][n] = W[n][d]; plain tiled transpose through shared memory
+    __shared__ uint32_t tile[32][33];
+    const uint32_t d0 = blockIdx.x * 32, n0 = blockIdx.y * 32;
+    for (uint32_t i = threadIdx.y; i < 32; i += blockDim.y) {
+        const uint32_t n = n0 + i, d = d0 + threadIdx.x;
+        uint32_t v = 0;
+        if (n < N && d < D)
+            v = esz == 2 ? (uint32_t)reinterpret_cast<const uint16_t *>(W)[(uint64_t)n * D + d]
+                         : reinterpret_cast<const uint32_t *>(W)[(uint64_t)n * D + d];
+        tile[i][threadIdx.x] = v;
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.y; i < 32; i += blockDim.y) {
+        const uint32_t d = d0 + i, n = n0 + threadIdx.x;
+        if (n < N && d < D) {
+            const uint32_t v = tile[threadIdx.x][i];
+            if (esz == 2) reinterpret_cast<uint16_t *>(WT)[(uint64_t)d * N + n] = (uint16_t)v;
+            else reinterpret_cast<uint32_t *>(WT)[(uint64_t)d * N + n] = v;
+        }
+    }
+}
+
+// sum[i] = sum over rows of A[x][i]; var[i] = mean of (A[x][i] - mean_i)^2.  One thread per node.
+__global__ void column_stats_kernel(const float *A, uint32_t n_rows, uint32_t N, double *sum, double *var)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    double s = 0.0;
+    for (uint32_t x = 0; x < n_rows; ++x) s = __dadd_rn(s, (double)A[(uint64_t)x * N + i]);
+    const double mean = __ddiv_rn(s, (double)n_rows);
+    double v = 0.0;
+    for (uint32_t x = 0; x < n_rows; ++x) {
+        const double d = __dsub_rn((double)A[(uint64_t)x * N + i], mean);
+        v = __dadd_rn(v, __dmul_rn(d, d));
+    }
+    sum[i] = s;
+    var[i] = __ddiv_rn(v, (double)n_rows);
+}
+
+// keys[b][x]: bit j = [activation of hash node (b, j) on row x > 0]
+__global__ void row_keys_kernel(const float *A, uint32_t n_rows, uint32_t N, const uint32_t *hash_nodes,
+                                uint32_t K, uint32_t L, uint32_t *keys)
+{
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (uint64_t)n_rows * L) return;
+    const uint32_t b = (uint32_t)(t / n_rows), x = (uint32_t)(t % n_rows);
+    uint32_t key = 0;
+    for (uint32_t j = 0; j < K; ++j)
+        if (A[(uint64_t)x * N + hash_nodes[b * K + j]] > 0.0f) key |= (1u << j);
+    keys[(uint64_t)b * n_rows + x] = key;
+}
+
+// One thread per (table, key): how many rows carry that key.
+__global__ void bucket_count_kernel(const uint32_t *keys, uint32_t n_rows, uint32_t nb, uint32_t L,
+                                    uint32_t *count)
+{
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= nb * L) return;
+    const uint32_t b = t / nb, key = t % nb;
+    uint32_t c = 0;
+    for (uint32_t x = 0; x < n_rows; ++x) c += (keys[(uint64_t)b * n_rows + x] == key) ? 1u : 0u;
+    count[t] = c;
+}
+
+// start[t] = exclusive prefix of count within a table (one block per table).
+__global__ void bucket_start_kernel(const uint32_t *count, uint32_t nb, uint32_t *start)
+{
+    __shared__ uint32_t carry;
+    const uint32_t b = blockIdx.x;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (uint32_t base = 0; base < nb; base += blockDim.x) {
+        // serial within the block is enough: nb <= 65536, build time only
+        if (threadIdx.x == 0) {
+            uint32_t run = carry;
+            const uint32_t end = min(nb, base + blockDim.x);
+            for (uint32_t k = base; k < end; ++k) {
+                start[b * nb + k] = run;
+                run += count[b * nb + k];
+            }
+            carry = run;
+        }
+        __syncthreads();
+    }
+}
+
+// One thread per (table, key): the rows of that bucket, in row order.
+__global__ void bucket_fill_kernel(const uint32_t *keys, uint32_t n_rows, uint32_t nb, uint32_t L,
+                                   const uint32_t *start, uint32_t *members)
+{
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= nb * L) return;
+    const uint32_t b = t / nb, key = t % nb;
+    uint32_t o = start[t];
+    for (uint32_t x = 0; x < n_rows; ++x)
+        if (keys[(uint64_t)b * n_rows + x] == key) members[(uint64_t)b * n_rows + o++] = x;
+}
+
+// score[bk][i] = sum over the bucket's rows (row order) of A[x][i], fp64.
+__global__ void bucket_score_kernel(const float *A, uint32_t n_rows, uint32_t N, uint32_t nb,
+                                    const uint32_t *start, const uint32_t *count, const uint32_t *members,
+                                    uint32_t bk0, double *score /* [segments in this pass][N] */)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t bk = bk0 + blockIdx.y;
+    if (i >= N) return;
+    const uint32_t b = bk / nb;
+    const uint32_t *mem = members + (uint64_t)b * n_rows + start[bk];
+    const uint32_t c = count[bk];
+    double s = 0.0;
+    for (uint32_t k = 0; k < c; ++k) s = __dadd_rn(s, (double)A[(uint64_t)mem[k] * N + i]);
+    score[(uint64_t)blockIdx.y * N + i] = s;
+}
+
+// Sort key: ascending unsigned order == descending score; zeros of either sign are equal.
+__device__ __forceinline__ uint64_t score_sort_key(double s)
+{
+    if (s == 0.0) s = 0.0;
+    uint64_t u = (uint64_t)__double_as_longlong(s);
+    u = (u >> 63) ? ~u : (u | 0x8000000000000000ull); // ascending-order image
+    return ~u;                                          // descending
+}
+
+// One block per segment: stable LSD radix sort (8 bits per pass) of the segment's
+// N (key, id) pairs; ids start ascending, so equal scores keep the lower id first.
+// seg_active[s] == 0 skips the segment.  The sorted ids end in ids_out[s][0..N).
+#define SORT_THREADS 256
+__global__ void __launch_bounds__(SORT_THREADS)
+segment_sort_kernel(const double *score, uint32_t N, const uint32_t *seg_active, uint64_t *keyA, uint64_t *keyB,
+                    uint32_t *idA, uint32_t *idB, uint32_t *ids_out)
+{
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t bin_base[256];
+    __shared__ uint32_t warp_cnt[SORT_THREADS / 32][256];
+    __shared__ uint32_t warp_off[SORT_THREADS / 32][256];
+    __shared__ uint32_t s_skip;
+    const uint32_t seg = blockIdx.x;
+    if (seg_active && !seg_active[seg]) return;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    uint64_t *ka = keyA + (uint64_t)seg * N, *kb = keyB + (uint64_t)seg * N;
+    uint32_t *ia = idA + (uint64_t)seg * N, *ib = idB + (uint64_t)seg * N;
+    const double *sc = score + (uint64_t)seg * N;
+    for (uint32_t i = threadIdx.x; i < N; i += blockDim.x) {
+        ka[i] = score_sort_key(sc[i]);
+        ia[i] = i;
+    }
+    for (uint32_t d = threadIdx.x; d < 256; d += blockDim.x)
+        for (uint32_t w = 0; w < SORT_THREADS / 32; ++w) warp_cnt[w][d] = 0;
+    __syncthreads();
+    for (uint32_t pass = 0; pass < 8; ++pass) {
+        const uint32_t shift = pass * 8;
+        for (uint32_t d = threadIdx.x; d < 256; d += blockDim.x) hist[d] = 0;
+        if (threadIdx.x == 0) s_skip = 0;
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < N; i += blockDim.x)
+            atomicAdd(&hist[(uint32_t)(ka[i] >> shift) & 255u], 1u);
+        __syncthreads();
+        if (threadIdx.x < 256 && hist[threadIdx.x] == N) s_skip = 1; // every key shares this digit
+        __syncthreads();
+        if (s_skip) { __syncthreads(); continue; }
+        if (threadIdx.x == 0) {
+            uint32_t run = 0;
+            for (uint32_t d = 0; d < 256; ++d) { bin_base[d] = run; run += hist[d]; }
+        }
+        __syncthreads();
+        for (uint32_t base = 0; base < N; base += blockDim.x) {
+            const uint32_t i = base + threadIdx.x;
+            const bool valid = i < N;
+            uint64_t key = 0;
+            uint32_t id = 0, digit = 0x100u + lane; // distinct dummies for lanes past the end
+            if (valid) { key = ka[i]; id = ia[i]; digit = (uint32_t)(key >> shift) & 255u; }
+            const uint32_t peers = __match_any_sync(SLONN_FULL_MASK, digit);
+            const uint32_t rank = __popc(peers & ((1u << lane) - 1u));
+            const bool leader = valid && rank == 0;
+            if (leader) warp_cnt[warp][digit] = __popc(peers);
+            __syncthreads();
+            if (threadIdx.x < 256) {
+                const uint32_t d = threadIdx.x;
+                uint32_t run = bin_base[d];
+                for (uint32_t w = 0; w < SORT_THREADS / 32; ++w) {
+                    warp_off[w][d] = run;
+                    run += warp_cnt[w][d];
+                }
+                bin_base[d] = run;
+            }
+            __syncthreads();
+            if (valid) {
+                const uint32_t dst = warp_off[warp][digit] + rank;
+                kb[dst] = key;
+                ib[dst] = id;
+            }
+            if (leader) warp_cnt[warp][digit] = 0;
+            __syncthreads();
+        }
+        uint64_t *tk = ka; ka = kb; kb = tk;
+        uint32_t *ti = ia; ia = ib; ib = ti;
+        __syncthreads();
+    }
+    uint32_t *out = ids_out + (uint64_t)seg * N;
+    for (uint32_t i = threadIdx.x; i < N; i += blockDim.x) out[i] = ia[i];
+}
+
+// tables[bk][0..cap) = the bucket's sorted ids, or the global ranking for a bucket no row reached.
+template <typename IDT>
+__global__ void fill_tables_kernel(const uint32_t *sorted /* [segs][N] */, const uint32_t *global_sorted,
+                                   const uint32_t *count, uint32_t bk0, uint32_t N, uint32_t cap, IDT *tables)
+{
+    const uint32_t bk = bk0 + blockIdx.y;
+    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= cap) return;
+    const uint32_t *src = count[bk] ? sorted + (uint64_t)blockIdx.y * N : global_sorted;
+    tables[(uint64_t)bk * cap + r] = (IDT)src[r];
+}
+
+// ---------------------------------------------------------------------------
+// host: hash-node sampling.  SplitMix64 stream; each draw takes one node from the
+// not-yet-drawn ones with probability proportional to its variance (inverse CDF in id
+// order); once no positive variance is left the draw is uniform over what remains.
+// ---------------------------------------------------------------------------
+struct sm64 {
+    uint64_t s;
+    uint64_t next()
+    {
+        s += 0x9E3779B97F4A7C15ull;
+        uint64_t z = s;
+        z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+        z ^= z >> 27; z *= 0x94D049BB133111EBull;
+        z ^= z >> 31;
+        return z;
+    }
+    double unit() { return (double)(next() >> 11) * 0x1.0p-53; }
+};
+
+void sample_hash_nodes(const std::vector<double> &var, uint32_t H, uint64_t seed, uint32_t layer, uint32_t *out)
+{
+    const uint32_t N = (uint32_t)var.size();
+    std::vector<char> used(N, 0);
+    sm64 rng{seed ^ (0xD6E8FEB86659FD93ull * (uint64_t)(layer + 1))};
+    for (uint32_t d = 0; d < H; ++d) {
+        const double u = rng.unit();
+        double mass = 0.0;
+        uint32_t left = 0;
+        for (uint32_t i = 0; i < N; ++i) {
+            if (used[i]) continue;
+            mass += var[i];
+            ++left;
+        }
+        uint32_t chosen = N;
+        if (mass > 0.0) {
+            const double target = u * mass;
+            double cum = 0.0;
+            uint32_t last_positive = N;
+            for (uint32_t i = 0; i < N && chosen == N; ++i) {
+                if (used[i] || !(var[i] > 0.0)) continue;
+                cum += var[i];
+                last_positive = i;
+                if (cum > target) chosen = i;
+            }
+            if (chosen == N) chosen = last_positive;
+        } else {
+            uint32_t skip = (uint32_t)(u * (double)left);
+            if (skip >= left) skip = left - 1;
+            for (uint32_t i = 0; i < N; ++i) {
+                if (used[i]) continue;
+                if (skip-- == 0) { chosen = i; break; }
+            }
+        }
+        used[chosen] = 1;
+        out[d] = chosen;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// tables of one layer from its complete calibration activations
+// ---------------------------------------------------------------------------
+int train_layer(slonn_model *m, uint32_t l, const float *A, uint32_t n_cal, uint64_t seed,
+                const uint32_t *override_nodes, cudaStream_t st)
+{
+    slonn_layer &ly = m->layer[l];
+    const uint32_t N = ly.N, K = m->K, L = m->L, H = m->H, nb = 1u << K, nseg = nb * L;
+    int rc = SLONN_OK;
+    double *d_sum = nullptr, *d_var = nullptr, *d_score = nullptr;
+    uint32_t *d_keys = nullptr, *d_count = nullptr, *d_start = nullptr, *d_members = nullptr;
+    uint64_t *d_keyA = nullptr, *d_keyB = nullptr;
+    uint32_t *d_idA = nullptr, *d_idB = nullptr, *d_sorted = nullptr, *d_gsorted = nullptr;
+    std::vector<double> var(N);
+
+    CK(cudaMalloc(&d_sum, sizeof(double) * N));
+    CK(cudaMalloc(&d_var, sizeof(double) * N));
+    column_stats_kernel<<<(N + 127) / 128, 128, 0, st>>>(A, n_cal, N, d_sum, d_var);
+    CK(cudaGetLastError());
+    CK(cudaMemcpyAsync(var.data(), d_var, sizeof(double) * N, cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+
+    if (override_nodes) {
+        for (uint32_t h = 0; h < H; ++h) {
+            if (override_nodes[h] >= N) { rc = SLONN_ERR_ARG; goto fail; }
+            for (uint32_t g = 0; g < h; ++g)
+                if (override_nodes[g] == override_nodes[h]) { rc = SLONN_ERR_ARG; goto fail; }
+            m->hash_nodes_host[l][h] = override_nodes[h];
+        }
+    } else {
+        sample_hash_nodes(var, H, seed, l, m->hash_nodes_host[l]);
+    }
+    CK(cudaMalloc(&ly.hash_nodes, sizeof(uint32_t) * H));
+    CK(cudaMemcpyAsync(ly.hash_nodes, m->hash_nodes_host[l], sizeof(uint32_t) * H, cudaMemcpyHostToDevice, st));
+
+    // rows -> buckets
+    CK(cudaMalloc(&d_keys, sizeof(uint32_t) * (uint64_t)n_cal * L));
+    CK(cudaMalloc(&d_members, sizeof(uint32_t) * (uint64_t)n_cal * L));
+    CK(cudaMalloc(&d_count, sizeof(uint32_t) * nseg));
+    CK(cudaMalloc(&d_start, sizeof(uint32_t) * nseg));
+    {
+        const uint64_t t = (uint64_t)n_cal * L;
+        row_keys_kernel<<<(uint32_t)((t + 255) / 256), 256, 0, st>>>(A, n_cal, N, ly.hash_nodes, K, L, d_keys);
+        CK(cudaGetLastError());
+        bucket_count_kernel<<<(nseg + 127) / 128, 128, 0, st>>>(d_keys, n_cal, nb, L, d_count);
+        CK(cudaGetLastError());
+        bucket_start_kernel<<<L, 256, 0, st>>>(d_count, nb, d_start);
+        CK(cudaGetLastError());
+        bucket_fill_kernel<<<(nseg + 127) / 128, 128, 0, st>>>(d_keys, n_cal, nb, L, d_start, d_members);
+        CK(cudaGetLastError());
+    }
+
+    // table storage
+    ly.cap = (m->list_cap == 0 || m->list_cap > N) ? N : m->list_cap;
+    ly.id_bytes = N <= 65536u ? 2u : 4u;
+    ly.table_bytes = (uint64_t)nseg * ly.cap * ly.id_bytes;
+    CK(cudaMalloc(&ly.tables, ly.table_bytes));
+
+    // global ranking (sum over all rows), used for buckets no row reached
+    CK(cudaMalloc(&d_gsorted, sizeof(uint32_t) * N));
+    {
+        uint64_t *gkA = nullptr, *gkB = nullptr;
+        uint32_t *giA = nullptr, *giB = nullptr;
+        bool ok = cudaMalloc(&gkA, 8ull * N) == cudaSuccess && cudaMalloc(&gkB, 8ull * N) == cudaSuccess &&
+                  cudaMalloc(&giA, 4ull * N) == cudaSuccess && cudaMalloc(&giB, 4ull * N) == cudaSuccess;
+        if (ok) {
+            segment_sort_kernel<<<1, SORT_THREADS, 0, st>>>(d_sum, N, nullptr, gkA, gkB, giA, giB, d_gsorted);
+            ok = cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(st) == cudaSuccess;
+        }
+        cudaFree(gkA); cudaFree(gkB); cudaFree(giA); cudaFree(giB);
+        if (!ok) { rc = SLONN_ERR_CUDA; goto fail; }
+    }
+
+    // buckets, a bounded number of segments at a time (36 bytes of scratch per node and segment)
+    {
+        uint64_t segs = (2ull << 30) / (36ull * N);
+        segs = std::max<uint64_t>(1, std::min<uint64_t>(segs, nseg));
+        const uint32_t S = (uint32_t)std::min<uint64_t>(segs, 65535);
+        CK(cudaMalloc(&d_score, sizeof(double) * (uint64_t)S * N));
+        CK(cudaMalloc(&d_keyA, 8ull * S * N));
+        CK(cudaMalloc(&d_keyB, 8ull * S * N));
+        CK(cudaMalloc(&d_idA, 4ull * S * N));
+        CK(cudaMalloc(&d_idB, 4ull * S * N));
+        CK(cudaMalloc(&d_sorted, 4ull * S * N));
+        for (uint32_t bk0 = 0; bk0 < nseg; bk0 += S) {
+            const uint32_t cnt = std::min(S, nseg - bk0);
+            bucket_score_kernel<<<dim3((N + 255) / 256, cnt), 256, 0, st>>>(A, n_cal, N, nb, d_start, d_count,
+                                                                            d_members, bk0, d_score);
+            CK(cudaGetLastError());
+            segment_sort_kernel<<<cnt, SORT_THREADS, 0, st>>>(d_score, N, d_count + bk0, d_keyA, d_keyB, d_idA,
+                                                              d_idB, d_sorted);
+            CK(cudaGetLastError());
+            const dim3 g((ly.cap + 255) / 256, cnt);
+            if (ly.id_bytes == 2)
+                fill_tables_kernel<uint16_t><<<g, 256, 0, st>>>(d_sorted, d_gsorted, d_count, bk0, N, ly.cap,
+                                                                (uint16_t *)ly.tables);
+            else
+                fill_tables_kernel<uint32_t><<<g, 256, 0, st>>>(d_sorted, d_gsorted, d_count, bk0, N, ly.cap,
+                                                                (uint32_t *)ly.tables);
+            CK(cudaGetLastError());
+        }
+        CK(cudaStreamSynchronize(st));
+    }
+fail:
+    cudaFree(d_sum); cudaFree(d_var); cudaFree(d_score); cudaFree(d_keys); cudaFree(d_count);
+    cudaFree(d_start); cudaFree(d_members); cudaFree(d_keyA); cudaFree(d_keyB); cudaFree(d_idA);
+    cudaFree(d_idB); cudaFree(d_sorted); cudaFree(d_gsorted);
+    return rc;
+}
+
+} // namespace
+
+// ---------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------
+extern "C" int slonn_version(void) { return SLONN_VERSION; }
+
+extern "C" const char *slonn_strerror(int code)
+{
+    switch (code) {
+    case SLONN_OK: return "ok";
+    case SLONN_ERR_ARG: return "bad argument";
+    case SLONN_ERR_DIM: return "bad dimension";
+    case SLONN_ERR_DTYPE: return "unknown weight type";
+    case SLONN_ERR_ALIGN: return "buffer or weight row not 16-byte aligned";
+    case SLONN_ERR_BUDGET: return "budget out of range";
+    case SLONN_ERR_NOMEM: return "out of memory";
+    case SLONN_ERR_CUDA: return "CUDA runtime error";
+    case SLONN_ERR_TIMEOUT: return "device-side wait timed out";
+    case SLONN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    default: return "unknown error";
+    }
+}
+
+extern "C" void slonn_free(slonn_model *m)
+{
+    if (!m || m->magic != SLONN_MAGIC) return;
+    for (uint32_t l = 0; l < m->n_layers; ++l) {
+        cudaFree(m->layer[l].tables);
+        cudaFree(m->layer[l].hash_nodes);
+        cudaFree(m->layer[l].WT);
+    }
+    m->magic = 0;
+    delete m;
+}
+
+extern "C" int slonn_model_info(const slonn_model *m, uint32_t layer, uint32_t *hash_nodes,
+                                const void **tables_dev, uint64_t *table_bytes, uint32_t *id_bytes, uint32_t *cap)
+{
+    if (!m || m->magic != SLONN_MAGIC || layer >= m->n_layers) return SLONN_ERR_ARG;
+    const slonn_layer &ly = m->layer[layer];
+    if (hash_nodes && ly.has_act) memcpy(hash_nodes, m->hash_nodes_host[layer], sizeof(uint32_t) * m->H);
+    if (tables_dev) *tables_dev = ly.tables;
+    if (table_bytes) *table_bytes = ly.table_bytes;
+    if (id_bytes) *id_bytes = ly.id_bytes;
+    if (cap) *cap = ly.cap;
+    return SLONN_OK;
+}
+
+extern "C" int slonn_model_tables_to_host(const slonn_model *m, uint32_t layer, void *dst_host, uint64_t dst_bytes)
+{
+    if (!m || m->magic != SLONN_MAGIC || layer >= m->n_layers || !dst_host) return SLONN_ERR_ARG;
+    const slonn_layer &ly = m->layer[layer];
+    if (!ly.has_act || !ly.tables) return SLONN_ERR_ARG;
+    if (dst_bytes < ly.table_bytes) return SLONN_ERR_WORKSPACE;
+    return cudaMemcpy(dst_host, ly.tables, ly.table_bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? SLONN_OK
+                                                                                                : SLONN_ERR_CUDA;
+}
+
+extern "C" int slonn_build(const slonn_build_desc *desc, const void *const *W, const float *const *bias,
+                           const slonn_rows *calib, void *stream, slonn_model **out)
+{
+    if (!desc || !W || !bias || !out || !desc->dims || !desc->has_activator) return SLONN_ERR_ARG;
+    if (desc->n_layers < 1 || desc->n_layers > SLONN_MAX_LAYERS) return SLONN_ERR_DIM;
+    if (desc->dtype != SLONN_F32 && desc->dtype != SLONN_BF16) return SLONN_ERR_DTYPE;
+    if (desc->K < 1 || desc->K > 16 || desc->L < 1 || desc->L > 8) return SLONN_ERR_DIM;
+    const uint32_t esz = desc->dtype == SLONN_BF16 ? 2u : 4u;
+    uint32_t n_act = 0;
+    for (uint32_t l = 0; l < desc->n_layers; ++l) {
+        const uint32_t D = desc->dims[l], N = desc->dims[l + 1];
+        if (D == 0 || N == 0) return SLONN_ERR_DIM;
+        if (!W[l] || !bias[l]) return SLONN_ERR_ARG;
+        const bool sparse0 = (l == 0 && desc->first_layer_sparse);
+        if (!sparse0 && (((uint64_t)D * esz) & 15u)) return SLONN_ERR_ALIGN;
+        if ((uintptr_t)W[l] & 15u) return SLONN_ERR_ALIGN;
+        if (desc->has_activator[l]) {
+            if (sparse0) return SLONN_ERR_ARG;
+            if (desc->K * desc->L > N) return SLONN_ERR_DIM;
+            ++n_act;
+        }
+    }
+    if (n_act) {
+        if (!calib || calib->n_rows == 0) return SLONN_ERR_ARG;
+        if (desc->first_layer_sparse ? (!calib->indptr || !calib->ids || !calib->vals) : !calib->dense)
+            return SLONN_ERR_ARG;
+        if (calib->dense && ((uintptr_t)calib->dense & 15u)) return SLONN_ERR_ALIGN;
+    }
+
+    slonn_model *m = new (std::nothrow) slonn_model;
+    if (!m) return SLONN_ERR_NOMEM;
+    memset(m, 0, sizeof(*m));
+    m->magic = SLONN_MAGIC;
+    cudaGetDevice(&m->device);
+    m->n_layers = desc->n_layers;
+    m->dtype = desc->dtype;
+    m->K = desc->K; m->L = desc->L; m->H = desc->K * desc->L;
+    m->list_cap = desc->list_cap;
+    m->first_sparse = desc->first_layer_sparse ? 1u : 0u;
+    for (uint32_t l = 0; l <= desc->n_layers; ++l) m->dims[l] = desc->dims[l];
+    for (uint32_t l = 0; l < desc->n_layers; ++l) {
+        slonn_layer &ly = m->layer[l];
+        ly.W = W[l]; ly.bias = bias[l]; ly.D = desc->dims[l]; ly.N = desc->dims[l + 1];
+        ly.has_act = desc->has_activator[l] ? 1u : 0u;
+        if (ly.has_act) m->act_index[l] = m->n_act++;
+    }
+
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = SLONN_OK;
+    float *cur = nullptr, *A = nullptr;
+    uint32_t *d_status = nullptr;
+    uint32_t last_needed = 0;
+    bool any = false;
+
+    if (m->first_sparse) {
+        slonn_layer &l0 = m->layer[0];
+        CK(cudaMalloc(&l0.WT, (uint64_t)l0.N * l0.D * esz));
+        transpose_kernel<<<dim3((l0.D + 31) / 32, (l0.N + 31) / 32), dim3(32, 8), 0, st>>>(l0.W, l0.WT, l0.N, l0.D, esz);
+        CK(cudaGetLastError());
+    }
+    for (uint32_t l = 0; l < m->n_layers; ++l)
+        if (m->layer[l].has_act) { last_needed = l; any = true; }
+    if (any) {
+        const uint32_t n_cal = calib->n_rows;
+        CK(cudaMalloc(&d_status, 4 * sizeof(uint32_t)));
+        CK(cudaMemsetAsync(d_status, 0, 4 * sizeof(uint32_t), st));
+        for (uint32_t l = 0; l <= last_needed; ++l) {
+            const slonn_layer &ly = m->layer[l];
+            const uint32_t relu = (l + 1 == m->n_layers) ? 0u : 1u;
+            CK(cudaMalloc(&A, sizeof(float) * (uint64_t)n_cal * ly.N));
+            if (l == 0 && m->first_sparse)
+                rc = slonn_forward_sparse_first(m, calib->indptr, calib->ids, calib->vals, n_cal, A, relu, d_status, st);
+            else
+                rc = slonn_forward_all_rows(m, l, l == 0 ? calib->dense : cur, n_cal, A, relu, st);
+            if (rc) goto fail;
+            if (ly.has_act) {
+                const uint32_t *ov = desc->hash_nodes_override ? desc->hash_nodes_override[l] : nullptr;
+                if ((rc = train_layer(m, l, A, n_cal, desc->seed, ov, st))) goto fail;
+            }
+            CK(cudaStreamSynchronize(st));
+            cudaFree(cur);
+            cur = A;
+            A = nullptr;
+        }
+        uint32_t hs[4];
+        CK(cudaMemcpy(hs, d_status, sizeof(hs), cudaMemcpyDeviceToHost));
+        if (hs[0]) { rc = -(int)hs[0]; goto fail; }
+    }
+    CK(cudaStreamSynchronize(st));
+    cudaFree(cur); cudaFree(A); cudaFree(d_status);
+    *out = m;
+    return SLONN_OK;
+fail:
+    cudaFree(cur); cudaFree(A); cudaFree(d_status);
+    slonn_free(m);
+    return rc;
+}

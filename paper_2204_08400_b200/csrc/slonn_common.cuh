@@ -1,0 +1,175 @@
+// Shared declarations of the SLO-NN library: the model object, launch parameter
+// blocks and the fixed-order warp dot product that every kernel uses.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/slonn.h"
+
+#define SLONN_FULL_MASK 0xffffffffu
+#define SLONN_MAGIC 0x534c4f4eu /* "SLON" */
+
+// ---- model -----------------------------------------------------------------
+
+struct slonn_layer {
+    const void *W;        // caller-owned, row-major [N][D]
+    const float *bias;    // caller-owned [N]
+    uint32_t D, N;
+    uint32_t has_act;
+    uint32_t cap;         // entries per bucket list
+    uint32_t id_bytes;    // 2 or 4
+    void *tables;         // library-owned [L][2^K][cap] ids
+    uint64_t table_bytes;
+    uint32_t *hash_nodes; // library-owned device copy, [L*K]
+    void *WT;             // library-owned transposed copy [D][N] (sparse-operand layer 0 only)
+};
+
+struct slonn_model {
+    uint32_t magic;
+    int device;
+    uint32_t n_layers;
+    uint32_t dims[SLONN_MAX_LAYERS + 1];
+    int32_t dtype;
+    uint32_t K, L, H;
+    uint32_t list_cap;
+    uint32_t first_sparse;
+    uint32_t n_act;
+    uint32_t act_index[SLONN_MAX_LAYERS]; // index of the layer among activator layers
+    slonn_layer layer[SLONN_MAX_LAYERS];
+    uint32_t hash_nodes_host[SLONN_MAX_LAYERS][128];
+};
+
+// ---- helpers ---------------------------------------------------------------
+
+// k% -> node count: nearest whole node, at least one (budget in basis points).
+__host__ __device__ __forceinline__ uint32_t slonn_budget_nodes(uint32_t bp, uint32_t N)
+{
+    uint64_t b = ((uint64_t)bp * N + 5000u) / 10000u;
+    if (b < 1) b = 1;
+    if (b > N) b = N;
+    return (uint32_t)b;
+}
+
+__device__ __forceinline__ void slonn_report(uint32_t *status, int code, uint32_t q, uint32_t layer)
+{
+    if (atomicCAS(status, 0u, (uint32_t)(-code)) == 0u) {
+        status[1] = q;
+        status[2] = layer;
+    }
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// Where input element j lives in the staged copy of a query's input vector.
+// fp32 weights: plain order.  bf16 weights: a 16-byte weight chunk holds 8
+// elements, so the 8 matching inputs are split into two float4 planes (first
+// four in plane 0, last four in plane 1) to keep 128-bit shared loads
+// conflict-free.
+template <bool BF16>
+__device__ __forceinline__ uint32_t xs_index(uint32_t j, uint32_t nchunks)
+{
+    if (BF16) return (((j >> 2) & 1u) * nchunks + (j >> 3)) * 4u + (j & 3u);
+    return j;
+}
+
+// Fixed-order dot products of R weight rows with the staged input, one warp.
+// Lane p owns partial sum p: it takes 16-byte chunks p, p+32, ... of each row
+// and accumulates their elements in ascending order with fused multiply-adds;
+// the xor butterfly then adds partials in the order 16, 8, 4, 2, 1.  Every lane
+// ends with the same sums.  Bias is added by the caller.
+template <bool BF16, int R>
+__device__ __forceinline__ void warp_dot_rows(const uint4 *const (&rows)[R], const float4 *xs4,
+                                              uint32_t nchunks, uint32_t lane, float (&acc)[R])
+{
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc[r] = 0.0f;
+#pragma unroll 2
+    for (uint32_t c = lane; c < nchunks; c += 32) {
+        uint4 w[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) w[r] = __ldg(rows[r] + c);
+        if (BF16) {
+            const float4 xa = xs4[c];
+            const float4 xb = xs4[nchunks + c];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float a = acc[r];
+                a = fmaf(bf16_lo(w[r].x), xa.x, a);
+                a = fmaf(bf16_hi(w[r].x), xa.y, a);
+                a = fmaf(bf16_lo(w[r].y), xa.z, a);
+                a = fmaf(bf16_hi(w[r].y), xa.w, a);
+                a = fmaf(bf16_lo(w[r].z), xb.x, a);
+                a = fmaf(bf16_hi(w[r].z), xb.y, a);
+                a = fmaf(bf16_lo(w[r].w), xb.z, a);
+                a = fmaf(bf16_hi(w[r].w), xb.w, a);
+                acc[r] = a;
+            }
+        } else {
+            const float4 xa = xs4[c];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float a = acc[r];
+                a = fmaf(__uint_as_float(w[r].x), xa.x, a);
+                a = fmaf(__uint_as_float(w[r].y), xa.y, a);
+                a = fmaf(__uint_as_float(w[r].z), xa.z, a);
+                a = fmaf(__uint_as_float(w[r].w), xa.w, a);
+                acc[r] = a;
+            }
+        }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) acc[r] = acc[r] + __shfl_xor_sync(SLONN_FULL_MASK, acc[r], off);
+    }
+}
+
+// ---- layer input descriptor --------------------------------------------------
+
+enum { SLONN_IN_DENSE = 0, SLONN_IN_LIST = 1 };
+
+struct slonn_input {
+    int kind;
+    const float *dense;     // DENSE: [n][D]
+    const uint64_t *indptr; // LIST: segment (q * ip_mul + ip_add) of ids / vals
+    const uint32_t *ids;
+    const float *vals;
+    uint32_t ip_mul, ip_add;
+};
+
+// Stages query q's input vector (D floats) into shared memory in xs_index order.
+// Must be called by the whole block; ends with a barrier.
+template <bool BF16>
+__device__ __forceinline__ void stage_input(const slonn_input &in, uint32_t q, uint32_t D,
+                                            uint32_t nchunks, float4 *xs4)
+{
+    const uint32_t nvec = D >> 2;
+    if (in.kind == SLONN_IN_DENSE) {
+        const float4 *src = reinterpret_cast<const float4 *>(in.dense + (uint64_t)q * D);
+        for (uint32_t i = threadIdx.x; i < nvec; i += blockDim.x) {
+            const float4 v = __ldg(src + i);
+            if (BF16) xs4[(i & 1u) * nchunks + (i >> 1)] = v;
+            else xs4[i] = v;
+        }
+    } else {
+        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (uint32_t i = threadIdx.x; i < nvec; i += blockDim.x) xs4[i] = z;
+        __syncthreads();
+        const uint64_t s0 = in.indptr[(uint64_t)q * in.ip_mul + in.ip_add];
+        const uint32_t len = (uint32_t)(in.indptr[(uint64_t)q * in.ip_mul + in.ip_add + 1] - s0);
+        float *xs = reinterpret_cast<float *>(xs4);
+        for (uint32_t i = threadIdx.x; i < len; i += blockDim.x) {
+            const uint32_t j = in.ids[s0 + i];
+            if (j < D) xs[xs_index<BF16>(j, nchunks)] = in.vals[s0 + i];
+        }
+    }
+    __syncthreads();
+}
+
+// ---- internal host entry points shared between translation units ---------------
+int slonn_forward_all_rows(const slonn_model *m, uint32_t l, const float *in_dense, uint32_t n, float *out,
+                           uint32_t relu, cudaStream_t st);
+int slonn_forward_sparse_first(const slonn_model *m, const uint64_t *indptr, const uint32_t *ids,
+                               const float *vals, uint32_t n, float *out, uint32_t relu, uint32_t *status,
+                               cudaStream_t st);

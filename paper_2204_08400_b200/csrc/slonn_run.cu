@@ -1,0 +1,400 @@
+// Host side of slonn_run: validates the batch, carves the workspace and
+// enqueues the per-layer kernels on the caller's stream.  No allocation, no
+// host synchronisation.
+#include <algorithm>
+#include <cstring>
+
+#include "slonn_run_kernels.cuh"
+
+namespace {
+
+inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+inline bool model_ok(const slonn_model *m) { return m && m->magic == SLONN_MAGIC; }
+
+inline uint32_t eff_max_bp(uint32_t max_bp) { return (max_bp == 0 || max_bp > 10000u) ? 10000u : max_bp; }
+
+// entries of the active CSR payload for n queries at max_bp
+uint64_t active_entries(const slonn_model *m, uint32_t n, uint32_t max_bp)
+{
+    uint64_t per = 0;
+    for (uint32_t l = 0; l < m->n_layers; ++l)
+        if (m->layer[l].has_act) per += slonn_budget_nodes(max_bp, m->layer[l].N);
+    return per * n;
+}
+
+// widest dense intermediate a non-activator hidden layer writes
+uint32_t dense_width(const slonn_model *m)
+{
+    uint32_t w = 0;
+    for (uint32_t l = 0; l + 1 < m->n_layers; ++l)
+        if (!m->layer[l].has_act) w = std::max(w, m->layer[l].N);
+    return w;
+}
+
+struct ws_layout {
+    uint64_t indptr, ids, vals, dense0, dense1, total;
+};
+
+ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp)
+{
+    ws_layout w;
+    const uint64_t ent = active_entries(m, n, max_bp);
+    uint64_t o = 0;
+    w.indptr = o; o = align_up(o + ((uint64_t)n * m->n_act + 1) * sizeof(uint64_t), 256);
+    w.ids = o; o = align_up(o + ent * sizeof(uint32_t), 256);
+    w.vals = o; o = align_up(o + ent * sizeof(float), 256);
+    const uint64_t db = align_up((uint64_t)n * dense_width(m) * sizeof(float), 256);
+    w.dense0 = o; o += db;
+    w.dense1 = o; o += db;
+    w.total = std::max<uint64_t>(o, 256);
+    return w;
+}
+
+template <typename K>
+int set_smem(K kernel, size_t bytes)
+{
+    if (bytes > 48 * 1024) {
+        if (bytes > 227 * 1024) return SLONN_ERR_DIM;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+            return SLONN_ERR_CUDA;
+    }
+    return SLONN_OK;
+}
+
+int launch_select(const slonn_model *m, const slonn_select_params &P, uint32_t n, cudaStream_t st)
+{
+    const size_t smem = (size_t)P.D * 4 + (size_t)((P.N + 31) / 32) * 4;
+    const bool bf = m->dtype == SLONN_BF16;
+    const bool id16 = m->layer[P.layer].id_bytes == 2;
+    int rc;
+    if (bf && id16) { if ((rc = set_smem(hash_select_kernel<true, uint16_t>, smem))) return rc;
+        hash_select_kernel<true, uint16_t><<<n, SLONN_THREADS, smem, st>>>(P); }
+    else if (bf) { if ((rc = set_smem(hash_select_kernel<true, uint32_t>, smem))) return rc;
+        hash_select_kernel<true, uint32_t><<<n, SLONN_THREADS, smem, st>>>(P); }
+    else if (id16) { if ((rc = set_smem(hash_select_kernel<false, uint16_t>, smem))) return rc;
+        hash_select_kernel<false, uint16_t><<<n, SLONN_THREADS, smem, st>>>(P); }
+    else { if ((rc = set_smem(hash_select_kernel<false, uint32_t>, smem))) return rc;
+        hash_select_kernel<false, uint32_t><<<n, SLONN_THREADS, smem, st>>>(P); }
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+// Rows per block: whole queries per block once the batch alone fills the GPU,
+// smaller row chunks for small batches so that every SM gets work.
+void gather_shape(uint32_t n, uint32_t max_rows, uint32_t *rows_per_cta, uint32_t *ctas_per_query)
+{
+    const uint32_t unit = (SLONN_THREADS / 32) * SLONN_ROWS_PER_WARP; // rows one block pass covers
+    const uint64_t want_ctas = 148ull * 16;                            // a few waves of resident blocks
+    uint64_t total_rows = (uint64_t)n * max_rows;
+    uint64_t rpc = (total_rows + want_ctas - 1) / want_ctas;
+    rpc = std::max<uint64_t>(unit, (rpc + unit - 1) / unit * unit);
+    if (rpc > max_rows) rpc = (max_rows + unit - 1) / unit * unit;
+    *rows_per_cta = (uint32_t)rpc;
+    *ctas_per_query = (uint32_t)((max_rows + rpc - 1) / rpc);
+}
+
+int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint32_t max_rows, cudaStream_t st)
+{
+    gather_shape(n, max_rows, &P.rows_per_cta, &P.ctas_per_query);
+    const size_t smem = (size_t)P.D * 4;
+    const uint64_t grid = (uint64_t)n * P.ctas_per_query;
+    if (grid == 0 || grid > 0x7fffffffull) return SLONN_ERR_DIM;
+    int rc;
+    if (m->dtype == SLONN_BF16) { if ((rc = set_smem(gather_dot_kernel<true>, smem))) return rc;
+        gather_dot_kernel<true><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(P); }
+    else { if ((rc = set_smem(gather_dot_kernel<false>, smem))) return rc;
+        gather_dot_kernel<false><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(P); }
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+} // namespace
+
+// ---- internal entry points used by the table builder --------------------------
+
+// Complete layer l (every node) for n dense input rows -> out [n][N_l].
+int slonn_forward_all_rows(const slonn_model *m, uint32_t l, const float *in_dense, uint32_t n, float *out,
+                           uint32_t relu, cudaStream_t st)
+{
+    const slonn_layer &ly = m->layer[l];
+    slonn_gather_params gp;
+    memset(&gp, 0, sizeof(gp));
+    gp.in.kind = SLONN_IN_DENSE; gp.in.dense = in_dense;
+    gp.W = ly.W; gp.bias = ly.bias; gp.D = ly.D; gp.N = ly.N;
+    gp.nchunks = ly.D * (m->dtype == SLONN_BF16 ? 2u : 4u) / 16u;
+    gp.use_list = 0; gp.out_dense = out; gp.out_stride = ly.N; gp.relu = relu;
+    return launch_gather(m, gp, n, ly.N, st);
+}
+
+// Complete layer 0 for n CSR rows -> out [n][N_0].
+int slonn_forward_sparse_first(const slonn_model *m, const uint64_t *indptr, const uint32_t *ids,
+                               const float *vals, uint32_t n, float *out, uint32_t relu, uint32_t *status,
+                               cudaStream_t st)
+{
+    const slonn_layer &ly = m->layer[0];
+    slonn_sparse_params sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.x_indptr = indptr; sp.x_ids = ids; sp.x_vals = vals;
+    sp.WT = ly.WT; sp.bias = ly.bias; sp.D = ly.D; sp.N = ly.N;
+    sp.out_dense = out; sp.out_stride = ly.N; sp.relu = relu;
+    sp.blocks_per_query = (ly.N + 127u) / 128u;
+    sp.status = status;
+    const uint64_t grid = (uint64_t)n * sp.blocks_per_query;
+    if (grid == 0 || grid > 0x7fffffffull) return SLONN_ERR_DIM;
+    if (m->dtype == SLONN_BF16) sparse_first_layer_kernel<true><<<(uint32_t)grid, 128, 0, st>>>(sp);
+    else sparse_first_layer_kernel<false><<<(uint32_t)grid, 128, 0, st>>>(sp);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+extern "C" int slonn_active_capacity(const slonn_model *m, uint32_t n, uint32_t max_bp, uint64_t *entries)
+{
+    if (!model_ok(m) || !entries) return SLONN_ERR_ARG;
+    *entries = active_entries(m, n, eff_max_bp(max_bp));
+    return SLONN_OK;
+}
+
+extern "C" int slonn_logit_stride(const slonn_model *m, uint32_t max_bp, uint32_t *stride)
+{
+    if (!model_ok(m) || !stride) return SLONN_ERR_ARG;
+    const slonn_layer &last = m->layer[m->n_layers - 1];
+    *stride = last.has_act ? slonn_budget_nodes(eff_max_bp(max_bp), last.N) : last.N;
+    return SLONN_OK;
+}
+
+extern "C" int slonn_workspace_bytes(const slonn_model *m, uint32_t n, uint32_t max_bp, uint64_t *bytes)
+{
+    if (!model_ok(m) || !bytes) return SLONN_ERR_ARG;
+    *bytes = carve(m, n, eff_max_bp(max_bp)).total;
+    return SLONN_OK;
+}
+
+extern "C" int slonn_run(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes,
+                         void *stream)
+{
+    if (!model_ok(m) || !b) return SLONN_ERR_ARG;
+    if (!b->budget_bp || !b->logits || !b->status) return SLONN_ERR_ARG;
+    if (m->first_sparse ? (!b->x_indptr || !b->x_ids || !b->x_vals) : !b->x_dense) return SLONN_ERR_ARG;
+    const slonn_layer &last = m->layer[m->n_layers - 1];
+    if (last.has_act && !b->logit_ids) return SLONN_ERR_ARG;
+    if (b->x_dense && ((uintptr_t)b->x_dense & 15u)) return SLONN_ERR_ALIGN;
+    const uint32_t n = b->n_queries;
+    const uint32_t max_bp = eff_max_bp(b->max_budget_bp);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(b->status, 0, 4 * sizeof(uint32_t), st) != cudaSuccess) return SLONN_ERR_CUDA;
+    if (n == 0) return SLONN_OK;
+
+    const ws_layout wl = carve(m, n, max_bp);
+    if (!workspace || ((uintptr_t)workspace & 255u) || ws_bytes < wl.total) return SLONN_ERR_WORKSPACE;
+    char *ws = (char *)workspace;
+    uint64_t *indptr = b->active_indptr ? b->active_indptr : (uint64_t *)(ws + wl.indptr);
+    uint32_t *ids = b->active_ids ? b->active_ids : (uint32_t *)(ws + wl.ids);
+    float *vals = b->active_vals ? b->active_vals : (float *)(ws + wl.vals);
+    float *dense[2] = {(float *)(ws + wl.dense0), (float *)(ws + wl.dense1)};
+
+    uint32_t stride = 0;
+    slonn_logit_stride(m, max_bp, &stride);
+
+    // offsets of every (query, activator layer) list
+    if (m->n_act) {
+        slonn_plan_params pp;
+        memset(&pp, 0, sizeof(pp));
+        pp.budget_bp = b->budget_bp; pp.n = n; pp.n_act = m->n_act; pp.max_bp = max_bp;
+        for (uint32_t l = 0; l < m->n_layers; ++l)
+            if (m->layer[l].has_act) {
+                const uint32_t a = m->act_index[l];
+                pp.act_N[a] = m->layer[l].N; pp.act_cap[a] = m->layer[l].cap; pp.act_layer[a] = l;
+            }
+        pp.indptr = indptr; pp.status = b->status;
+        plan_kernel<<<1, 1024, 0, st>>>(pp);
+        if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+    }
+
+    // input := x
+    slonn_input in;
+    memset(&in, 0, sizeof(in));
+    in.kind = SLONN_IN_DENSE;
+    in.dense = b->x_dense;
+    int dense_cur = 0;
+
+    for (uint32_t l = 0; l < m->n_layers; ++l) {
+        const slonn_layer &ly = m->layer[l];
+        const bool is_last = (l + 1 == m->n_layers);
+        const uint32_t esz = m->dtype == SLONN_BF16 ? 2u : 4u;
+        const uint32_t nchunks = ly.D * esz / 16u;
+        int rc;
+        if (l == 0 && m->first_sparse) {
+            float *o = is_last ? b->logits : dense[dense_cur];
+            if ((rc = slonn_forward_sparse_first(m, b->x_indptr, b->x_ids, b->x_vals, n, o, is_last ? 0u : 1u,
+                                                 b->status, st)))
+                return rc;
+            in.kind = SLONN_IN_DENSE; in.dense = o;
+            dense_cur ^= 1;
+            continue;
+        }
+        slonn_gather_params gp;
+        memset(&gp, 0, sizeof(gp));
+        gp.in = in; gp.W = ly.W; gp.bias = ly.bias; gp.D = ly.D; gp.N = ly.N; gp.nchunks = nchunks;
+        gp.n_act = m->n_act; gp.indptr = indptr; gp.ids = ids;
+        gp.relu = is_last ? 0u : 1u;
+        uint32_t max_rows = ly.N;
+        if (ly.has_act) {
+            const uint32_t a = m->act_index[l];
+            slonn_select_params sp;
+            memset(&sp, 0, sizeof(sp));
+            sp.in = in; sp.W = ly.W; sp.bias = ly.bias; sp.D = ly.D; sp.N = ly.N; sp.nchunks = nchunks;
+            sp.hash_nodes = ly.hash_nodes; sp.tables = ly.tables; sp.cap = ly.cap; sp.K = m->K; sp.L = m->L;
+            sp.n_act = m->n_act; sp.a = a; sp.layer = l; sp.indptr = indptr; sp.out_ids = ids;
+            sp.codes = b->codes; sp.status = b->status;
+            if ((rc = launch_select(m, sp, n, st))) return rc;
+            gp.use_list = 1; gp.a = a; gp.out_vals = vals;
+            if (is_last) { gp.out_dense = b->logits; gp.out_dense_ids = b->logit_ids; gp.out_stride = stride; }
+            max_rows = slonn_budget_nodes(max_bp, ly.N);
+            if ((rc = launch_gather(m, gp, n, max_rows, st))) return rc;
+            in.kind = SLONN_IN_LIST; in.indptr = indptr; in.ids = ids; in.vals = vals;
+            in.ip_mul = m->n_act; in.ip_add = a;
+        } else {
+            gp.use_list = 0;
+            gp.out_dense = is_last ? b->logits : dense[dense_cur];
+            gp.out_stride = ly.N;
+            if ((rc = launch_gather(m, gp, n, max_rows, st))) return rc;
+            in.kind = SLONN_IN_DENSE; in.dense = gp.out_dense;
+            dense_cur ^= 1;
+        }
+    }
+
+    if (b->pred) {
+        slonn_argmax_params ap;
+        memset(&ap, 0, sizeof(ap));
+        ap.logits = b->logits; ap.stride = stride; ap.n = n; ap.pred = b->pred;
+        if (last.has_act) {
+            ap.logit_ids = b->logit_ids; ap.indptr = indptr; ap.n_act = m->n_act;
+            ap.a = m->act_index[m->n_layers - 1];
+        } else {
+            ap.fixed_len = last.N;
+        }
+        argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
+        if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+    }
+    return SLONN_OK;
+}
+
+// ---- host-buffer variant -----------------------------------------------------
+
+namespace {
+struct host_layout {
+    uint64_t x, indptr_in, ids_in, vals_in, bp, logits, logit_ids, pred, codes, a_indptr, a_ids, a_vals, status,
+        inner, total;
+};
+
+host_layout carve_host(const slonn_model *m, uint32_t n, uint32_t max_bp, uint64_t x_nnz)
+{
+    host_layout h;
+    memset(&h, 0, sizeof(h));
+    uint32_t stride = 0;
+    slonn_logit_stride(m, max_bp, &stride);
+    const uint64_t ent = active_entries(m, n, max_bp);
+    uint64_t o = 0;
+    auto take = [&](uint64_t bytes) { uint64_t at = o; o = align_up(o + bytes, 256); return at; };
+    if (m->first_sparse) {
+        h.indptr_in = take(((uint64_t)n + 1) * 8);
+        h.ids_in = take(x_nnz * 4);
+        h.vals_in = take(x_nnz * 4);
+    } else {
+        h.x = take((uint64_t)n * m->dims[0] * 4);
+    }
+    h.bp = take((uint64_t)n * 2);
+    h.logits = take((uint64_t)n * stride * 4);
+    h.logit_ids = take((uint64_t)n * stride * 4);
+    h.pred = take((uint64_t)n * 4);
+    h.codes = take((uint64_t)n * m->n_act * m->L * 2);
+    h.a_indptr = take(((uint64_t)n * m->n_act + 1) * 8);
+    h.a_ids = take(ent * 4);
+    h.a_vals = take(ent * 4);
+    h.status = take(16);
+    h.inner = o;
+    h.total = o + carve(m, n, max_bp).total;
+    return h;
+}
+} // namespace
+
+extern "C" int slonn_host_workspace_bytes(const slonn_model *m, uint32_t n, uint32_t max_bp, uint64_t x_nnz,
+                                          uint64_t *bytes)
+{
+    if (!model_ok(m) || !bytes) return SLONN_ERR_ARG;
+    *bytes = carve_host(m, n, eff_max_bp(max_bp), x_nnz).total;
+    return SLONN_OK;
+}
+
+extern "C" int slonn_run_host(const slonn_model *m, const slonn_batch *hb, void *workspace, uint64_t ws_bytes,
+                              void *stream, uint64_t *h2d_bytes, uint64_t *d2h_bytes)
+{
+    if (!model_ok(m) || !hb) return SLONN_ERR_ARG;
+    if (!hb->budget_bp || !hb->logits || !hb->status) return SLONN_ERR_ARG;
+    if (m->first_sparse ? (!hb->x_indptr || !hb->x_ids || !hb->x_vals) : !hb->x_dense) return SLONN_ERR_ARG;
+    const slonn_layer &last = m->layer[m->n_layers - 1];
+    if (last.has_act && !hb->logit_ids) return SLONN_ERR_ARG;
+    const uint32_t n = hb->n_queries;
+    const uint32_t max_bp = eff_max_bp(hb->max_budget_bp);
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint64_t x_nnz = m->first_sparse ? hb->x_indptr[n] : 0; // host array: readable here
+    const host_layout hl = carve_host(m, n, max_bp, x_nnz);
+    if (!workspace || ((uintptr_t)workspace & 255u) || ws_bytes < hl.total) return SLONN_ERR_WORKSPACE;
+    char *ws = (char *)workspace;
+    uint32_t stride = 0;
+    slonn_logit_stride(m, max_bp, &stride);
+    const uint64_t ent = active_entries(m, n, max_bp);
+    uint64_t up = 0, down = 0;
+#define H2D(dst, src, bytes)                                                                      \
+    do {                                                                                          \
+        if ((bytes) && cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyHostToDevice, st) != cudaSuccess) \
+            return SLONN_ERR_CUDA;                                                                \
+        up += (bytes);                                                                            \
+    } while (0)
+#define D2H(dst, src, bytes)                                                                      \
+    do {                                                                                          \
+        if ((bytes) && cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToHost, st) != cudaSuccess) \
+            return SLONN_ERR_CUDA;                                                                \
+        down += (bytes);                                                                          \
+    } while (0)
+
+    slonn_batch db = *hb;
+    if (m->first_sparse) {
+        H2D(ws + hl.indptr_in, hb->x_indptr, ((uint64_t)n + 1) * 8);
+        H2D(ws + hl.ids_in, hb->x_ids, x_nnz * 4);
+        H2D(ws + hl.vals_in, hb->x_vals, x_nnz * 4);
+        db.x_dense = nullptr;
+        db.x_indptr = (const uint64_t *)(ws + hl.indptr_in);
+        db.x_ids = (const uint32_t *)(ws + hl.ids_in);
+        db.x_vals = (const float *)(ws + hl.vals_in);
+    } else {
+        H2D(ws + hl.x, hb->x_dense, (uint64_t)n * m->dims[0] * 4);
+        db.x_dense = (const float *)(ws + hl.x);
+    }
+    H2D(ws + hl.bp, hb->budget_bp, (uint64_t)n * 2);
+    db.budget_bp = (const uint16_t *)(ws + hl.bp);
+    db.logits = (float *)(ws + hl.logits);
+    db.logit_ids = last.has_act ? (uint32_t *)(ws + hl.logit_ids) : nullptr;
+    db.pred = hb->pred ? (uint32_t *)(ws + hl.pred) : nullptr;
+    db.codes = hb->codes ? (uint16_t *)(ws + hl.codes) : nullptr;
+    db.active_indptr = (uint64_t *)(ws + hl.a_indptr);
+    db.active_ids = (uint32_t *)(ws + hl.a_ids);
+    db.active_vals = (float *)(ws + hl.a_vals);
+    db.status = (uint32_t *)(ws + hl.status);
+
+    const int rc = slonn_run(m, &db, ws + hl.inner, ws_bytes - hl.inner, st);
+    if (rc) return rc;
+
+    D2H(hb->logits, db.logits, (uint64_t)n * stride * 4);
+    if (last.has_act) D2H(hb->logit_ids, db.logit_ids, (uint64_t)n * stride * 4);
+    if (hb->pred) D2H(hb->pred, db.pred, (uint64_t)n * 4);
+    if (hb->codes) D2H(hb->codes, db.codes, (uint64_t)n * m->n_act * m->L * 2);
+    if (hb->active_indptr) D2H(hb->active_indptr, db.active_indptr, ((uint64_t)n * m->n_act + 1) * 8);
+    if (hb->active_ids) D2H(hb->active_ids, db.active_ids, ent * 4);
+    if (hb->active_vals) D2H(hb->active_vals, db.active_vals, ent * 4);
+    D2H(hb->status, db.status, 16);
+#undef H2D
+#undef D2H
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SLONN_ERR_CUDA;
+    if (h2d_bytes) *h2d_bytes = up;
+    if (d2h_bytes) *d2h_bytes = down;
+    return SLONN_OK;
+}

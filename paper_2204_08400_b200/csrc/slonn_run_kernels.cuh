@@ -1,0 +1,431 @@
+// Kernels of the SLO-aware forward pass (Fig. 2 steps 1, 3, 4 of the paper):
+//   plan_kernel              budgets -> per (query, activator layer) list offsets
+//   hash_select_kernel       FreeHash bits -> keys -> bucket lists -> first B distinct ids
+//   gather_dot_kernel        the selected rows' dot products, bias, activation
+//   sparse_first_layer_kernel  layer 0 fed by CSR rows (transposed weights)
+//   argmax_kernel            prediction over the computed logits
+#pragma once
+#include "slonn_common.cuh"
+
+#define SLONN_THREADS 256
+#define SLONN_ROWS_PER_WARP 4
+
+// ---------------------------------------------------------------------------
+// block-wide exclusive scan of one value per thread (blockDim.x <= 1024)
+// ---------------------------------------------------------------------------
+template <typename T>
+__device__ __forceinline__ T block_exclusive_scan(T v, T *warp_sums /* [32] shared */, T *total)
+{
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    T incl = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        T t = __shfl_up_sync(SLONN_FULL_MASK, incl, off);
+        if (lane >= (uint32_t)off) incl += t;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t nw = (blockDim.x + 31u) >> 5;
+        T w = lane < nw ? warp_sums[lane] : (T)0;
+        T wi = w;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            T t = __shfl_up_sync(SLONN_FULL_MASK, wi, off);
+            if (lane >= (uint32_t)off) wi += t;
+        }
+        warp_sums[lane] = wi - w; // exclusive warp offsets
+        if (lane == 31) *total = wi;
+    }
+    __syncthreads();
+    const T res = warp_sums[warp] + incl - v;
+    __syncthreads();
+    return res;
+}
+
+// ---------------------------------------------------------------------------
+// plan: node counts and offsets from the budgets (one block)
+// ---------------------------------------------------------------------------
+struct slonn_plan_params {
+    const uint16_t *budget_bp;
+    uint32_t n, n_act, max_bp;
+    uint32_t act_N[SLONN_MAX_LAYERS];
+    uint32_t act_cap[SLONN_MAX_LAYERS];
+    uint32_t act_layer[SLONN_MAX_LAYERS];
+    uint64_t *indptr; // [n * n_act + 1]
+    uint32_t *status;
+};
+
+__device__ __forceinline__ uint32_t plan_count(const slonn_plan_params &P, uint64_t e, bool check)
+{
+    const uint32_t q = (uint32_t)(e / P.n_act), a = (uint32_t)(e % P.n_act);
+    uint32_t bp = P.budget_bp[q];
+    bool bad = (bp < 1u) || (bp > 10000u) || (bp > P.max_bp);
+    if (bp < 1u) bp = 1u;
+    if (bp > P.max_bp) bp = P.max_bp;
+    const uint32_t B = slonn_budget_nodes(bp, P.act_N[a]);
+    if (B > P.act_cap[a] && B != P.act_N[a]) bad = true;
+    if (bad && check) slonn_report(P.status, SLONN_ERR_BUDGET, q, P.act_layer[a]);
+    return B;
+}
+
+__global__ void __launch_bounds__(1024) plan_kernel(slonn_plan_params P)
+{
+    __shared__ uint64_t warp_sums[32];
+    __shared__ uint64_t total;
+    const uint64_t M = (uint64_t)P.n * P.n_act;
+    const uint64_t per = (M + blockDim.x - 1) / blockDim.x;
+    const uint64_t e0 = (uint64_t)threadIdx.x * per;
+    const uint64_t e1 = e0 + per < M ? e0 + per : M;
+    uint64_t local = 0;
+    for (uint64_t e = e0; e < e1; ++e) local += plan_count(P, e, true);
+    uint64_t run = block_exclusive_scan<uint64_t>(local, warp_sums, &total);
+    for (uint64_t e = e0; e < e1; ++e) {
+        P.indptr[e] = run;
+        run += plan_count(P, e, false);
+    }
+    if (threadIdx.x == 0) P.indptr[M] = total;
+}
+
+// ---------------------------------------------------------------------------
+// hash + select: one block per query
+// ---------------------------------------------------------------------------
+struct slonn_select_params {
+    slonn_input in;
+    const void *W;
+    const float *bias;
+    uint32_t D, N, nchunks;
+    const uint32_t *hash_nodes; // device [L*K]
+    const void *tables;         // [L][2^K][cap]
+    uint32_t cap, K, L;
+    uint32_t n_act, a, layer;
+    const uint64_t *indptr;     // offsets of (q, a)
+    uint32_t *out_ids;          // CSR payload
+    uint16_t *codes;            // nullable [n][n_act][L]
+    uint32_t *status;
+};
+
+template <typename IDT>
+__device__ __forceinline__ uint32_t table_entry(const void *tables, uint32_t cap, uint32_t K,
+                                                uint32_t b, uint32_t key, uint32_t r)
+{
+    const IDT *t = reinterpret_cast<const IDT *>(tables);
+    return (uint32_t)__ldg(t + (((uint64_t)b << K) + key) * cap + r);
+}
+
+template <bool BF16, typename IDT>
+__global__ void __launch_bounds__(SLONN_THREADS) hash_select_kernel(slonn_select_params P)
+{
+    extern __shared__ float4 smem4[];
+    float4 *xs4 = smem4;
+    uint32_t *bitmap = reinterpret_cast<uint32_t *>(smem4 + (P.D >> 2));
+    __shared__ float zh[128];
+    __shared__ uint32_t keys[8];
+    __shared__ uint32_t scan_ws[32];
+    __shared__ uint32_t scan_total;
+    __shared__ uint32_t s_total;
+
+    const uint32_t q = blockIdx.x;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const uint32_t H = P.K * P.L;
+    const uint64_t off = P.indptr[(uint64_t)q * P.n_act + P.a];
+    const uint32_t B = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - off);
+    const uint32_t nwords = (P.N + 31u) >> 5;
+
+    // (1) FreeHash: z_h = w_h . x + b_h for the layer's K*L hash nodes
+    stage_input<BF16>(P.in, q, P.D, P.nchunks, xs4);
+    const uint32_t row_u4 = P.nchunks; // uint4 per weight row
+    for (uint32_t h0 = warp * SLONN_ROWS_PER_WARP; h0 < H; h0 += nwarps * SLONN_ROWS_PER_WARP) {
+        const uint4 *rows[SLONN_ROWS_PER_WARP];
+        uint32_t node[SLONN_ROWS_PER_WARP];
+#pragma unroll
+        for (int r = 0; r < SLONN_ROWS_PER_WARP; ++r) {
+            const uint32_t h = min(h0 + r, H - 1);
+            node[r] = __ldg(P.hash_nodes + h);
+            rows[r] = reinterpret_cast<const uint4 *>(P.W) + (uint64_t)node[r] * row_u4;
+        }
+        float acc[SLONN_ROWS_PER_WARP];
+        warp_dot_rows<BF16, SLONN_ROWS_PER_WARP>(rows, xs4, P.nchunks, lane, acc);
+#pragma unroll
+        for (int r = 0; r < SLONN_ROWS_PER_WARP; ++r)
+            if (lane == (uint32_t)r && h0 + r < H) zh[h0 + r] = acc[r] + __ldg(P.bias + node[r]);
+    }
+    for (uint32_t i = threadIdx.x; i < nwords; i += blockDim.x) bitmap[i] = 0u;
+    __syncthreads();
+
+    // (2) keys: bit j of key_b = [z of hash function j of table b > 0]
+    if (threadIdx.x < P.L) {
+        uint32_t key = 0;
+        for (uint32_t j = 0; j < P.K; ++j)
+            if (zh[threadIdx.x * P.K + j] > 0.0f) key |= (1u << j);
+        keys[threadIdx.x] = key;
+        if (P.codes) P.codes[((uint64_t)q * P.n_act + P.a) * P.L + threadIdx.x] = (uint16_t)key;
+    }
+    if (threadIdx.x == 0) s_total = 0;
+    __syncthreads();
+
+    uint32_t *out = P.out_ids + off;
+    if (B == P.N) { // every node
+        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
+        return;
+    }
+    if (B > P.cap) { // reported by the plan; keep the output in range
+        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
+        return;
+    }
+
+    // (3)+(4) read the L lists rank by rank; the first B distinct ids are the active set.
+    // Position pos = rank * L + table.  A block-wide step marks blockDim.x positions
+    // at once; the step that would pass B is undone and replayed 32 positions at a
+    // time by warp 0, which cuts exactly at B.
+    const uint32_t npos = B * P.L; // B distinct ids are always found within rank < B
+    uint32_t total = 0;
+    for (uint32_t base = 0; base < npos; base += blockDim.x) {
+        const uint32_t pos = base + threadIdx.x;
+        const bool valid = pos < npos;
+        uint32_t id = 0;
+        bool won = false;
+        if (valid) {
+            const uint32_t r = pos / P.L, b = pos - r * P.L;
+            id = table_entry<IDT>(P.tables, P.cap, P.K, b, keys[b], r);
+            if (id < P.N) {
+                const uint32_t bit = 1u << (id & 31u);
+                won = (atomicOr(&bitmap[id >> 5], bit) & bit) == 0u;
+            }
+        }
+        const uint32_t cnt = (uint32_t)__syncthreads_count(won);
+        if (total + cnt < B) { total += cnt; continue; }
+        if (total + cnt == B) { total = B; break; }
+        // crossing step: undo, then replay in order
+        if (won) atomicAnd(&bitmap[id >> 5], ~(1u << (id & 31u)));
+        __syncthreads();
+        if (warp == 0) {
+            for (uint32_t sub = 0; sub < blockDim.x && total < B; sub += 32) {
+                const uint32_t p2 = base + sub + lane;
+                const bool v2 = p2 < npos;
+                uint32_t id2 = 0xffffffffu - lane; // distinct dummies
+                bool fresh = false;
+                if (v2) {
+                    const uint32_t r = p2 / P.L, b = p2 - r * P.L;
+                    id2 = table_entry<IDT>(P.tables, P.cap, P.K, b, keys[b], r);
+                    if (id2 < P.N) fresh = ((bitmap[id2 >> 5] >> (id2 & 31u)) & 1u) == 0u;
+                }
+                const uint32_t same = __match_any_sync(SLONN_FULL_MASK, id2);
+                const bool first = (uint32_t)(__ffs(same) - 1) == lane;
+                const bool take = fresh && first;
+                const uint32_t bal = __ballot_sync(SLONN_FULL_MASK, take);
+                const uint32_t need = B - total;
+                const uint32_t rank = __popc(bal & ((1u << lane) - 1u));
+                if (take && rank < need) atomicOr(&bitmap[id2 >> 5], 1u << (id2 & 31u));
+                const uint32_t c = (uint32_t)__popc(bal);
+                total += c < need ? c : need;
+                __syncwarp();
+            }
+            if (lane == 0) s_total = total;
+        }
+        __syncthreads();
+        total = s_total;
+        break;
+    }
+    __syncthreads();
+    if (total != B) { // cannot happen with well-formed tables; keep the output in range
+        if (threadIdx.x == 0) slonn_report(P.status, SLONN_ERR_ARG, q, P.layer);
+        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
+        return;
+    }
+
+    // emit ascending ids: popcount prefix over the bitmap words
+    const uint32_t wpt = (nwords + blockDim.x - 1) / blockDim.x;
+    const uint32_t w0 = threadIdx.x * wpt;
+    const uint32_t w1 = min(w0 + wpt, nwords);
+    uint32_t cnt = 0;
+    for (uint32_t w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+    uint32_t o = block_exclusive_scan<uint32_t>(cnt, scan_ws, &scan_total);
+    for (uint32_t w = w0; w < w1; ++w) {
+        uint32_t bits = bitmap[w];
+        while (bits) {
+            const uint32_t t = __ffs(bits) - 1;
+            bits &= bits - 1;
+            out[o++] = (w << 5) + t;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// gather-dot: the selected rows of one layer
+// ---------------------------------------------------------------------------
+struct slonn_gather_params {
+    slonn_input in;
+    const void *W;
+    const float *bias;
+    uint32_t D, N, nchunks;
+    uint32_t use_list;        // 1: rows = active ids of (q, a); 0: every row
+    uint32_t n_act, a;
+    const uint64_t *indptr;
+    const uint32_t *ids;      // CSR payload (use_list)
+    float *out_vals;          // CSR payload (use_list), nullable
+    float *out_dense;         // [n][N] (!use_list), or strided copy [n][out_stride] (use_list), nullable
+    uint32_t *out_dense_ids;  // [n][out_stride] ids beside the strided copy, nullable
+    uint32_t out_stride;
+    uint32_t relu;
+    uint32_t rows_per_cta, ctas_per_query;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_params P)
+{
+    extern __shared__ float4 smem4[];
+    const uint32_t q = blockIdx.x / P.ctas_per_query;
+    const uint32_t chunk = blockIdx.x - q * P.ctas_per_query;
+    uint64_t off = 0;
+    uint32_t B = P.N;
+    if (P.use_list) {
+        off = P.indptr[(uint64_t)q * P.n_act + P.a];
+        B = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - off);
+    }
+    const uint32_t r0 = chunk * P.rows_per_cta;
+    if (r0 >= B) return;
+    const uint32_t r1 = min(B, r0 + P.rows_per_cta);
+
+    stage_input<BF16>(P.in, q, P.D, P.nchunks, smem4);
+
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (uint32_t r = r0 + warp * SLONN_ROWS_PER_WARP; r < r1; r += nwarps * SLONN_ROWS_PER_WARP) {
+        const uint4 *rows[SLONN_ROWS_PER_WARP];
+        uint32_t node[SLONN_ROWS_PER_WARP];
+#pragma unroll
+        for (int k = 0; k < SLONN_ROWS_PER_WARP; ++k) {
+            const uint32_t rr = min(r + k, r1 - 1);
+            node[k] = P.use_list ? __ldg(P.ids + off + rr) : rr;
+            rows[k] = reinterpret_cast<const uint4 *>(P.W) + (uint64_t)node[k] * P.nchunks;
+        }
+        float acc[SLONN_ROWS_PER_WARP];
+        warp_dot_rows<BF16, SLONN_ROWS_PER_WARP>(rows, smem4, P.nchunks, lane, acc);
+#pragma unroll
+        for (int k = 0; k < SLONN_ROWS_PER_WARP; ++k) {
+            if (lane == (uint32_t)k && r + k < r1) {
+                float z = acc[k] + __ldg(P.bias + node[k]);
+                if (P.relu) z = z > 0.0f ? z : 0.0f;
+                if (P.use_list) {
+                    if (P.out_vals) P.out_vals[off + r + k] = z;
+                    if (P.out_dense) {
+                        P.out_dense[(uint64_t)q * P.out_stride + r + k] = z;
+                        if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q * P.out_stride + r + k] = node[k];
+                    }
+                } else {
+                    P.out_dense[(uint64_t)q * P.out_stride + node[k]] = z;
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// layer 0 fed by CSR rows (sparse operand): thread n owns output node n and walks
+// the row's nonzeros in id order; nonzero number j goes to partial sum j mod 32.
+// WT is the transposed weight copy [D][N], so each nonzero reads one contiguous row.
+// ---------------------------------------------------------------------------
+struct slonn_sparse_params {
+    const uint64_t *x_indptr;
+    const uint32_t *x_ids;
+    const float *x_vals;
+    const void *WT;
+    const float *bias;
+    uint32_t D, N;
+    float *out_dense; // [n][out_stride]
+    uint32_t out_stride;
+    uint32_t relu;
+    uint32_t blocks_per_query; // ceil(N / 128)
+    uint32_t *status;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(128) sparse_first_layer_kernel(slonn_sparse_params P)
+{
+    __shared__ uint32_t s_ids[128];
+    __shared__ float s_vals[128];
+    const uint32_t q = blockIdx.x / P.blocks_per_query;
+    const uint32_t n = (blockIdx.x - q * P.blocks_per_query) * blockDim.x + threadIdx.x;
+    const uint64_t s0 = P.x_indptr[q];
+    const uint32_t nnz = (uint32_t)(P.x_indptr[q + 1] - s0);
+    float acc[32];
+#pragma unroll
+    for (int p = 0; p < 32; ++p) acc[p] = 0.0f;
+    for (uint32_t base = 0; base < nnz; base += 128) {
+        __syncthreads();
+        if (base + threadIdx.x < nnz) {
+            uint32_t id = P.x_ids[s0 + base + threadIdx.x];
+            float v = P.x_vals[s0 + base + threadIdx.x];
+            if (id >= P.D) { slonn_report(P.status, SLONN_ERR_ARG, q, 0); id = 0; v = 0.0f; }
+            s_ids[threadIdx.x] = id;
+            s_vals[threadIdx.x] = v;
+        }
+        __syncthreads();
+        if (n < P.N) {
+            const uint32_t m = min(128u, nnz - base);
+#pragma unroll
+            for (uint32_t jb = 0; jb < 128; jb += 32) {
+#pragma unroll
+                for (uint32_t p = 0; p < 32; ++p) {
+                    if (jb + p < m) {
+                        const uint64_t idx = (uint64_t)s_ids[jb + p] * P.N + n;
+                        float w;
+                        if (BF16) w = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(P.WT) + idx) << 16);
+                        else w = __ldg(reinterpret_cast<const float *>(P.WT) + idx);
+                        acc[p] = fmaf(w, s_vals[jb + p], acc[p]);
+                    }
+                }
+            }
+        }
+    }
+    if (n >= P.N) return;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+#pragma unroll
+        for (int p = 0; p < off; ++p) acc[p] = acc[p] + acc[p + off];
+    }
+    float z = acc[0] + __ldg(P.bias + n);
+    if (P.relu) z = z > 0.0f ? z : 0.0f;
+    P.out_dense[(uint64_t)q * P.out_stride + n] = z;
+}
+
+// ---------------------------------------------------------------------------
+// argmax over each query's computed logits (one warp per query)
+// ---------------------------------------------------------------------------
+struct slonn_argmax_params {
+    const float *logits;       // [n][stride]
+    const uint32_t *logit_ids; // nullable: position -> node id
+    uint32_t stride, n;
+    uint32_t fixed_len;        // used when indptr == NULL
+    const uint64_t *indptr;    // budgeted last layer: length of (q, a)
+    uint32_t n_act, a;
+    uint32_t *pred;
+};
+
+__global__ void __launch_bounds__(256) argmax_kernel(slonn_argmax_params P)
+{
+    const uint32_t q = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const uint32_t lane = threadIdx.x & 31u;
+    if (q >= P.n) return;
+    uint32_t len = P.fixed_len;
+    if (P.indptr)
+        len = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - P.indptr[(uint64_t)q * P.n_act + P.a]);
+    const float *lg = P.logits + (uint64_t)q * P.stride;
+    float best = 0.0f;
+    uint32_t bi = 0xffffffffu;
+    for (uint32_t i = lane; i < len; i += 32) {
+        const float v = lg[i];
+        if (bi == 0xffffffffu || v > best) { best = v; bi = i; }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const float ob = __shfl_xor_sync(SLONN_FULL_MASK, best, off);
+        const uint32_t oi = __shfl_xor_sync(SLONN_FULL_MASK, bi, off);
+        if (oi != 0xffffffffu && (bi == 0xffffffffu || ob > best || (ob == best && oi < bi))) {
+            best = ob;
+            bi = oi;
+        }
+    }
+    if (lane == 0 && bi != 0xffffffffu)
+        P.pred[q] = P.logit_ids ? P.logit_ids[(uint64_t)q * P.stride + bi] : bi;
+}

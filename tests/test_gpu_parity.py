@@ -1,0 +1,197 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on
+the same seeded inputs.  Integer results (hash codes, bucket contents, active
+sets, argmax) must be bit-exact; logits within 1e-5 (fp32 weights) / 2e-2 (bf16
+weights) of the fp64 oracle, relative to the largest logit of the query."""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2204_08400_b200 import workloads as wl_mod
+from paper_2204_08400_b200.workloads import Workload
+from parity_util import assert_build_parity, assert_run_parity, oracle_model, oracle_run, take_queries
+
+pytestmark = pytest.mark.gpu
+
+
+def custom_workload(seed, dims, has_act, dtype, n, n_cal, K, L, law="relu_normal", bias_scale=0.2,
+                    list_cap=0, budgets=(500, 1000, 2500, 5000, 10000)):
+    W_f32, W_store, bias = wl_mod.draw_mlp(dims, seed, dtype, bias_scale=bias_scale)
+    x = wl_mod.draw_dense_inputs(n, dims[0], seed + 1, law)
+    calib = wl_mod.draw_dense_inputs(n_cal, dims[0], seed + 2, law)
+    bp = wl_mod.draw_mixed_budgets(n, seed + 3, budgets)
+    return Workload(name="custom", dims=list(dims), has_act=list(has_act), dtype=dtype, W_f32=W_f32,
+                    W_store=W_store, bias=bias, first_sparse=False, calib=calib, x=x, budget_bp=bp,
+                    K=K, L=L, seed=seed + 4, list_cap=list_cap)
+
+
+def check(wl, n_cal=None, sample=None, expect_build=True):
+    from paper_2204_08400_b200 import harness
+    dm = harness.DeviceModel(wl, n_cal=n_cal)
+    om = oracle_model(wl, n_cal=n_cal)
+    if expect_build:
+        assert_build_parity(dm, om, wl)
+    g = harness.run_once(dm, wl.x, wl.budget_bp)
+    n_act = sum(wl.has_act)
+    if sample is None:
+        x, bp = wl.x, wl.budget_bp
+    else:
+        x, bp = take_queries(wl, sample), wl.budget_bp[sample]
+        g = slice_results(g, sample, n_act)
+    o32 = oracle_run(om, wl, x, bp, orc.CANON32)
+    o64 = oracle_run(om, wl, x, bp, orc.REF64)
+    info = assert_run_parity(g, o32, o64, wl, n_act, bool(wl.has_act[-1]))
+    dm.free()
+    return info
+
+
+def slice_results(g, idx, n_act):
+    """Restrict full-batch GPU results to the sampled queries (CSR payload re-packed)."""
+    idx = np.asarray(idx)
+    ip = g["active_indptr"].astype(np.int64)
+    out = {"status": g["status"], "logits": g["logits"][idx], "pred": g["pred"][idx],
+           "codes": g["codes"][idx], "logit_stride": g["logit_stride"]}
+    if "logit_ids" in g:
+        out["logit_ids"] = g["logit_ids"][idx]
+    nip = [0]
+    ids, vals = [], []
+    for q in idx:
+        for a in range(n_act):
+            s, e = ip[q * n_act + a], ip[q * n_act + a + 1]
+            ids.append(g["active_ids"][s:e]); vals.append(g["active_vals"][s:e])
+            nip.append(nip[-1] + int(e - s))
+    out["active_indptr"] = np.asarray(nip, dtype=np.uint64)
+    out["active_ids"] = np.concatenate(ids) if ids else np.zeros(0, np.uint32)
+    out["active_vals"] = np.concatenate(vals) if vals else np.zeros(0, np.float32)
+    return out
+
+
+# ---- small shapes spanning several tiles and ragged tails ----------------------
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_small_mlp_mixed_budgets(dtype):
+    wl = custom_workload(50, [136, 200, 96, 24], [1, 1, 0], dtype, n=300, n_cal=700, K=4, L=2)
+    check(wl)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_three_tables_and_output_activator(dtype):
+    wl = custom_workload(51, [72, 160, 328], [1, 1], dtype, n=120, n_cal=500, K=3, L=3,
+                         budgets=(100, 700, 3300, 10000))
+    check(wl)
+
+
+def test_single_table_single_bit():
+    wl = custom_workload(52, [40, 64, 8], [1, 0], "f32", n=64, n_cal=100, K=1, L=1)
+    check(wl)
+
+
+def test_list_cap():
+    wl = custom_workload(53, [64, 256, 16], [1, 0], "bf16", n=200, n_cal=600, K=5, L=2, list_cap=70,
+                         budgets=(100, 1000, 2500, 10000))   # B = 3, 26, 64, 256 (all)
+    check(wl)
+
+
+def test_no_activators_is_the_dense_network():
+    wl = custom_workload(54, [96, 128, 40], [0, 0], "f32", n=77, n_cal=10, K=2, L=1)
+    check(wl)
+
+
+# ---- the benchmark shapes -------------------------------------------------------
+
+def test_c1_full():
+    for bp in (1000, 2500, 5000, 10000):
+        wl = wl_mod.load("c1", budget_bp=bp, n_cal=4096)
+        check(wl, expect_build=(bp == 1000))
+
+
+def test_c2_reduced_queries_all_budgets():
+    for bp in (500, 1000, 2500, 5000, 10000):
+        wl = wl_mod.load("c2", n_queries=1024, n_cal=2048, budget_bp=bp)
+        check(wl, expect_build=(bp == 500))
+
+
+def test_c3_narrow_output():
+    # same structure as the wide-output net with a 20,000-node output layer
+    for bp in (100, 500, 1000):
+        wl = wl_mod.load("c3", n_queries=64, n_cal=512, budget_bp=bp, dims=[100000, 128, 20000])
+        check(wl, expect_build=(bp == 100))
+
+
+def test_c4_narrow_batches():
+    for n in (1, 64):
+        wl = wl_mod.load("c4", n_queries=n, n_cal=1024, budget_bp=2500, dims=[512] + [512] * 8 + [104])
+        check(wl, expect_build=(n == 1))
+
+
+def test_c5_mixed_budgets_reduced():
+    wl = wl_mod.load("c5", n_queries=512, n_cal=1024, dims=[512, 1024, 1024, 200])
+    assert len(set(wl.budget_bp.tolist())) == 5
+    check(wl)
+
+
+# ---- edge cases -----------------------------------------------------------------
+
+def test_empty_batch_and_single_query():
+    from paper_2204_08400_b200 import harness
+    wl = custom_workload(55, [32, 64, 8], [1, 0], "f32", n=1, n_cal=50, K=2, L=2)
+    dm = harness.DeviceModel(wl)
+    g = harness.run_once(dm, wl.x[:0], wl.budget_bp[:0], max_budget_bp=10000)
+    assert g["status"][0] == 0 and g["pred"].size == 0
+    dm.free()
+    check(wl)
+
+
+def test_one_node_budget():
+    wl = custom_workload(56, [48, 96, 16], [1, 0], "bf16", n=40, n_cal=200, K=3, L=2, budgets=(1, 50))
+    check(wl)
+
+
+def test_invalid_budget_is_reported_not_fatal():
+    from paper_2204_08400_b200 import harness
+    wl = custom_workload(57, [32, 64, 8], [1, 0], "f32", n=16, n_cal=80, K=2, L=2, budgets=(2500,))
+    dm = harness.DeviceModel(wl)
+    bp = wl.budget_bp.copy()
+    bp[5] = 0
+    g = harness.run_once(dm, wl.x, bp, max_budget_bp=5000)
+    assert g["status"][0] == 5 and g["status"][1] == 5     # SLONN_ERR_BUDGET at query 5
+    bp[5] = 2500
+    g = harness.run_once(dm, wl.x, bp, max_budget_bp=5000)
+    assert g["status"][0] == 0
+    dm.free()
+
+
+def test_runs_are_deterministic():
+    from paper_2204_08400_b200 import harness
+    wl = custom_workload(58, [136, 200, 96, 24], [1, 1, 0], "bf16", n=256, n_cal=300, K=4, L=2)
+    dm = harness.DeviceModel(wl)
+    a = harness.run_once(dm, wl.x, wl.budget_bp)
+    b = harness.run_once(dm, wl.x, wl.budget_bp)
+    for k in ("logits", "pred", "codes", "active_ids", "active_vals"):
+        assert np.array_equal(a[k], b[k])
+    dm.free()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    import torch
+    from paper_2204_08400_b200 import binding as sl, harness
+    wl = custom_workload(59, [64, 128, 24], [1, 0], "f32", n=100, n_cal=200, K=3, L=2)
+    dm = harness.DeviceModel(wl)
+    want = harness.run_once(dm, wl.x, wl.budget_bp)
+    n = wl.n_queries
+    max_bp = int(wl.budget_bp.max())
+    stride = sl.slonn_logit_stride(dm.model, max_bp)
+    logits = np.zeros((n, stride), np.float32)
+    pred = np.zeros(n, np.uint32)
+    status = np.ones(4, np.uint32)
+    codes = np.zeros((n, 1, 2), np.uint16)
+    nb = sl.slonn_host_workspace_bytes(dm.model, n, max_bp)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dm.device)
+    hb = sl.make_batch(n, np.ascontiguousarray(wl.budget_bp), logits, status, x_dense=np.ascontiguousarray(wl.x),
+                       max_budget_bp=max_bp, pred=pred, codes=codes)
+    up, down = sl.slonn_run_host(dm.model, hb, ws, nb)
+    assert status[0] == 0
+    assert up == wl.x.nbytes + wl.budget_bp.nbytes
+    assert down == logits.nbytes + pred.nbytes + codes.nbytes + 16
+    assert np.array_equal(logits, want["logits"]) and np.array_equal(pred, want["pred"])
+    assert np.array_equal(codes, want["codes"])
+    dm.free()
