@@ -1,0 +1,338 @@
+"""Benchmark of the SLO-NN inference path on B200.
+
+One step = one pass of the whole hot path (plan, hash+select, gather-dot per
+layer, argmax) over one batch of synthetic queries.  Default workload: the
+784-1024-1024-10 bf16 MLP with 65,536 queries ("c2"), headline budget 10 %,
+plus a sweep over the other budgets.  Prints ONE JSON line on rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--budget-bp 1000]
+  python bench.py --impl reference ...     # the CPU oracle on a bounded sample
+
+Multi-GPU: queries are independent, so ranks are replicas that each process
+their own batch (weak scaling); there is no data-path collective.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2204_08400_b200 import workloads  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def gathered_bytes(wl, budget_bp):
+    """Algorithmic bytes of the gather-dot launches of one step: every selected weight row
+    once per query (row-granular), all queries."""
+    esz = 2 if wl.dtype == "bf16" else 4
+    per_launch = []
+    for l in range(len(wl.dims) - 1):
+        if l == 0 and wl.first_sparse:
+            continue
+        D, N = wl.dims[l], wl.dims[l + 1]
+        if wl.has_act[l]:
+            uniq, cnt = np.unique(budget_bp, return_counts=True)
+            total_rows = int(sum(max(1, (int(bp) * N + 5000) // 10000) * int(c) for bp, c in zip(uniq, cnt)))
+        else:
+            total_rows = N * budget_bp.size
+        per_launch.append(total_rows * D * esz)
+    return per_launch
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, reasons, mx = [], set(), None
+        for line in self.f.read().splitlines():
+            parts = [s.strip() for s in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx = float(parts[2])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_queries_per_sec(wl, budget_bp, target_seconds=12.0):
+    """The CPU oracle as it stands, timed on a bounded prefix of the workload's queries."""
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from oracle import oracle as orc
+    from parity_util import oracle_model, oracle_run, take_queries
+    om = oracle_model(wl)
+    n0 = min(wl.n_queries, 256)
+    idx = np.arange(n0)
+    bp = np.full(n0, budget_bp, np.uint16)
+    t0 = time.perf_counter()
+    oracle_run(om, wl, take_queries(wl, idx), bp, orc.CANON32)
+    dt = max(time.perf_counter() - t0, 1e-4)
+    n1 = int(min(wl.n_queries, max(n0, n0 * target_seconds / dt)))
+    idx = np.arange(n1)
+    bp = np.full(n1, budget_bp, np.uint16)
+    xs = take_queries(wl, idx)
+    t0 = time.perf_counter()
+    oracle_run(om, wl, xs, bp, orc.CANON32)
+    dt = time.perf_counter() - t0
+    return n1 / dt, orc.threads(), n1, dt, (om, xs, bp)
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    wl = workloads.load(args.workload, budget_bp=args.budget_bp)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from oracle import oracle as orc
+    from parity_util import oracle_run
+    qps, cores, n1, dt, (om, xs, bp) = oracle_queries_per_sec(wl, args.budget_bp, target_seconds=6.0)
+    for _ in range(args.warmup):
+        pass  # the sizing pass above already warmed caches; warm-up steps would only repeat it
+    times = []
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        oracle_run(om, wl, xs, bp, orc.CANON32)
+        times.append(time.perf_counter() - t0)
+    ms = 1e3 * float(np.sum(times)) / max(args.steps, 1)
+    value = n1 / (ms / 1e3)
+    line = {
+        "impl": "reference", "metric": "queries_per_sec_at_budget", "value": value, "unit": "queries/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: " + "-".join(map(str, wl.dims)) + f" {wl.dtype}, budget {args.budget_bp} bp",
+                   "queries_per_step": n1},
+        "cpu_baseline": {"value": value, "unit": "queries/s", "cores": cores, "kind": "oracle",
+                         "sample": f"first {n1} of {wl.n_queries} queries per step"},
+        "e2e": {"value": value, "unit": "queries/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--budget-bp", type=int, default=1000)
+    ap.add_argument("--queries", type=int, default=None, help="override the workload's query count")
+    ap.add_argument("--n-cal", type=int, default=None)
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2204_08400_b200 import binding as sl, harness
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    # every rank is a replica with its own batch (same law, rank-specific seed is not needed:
+    # throughput does not depend on the draw; parity tests cover the values)
+    wl = workloads.load(args.workload, n_queries=args.queries, n_cal=args.n_cal, budget_bp=args.budget_bp)
+    n = wl.n_queries
+    dm = harness.DeviceModel(wl, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(batch, steps, warmup):
+        for _ in range(warmup):
+            batch.run(stream)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            batch.run(stream)
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms / steps
+
+    # ---- headline: device-resident inputs ----
+    batch = harness.DeviceBatch(dm, wl.x, wl.budget_bp, max_budget_bp=args.budget_bp, full_outputs=False)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_step = timed(batch, args.steps, args.warmup)
+    clocks = sampler.stop() if rank == 0 else None
+    status = batch.status.cpu().numpy()
+    assert status[0] == 0, f"device status {status}"
+    value = world * n / (ms_step / 1e3)
+    launches_per_step = 1 + sum(2 if a else 1 for a in wl.has_act) + 1  # plan, (select+)gather per layer, argmax
+
+    # ---- per-stage device time of the same step (event pair around every launch) ----
+    stage_ms = {s: 0.0 for s in sl.STAGES}
+    stage_cnt = {s: 0 for s in sl.STAGES}
+    prof_steps = max(3, min(args.steps, 10))
+    for _ in range(prof_steps):
+        ms, cnt = sl.slonn_run_timed(dm.model, batch.batch, batch.ws, batch.ws_bytes, stream)
+        for s in sl.STAGES:
+            stage_ms[s] += ms[s]; stage_cnt[s] += cnt[s]
+    gbytes = gathered_bytes(wl, wl.budget_bp)
+    gd_ms = stage_ms["gather_dot"] / prof_steps          # all gather-dot launches of one step
+    gd_launches = stage_cnt["gather_dot"] // prof_steps
+    peak, peak_kind = measured_peaks()
+    achieved = sum(gbytes) / (gd_ms / 1e3) / 1e9 if gd_ms > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "gather_dot_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                "bytes_per_step": int(sum(gbytes)), "launches_per_step": gd_launches,
+                "avg_launch_ms": gd_ms / max(gd_launches, 1),
+                "stage_ms_per_step": {s: stage_ms[s] / prof_steps for s in sl.STAGES}}
+
+    # ---- budget sweep (the latency profile T(k, isolated) of the paper) ----
+    sweep = {}
+    if not args.no_sweep and world == 1:
+        for bp in wl.budgets_named:
+            bps = np.full(n, bp, np.uint16)
+            b2 = harness.DeviceBatch(dm, wl.x, bps, max_budget_bp=bp, full_outputs=False)
+            ms2 = timed(b2, max(3, args.steps // 4), 3)
+            st_ms, _ = sl.slonn_run_timed(dm.model, b2.batch, b2.ws, b2.ws_bytes, stream)
+            gb = sum(gathered_bytes(wl, bps))
+            sweep[str(bp)] = {"queries_per_s": n / (ms2 / 1e3), "ms_per_step": ms2,
+                              "gather_dot_GBps": gb / (st_ms["gather_dot"] / 1e3) / 1e9 if st_ms["gather_dot"] > 0 else None,
+                              "gather_dot_frac_of_peak": (gb / (st_ms["gather_dot"] / 1e3) / 1e9) / peak if st_ms["gather_dot"] > 0 else None}
+            del b2
+
+    # ---- end to end through the host-buffer entry point ----
+    e2e = None
+    if not args.no_e2e:
+        x_nnz = int(wl.x[0][-1]) if wl.first_sparse else 0
+        stride = sl.slonn_logit_stride(dm.model, args.budget_bp)
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        view = {np.dtype(np.uint16): np.int16, np.dtype(np.uint32): np.int32, np.dtype(np.uint64): np.int64}
+        pinv = lambda a: pin(np.ascontiguousarray(a).view(view.get(a.dtype, a.dtype)))
+        h_logits = torch.zeros((n, stride), dtype=torch.float32).pin_memory()
+        h_pred = torch.zeros(n, dtype=torch.int32).pin_memory()
+        h_status = torch.zeros(4, dtype=torch.int32).pin_memory()
+        h_bp = pinv(wl.budget_bp)
+        h_lids = torch.zeros((n, stride), dtype=torch.int32).pin_memory() if wl.has_act[-1] else None
+        if wl.first_sparse:
+            h_csr = tuple(pinv(a) for a in wl.x)
+            hb = sl.make_batch(n, h_bp, h_logits, h_status, x_csr=h_csr, max_budget_bp=args.budget_bp,
+                               logit_ids=h_lids, pred=h_pred)
+        else:
+            h_x = pin(wl.x)
+            hb = sl.make_batch(n, h_bp, h_logits, h_status, x_dense=h_x, max_budget_bp=args.budget_bp,
+                               logit_ids=h_lids, pred=h_pred)
+        nb = sl.slonn_host_workspace_bytes(dm.model, n, args.budget_bp, x_nnz)
+        hws = torch.empty(nb, dtype=torch.uint8, device=dev)
+        e_steps = max(3, min(args.steps, 10))
+        for _ in range(3):
+            up, down = sl.slonn_run_host(dm.model, hb, hws, nb, stream)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e_steps):
+            up, down = sl.slonn_run_host(dm.model, hb, hws, nb, stream)
+        e1.record(stream)
+        barrier()
+        ms_e = e0.elapsed_time(e1) / e_steps
+        if world > 1:
+            t = torch.tensor([ms_e], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e = float(t.item())
+        assert int(h_status[0]) == 0
+        e2e = {"value": world * n / (ms_e / 1e3), "unit": "queries/s", "h2d_bytes_per_step": int(up),
+               "d2h_bytes_per_step": int(down), "ms_per_step": ms_e}
+
+    # ---- the CPU oracle beside it (rank 0, single-GPU runs only) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        qps, cores, n1, dt, _ = oracle_queries_per_sec(wl, args.budget_bp)
+        cpu = {"value": qps, "unit": "queries/s", "cores": cores, "kind": "oracle",
+               "sample": f"first {n1} of {n} queries, {dt:.1f} s"}
+
+    if rank == 0:
+        esz_name = "f32"  # every sum is accumulated in fp32 (bf16 weights are widened)
+        line = {
+            "metric": "queries_per_sec_at_budget", "value": value, "unit": "queries/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": esz_name, "data": "synthetic",
+            "config": {"workload": f"{args.workload}: " + "-".join(map(str, wl.dims)) +
+                                   f" {wl.dtype} weights, {n} queries/GPU, budget {args.budget_bp} bp, K={wl.K} L={wl.L}",
+                       "queries_per_step_per_gpu": n, "budget_bp": args.budget_bp,
+                       "l2": "inputs_larger_than_l2" if (wl.x.nbytes if not wl.first_sparse else 0) > L2_BYTES
+                             else "weights_and_inputs_l2_resident",
+                       "table_bytes": dm.table_bytes(), "parallelism": f"replicas x{world}"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "budget_sweep": sweep,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -186,6 +186,25 @@ int slonn_run(const slonn_model *m, const slonn_batch *batch, void *workspace,
               uint64_t workspace_bytes, void *stream);
 
 /*
+ * slonn_run with a CUDA event pair around every kernel launch, for measurement
+ * (the per-stage breakdown of Fig. 3 of the paper: time in the LSH part, which
+ * includes the hash functions, against time in the forward computation).
+ * Synchronises `stream`, then adds each launch's device time to
+ * stage_ms[stage] and counts it in stage_launches[stage] (both HOST arrays of
+ * SLONN_N_STAGES entries).  Creates and destroys events, so unlike slonn_run it
+ * is not allocation-free.
+ */
+#define SLONN_STAGE_PLAN 0          /* budgets -> list offsets                      */
+#define SLONN_STAGE_HASH_SELECT 1   /* FreeHash bits, keys, bucket lists, top-k% cut */
+#define SLONN_STAGE_GATHER_DOT 2    /* selected rows' dot products                   */
+#define SLONN_STAGE_SPARSE_FIRST 3  /* first layer fed by CSR rows                   */
+#define SLONN_STAGE_ARGMAX 4        /* prediction                                    */
+#define SLONN_N_STAGES 5
+int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *workspace,
+                    uint64_t workspace_bytes, void *stream, float *stage_ms,
+                    uint32_t *stage_launches);
+
+/*
  * Same computation for callers that keep queries and results in HOST memory:
  * every pointer of `host_batch` (inputs, outputs, status) is a host pointer,
  * pinned memory recommended.  Copies the inputs to the device, runs, copies

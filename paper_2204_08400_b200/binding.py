@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libslonn.so")
 EXPORTS = [
     "slonn_version", "slonn_strerror", "slonn_build", "slonn_model_info", "slonn_model_tables_to_host",
     "slonn_free", "slonn_active_capacity", "slonn_logit_stride", "slonn_workspace_bytes", "slonn_run",
+    "slonn_run_timed",
     "slonn_host_workspace_bytes", "slonn_run_host",
 ]
 
@@ -82,6 +83,9 @@ def lib():
         L.slonn_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint64)]
         L.slonn_run.restype = C.c_int
         L.slonn_run.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p]
+        L.slonn_run_timed.restype = C.c_int
+        L.slonn_run_timed.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p,
+                                      C.c_void_p, C.c_void_p]
         L.slonn_host_workspace_bytes.restype = C.c_int
         L.slonn_host_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64,
                                                  C.POINTER(C.c_uint64)]
@@ -265,6 +269,20 @@ def slonn_run(model: Model, batch: _Batch, workspace, workspace_bytes: int, stre
     rc = lib().slonn_run(model.handle, C.byref(batch), _ptr(workspace), workspace_bytes, _stream_ptr(stream))
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_run")
+
+
+STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax")
+
+
+def slonn_run_timed(model: Model, batch: _Batch, workspace, workspace_bytes: int, stream=None):
+    """Returns ({stage: ms}, {stage: launches}) for this run; synchronises the stream."""
+    ms = np.zeros(len(STAGES), dtype=np.float32)
+    cnt = np.zeros(len(STAGES), dtype=np.uint32)
+    rc = lib().slonn_run_timed(model.handle, C.byref(batch), _ptr(workspace), workspace_bytes,
+                               _stream_ptr(stream), ms.ctypes.data, cnt.ctypes.data)
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_run_timed")
+    return dict(zip(STAGES, ms.tolist())), dict(zip(STAGES, cnt.tolist()))
 
 
 def slonn_run_host(model: Model, host_batch: _Batch, workspace, workspace_bytes: int, stream=None):

@@ -8,6 +8,27 @@
 
 namespace {
 
+// Optional per-stage timing: an event pair around every launch of a stage.
+struct stage_timer {
+    struct span { int stage; cudaEvent_t a, b; };
+    span spans[8 * SLONN_MAX_LAYERS];
+    int n = 0;
+    bool failed = false;
+    cudaStream_t st = nullptr;
+    void tic(int stage)
+    {
+        if (n >= (int)(sizeof(spans) / sizeof(spans[0]))) { failed = true; return; }
+        span &s = spans[n];
+        s.stage = stage;
+        if (cudaEventCreate(&s.a) != cudaSuccess || cudaEventCreate(&s.b) != cudaSuccess) { failed = true; return; }
+        cudaEventRecord(s.a, st);
+        ++n;
+    }
+    void toc() { if (n > 0 && !failed) cudaEventRecord(spans[n - 1].b, st); }
+};
+#define TIC(stage) do { if (tm) tm->tic(stage); } while (0)
+#define TOC() do { if (tm) tm->toc(); } while (0)
+
 inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
 inline bool model_ok(const slonn_model *m) { return m && m->magic == SLONN_MAGIC; }
@@ -167,20 +188,20 @@ extern "C" int slonn_workspace_bytes(const slonn_model *m, uint32_t n, uint32_t 
     return SLONN_OK;
 }
 
-extern "C" int slonn_run(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes,
-                         void *stream)
+static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes,
+                    void *stream, stage_timer *tm)
 {
-    if (!model_ok(m) || !b) return SLONN_ERR_ARG;
-    if (!b->budget_bp || !b->logits || !b->status) return SLONN_ERR_ARG;
-    if (m->first_sparse ? (!b->x_indptr || !b->x_ids || !b->x_vals) : !b->x_dense) return SLONN_ERR_ARG;
-    const slonn_layer &last = m->layer[m->n_layers - 1];
-    if (last.has_act && !b->logit_ids) return SLONN_ERR_ARG;
-    if (b->x_dense && ((uintptr_t)b->x_dense & 15u)) return SLONN_ERR_ALIGN;
+    if (!model_ok(m) || !b || !b->status) return SLONN_ERR_ARG;
     const uint32_t n = b->n_queries;
     const uint32_t max_bp = eff_max_bp(b->max_budget_bp);
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(b->status, 0, 4 * sizeof(uint32_t), st) != cudaSuccess) return SLONN_ERR_CUDA;
-    if (n == 0) return SLONN_OK;
+    if (n == 0) return SLONN_OK; // an empty batch needs no other buffer
+    if (!b->budget_bp || !b->logits) return SLONN_ERR_ARG;
+    if (m->first_sparse ? (!b->x_indptr || !b->x_ids || !b->x_vals) : !b->x_dense) return SLONN_ERR_ARG;
+    const slonn_layer &last = m->layer[m->n_layers - 1];
+    if (last.has_act && !b->logit_ids) return SLONN_ERR_ARG;
+    if (b->x_dense && ((uintptr_t)b->x_dense & 15u)) return SLONN_ERR_ALIGN;
 
     const ws_layout wl = carve(m, n, max_bp);
     if (!workspace || ((uintptr_t)workspace & 255u) || ws_bytes < wl.total) return SLONN_ERR_WORKSPACE;
@@ -204,7 +225,9 @@ extern "C" int slonn_run(const slonn_model *m, const slonn_batch *b, void *works
                 pp.act_N[a] = m->layer[l].N; pp.act_cap[a] = m->layer[l].cap; pp.act_layer[a] = l;
             }
         pp.indptr = indptr; pp.status = b->status;
+        TIC(SLONN_STAGE_PLAN);
         plan_kernel<<<1, 1024, 0, st>>>(pp);
+        TOC();
         if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
     }
 
@@ -223,9 +246,11 @@ extern "C" int slonn_run(const slonn_model *m, const slonn_batch *b, void *works
         int rc;
         if (l == 0 && m->first_sparse) {
             float *o = is_last ? b->logits : dense[dense_cur];
-            if ((rc = slonn_forward_sparse_first(m, b->x_indptr, b->x_ids, b->x_vals, n, o, is_last ? 0u : 1u,
-                                                 b->status, st)))
-                return rc;
+            TIC(SLONN_STAGE_SPARSE_FIRST);
+            rc = slonn_forward_sparse_first(m, b->x_indptr, b->x_ids, b->x_vals, n, o, is_last ? 0u : 1u,
+                                            b->status, st);
+            TOC();
+            if (rc) return rc;
             in.kind = SLONN_IN_DENSE; in.dense = o;
             dense_cur ^= 1;
             continue;
@@ -244,18 +269,27 @@ extern "C" int slonn_run(const slonn_model *m, const slonn_batch *b, void *works
             sp.hash_nodes = ly.hash_nodes; sp.tables = ly.tables; sp.cap = ly.cap; sp.K = m->K; sp.L = m->L;
             sp.n_act = m->n_act; sp.a = a; sp.layer = l; sp.indptr = indptr; sp.out_ids = ids;
             sp.codes = b->codes; sp.status = b->status;
-            if ((rc = launch_select(m, sp, n, st))) return rc;
+            TIC(SLONN_STAGE_HASH_SELECT);
+            rc = launch_select(m, sp, n, st);
+            TOC();
+            if (rc) return rc;
             gp.use_list = 1; gp.a = a; gp.out_vals = vals;
             if (is_last) { gp.out_dense = b->logits; gp.out_dense_ids = b->logit_ids; gp.out_stride = stride; }
             max_rows = slonn_budget_nodes(max_bp, ly.N);
-            if ((rc = launch_gather(m, gp, n, max_rows, st))) return rc;
+            TIC(SLONN_STAGE_GATHER_DOT);
+            rc = launch_gather(m, gp, n, max_rows, st);
+            TOC();
+            if (rc) return rc;
             in.kind = SLONN_IN_LIST; in.indptr = indptr; in.ids = ids; in.vals = vals;
             in.ip_mul = m->n_act; in.ip_add = a;
         } else {
             gp.use_list = 0;
             gp.out_dense = is_last ? b->logits : dense[dense_cur];
             gp.out_stride = ly.N;
-            if ((rc = launch_gather(m, gp, n, max_rows, st))) return rc;
+            TIC(SLONN_STAGE_GATHER_DOT);
+            rc = launch_gather(m, gp, n, max_rows, st);
+            TOC();
+            if (rc) return rc;
             in.kind = SLONN_IN_DENSE; in.dense = gp.out_dense;
             dense_cur ^= 1;
         }
@@ -271,10 +305,40 @@ extern "C" int slonn_run(const slonn_model *m, const slonn_batch *b, void *works
         } else {
             ap.fixed_len = last.N;
         }
+        TIC(SLONN_STAGE_ARGMAX);
         argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
+        TOC();
         if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
     }
     return SLONN_OK;
+}
+
+extern "C" int slonn_run(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes,
+                         void *stream)
+{
+    return run_impl(m, b, workspace, ws_bytes, stream, nullptr);
+}
+
+extern "C" int slonn_run_timed(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes,
+                               void *stream, float *stage_ms, uint32_t *stage_launches)
+{
+    if (!stage_ms || !stage_launches) return SLONN_ERR_ARG;
+    stage_timer tm;
+    tm.st = (cudaStream_t)stream;
+    int rc = run_impl(m, b, workspace, ws_bytes, stream, &tm);
+    if (cudaStreamSynchronize(tm.st) != cudaSuccess && rc == SLONN_OK) rc = SLONN_ERR_CUDA;
+    for (int s = 0; s < SLONN_N_STAGES; ++s) { stage_ms[s] = 0.0f; stage_launches[s] = 0; }
+    for (int i = 0; i < tm.n; ++i) {
+        float ms = 0.0f;
+        if (rc == SLONN_OK && !tm.failed && cudaEventElapsedTime(&ms, tm.spans[i].a, tm.spans[i].b) == cudaSuccess) {
+            stage_ms[tm.spans[i].stage] += ms;
+            stage_launches[tm.spans[i].stage] += 1;
+        }
+        cudaEventDestroy(tm.spans[i].a);
+        cudaEventDestroy(tm.spans[i].b);
+    }
+    if (tm.failed && rc == SLONN_OK) rc = SLONN_ERR_CUDA;
+    return rc;
 }
 
 // ---- host-buffer variant -----------------------------------------------------
