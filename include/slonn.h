@@ -186,6 +186,39 @@ int slonn_run(const slonn_model *m, const slonn_batch *batch, void *workspace,
               uint64_t workspace_bytes, void *stream);
 
 /*
+ * slonn_run without a caller-provided workspace.  (The paper has no counterpart;
+ * this exists for deployment.)
+ *
+ * Who needs it: code that has to serve queries but is not allowed to obtain
+ * device memory -- a request handler in a serving process whose device memory
+ * was partitioned at start-up and where later cudaMalloc calls are forbidden or
+ * would stall every stream; a plug-in inside a host program whose own allocator
+ * owns the GPU; a C caller with no allocator at hand at all.  Such a caller still
+ * passes its input and output buffers in `batch`, exactly as for slonn_run, but
+ * the intermediate lists and activations go to a fixed scratch area of
+ * SLONN_STATIC_WORKSPACE_BYTES that is compiled into the library as a device
+ * array (each GPU that loads the library holds those bytes until the process
+ * ends).  The call performs no cudaMalloc / cudaFree and uses no allocating
+ * library routine.
+ *
+ *   - The batch must fit: if slonn_workspace_bytes(m, n_queries, max_budget_bp)
+ *     exceeds SLONN_STATIC_WORKSPACE_BYTES the call returns SLONN_ERR_WORKSPACE
+ *     and launches nothing.  Use smaller batches or slonn_run.
+ *   - The model's device must be the current device (else SLONN_ERR_ARG).
+ *   - The first call on each device looks up the scratch area's device address
+ *     (a one-time set-up step under a lock).  Make that first call during
+ *     start-up, before any stream capture begins.
+ *   - All calls on a device share the one scratch area and it keeps whatever the
+ *     previous call left there.  Nothing in it needs to start at zero (every
+ *     entry is written before it is read within a call), but two calls whose
+ *     kernels overlap on the GPU -- different streams, or different host threads
+ *     -- race on it: serialise them on one stream.
+ * Results are identical to slonn_run's.
+ */
+#define SLONN_STATIC_WORKSPACE_BYTES (16u << 20)
+int slonn_run_static(const slonn_model *m, const slonn_batch *batch, void *stream);
+
+/*
  * slonn_run with a CUDA event pair around every kernel launch, for measurement
  * (the per-stage breakdown of Fig. 3 of the paper: time in the LSH part, which
  * includes the hash functions, against time in the forward computation).

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libslonn.so")
 EXPORTS = [
     "slonn_version", "slonn_strerror", "slonn_build", "slonn_model_info", "slonn_model_tables_to_host",
     "slonn_free", "slonn_active_capacity", "slonn_logit_stride", "slonn_workspace_bytes", "slonn_run",
-    "slonn_run_timed",
+    "slonn_run_timed", "slonn_run_static",
     "slonn_host_workspace_bytes", "slonn_run_host",
 ]
 
@@ -83,6 +83,8 @@ def lib():
         L.slonn_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint64)]
         L.slonn_run.restype = C.c_int
         L.slonn_run.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p]
+        L.slonn_run_static.restype = C.c_int
+        L.slonn_run_static.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p]
         L.slonn_run_timed.restype = C.c_int
         L.slonn_run_timed.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p,
                                       C.c_void_p, C.c_void_p]
@@ -269,6 +271,20 @@ def slonn_run(model: Model, batch: _Batch, workspace, workspace_bytes: int, stre
     rc = lib().slonn_run(model.handle, C.byref(batch), _ptr(workspace), workspace_bytes, _stream_ptr(stream))
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_run")
+
+
+STATIC_WORKSPACE_BYTES = 16 << 20
+
+
+def slonn_run_static(model: Model, batch: _Batch, stream=None) -> None:
+    """slonn_run for callers that may not allocate device memory: no workspace argument, the
+    library's built-in scratch area (STATIC_WORKSPACE_BYTES) is used instead.  Raises
+    SlonnError(SLONN_ERR_WORKSPACE) when the batch needs more than that.  Calls on one device
+    share the scratch area, so keep them on one stream; make the first call before any stream
+    capture starts."""
+    rc = lib().slonn_run_static(model.handle, C.byref(batch), _stream_ptr(stream))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_run_static")
 
 
 STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax")

@@ -3,6 +3,7 @@
 // host synchronisation.
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 
 #include "slonn_run_kernels.cuh"
 
@@ -339,6 +340,39 @@ extern "C" int slonn_run_timed(const slonn_model *m, const slonn_batch *b, void 
     }
     if (tm.failed && rc == SLONN_OK) rc = SLONN_ERR_CUDA;
     return rc;
+}
+
+// ---- run on the library's own fixed scratch area --------------------------------
+
+// Scratch of slonn_run_static.  It lives in the library image, so every GPU that loads the
+// library carries these bytes until the process exits.  In host code this name is only a
+// stand-in for the symbol, not an address a kernel can use: the device address is looked up
+// once per device with cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char slonn_static_scratch[SLONN_STATIC_WORKSPACE_BYTES];
+
+namespace {
+std::mutex g_static_mu;
+void *g_static_ptr[64]; // device address of slonn_static_scratch, per device ordinal
+} // namespace
+
+extern "C" int slonn_run_static(const slonn_model *m, const slonn_batch *b, void *stream)
+{
+    if (!model_ok(m) || !b) return SLONN_ERR_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SLONN_ERR_CUDA;
+    if (dev != m->device || dev < 0 || dev >= 64) return SLONN_ERR_ARG; // the model's device must be current
+    const uint64_t need = carve(m, b->n_queries, eff_max_bp(b->max_budget_bp)).total;
+    if (need > SLONN_STATIC_WORKSPACE_BYTES) return SLONN_ERR_WORKSPACE;
+    void *ws = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        ws = g_static_ptr[dev];
+        if (!ws) { // first call on this device: resolve the symbol with this device current
+            if (cudaGetSymbolAddress(&ws, slonn_static_scratch) != cudaSuccess || !ws) return SLONN_ERR_CUDA;
+            g_static_ptr[dev] = ws;
+        }
+    }
+    return run_impl(m, b, ws, SLONN_STATIC_WORKSPACE_BYTES, stream, nullptr);
 }
 
 // ---- host-buffer variant -----------------------------------------------------
