@@ -37,6 +37,12 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def hash_bytes(wl, n):
+    """Weight bytes of the FreeHash rows of one step: K*L rows per query and activator layer."""
+    esz = 2 if wl.dtype == "bf16" else 4
+    return sum(wl.K * wl.L * wl.dims[l] * esz * n for l in range(len(wl.dims) - 1) if wl.has_act[l])
+
+
 def gathered_bytes(wl, budget_bp):
     """Algorithmic bytes of the gather-dot launches of one step: every selected weight row
     once per query (row-granular), all queries."""
@@ -234,7 +240,7 @@ def main():
     status = batch.status.cpu().numpy()
     assert status[0] == 0, f"device status {status}"
     value = world * n / (ms_step / 1e3)
-    launches_per_step = 1 + sum(2 if a else 1 for a in wl.has_act) + 1  # plan, (select+)gather per layer, argmax
+    launches_per_step = None  # counted below from the per-stage launch counters
 
     # ---- per-stage device time of the same step (event pair around every launch) ----
     stage_ms = {s: 0.0 for s in sl.STAGES}
@@ -244,15 +250,24 @@ def main():
         ms, cnt = sl.slonn_run_timed(dm.model, batch.batch, batch.ws, batch.ws_bytes, stream)
         for s in sl.STAGES:
             stage_ms[s] += ms[s]; stage_cnt[s] += cnt[s]
-    gbytes = gathered_bytes(wl, wl.budget_bp)
-    gd_ms = stage_ms["gather_dot"] / prof_steps          # all gather-dot launches of one step
-    gd_launches = stage_cnt["gather_dot"] // prof_steps
+    def stage_roofline(ms_by_stage, cnt_by_stage, bps, steps):
+        """Dominant kernel of the step and its achieved rate on the weight bytes it must touch."""
+        gb = sum(gathered_bytes(wl, bps))
+        if ms_by_stage["fused"] > 0:     # one launch does hash + select + gather for every layer
+            kernel, ms, launches, nbytes = "fused_network_kernel", ms_by_stage["fused"], cnt_by_stage["fused"], gb + hash_bytes(wl, bps.size)
+        else:
+            kernel, ms, launches, nbytes = "gather_dot_kernel", ms_by_stage["gather_dot"], cnt_by_stage["gather_dot"], gb
+        ms /= steps
+        launches //= steps
+        ach = nbytes / (ms / 1e3) / 1e9 if ms > 0 else 0.0
+        return kernel, ms, launches, nbytes, ach
+
     peak, peak_kind = measured_peaks()
-    achieved = sum(gbytes) / (gd_ms / 1e3) / 1e9 if gd_ms > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "gather_dot_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    kernel, k_ms, k_launches, k_bytes, achieved = stage_roofline(stage_ms, stage_cnt, wl.budget_bp, prof_steps)
+    roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
-                "bytes_per_step": int(sum(gbytes)), "launches_per_step": gd_launches,
-                "avg_launch_ms": gd_ms / max(gd_launches, 1),
+                "bytes_per_step": int(k_bytes), "launches_per_step": k_launches,
+                "avg_launch_ms": k_ms / max(k_launches, 1),
                 "stage_ms_per_step": {s: stage_ms[s] / prof_steps for s in sl.STAGES}}
 
     # ---- budget sweep (the latency profile T(k, isolated) of the paper) ----
@@ -262,11 +277,10 @@ def main():
             bps = np.full(n, bp, np.uint16)
             b2 = harness.DeviceBatch(dm, wl.x, bps, max_budget_bp=bp, full_outputs=False)
             ms2 = timed(b2, max(3, args.steps // 4), 3)
-            st_ms, _ = sl.slonn_run_timed(dm.model, b2.batch, b2.ws, b2.ws_bytes, stream)
-            gb = sum(gathered_bytes(wl, bps))
-            sweep[str(bp)] = {"queries_per_s": n / (ms2 / 1e3), "ms_per_step": ms2,
-                              "gather_dot_GBps": gb / (st_ms["gather_dot"] / 1e3) / 1e9 if st_ms["gather_dot"] > 0 else None,
-                              "gather_dot_frac_of_peak": (gb / (st_ms["gather_dot"] / 1e3) / 1e9) / peak if st_ms["gather_dot"] > 0 else None}
+            st_ms, st_cnt = sl.slonn_run_timed(dm.model, b2.batch, b2.ws, b2.ws_bytes, stream)
+            k2, _, _, _, ach2 = stage_roofline(st_ms, st_cnt, bps, 1)
+            sweep[str(bp)] = {"queries_per_s": n / (ms2 / 1e3), "ms_per_step": ms2, "kernel": k2,
+                              "weight_GBps": ach2, "frac_of_peak": ach2 / peak}
             del b2
 
     # ---- end to end through the host-buffer entry point ----
@@ -330,7 +344,8 @@ def main():
                        "l2": "inputs_larger_than_l2" if (wl.x.nbytes if not wl.first_sparse else 0) > L2_BYTES
                              else "weights_and_inputs_l2_resident",
                        "table_bytes": dm.table_bytes(), "parallelism": f"replicas x{world}"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks, "e2e": e2e,
+            "gpu_launches": (sum(stage_cnt.values()) // prof_steps + (1 if stage_cnt["plan"] else 0)) * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "budget_sweep": sweep,
         }
         print(json.dumps(line), flush=True)

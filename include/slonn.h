@@ -165,7 +165,16 @@ typedef struct {
     uint32_t *status;              /* required. [4] words: [0] first error code seen on the   */
                                    /* device (0 = ok, else -SLONN_ERR_*), [1] query index,    */
                                    /* [2] layer index, [3] reserved.  Cleared by slonn_run    */
+    uint32_t kernel_path;          /* HOST value: SLONN_PATH_AUTO, or force one of the two    */
+                                   /* kernel families (results are identical; for testing and */
+                                   /* tuning).  _FUSED on a network it cannot take returns    */
+                                   /* SLONN_ERR_DIM                                           */
 } slonn_batch;
+
+#define SLONN_PATH_AUTO 0    /* library chooses                                               */
+#define SLONN_PATH_STAGED 1  /* one block per query and stage: any width, any batch size      */
+#define SLONN_PATH_FUSED 2   /* one warp per query through all layers: widths <= 1024 inputs, */
+                             /* <= 4096 nodes per layer, dense first layer                    */
 
 /* Number of entries active_ids / active_vals need for n queries at max_budget_bp. */
 int slonn_active_capacity(const slonn_model *m, uint32_t n_queries, uint32_t max_budget_bp,
@@ -232,7 +241,8 @@ int slonn_run_static(const slonn_model *m, const slonn_batch *batch, void *strea
 #define SLONN_STAGE_GATHER_DOT 2    /* selected rows' dot products                   */
 #define SLONN_STAGE_SPARSE_FIRST 3  /* first layer fed by CSR rows                   */
 #define SLONN_STAGE_ARGMAX 4        /* prediction                                    */
-#define SLONN_N_STAGES 5
+#define SLONN_STAGE_FUSED 5         /* all of 1, 2, 4 in the one-warp-per-query kernel */
+#define SLONN_N_STAGES 6
 int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *workspace,
                     uint64_t workspace_bytes, void *stream, float *stage_ms,
                     uint32_t *stage_launches);

@@ -48,7 +48,8 @@ class _Batch(C.Structure):
                 ("x_ids", C.c_void_p), ("x_vals", C.c_void_p), ("budget_bp", C.c_void_p),
                 ("max_budget_bp", C.c_uint32), ("logits", C.c_void_p), ("logit_ids", C.c_void_p),
                 ("pred", C.c_void_p), ("codes", C.c_void_p), ("active_indptr", C.c_void_p),
-                ("active_ids", C.c_void_p), ("active_vals", C.c_void_p), ("status", C.c_void_p)]
+                ("active_ids", C.c_void_p), ("active_vals", C.c_void_p), ("status", C.c_void_p),
+                ("kernel_path", C.c_uint32)]
 
 
 _lib = None
@@ -252,7 +253,7 @@ def slonn_host_workspace_bytes(model: Model, n_queries: int, max_budget_bp: int 
 
 def make_batch(n_queries: int, budget_bp, logits, status, x_dense=None, x_csr=None, max_budget_bp: int = 0,
                logit_ids=None, pred=None, codes=None, active_indptr=None, active_ids=None,
-               active_vals=None) -> _Batch:
+               active_vals=None, kernel_path: int = 0) -> _Batch:
     """Fills a slonn_batch from tensors/arrays (device for slonn_run, host for slonn_run_host)."""
     b = _Batch()
     b.n_queries = n_queries
@@ -264,6 +265,7 @@ def make_batch(n_queries: int, budget_bp, logits, status, x_dense=None, x_csr=No
     b.logits, b.logit_ids, b.pred, b.codes = _ptr(logits), _ptr(logit_ids), _ptr(pred), _ptr(codes)
     b.active_indptr, b.active_ids, b.active_vals = _ptr(active_indptr), _ptr(active_ids), _ptr(active_vals)
     b.status = _ptr(status)
+    b.kernel_path = kernel_path
     return b
 
 
@@ -287,7 +289,8 @@ def slonn_run_static(model: Model, batch: _Batch, stream=None) -> None:
         raise SlonnError(rc, "slonn_run_static")
 
 
-STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax")
+STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused")
+PATH_AUTO, PATH_STAGED, PATH_FUSED = 0, 1, 2
 
 
 def slonn_run_timed(model: Model, batch: _Batch, workspace, workspace_bytes: int, stream=None):

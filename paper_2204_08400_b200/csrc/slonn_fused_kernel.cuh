@@ -1,0 +1,325 @@
+// Whole-network kernel for narrow layers: one warp carries one query through
+// every layer (hash -> keys -> bucket lists -> top-k% -> selected rows ->
+// next layer) with the layer input held in registers.  Used when every layer's
+// input width is at most 1024 and every activator layer at most 4096 nodes
+// wide; wider networks use the per-stage kernels.
+//
+// Same arithmetic as everywhere else in the library: lane p owns partial sum
+// p and takes 16-byte weight chunks p, p+32, ... in ascending order; xor
+// butterfly 16, 8, 4, 2, 1; bias last.
+#pragma once
+#include "slonn_common.cuh"
+
+#define SLONN_FUSED_ROWS 4
+#define SLONN_FUSED_WARPS 4
+#define SLONN_FUSED_MAX_D 1024
+#define SLONN_FUSED_MAX_N 4096
+
+struct slonn_fused_layer {
+    const void *W;
+    const float *bias;
+    const uint32_t *hash_nodes;
+    const void *tables;
+    uint32_t D, N, nchunks, cap;
+    uint32_t has_act, a, relu, id_bytes;
+};
+
+struct slonn_fused_params {
+    slonn_fused_layer layer[SLONN_MAX_LAYERS];
+    uint32_t n_layers, n, n_act, K, L;
+    const float *x;          // [n][D0]
+    const uint64_t *indptr;  // [n * n_act + 1]
+    uint32_t *out_ids;       // CSR payload, nullable
+    float *out_vals;         // CSR payload, nullable
+    uint16_t *codes;         // nullable
+    float *logits;
+    uint32_t logit_stride;
+    uint32_t *logit_ids;     // budgeted last layer only
+    uint32_t *pred;          // nullable
+    uint32_t *status;
+    uint32_t xbuf_floats, ids_cap, bitmap_words, warp_bytes; // per-warp shared memory carve
+};
+
+template <bool BF16>
+struct fused_traits {
+    static constexpr int VPC = BF16 ? 8 : 4; // input values per 16-byte weight chunk
+};
+
+// x registers <- dense global row
+template <bool BF16, int NC>
+__device__ __forceinline__ void fused_load_x_global(float (&xr)[NC * fused_traits<BF16>::VPC], const float *row,
+                                                    uint32_t nchunks, uint32_t lane)
+{
+    constexpr int VPC = fused_traits<BF16>::VPC;
+    const float4 *x4 = reinterpret_cast<const float4 *>(row);
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+        const uint32_t c = lane + 32u * i;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (c < nchunks) {
+            if (BF16) { a = __ldg(x4 + 2 * c); b = __ldg(x4 + 2 * c + 1); }
+            else a = __ldg(x4 + c);
+        }
+        xr[i * VPC + 0] = a.x; xr[i * VPC + 1] = a.y; xr[i * VPC + 2] = a.z; xr[i * VPC + 3] = a.w;
+        if (BF16) { xr[i * VPC + 4] = b.x; xr[i * VPC + 5] = b.y; xr[i * VPC + 6] = b.z; xr[i * VPC + 7] = b.w; }
+    }
+}
+
+// x registers <- this warp's staged vector (xs_index layout for `nchunks`)
+template <bool BF16, int NC>
+__device__ __forceinline__ void fused_load_x_shared(float (&xr)[NC * fused_traits<BF16>::VPC], const float4 *xs4,
+                                                    uint32_t nchunks, uint32_t lane)
+{
+    constexpr int VPC = fused_traits<BF16>::VPC;
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+        const uint32_t c = lane + 32u * i;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (c < nchunks) {
+            a = xs4[c];
+            if (BF16) b = xs4[nchunks + c];
+        }
+        xr[i * VPC + 0] = a.x; xr[i * VPC + 1] = a.y; xr[i * VPC + 2] = a.z; xr[i * VPC + 3] = a.w;
+        if (BF16) { xr[i * VPC + 4] = b.x; xr[i * VPC + 5] = b.y; xr[i * VPC + 6] = b.z; xr[i * VPC + 7] = b.w; }
+    }
+}
+
+// Fixed-order dot products of R rows against the register-resident input.
+template <bool BF16, int NC, int R>
+__device__ __forceinline__ void fused_dot_rows(const uint4 *const (&rows)[R],
+                                               const float (&xr)[NC * fused_traits<BF16>::VPC], uint32_t nchunks,
+                                               uint32_t lane, float (&acc)[R])
+{
+    constexpr int VPC = fused_traits<BF16>::VPC;
+    constexpr int G = NC < 2 ? NC : 2; // rounds whose loads are issued together
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc[r] = 0.0f;
+#pragma unroll
+    for (int i0 = 0; i0 < NC; i0 += G) {
+        uint4 w[G][R];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const uint32_t c = lane + 32u * (i0 + g);
+            if (c < nchunks) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) w[g][r] = __ldg(rows[r] + c);
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const int i = i0 + g;
+            const uint32_t c = lane + 32u * i;
+            if (c < nchunks) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float a = acc[r];
+                    if (BF16) {
+                        a = fmaf(bf16_lo(w[g][r].x), xr[i * VPC + 0], a);
+                        a = fmaf(bf16_hi(w[g][r].x), xr[i * VPC + 1], a);
+                        a = fmaf(bf16_lo(w[g][r].y), xr[i * VPC + 2], a);
+                        a = fmaf(bf16_hi(w[g][r].y), xr[i * VPC + 3], a);
+                        a = fmaf(bf16_lo(w[g][r].z), xr[i * VPC + 4], a);
+                        a = fmaf(bf16_hi(w[g][r].z), xr[i * VPC + 5], a);
+                        a = fmaf(bf16_lo(w[g][r].w), xr[i * VPC + 6], a);
+                        a = fmaf(bf16_hi(w[g][r].w), xr[i * VPC + 7], a);
+                    } else {
+                        a = fmaf(__uint_as_float(w[g][r].x), xr[i * VPC + 0], a);
+                        a = fmaf(__uint_as_float(w[g][r].y), xr[i * VPC + 1], a);
+                        a = fmaf(__uint_as_float(w[g][r].z), xr[i * VPC + 2], a);
+                        a = fmaf(__uint_as_float(w[g][r].w), xr[i * VPC + 3], a);
+                    }
+                    acc[r] = a;
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) acc[r] = acc[r] + __shfl_xor_sync(SLONN_FULL_MASK, acc[r], off);
+    }
+}
+
+template <typename IDT>
+__device__ __forceinline__ uint32_t fused_table_entry(const void *tables, uint32_t cap, uint32_t K, uint32_t b,
+                                                      uint32_t key, uint32_t r)
+{
+    const IDT *t = reinterpret_cast<const IDT *>(tables);
+    return (uint32_t)__ldg(t + (((uint64_t)b << K) + key) * cap + r);
+}
+
+// First B distinct ids of the rank-interleaved bucket lists -> ids_s[0..B) ascending.
+// mykey: lane b holds the key of table b.  One warp, no block barrier.
+__device__ __forceinline__ void fused_select(const slonn_fused_layer &ly, uint32_t K, uint32_t L, uint32_t mykey,
+                                             uint32_t B, uint32_t *bitmap, uint16_t *ids_s, uint32_t lane)
+{
+    const uint32_t nwords = (ly.N + 31u) >> 5;
+    for (uint32_t w = lane; w < nwords; w += 32) bitmap[w] = 0u;
+    __syncwarp();
+    const uint32_t npos = B * L;
+    uint32_t total = 0;
+    for (uint32_t base = 0; base < npos && total < B; base += 32) {
+        const uint32_t pos = base + lane;
+        uint32_t id = 0xffffffffu - lane; // distinct dummies for lanes past the end
+        bool fresh = false;
+        const uint32_t r = pos / L, b = pos - r * L;
+        const uint32_t key = __shfl_sync(SLONN_FULL_MASK, mykey, b & 31u);
+        if (pos < npos) {
+            id = ly.id_bytes == 2 ? fused_table_entry<uint16_t>(ly.tables, ly.cap, K, b, key, r)
+                                  : fused_table_entry<uint32_t>(ly.tables, ly.cap, K, b, key, r);
+            if (id < ly.N) fresh = ((bitmap[id >> 5] >> (id & 31u)) & 1u) == 0u;
+        }
+        const uint32_t same = __match_any_sync(SLONN_FULL_MASK, id);
+        const bool take = fresh && ((uint32_t)(__ffs(same) - 1) == lane);
+        const uint32_t bal = __ballot_sync(SLONN_FULL_MASK, take);
+        const uint32_t need = B - total;
+        const uint32_t rank = __popc(bal & ((1u << lane) - 1u));
+        if (take && rank < need) atomicOr(&bitmap[id >> 5], 1u << (id & 31u));
+        const uint32_t c = (uint32_t)__popc(bal);
+        total += c < need ? c : need;
+        __syncwarp();
+    }
+    uint32_t running = 0;
+    for (uint32_t w0 = 0; w0 < nwords; w0 += 32) {
+        const uint32_t w = w0 + lane;
+        uint32_t bits = w < nwords ? bitmap[w] : 0u;
+        const uint32_t cnt = __popc(bits);
+        uint32_t incl = cnt;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t t = __shfl_up_sync(SLONN_FULL_MASK, incl, off);
+            if (lane >= (uint32_t)off) incl += t;
+        }
+        uint32_t o = running + incl - cnt;
+        while (bits) {
+            const uint32_t t = __ffs(bits) - 1;
+            bits &= bits - 1;
+            if (o < B) ids_s[o] = (uint16_t)((w << 5) + t);
+            ++o;
+        }
+        running += __shfl_sync(SLONN_FULL_MASK, incl, 31);
+    }
+    __syncwarp();
+}
+
+template <bool BF16, int NC>
+__global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32) fused_network_kernel(const __grid_constant__ slonn_fused_params P)
+{
+    constexpr int VPC = fused_traits<BF16>::VPC;
+    constexpr int R = SLONN_FUSED_ROWS;
+    extern __shared__ float4 smem4[];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t q = blockIdx.x * SLONN_FUSED_WARPS + warp;
+    if (q >= P.n) return;
+    unsigned char *wbase = reinterpret_cast<unsigned char *>(smem4) + (size_t)warp * P.warp_bytes;
+    float4 *xbuf4 = reinterpret_cast<float4 *>(wbase);
+    float *xbuf = reinterpret_cast<float *>(wbase);
+    uint16_t *ids_s = reinterpret_cast<uint16_t *>(wbase + (size_t)P.xbuf_floats * 4);
+    uint32_t *bitmap = reinterpret_cast<uint32_t *>(wbase + (size_t)P.xbuf_floats * 4 + (size_t)P.ids_cap * 2);
+
+    float xr[NC * VPC];
+    float best = 0.0f;          // running argmax over the last layer (per lane)
+    uint32_t best_id = 0xffffffffu;
+
+    for (uint32_t l = 0; l < P.n_layers; ++l) {
+        const slonn_fused_layer &ly = P.layer[l];
+        const bool is_last = (l + 1 == P.n_layers);
+        // input := previous activation (registers)
+        if (l == 0) fused_load_x_global<BF16, NC>(xr, P.x + (uint64_t)q * ly.D, ly.nchunks, lane);
+        else fused_load_x_shared<BF16, NC>(xr, xbuf4, ly.nchunks, lane);
+        __syncwarp();
+        uint32_t next_chunks = 0;
+        if (!is_last) { // clear the staging vector the selected nodes' activations go to
+            next_chunks = P.layer[l + 1].nchunks;
+            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (uint32_t i = lane; i < (ly.N >> 2); i += 32) xbuf4[i] = z;
+            __syncwarp();
+        }
+
+        uint32_t B = ly.N;
+        uint64_t off = 0;
+        bool implicit_ids = true;
+        if (ly.has_act) {
+            off = P.indptr[(uint64_t)q * P.n_act + ly.a];
+            B = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + ly.a + 1] - off);
+            // FreeHash: signs of the K*L sampled nodes' pre-activations
+            const uint32_t H = P.K * P.L;
+            uint32_t mykey = 0;
+            for (uint32_t h0 = 0; h0 < H; h0 += R) {
+                const uint4 *rows[R];
+                uint32_t node[R];
+#pragma unroll
+                for (int k = 0; k < R; ++k) {
+                    node[k] = __ldg(ly.hash_nodes + min(h0 + k, H - 1));
+                    rows[k] = reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)node[k] * ly.nchunks;
+                }
+                float acc[R];
+                fused_dot_rows<BF16, NC, R>(rows, xr, ly.nchunks, lane, acc);
+#pragma unroll
+                for (int k = 0; k < R; ++k) {
+                    const uint32_t h = h0 + k;
+                    if (h < H) {
+                        const float z = acc[k] + __ldg(ly.bias + node[k]);
+                        const uint32_t tb = h / P.K, j = h - tb * P.K;
+                        if (lane == tb && z > 0.0f) mykey |= (1u << j);
+                    }
+                }
+            }
+            if (P.codes && lane < P.L) P.codes[((uint64_t)q * P.n_act + ly.a) * P.L + lane] = (uint16_t)mykey;
+            if (B != ly.N && B <= ly.cap) {
+                fused_select(ly, P.K, P.L, mykey, B, bitmap, ids_s, lane);
+                implicit_ids = false;
+            }
+            if (P.out_ids) {
+                for (uint32_t i = lane; i < B; i += 32) P.out_ids[off + i] = implicit_ids ? i : (uint32_t)ids_s[i];
+            }
+        }
+
+        // the selected rows
+        for (uint32_t r0 = 0; r0 < B; r0 += R) {
+            const uint4 *rows[R];
+            uint32_t node[R];
+#pragma unroll
+            for (int k = 0; k < R; ++k) {
+                const uint32_t rr = min(r0 + k, B - 1);
+                node[k] = implicit_ids ? rr : (uint32_t)ids_s[rr];
+                rows[k] = reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)node[k] * ly.nchunks;
+            }
+            float acc[R];
+            fused_dot_rows<BF16, NC, R>(rows, xr, ly.nchunks, lane, acc);
+#pragma unroll
+            for (int k = 0; k < R; ++k) {
+                if (lane == (uint32_t)k && r0 + k < B) {
+                    float z = acc[k] + __ldg(ly.bias + node[k]);
+                    if (ly.relu) z = z > 0.0f ? z : 0.0f;
+                    if (ly.has_act && P.out_vals) P.out_vals[off + r0 + k] = z;
+                    if (!is_last) {
+                        xbuf[xs_index<BF16>(node[k], next_chunks)] = z;
+                    } else {
+                        if (ly.has_act) {
+                            P.logits[(uint64_t)q * P.logit_stride + r0 + k] = z;
+                            P.logit_ids[(uint64_t)q * P.logit_stride + r0 + k] = node[k];
+                        } else {
+                            P.logits[(uint64_t)q * P.logit_stride + node[k]] = z;
+                        }
+                        if (best_id == 0xffffffffu || z > best) { best = z; best_id = node[k]; }
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    }
+
+    if (P.pred) { // lowest node id among the largest logits
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            const float ob = __shfl_xor_sync(SLONN_FULL_MASK, best, off);
+            const uint32_t oi = __shfl_xor_sync(SLONN_FULL_MASK, best_id, off);
+            if (oi != 0xffffffffu && (best_id == 0xffffffffu || ob > best || (ob == best && oi < best_id))) {
+                best = ob;
+                best_id = oi;
+            }
+        }
+        if (lane == 0 && best_id != 0xffffffffu) P.pred[q] = best_id;
+    }
+}

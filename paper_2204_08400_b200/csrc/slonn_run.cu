@@ -5,6 +5,7 @@
 #include <cstring>
 #include <mutex>
 
+#include "slonn_fused_kernel.cuh"
 #include "slonn_run_kernels.cuh"
 
 namespace {
@@ -55,7 +56,7 @@ uint32_t dense_width(const slonn_model *m)
 }
 
 struct ws_layout {
-    uint64_t indptr, ids, vals, dense0, dense1, total;
+    uint64_t indptr, plan_sums, ids, vals, dense0, dense1, total;
 };
 
 ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp)
@@ -64,6 +65,8 @@ ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp)
     const uint64_t ent = active_entries(m, n, max_bp);
     uint64_t o = 0;
     w.indptr = o; o = align_up(o + ((uint64_t)n * m->n_act + 1) * sizeof(uint64_t), 256);
+    const uint64_t tiles = ((uint64_t)n * m->n_act + SLONN_PLAN_TILE - 1) / SLONN_PLAN_TILE;
+    w.plan_sums = o; o = align_up(o + (tiles + 1) * sizeof(uint64_t), 256);
     w.ids = o; o = align_up(o + ent * sizeof(uint32_t), 256);
     w.vals = o; o = align_up(o + ent * sizeof(float), 256);
     const uint64_t db = align_up((uint64_t)n * dense_width(m) * sizeof(float), 256);
@@ -127,6 +130,70 @@ int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint
     else { if ((rc = set_smem(gather_dot_kernel<false>, smem))) return rc;
         gather_dot_kernel<false><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(P); }
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+// ---- whole-network kernel for narrow layers -----------------------------------
+
+bool fused_eligible(const slonn_model *m)
+{
+    if (m->first_sparse) return false;
+    for (uint32_t l = 0; l < m->n_layers; ++l) {
+        const slonn_layer &ly = m->layer[l];
+        if (ly.D > SLONN_FUSED_MAX_D || ly.N > SLONN_FUSED_MAX_N) return false;
+    }
+    return true;
+}
+
+template <bool BF16, int NC>
+int launch_fused_t(const slonn_fused_params &P, cudaStream_t st)
+{
+    const size_t smem = (size_t)P.warp_bytes * SLONN_FUSED_WARPS;
+    int rc = set_smem(fused_network_kernel<BF16, NC>, smem);
+    if (rc) return rc;
+    const uint32_t grid = (P.n + SLONN_FUSED_WARPS - 1) / SLONN_FUSED_WARPS;
+    fused_network_kernel<BF16, NC><<<grid, SLONN_FUSED_WARPS * 32, smem, st>>>(P);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *indptr, uint32_t stride, cudaStream_t st)
+{
+    slonn_fused_params P;
+    memset(&P, 0, sizeof(P));
+    const uint32_t esz = m->dtype == SLONN_BF16 ? 2u : 4u;
+    uint32_t max_rounds = 1, xbuf = 4, ids_cap = 8, words = 1;
+    for (uint32_t l = 0; l < m->n_layers; ++l) {
+        const slonn_layer &ly = m->layer[l];
+        slonn_fused_layer &f = P.layer[l];
+        f.W = ly.W; f.bias = ly.bias; f.hash_nodes = ly.hash_nodes; f.tables = ly.tables;
+        f.D = ly.D; f.N = ly.N; f.nchunks = ly.D * esz / 16u; f.cap = ly.cap;
+        f.has_act = ly.has_act; f.a = m->act_index[l]; f.relu = (l + 1 == m->n_layers) ? 0u : 1u;
+        f.id_bytes = ly.id_bytes;
+        max_rounds = std::max(max_rounds, (f.nchunks + 31u) / 32u);
+        if (l > 0) xbuf = std::max(xbuf, (ly.D + 3u) / 4u * 4u);
+        if (ly.has_act) {
+            ids_cap = std::max(ids_cap, (ly.N + 7u) / 8u * 8u);
+            words = std::max(words, (ly.N + 31u) / 32u);
+        }
+    }
+    P.n_layers = m->n_layers; P.n = b->n_queries; P.n_act = m->n_act; P.K = m->K; P.L = m->L;
+    P.x = b->x_dense; P.indptr = indptr;
+    P.out_ids = b->active_ids; P.out_vals = b->active_vals; P.codes = b->codes;
+    P.logits = b->logits; P.logit_stride = stride; P.logit_ids = b->logit_ids; P.pred = b->pred;
+    P.status = b->status;
+    P.xbuf_floats = xbuf; P.ids_cap = ids_cap; P.bitmap_words = words;
+    P.warp_bytes = (uint32_t)align_up((uint64_t)xbuf * 4 + (uint64_t)ids_cap * 2 + (uint64_t)words * 4, 16);
+    const bool bf = m->dtype == SLONN_BF16;
+    if (bf) {
+        if (max_rounds <= 1) return launch_fused_t<true, 1>(P, st);
+        if (max_rounds <= 2) return launch_fused_t<true, 2>(P, st);
+        if (max_rounds <= 4) return launch_fused_t<true, 4>(P, st);
+    } else {
+        if (max_rounds <= 1) return launch_fused_t<false, 1>(P, st);
+        if (max_rounds <= 2) return launch_fused_t<false, 2>(P, st);
+        if (max_rounds <= 4) return launch_fused_t<false, 4>(P, st);
+        if (max_rounds <= 8) return launch_fused_t<false, 8>(P, st);
+    }
+    return SLONN_ERR_DIM;
 }
 
 } // namespace
@@ -226,10 +293,24 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
                 pp.act_N[a] = m->layer[l].N; pp.act_cap[a] = m->layer[l].cap; pp.act_layer[a] = l;
             }
         pp.indptr = indptr; pp.status = b->status;
+        const uint64_t tiles = ((uint64_t)n * m->n_act + SLONN_PLAN_TILE - 1) / SLONN_PLAN_TILE;
+        uint64_t *tile_sums = (uint64_t *)(ws + wl.plan_sums);
         TIC(SLONN_STAGE_PLAN);
-        plan_kernel<<<1, 1024, 0, st>>>(pp);
+        plan_partial_kernel<<<(uint32_t)tiles, SLONN_PLAN_THREADS, 0, st>>>(pp, tile_sums);
+        plan_final_kernel<<<(uint32_t)tiles, SLONN_PLAN_THREADS, 0, st>>>(pp, tile_sums);
         TOC();
         if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+    }
+
+    // narrow networks with enough queries to fill the GPU: one warp per query, every layer in one launch
+    if (b->kernel_path > SLONN_PATH_FUSED) return SLONN_ERR_ARG;
+    if (b->kernel_path == SLONN_PATH_FUSED && !fused_eligible(m)) return SLONN_ERR_DIM;
+    if (b->kernel_path == SLONN_PATH_FUSED ||
+        (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n >= 512)) {
+        TIC(SLONN_STAGE_FUSED);
+        const int rc = launch_fused(m, b, indptr, stride, st);
+        TOC();
+        return rc;
     }
 
     // input := x

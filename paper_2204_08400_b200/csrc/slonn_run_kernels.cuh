@@ -1,5 +1,5 @@
 // Kernels of the SLO-aware forward pass (Fig. 2 steps 1, 3, 4 of the paper):
-//   plan_kernel              budgets -> per (query, activator layer) list offsets
+//   plan_*_kernel            budgets -> per (query, activator layer) list offsets
 //   hash_select_kernel       FreeHash bits -> keys -> bucket lists -> first B distinct ids
 //   gather_dot_kernel        the selected rows' dot products, bias, activation
 //   sparse_first_layer_kernel  layer 0 fed by CSR rows (transposed weights)
@@ -69,22 +69,50 @@ __device__ __forceinline__ uint32_t plan_count(const slonn_plan_params &P, uint6
     return B;
 }
 
-__global__ void __launch_bounds__(1024) plan_kernel(slonn_plan_params P)
+// Two launches: per-tile sums, then each tile's prefix (tile base = sum of the tiles before it).
+#define SLONN_PLAN_THREADS 256
+#define SLONN_PLAN_PER_THREAD 8
+#define SLONN_PLAN_TILE (SLONN_PLAN_THREADS * SLONN_PLAN_PER_THREAD)
+
+__global__ void __launch_bounds__(SLONN_PLAN_THREADS) plan_partial_kernel(slonn_plan_params P, uint64_t *tile_sums)
 {
     __shared__ uint64_t warp_sums[32];
     __shared__ uint64_t total;
     const uint64_t M = (uint64_t)P.n * P.n_act;
-    const uint64_t per = (M + blockDim.x - 1) / blockDim.x;
-    const uint64_t e0 = (uint64_t)threadIdx.x * per;
-    const uint64_t e1 = e0 + per < M ? e0 + per : M;
+    const uint64_t e0 = (uint64_t)blockIdx.x * SLONN_PLAN_TILE + (uint64_t)threadIdx.x * SLONN_PLAN_PER_THREAD;
     uint64_t local = 0;
-    for (uint64_t e = e0; e < e1; ++e) local += plan_count(P, e, true);
-    uint64_t run = block_exclusive_scan<uint64_t>(local, warp_sums, &total);
-    for (uint64_t e = e0; e < e1; ++e) {
-        P.indptr[e] = run;
-        run += plan_count(P, e, false);
+    for (uint32_t k = 0; k < SLONN_PLAN_PER_THREAD; ++k)
+        if (e0 + k < M) local += plan_count(P, e0 + k, true);
+    block_exclusive_scan<uint64_t>(local, warp_sums, &total);
+    if (threadIdx.x == 0) tile_sums[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(SLONN_PLAN_THREADS) plan_final_kernel(slonn_plan_params P, const uint64_t *tile_sums)
+{
+    __shared__ uint64_t warp_sums[32];
+    __shared__ uint64_t total;
+    __shared__ uint64_t base_total;
+    const uint64_t M = (uint64_t)P.n * P.n_act;
+    // base of this tile: sum of all earlier tiles
+    uint64_t part = 0;
+    for (uint32_t t = threadIdx.x; t < blockIdx.x; t += blockDim.x) part += tile_sums[t];
+    block_exclusive_scan<uint64_t>(part, warp_sums, &base_total);
+    const uint64_t base = base_total;
+    const uint64_t e0 = (uint64_t)blockIdx.x * SLONN_PLAN_TILE + (uint64_t)threadIdx.x * SLONN_PLAN_PER_THREAD;
+    uint32_t cnt[SLONN_PLAN_PER_THREAD];
+    uint64_t local = 0;
+#pragma unroll
+    for (uint32_t k = 0; k < SLONN_PLAN_PER_THREAD; ++k) {
+        cnt[k] = (e0 + k < M) ? plan_count(P, e0 + k, false) : 0u;
+        local += cnt[k];
     }
-    if (threadIdx.x == 0) P.indptr[M] = total;
+    uint64_t run = base + block_exclusive_scan<uint64_t>(local, warp_sums, &total);
+#pragma unroll
+    for (uint32_t k = 0; k < SLONN_PLAN_PER_THREAD; ++k) {
+        if (e0 + k < M) P.indptr[e0 + k] = run;
+        run += cnt[k];
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) P.indptr[M] = base + total;
 }
 
 // ---------------------------------------------------------------------------

@@ -62,7 +62,8 @@ class DeviceModel:
 class DeviceBatch:
     """Device buffers of one batch: inputs uploaded once, outputs preallocated."""
 
-    def __init__(self, dm: DeviceModel, x, budget_bp: np.ndarray, max_budget_bp: int = 0, full_outputs=True):
+    def __init__(self, dm: DeviceModel, x, budget_bp: np.ndarray, max_budget_bp: int = 0, full_outputs=True,
+                 kernel_path: int = 0):
         dev = dm.device
         self.dm = dm
         m = dm.model
@@ -93,7 +94,7 @@ class DeviceBatch:
         self.batch = sl.make_batch(self.n, self.bp, self.logits, self.status, x_dense=self.x_dense,
                                    x_csr=self.x_csr, max_budget_bp=self.max_bp, logit_ids=self.logit_ids,
                                    pred=self.pred, codes=self.codes, active_indptr=self.indptr,
-                                   active_ids=self.ids, active_vals=self.vals)
+                                   active_ids=self.ids, active_vals=self.vals, kernel_path=kernel_path)
 
     def run(self, stream=None):
         sl.slonn_run(self.dm.model, self.batch, self.ws, self.ws_bytes, stream)
@@ -118,7 +119,7 @@ class DeviceBatch:
         return out
 
 
-def run_once(dm: DeviceModel, x, budget_bp: np.ndarray, max_budget_bp: int = 0) -> dict:
-    b = DeviceBatch(dm, x, budget_bp, max_budget_bp)
+def run_once(dm: DeviceModel, x, budget_bp: np.ndarray, max_budget_bp: int = 0, kernel_path: int = 0) -> dict:
+    b = DeviceBatch(dm, x, budget_bp, max_budget_bp, kernel_path=kernel_path)
     b.run()
     return b.results()

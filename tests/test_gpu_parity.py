@@ -24,22 +24,31 @@ def custom_workload(seed, dims, has_act, dtype, n, n_cal, K, L, law="relu_normal
                     K=K, L=L, seed=seed + 4, list_cap=list_cap)
 
 
+def kernel_paths(wl):
+    """Both kernel families where the network fits the one-warp-per-query kernel, else the staged one."""
+    fused_ok = (not wl.first_sparse) and max(wl.dims[:-1]) <= 1024 and max(wl.dims[1:]) <= 4096
+    return (1, 2) if fused_ok else (1,)
+
+
 def check(wl, n_cal=None, sample=None, expect_build=True):
     from paper_2204_08400_b200 import harness
     dm = harness.DeviceModel(wl, n_cal=n_cal)
     om = oracle_model(wl, n_cal=n_cal)
     if expect_build:
         assert_build_parity(dm, om, wl)
-    g = harness.run_once(dm, wl.x, wl.budget_bp)
     n_act = sum(wl.has_act)
     if sample is None:
         x, bp = wl.x, wl.budget_bp
     else:
         x, bp = take_queries(wl, sample), wl.budget_bp[sample]
-        g = slice_results(g, sample, n_act)
     o32 = oracle_run(om, wl, x, bp, orc.CANON32)
     o64 = oracle_run(om, wl, x, bp, orc.REF64)
-    info = assert_run_parity(g, o32, o64, wl, n_act, bool(wl.has_act[-1]))
+    info = None
+    for path in kernel_paths(wl):
+        g = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=path)
+        if sample is not None:
+            g = slice_results(g, sample, n_act)
+        info = assert_run_parity(g, o32, o64, wl, n_act, bool(wl.has_act[-1]))
     dm.free()
     return info
 
@@ -150,13 +159,14 @@ def test_invalid_budget_is_reported_not_fatal():
     from paper_2204_08400_b200 import harness
     wl = custom_workload(57, [32, 64, 8], [1, 0], "f32", n=16, n_cal=80, K=2, L=2, budgets=(2500,))
     dm = harness.DeviceModel(wl)
-    bp = wl.budget_bp.copy()
-    bp[5] = 0
-    g = harness.run_once(dm, wl.x, bp, max_budget_bp=5000)
-    assert g["status"][0] == 5 and g["status"][1] == 5     # SLONN_ERR_BUDGET at query 5
-    bp[5] = 2500
-    g = harness.run_once(dm, wl.x, bp, max_budget_bp=5000)
-    assert g["status"][0] == 0
+    for path in (1, 2):
+        bp = wl.budget_bp.copy()
+        bp[5] = 0
+        g = harness.run_once(dm, wl.x, bp, max_budget_bp=5000, kernel_path=path)
+        assert g["status"][0] == 5 and g["status"][1] == 5     # SLONN_ERR_BUDGET at query 5
+        bp[5] = 2500
+        g = harness.run_once(dm, wl.x, bp, max_budget_bp=5000, kernel_path=path)
+        assert g["status"][0] == 0
     dm.free()
 
 
@@ -164,10 +174,10 @@ def test_runs_are_deterministic():
     from paper_2204_08400_b200 import harness
     wl = custom_workload(58, [136, 200, 96, 24], [1, 1, 0], "bf16", n=256, n_cal=300, K=4, L=2)
     dm = harness.DeviceModel(wl)
-    a = harness.run_once(dm, wl.x, wl.budget_bp)
-    b = harness.run_once(dm, wl.x, wl.budget_bp)
-    for k in ("logits", "pred", "codes", "active_ids", "active_vals"):
-        assert np.array_equal(a[k], b[k])
+    runs = [harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=p) for p in (1, 1, 2, 2, 0)]
+    for b in runs[1:]:
+        for k in ("logits", "pred", "codes", "active_ids", "active_vals"):
+            assert np.array_equal(runs[0][k], b[k])
     dm.free()
 
 
@@ -195,3 +205,19 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert np.array_equal(logits, want["logits"]) and np.array_equal(pred, want["pred"])
     assert np.array_equal(codes, want["codes"])
     dm.free()
+
+
+def test_fused_path_refuses_wide_networks():
+    from paper_2204_08400_b200 import binding as sl, harness
+    wl = custom_workload(60, [2048, 64, 8], [1, 0], "f32", n=4, n_cal=40, K=2, L=2)
+    dm = harness.DeviceModel(wl)
+    with pytest.raises(sl.SlonnError) as e:
+        harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=2)
+    assert e.value.code == sl.ERR["DIM"]
+    dm.free()
+
+
+def test_plan_offsets_span_many_tiles():
+    # more (query, layer) entries than one plan tile, mixed budgets: offsets must equal the oracle's
+    wl = custom_workload(61, [32, 64, 40, 8], [1, 1, 0], "f32", n=5000, n_cal=100, K=2, L=2)
+    check(wl)
