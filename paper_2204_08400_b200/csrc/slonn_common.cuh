@@ -61,6 +61,54 @@ __device__ __forceinline__ void slonn_report(uint32_t *status, int code, uint32_
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
+// Element e (compile-time) of a 16-byte weight chunk, widened to fp32.
+template <bool BF16, int E>
+__device__ __forceinline__ float chunk_elem(const uint4 &w)
+{
+    if (BF16) {
+        const uint32_t u = (E >> 1) == 0 ? w.x : (E >> 1) == 1 ? w.y : (E >> 1) == 2 ? w.z : w.w;
+        return (E & 1) ? bf16_hi(u) : bf16_lo(u);
+    }
+    return __uint_as_float(E == 0 ? w.x : E == 1 ? w.y : E == 2 ? w.z : w.w);
+}
+
+// acc[r] = fmaf(w[r][E], x[E], acc[r]) for every row, elements in ascending order; rows are
+// interleaved so that consecutive instructions belong to independent accumulation chains.
+template <bool BF16, int R, int E, int VPC>
+struct chunk_fma {
+    __device__ static __forceinline__ void run(const uint4 (&w)[R], const float *x, float (&acc)[R])
+    {
+#pragma unroll
+        for (int r = 0; r < R; ++r) acc[r] = fmaf(chunk_elem<BF16, E>(w[r]), x[E], acc[r]);
+        chunk_fma<BF16, R, E + 1, VPC>::run(w, x, acc);
+    }
+};
+template <bool BF16, int R, int VPC>
+struct chunk_fma<BF16, R, VPC, VPC> {
+    __device__ static __forceinline__ void run(const uint4 (&)[R], const float *, float (&)[R]) {}
+};
+
+// Sums of 4 rows' 32 partials with 6 shuffles instead of 20.  Same additions as the xor
+// butterfly 16, 8, 4, 2, 1 of each row (each step adds the same two operands), but after
+// stride 16 a lane only carries two of the rows and after stride 8 one.  Returns the sum of
+// row (lane >> 3); the 8 lanes of a group hold the same value.
+__device__ __forceinline__ float reduce_rows4(const float (&a)[4], uint32_t lane)
+{
+    const bool hi16 = (lane & 16u) != 0u;
+    float k0 = hi16 ? a[2] : a[0], k1 = hi16 ? a[3] : a[1];
+    const float s0 = hi16 ? a[0] : a[2], s1 = hi16 ? a[1] : a[3];
+    k0 = k0 + __shfl_xor_sync(SLONN_FULL_MASK, s0, 16);
+    k1 = k1 + __shfl_xor_sync(SLONN_FULL_MASK, s1, 16);
+    const bool hi8 = (lane & 8u) != 0u;
+    float k = hi8 ? k1 : k0;
+    const float s = hi8 ? k0 : k1;
+    k = k + __shfl_xor_sync(SLONN_FULL_MASK, s, 8);
+    k = k + __shfl_xor_sync(SLONN_FULL_MASK, k, 4);
+    k = k + __shfl_xor_sync(SLONN_FULL_MASK, k, 2);
+    k = k + __shfl_xor_sync(SLONN_FULL_MASK, k, 1);
+    return k;
+}
+
 // Where input element j lives in the staged copy of a query's input vector.
 // fp32 weights: plain order.  bf16 weights: a 16-byte weight chunk holds 8
 // elements, so the 8 matching inputs are split into two float4 planes (first

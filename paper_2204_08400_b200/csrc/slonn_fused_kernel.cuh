@@ -5,8 +5,8 @@
 // wide; wider networks use the per-stage kernels.
 //
 // Same arithmetic as everywhere else in the library: lane p owns partial sum
-// p and takes 16-byte weight chunks p, p+32, ... in ascending order; xor
-// butterfly 16, 8, 4, 2, 1; bias last.
+// p and takes 16-byte weight chunks p, p+32, ... in ascending order; partials
+// are added pairwise with strides 16, 8, 4, 2, 1; bias last.
 #pragma once
 #include "slonn_common.cuh"
 
@@ -84,7 +84,8 @@ __device__ __forceinline__ void fused_load_x_shared(float (&xr)[NC * fused_trait
     }
 }
 
-// Fixed-order dot products of R rows against the register-resident input.
+// Fixed-order partial sums of R rows against the register-resident input: lane p ends
+// with partial p of every row (the caller reduces them).
 template <bool BF16, int NC, int R>
 __device__ __forceinline__ void fused_dot_rows(const uint4 *const (&rows)[R],
                                                const float (&xr)[NC * fused_traits<BF16>::VPC], uint32_t nchunks,
@@ -107,36 +108,9 @@ __device__ __forceinline__ void fused_dot_rows(const uint4 *const (&rows)[R],
         }
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-            const int i = i0 + g;
-            const uint32_t c = lane + 32u * i;
-            if (c < nchunks) {
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    float a = acc[r];
-                    if (BF16) {
-                        a = fmaf(bf16_lo(w[g][r].x), xr[i * VPC + 0], a);
-                        a = fmaf(bf16_hi(w[g][r].x), xr[i * VPC + 1], a);
-                        a = fmaf(bf16_lo(w[g][r].y), xr[i * VPC + 2], a);
-                        a = fmaf(bf16_hi(w[g][r].y), xr[i * VPC + 3], a);
-                        a = fmaf(bf16_lo(w[g][r].z), xr[i * VPC + 4], a);
-                        a = fmaf(bf16_hi(w[g][r].z), xr[i * VPC + 5], a);
-                        a = fmaf(bf16_lo(w[g][r].w), xr[i * VPC + 6], a);
-                        a = fmaf(bf16_hi(w[g][r].w), xr[i * VPC + 7], a);
-                    } else {
-                        a = fmaf(__uint_as_float(w[g][r].x), xr[i * VPC + 0], a);
-                        a = fmaf(__uint_as_float(w[g][r].y), xr[i * VPC + 1], a);
-                        a = fmaf(__uint_as_float(w[g][r].z), xr[i * VPC + 2], a);
-                        a = fmaf(__uint_as_float(w[g][r].w), xr[i * VPC + 3], a);
-                    }
-                    acc[r] = a;
-                }
-            }
+            const uint32_t c = lane + 32u * (i0 + g);
+            if (c < nchunks) chunk_fma<BF16, R, 0, VPC>::run(w[g], &xr[(i0 + g) * VPC], acc);
         }
-    }
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-#pragma unroll
-        for (int r = 0; r < R; ++r) acc[r] = acc[r] + __shfl_xor_sync(SLONN_FULL_MASK, acc[r], off);
     }
 }
 
@@ -203,7 +177,7 @@ __device__ __forceinline__ void fused_select(const slonn_fused_layer &ly, uint32
 }
 
 template <bool BF16, int NC>
-__global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32) fused_network_kernel(const __grid_constant__ slonn_fused_params P)
+__global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, 4) fused_network_kernel(const __grid_constant__ slonn_fused_params P)
 {
     constexpr int VPC = fused_traits<BF16>::VPC;
     constexpr int R = SLONN_FUSED_ROWS;
@@ -247,21 +221,23 @@ __global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32) fused_network_kernel(c
             uint32_t mykey = 0;
             for (uint32_t h0 = 0; h0 < H; h0 += R) {
                 const uint4 *rows[R];
-                uint32_t node[R];
 #pragma unroll
                 for (int k = 0; k < R; ++k) {
-                    node[k] = __ldg(ly.hash_nodes + min(h0 + k, H - 1));
-                    rows[k] = reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)node[k] * ly.nchunks;
+                    const uint32_t nd = __ldg(ly.hash_nodes + min(h0 + k, H - 1));
+                    rows[k] = reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)nd * ly.nchunks;
                 }
                 float acc[R];
                 fused_dot_rows<BF16, NC, R>(rows, xr, ly.nchunks, lane, acc);
+                // lanes 8k..8k+7 hold the sum of row k; collect the R signs with one ballot
+                const uint32_t mynode = __ldg(ly.hash_nodes + min(h0 + (lane >> 3), H - 1));
+                const float z = reduce_rows4(acc, lane) + __ldg(ly.bias + mynode);
+                const uint32_t signs = __ballot_sync(SLONN_FULL_MASK, z > 0.0f);
 #pragma unroll
                 for (int k = 0; k < R; ++k) {
                     const uint32_t h = h0 + k;
                     if (h < H) {
-                        const float z = acc[k] + __ldg(ly.bias + node[k]);
                         const uint32_t tb = h / P.K, j = h - tb * P.K;
-                        if (lane == tb && z > 0.0f) mykey |= (1u << j);
+                        if (lane == tb && ((signs >> (8 * k)) & 1u)) mykey |= (1u << j);
                     }
                 }
             }
@@ -278,32 +254,31 @@ __global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32) fused_network_kernel(c
         // the selected rows
         for (uint32_t r0 = 0; r0 < B; r0 += R) {
             const uint4 *rows[R];
-            uint32_t node[R];
 #pragma unroll
             for (int k = 0; k < R; ++k) {
                 const uint32_t rr = min(r0 + k, B - 1);
-                node[k] = implicit_ids ? rr : (uint32_t)ids_s[rr];
-                rows[k] = reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)node[k] * ly.nchunks;
+                const uint32_t nd = implicit_ids ? rr : (uint32_t)ids_s[rr];
+                rows[k] = reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)nd * ly.nchunks;
             }
             float acc[R];
             fused_dot_rows<BF16, NC, R>(rows, xr, ly.nchunks, lane, acc);
-#pragma unroll
-            for (int k = 0; k < R; ++k) {
-                if (lane == (uint32_t)k && r0 + k < B) {
-                    float z = acc[k] + __ldg(ly.bias + node[k]);
-                    if (ly.relu) z = z > 0.0f ? z : 0.0f;
-                    if (ly.has_act && P.out_vals) P.out_vals[off + r0 + k] = z;
-                    if (!is_last) {
-                        xbuf[xs_index<BF16>(node[k], next_chunks)] = z;
+            const float sum = reduce_rows4(acc, lane); // row r0 + (lane >> 3)
+            const uint32_t r = r0 + (lane >> 3);
+            if ((lane & 7u) == 0u && r < B) {
+                const uint32_t nd = implicit_ids ? r : (uint32_t)ids_s[r];
+                float z = sum + __ldg(ly.bias + nd);
+                if (ly.relu) z = z > 0.0f ? z : 0.0f;
+                if (ly.has_act && P.out_vals) P.out_vals[off + r] = z;
+                if (!is_last) {
+                    xbuf[xs_index<BF16>(nd, next_chunks)] = z;
+                } else {
+                    if (ly.has_act) {
+                        P.logits[(uint64_t)q * P.logit_stride + r] = z;
+                        P.logit_ids[(uint64_t)q * P.logit_stride + r] = nd;
                     } else {
-                        if (ly.has_act) {
-                            P.logits[(uint64_t)q * P.logit_stride + r0 + k] = z;
-                            P.logit_ids[(uint64_t)q * P.logit_stride + r0 + k] = node[k];
-                        } else {
-                            P.logits[(uint64_t)q * P.logit_stride + node[k]] = z;
-                        }
-                        if (best_id == 0xffffffffu || z > best) { best = z; best_id = node[k]; }
+                        P.logits[(uint64_t)q * P.logit_stride + nd] = z;
                     }
+                    if (best_id == 0xffffffffu || z > best) { best = z; best_id = nd; }
                 }
             }
         }
