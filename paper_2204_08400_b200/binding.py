@@ -15,7 +15,7 @@ ERR = {"ARG": -1, "DIM": -2, "DTYPE": -3, "ALIGN": -4, "BUDGET": -5, "NOMEM": -6
        "TIMEOUT": -8, "WORKSPACE": -9}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libslonn.so")
+LIB_PATH = os.environ.get("SLONN_LIB", os.path.join(_HERE, "libslonn.so"))  # SLONN_LIB: another build of the library
 
 EXPORTS = [
     "slonn_version", "slonn_strerror", "slonn_build", "slonn_model_info", "slonn_model_tables_to_host",

@@ -10,8 +10,16 @@
 #pragma once
 #include "slonn_common.cuh"
 
-#define SLONN_FUSED_ROWS 4
-#define SLONN_FUSED_WARPS 4
+#define SLONN_FUSED_ROWS 4          // rows per pass; the 6-shuffle reduction is written for 4
+#ifndef SLONN_FUSED_WARPS
+#define SLONN_FUSED_WARPS 4         // queries (warps) per block
+#endif
+#ifndef SLONN_FUSED_GROUP
+#define SLONN_FUSED_GROUP 1         // 32-chunk rounds whose loads are issued together
+#endif
+#ifndef SLONN_FUSED_MIN_BLOCKS
+#define SLONN_FUSED_MIN_BLOCKS 5    // resident blocks per SM the register allocation must allow
+#endif
 #define SLONN_FUSED_MAX_D 1024
 #define SLONN_FUSED_MAX_N 4096
 
@@ -92,7 +100,7 @@ __device__ __forceinline__ void fused_dot_rows(const uint4 *const (&rows)[R],
                                                uint32_t lane, float (&acc)[R])
 {
     constexpr int VPC = fused_traits<BF16>::VPC;
-    constexpr int G = NC < 2 ? NC : 2; // rounds whose loads are issued together
+    constexpr int G = NC < SLONN_FUSED_GROUP ? NC : SLONN_FUSED_GROUP; // rounds whose loads are issued together
 #pragma unroll
     for (int r = 0; r < R; ++r) acc[r] = 0.0f;
 #pragma unroll
@@ -177,7 +185,7 @@ __device__ __forceinline__ void fused_select(const slonn_fused_layer &ly, uint32
 }
 
 template <bool BF16, int NC>
-__global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, 4) fused_network_kernel(const __grid_constant__ slonn_fused_params P)
+__global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, SLONN_FUSED_MIN_BLOCKS) fused_network_kernel(const __grid_constant__ slonn_fused_params P)
 {
     constexpr int VPC = fused_traits<BF16>::VPC;
     constexpr int R = SLONN_FUSED_ROWS;
