@@ -186,7 +186,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2204_08400_b200 import binding as sl, harness
+    from paper_2204_08400_b200 import binding as sl, harness, replicas
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
@@ -219,12 +219,7 @@ def main():
             batch.run(stream)
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms / steps
+        return replicas.slowest_rank_ms(e0.elapsed_time(e1), dev) / steps
 
     # ---- headline: device-resident inputs ----
     batch = harness.DeviceBatch(dm, wl.x, wl.budget_bp, max_budget_bp=args.budget_bp, full_outputs=False)
@@ -239,7 +234,8 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     status = batch.status.cpu().numpy()
     assert status[0] == 0, f"device status {status}"
-    value = world * n / (ms_step / 1e3)
+    n_all = replicas.total_units(n, dev)          # queries all ranks processed in one step
+    value = n_all / (ms_step / 1e3)
     launches_per_step = None  # counted below from the per-stage launch counters
 
     # ---- per-stage device time of the same step (event pair around every launch) ----
@@ -316,13 +312,9 @@ def main():
             up, down = sl.slonn_run_host(dm.model, hb, hws, nb, stream)
         e1.record(stream)
         barrier()
-        ms_e = e0.elapsed_time(e1) / e_steps
-        if world > 1:
-            t = torch.tensor([ms_e], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e = float(t.item())
+        ms_e = replicas.slowest_rank_ms(e0.elapsed_time(e1), dev) / e_steps
         assert int(h_status[0]) == 0
-        e2e = {"value": world * n / (ms_e / 1e3), "unit": "queries/s", "h2d_bytes_per_step": int(up),
+        e2e = {"value": n_all / (ms_e / 1e3), "unit": "queries/s", "h2d_bytes_per_step": int(up),
                "d2h_bytes_per_step": int(down), "ms_per_step": ms_e}
 
     # ---- the CPU oracle beside it (rank 0, single-GPU runs only) ----

@@ -121,15 +121,17 @@ __device__ __forceinline__ uint32_t xs_index(uint32_t j, uint32_t nchunks)
     return j;
 }
 
-// Fixed-order dot products of R weight rows with the staged input, one warp.
+// Fixed-order partial sums of R weight rows with the staged input, one warp.
 // Lane p owns partial sum p: it takes 16-byte chunks p, p+32, ... of each row
-// and accumulates their elements in ascending order with fused multiply-adds;
-// the xor butterfly then adds partials in the order 16, 8, 4, 2, 1.  Every lane
-// ends with the same sums.  Bias is added by the caller.
+// and accumulates their elements in ascending order with fused multiply-adds
+// (rows interleaved, so neighbouring instructions are independent).  The caller
+// adds the 32 partials of each row in the order 16, 8, 4, 2, 1 (reduce_rows4)
+// and then the bias.
 template <bool BF16, int R>
 __device__ __forceinline__ void warp_dot_rows(const uint4 *const (&rows)[R], const float4 *xs4,
                                               uint32_t nchunks, uint32_t lane, float (&acc)[R])
 {
+    constexpr int VPC = BF16 ? 8 : 4;
 #pragma unroll
     for (int r = 0; r < R; ++r) acc[r] = 0.0f;
 #pragma unroll 2
@@ -137,39 +139,14 @@ __device__ __forceinline__ void warp_dot_rows(const uint4 *const (&rows)[R], con
         uint4 w[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) w[r] = __ldg(rows[r] + c);
+        float x[VPC];
+        const float4 xa = xs4[c];
+        x[0] = xa.x; x[1] = xa.y; x[2] = xa.z; x[3] = xa.w;
         if (BF16) {
-            const float4 xa = xs4[c];
             const float4 xb = xs4[nchunks + c];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                float a = acc[r];
-                a = fmaf(bf16_lo(w[r].x), xa.x, a);
-                a = fmaf(bf16_hi(w[r].x), xa.y, a);
-                a = fmaf(bf16_lo(w[r].y), xa.z, a);
-                a = fmaf(bf16_hi(w[r].y), xa.w, a);
-                a = fmaf(bf16_lo(w[r].z), xb.x, a);
-                a = fmaf(bf16_hi(w[r].z), xb.y, a);
-                a = fmaf(bf16_lo(w[r].w), xb.z, a);
-                a = fmaf(bf16_hi(w[r].w), xb.w, a);
-                acc[r] = a;
-            }
-        } else {
-            const float4 xa = xs4[c];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                float a = acc[r];
-                a = fmaf(__uint_as_float(w[r].x), xa.x, a);
-                a = fmaf(__uint_as_float(w[r].y), xa.y, a);
-                a = fmaf(__uint_as_float(w[r].z), xa.z, a);
-                a = fmaf(__uint_as_float(w[r].w), xa.w, a);
-                acc[r] = a;
-            }
+            x[VPC - 4] = xb.x; x[VPC - 3] = xb.y; x[VPC - 2] = xb.z; x[VPC - 1] = xb.w;
         }
-    }
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-#pragma unroll
-        for (int r = 0; r < R; ++r) acc[r] = acc[r] + __shfl_xor_sync(SLONN_FULL_MASK, acc[r], off);
+        chunk_fma<BF16, R, 0, VPC>::run(w, x, acc);
     }
 }
 

@@ -8,7 +8,7 @@
 #include "slonn_common.cuh"
 
 #define SLONN_THREADS 256
-#define SLONN_ROWS_PER_WARP 4
+#define SLONN_ROWS_PER_WARP 4 // the 6-shuffle reduction (reduce_rows4) is written for 4 rows
 
 // ---------------------------------------------------------------------------
 // block-wide exclusive scan of one value per thread (blockDim.x <= 1024)
@@ -165,18 +165,16 @@ __global__ void __launch_bounds__(SLONN_THREADS) hash_select_kernel(slonn_select
     const uint32_t row_u4 = P.nchunks; // uint4 per weight row
     for (uint32_t h0 = warp * SLONN_ROWS_PER_WARP; h0 < H; h0 += nwarps * SLONN_ROWS_PER_WARP) {
         const uint4 *rows[SLONN_ROWS_PER_WARP];
-        uint32_t node[SLONN_ROWS_PER_WARP];
 #pragma unroll
         for (int r = 0; r < SLONN_ROWS_PER_WARP; ++r) {
-            const uint32_t h = min(h0 + r, H - 1);
-            node[r] = __ldg(P.hash_nodes + h);
-            rows[r] = reinterpret_cast<const uint4 *>(P.W) + (uint64_t)node[r] * row_u4;
+            const uint32_t nd = __ldg(P.hash_nodes + min(h0 + r, H - 1));
+            rows[r] = reinterpret_cast<const uint4 *>(P.W) + (uint64_t)nd * row_u4;
         }
         float acc[SLONN_ROWS_PER_WARP];
         warp_dot_rows<BF16, SLONN_ROWS_PER_WARP>(rows, xs4, P.nchunks, lane, acc);
-#pragma unroll
-        for (int r = 0; r < SLONN_ROWS_PER_WARP; ++r)
-            if (lane == (uint32_t)r && h0 + r < H) zh[h0 + r] = acc[r] + __ldg(P.bias + node[r]);
+        const float sum = reduce_rows4(acc, lane); // row h0 + (lane >> 3)
+        const uint32_t h = h0 + (lane >> 3);
+        if ((lane & 7u) == 0u && h < H) zh[h] = sum + __ldg(P.bias + __ldg(P.hash_nodes + h));
     }
     for (uint32_t i = threadIdx.x; i < nwords; i += blockDim.x) bitmap[i] = 0u;
     __syncthreads();
@@ -320,29 +318,28 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     for (uint32_t r = r0 + warp * SLONN_ROWS_PER_WARP; r < r1; r += nwarps * SLONN_ROWS_PER_WARP) {
         const uint4 *rows[SLONN_ROWS_PER_WARP];
-        uint32_t node[SLONN_ROWS_PER_WARP];
 #pragma unroll
         for (int k = 0; k < SLONN_ROWS_PER_WARP; ++k) {
             const uint32_t rr = min(r + k, r1 - 1);
-            node[k] = P.use_list ? __ldg(P.ids + off + rr) : rr;
-            rows[k] = reinterpret_cast<const uint4 *>(P.W) + (uint64_t)node[k] * P.nchunks;
+            const uint32_t nd = P.use_list ? __ldg(P.ids + off + rr) : rr;
+            rows[k] = reinterpret_cast<const uint4 *>(P.W) + (uint64_t)nd * P.nchunks;
         }
         float acc[SLONN_ROWS_PER_WARP];
         warp_dot_rows<BF16, SLONN_ROWS_PER_WARP>(rows, smem4, P.nchunks, lane, acc);
-#pragma unroll
-        for (int k = 0; k < SLONN_ROWS_PER_WARP; ++k) {
-            if (lane == (uint32_t)k && r + k < r1) {
-                float z = acc[k] + __ldg(P.bias + node[k]);
-                if (P.relu) z = z > 0.0f ? z : 0.0f;
-                if (P.use_list) {
-                    if (P.out_vals) P.out_vals[off + r + k] = z;
-                    if (P.out_dense) {
-                        P.out_dense[(uint64_t)q * P.out_stride + r + k] = z;
-                        if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q * P.out_stride + r + k] = node[k];
-                    }
-                } else {
-                    P.out_dense[(uint64_t)q * P.out_stride + node[k]] = z;
+        const float sum = reduce_rows4(acc, lane); // row r + (lane >> 3)
+        const uint32_t mr = r + (lane >> 3);
+        if ((lane & 7u) == 0u && mr < r1) {
+            const uint32_t nd = P.use_list ? __ldg(P.ids + off + mr) : mr;
+            float z = sum + __ldg(P.bias + nd);
+            if (P.relu) z = z > 0.0f ? z : 0.0f;
+            if (P.use_list) {
+                if (P.out_vals) P.out_vals[off + mr] = z;
+                if (P.out_dense) {
+                    P.out_dense[(uint64_t)q * P.out_stride + mr] = z;
+                    if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q * P.out_stride + mr] = nd;
                 }
+            } else {
+                P.out_dense[(uint64_t)q * P.out_stride + nd] = z;
             }
         }
     }

@@ -138,6 +138,36 @@ def test_c5_mixed_budgets_reduced():
     check(wl)
 
 
+# ---- full sizes, in the launch configuration the benchmark times, on sampled queries ----
+
+def test_c2_full_size_sampled():
+    wl = wl_mod.load("c2", budget_bp=1000)                      # 65,536 queries, 16,384 calibration rows
+    sample = np.unique(np.linspace(0, wl.n_queries - 1, 192).astype(np.int64))
+    info = check(wl, sample=sample)
+    assert info["decision_disagreements"] <= 2
+
+
+def test_c5_full_widths_mixed_budgets_sampled():
+    wl = wl_mod.load("c5", n_queries=8192, n_cal=512)            # one batch of the mixed-budget stream
+    sample = np.unique(np.linspace(0, wl.n_queries - 1, 48).astype(np.int64))
+    check(wl, n_cal=512, sample=sample)
+
+
+def test_c4_full_widths_batch_sizes_sampled():
+    import dataclasses
+    full = wl_mod.load("c4", n_queries=64, n_cal=192, budget_bp=1000)
+    for n, k in ((1, 1), (64, 8)):
+        wl = dataclasses.replace(full, x=full.x[:n], budget_bp=full.budget_bp[:n])
+        sample = np.unique(np.linspace(0, n - 1, k).astype(np.int64))
+        check(wl, n_cal=192, sample=sample, expect_build=(n == 1))
+
+
+def test_c3_full_width_output_layer_sampled():
+    wl = wl_mod.load("c3", n_queries=256, n_cal=256, budget_bp=1000, list_cap=20000)
+    sample = np.arange(0, 256, 32)
+    check(wl, n_cal=256, sample=sample)
+
+
 # ---- edge cases -----------------------------------------------------------------
 
 def test_empty_batch_and_single_query():
