@@ -115,13 +115,13 @@ def oracle_queries_per_sec(wl, budget_bp, target_seconds=12.0):
     om = oracle_model(wl)
     n0 = min(wl.n_queries, 256)
     idx = np.arange(n0)
-    bp = np.full(n0, budget_bp, np.uint16)
+    bp = wl.budget_bp[:n0] if budget_bp is None else np.full(n0, budget_bp, np.uint16)
     t0 = time.perf_counter()
     oracle_run(om, wl, take_queries(wl, idx), bp, orc.CANON32)
     dt = max(time.perf_counter() - t0, 1e-4)
     n1 = int(min(wl.n_queries, max(n0, n0 * target_seconds / dt)))
     idx = np.arange(n1)
-    bp = np.full(n1, budget_bp, np.uint16)
+    bp = wl.budget_bp[:n1] if budget_bp is None else np.full(n1, budget_bp, np.uint16)
     xs = take_queries(wl, idx)
     t0 = time.perf_counter()
     oracle_run(om, wl, xs, bp, orc.CANON32)
@@ -132,11 +132,13 @@ def oracle_queries_per_sec(wl, budget_bp, target_seconds=12.0):
 def run_reference(args, rank, world):
     if rank != 0:
         return
-    wl = workloads.load(args.workload, budget_bp=args.budget_bp)
+    wl = workloads.load(args.workload, n_queries=args.queries, n_cal=args.n_cal,
+                        budget_bp=args.budget_bp if args.budget_bp else None)
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     from oracle import oracle as orc
     from parity_util import oracle_run
-    qps, cores, n1, dt, (om, xs, bp) = oracle_queries_per_sec(wl, args.budget_bp, target_seconds=6.0)
+    qps, cores, n1, dt, (om, xs, bp) = oracle_queries_per_sec(wl, args.budget_bp if args.budget_bp else None,
+                                                              target_seconds=6.0)
     for _ in range(args.warmup):
         pass  # the sizing pass above already warmed caches; warm-up steps would only repeat it
     times = []
@@ -167,7 +169,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2")
-    ap.add_argument("--budget-bp", type=int, default=1000)
+    ap.add_argument("--budget-bp", type=int, default=1000,
+                    help="budget of every query in basis points; 0 = the workload's mixed per-query budgets (c5)")
     ap.add_argument("--queries", type=int, default=None, help="override the workload's query count")
     ap.add_argument("--n-cal", type=int, default=None)
     ap.add_argument("--no-sweep", action="store_true")
@@ -198,7 +201,9 @@ def main():
 
     # every rank is a replica with its own batch (same law, rank-specific seed is not needed:
     # throughput does not depend on the draw; parity tests cover the values)
-    wl = workloads.load(args.workload, n_queries=args.queries, n_cal=args.n_cal, budget_bp=args.budget_bp)
+    wl = workloads.load(args.workload, n_queries=args.queries, n_cal=args.n_cal,
+                        budget_bp=args.budget_bp if args.budget_bp else None)
+    max_bp = int(wl.budget_bp.max())
     n = wl.n_queries
     dm = harness.DeviceModel(wl, device=dev)
     stream = torch.cuda.current_stream(dev)
@@ -222,7 +227,7 @@ def main():
         return replicas.slowest_rank_ms(e0.elapsed_time(e1), dev) / steps
 
     # ---- headline: device-resident inputs ----
-    batch = harness.DeviceBatch(dm, wl.x, wl.budget_bp, max_budget_bp=args.budget_bp, full_outputs=False)
+    batch = harness.DeviceBatch(dm, wl.x, wl.budget_bp, max_budget_bp=max_bp, full_outputs=False)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -283,7 +288,7 @@ def main():
     e2e = None
     if not args.no_e2e:
         x_nnz = int(wl.x[0][-1]) if wl.first_sparse else 0
-        stride = sl.slonn_logit_stride(dm.model, args.budget_bp)
+        stride = sl.slonn_logit_stride(dm.model, max_bp)
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
         view = {np.dtype(np.uint16): np.int16, np.dtype(np.uint32): np.int32, np.dtype(np.uint64): np.int64}
         pinv = lambda a: pin(np.ascontiguousarray(a).view(view.get(a.dtype, a.dtype)))
@@ -294,13 +299,13 @@ def main():
         h_lids = torch.zeros((n, stride), dtype=torch.int32).pin_memory() if wl.has_act[-1] else None
         if wl.first_sparse:
             h_csr = tuple(pinv(a) for a in wl.x)
-            hb = sl.make_batch(n, h_bp, h_logits, h_status, x_csr=h_csr, max_budget_bp=args.budget_bp,
+            hb = sl.make_batch(n, h_bp, h_logits, h_status, x_csr=h_csr, max_budget_bp=max_bp,
                                logit_ids=h_lids, pred=h_pred)
         else:
             h_x = pin(wl.x)
-            hb = sl.make_batch(n, h_bp, h_logits, h_status, x_dense=h_x, max_budget_bp=args.budget_bp,
+            hb = sl.make_batch(n, h_bp, h_logits, h_status, x_dense=h_x, max_budget_bp=max_bp,
                                logit_ids=h_lids, pred=h_pred)
-        nb = sl.slonn_host_workspace_bytes(dm.model, n, args.budget_bp, x_nnz)
+        nb = sl.slonn_host_workspace_bytes(dm.model, n, max_bp, x_nnz)
         hws = torch.empty(nb, dtype=torch.uint8, device=dev)
         e_steps = max(3, min(args.steps, 10))
         for _ in range(3):
@@ -320,7 +325,7 @@ def main():
     # ---- the CPU oracle beside it (rank 0, single-GPU runs only) ----
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        qps, cores, n1, dt, _ = oracle_queries_per_sec(wl, args.budget_bp)
+        qps, cores, n1, dt, _ = oracle_queries_per_sec(wl, None if not args.budget_bp else args.budget_bp)
         cpu = {"value": qps, "unit": "queries/s", "cores": cores, "kind": "oracle",
                "sample": f"first {n1} of {n} queries, {dt:.1f} s"}
 
@@ -331,7 +336,8 @@ def main():
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": esz_name, "data": "synthetic",
             "config": {"workload": f"{args.workload}: " + "-".join(map(str, wl.dims)) +
-                                   f" {wl.dtype} weights, {n} queries/GPU, budget {args.budget_bp} bp, K={wl.K} L={wl.L}",
+                                   f" {wl.dtype} weights, {n} queries/GPU, budget " +
+                                   (f"{args.budget_bp} bp" if args.budget_bp else "mixed 5/10/25/50/100 %") + f", K={wl.K} L={wl.L}",
                        "queries_per_step_per_gpu": n, "budget_bp": args.budget_bp,
                        "l2": "inputs_larger_than_l2" if (wl.x.nbytes if not wl.first_sparse else 0) > L2_BYTES
                              else "weights_and_inputs_l2_resident",

@@ -195,6 +195,24 @@ int slonn_run(const slonn_model *m, const slonn_batch *batch, void *workspace,
               uint64_t workspace_bytes, void *stream);
 
 /*
+ * One dense layer on the tensor cores: out = act(X * W^T + bias), the case in which every
+ * node of a layer is computed (Sec. 3.4: with all nodes computed an SLO-NN does exactly the
+ * work of the full network).  bf16 operands, fp32 accumulation in tensor memory.
+ *   x_bf16  : [M][D] bf16 bit patterns, row-major      w_bf16 : [N][D] bf16, row-major
+ *   bias    : [N] fp32, nullable                       relu   : 1 = max(., 0), 0 = identity
+ *   out_f32 : [M][N] fp32, nullable                    out_bf16 : [M][N] bf16 (rounded to
+ *             nearest even), nullable; at least one of the two
+ *   status  : [4] device words, nullable; cleared, then [0] = -SLONN_ERR_TIMEOUT if a bounded
+ *             on-chip wait ran out
+ * D * 2 bytes must be a multiple of 16 and both matrices 16-byte aligned.  Asynchronous on
+ * `stream`.  The accumulation order of the tensor core is unspecified, so results agree with
+ * the fixed-order kernels to rounding (about 1e-6 relative per sum), not bit for bit.
+ */
+int slonn_dense_layer(const void *x_bf16, const void *w_bf16, const float *bias, uint32_t M,
+                      uint32_t N, uint32_t D, uint32_t relu, float *out_f32, void *out_bf16,
+                      uint32_t *status, void *stream);
+
+/*
  * slonn_run without a caller-provided workspace.  (The paper has no counterpart;
  * this exists for deployment.)
  *

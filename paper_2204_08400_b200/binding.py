@@ -20,7 +20,7 @@ LIB_PATH = os.environ.get("SLONN_LIB", os.path.join(_HERE, "libslonn.so"))  # SL
 EXPORTS = [
     "slonn_version", "slonn_strerror", "slonn_build", "slonn_model_info", "slonn_model_tables_to_host",
     "slonn_free", "slonn_active_capacity", "slonn_logit_stride", "slonn_workspace_bytes", "slonn_run",
-    "slonn_run_timed", "slonn_run_static",
+    "slonn_run_timed", "slonn_run_static", "slonn_dense_layer",
     "slonn_host_workspace_bytes", "slonn_run_host",
 ]
 
@@ -86,6 +86,9 @@ def lib():
         L.slonn_run.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p]
         L.slonn_run_static.restype = C.c_int
         L.slonn_run_static.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p]
+        L.slonn_dense_layer.restype = C.c_int
+        L.slonn_dense_layer.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32,
+                                        C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.slonn_run_timed.restype = C.c_int
         L.slonn_run_timed.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p,
                                       C.c_void_p, C.c_void_p]
@@ -273,6 +276,15 @@ def slonn_run(model: Model, batch: _Batch, workspace, workspace_bytes: int, stre
     rc = lib().slonn_run(model.handle, C.byref(batch), _ptr(workspace), workspace_bytes, _stream_ptr(stream))
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_run")
+
+
+def slonn_dense_layer(x_bf16, w_bf16, bias, M: int, N: int, D: int, relu: bool, out_f32=None, out_bf16=None,
+                      status=None, stream=None) -> None:
+    """out = act(X W^T + bias) on the tensor cores; device tensors, bf16 bit patterns for X, W, out_bf16."""
+    rc = lib().slonn_dense_layer(_ptr(x_bf16), _ptr(w_bf16), _ptr(bias), M, N, D, int(bool(relu)), _ptr(out_f32),
+                                 _ptr(out_bf16), _ptr(status), _stream_ptr(stream))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_dense_layer")
 
 
 STATIC_WORKSPACE_BYTES = 16 << 20

@@ -1,0 +1,301 @@
+// Dense layer on the 5th-generation tensor cores: C = act(A * W^T + bias) with bf16
+// operands and fp32 accumulation.  This is the "all nodes computed" case of the paper
+// (Sec. 3.4: at a 100 % budget an SLO-NN is the full network), the one stage of the path that
+// is a dense contraction.
+//
+// One 128x128 output tile per block, K in steps of 64 (one 128-byte swizzle atom):
+//   warp 0 / one lane : TMA producer, cp.async.bulk.tensor 2-D tile loads into a 4-stage ring
+//   warp 1 / one lane : tcgen05.mma issuer, accumulator in tensor memory (128 lanes x 128 columns)
+//   warps 0-3         : epilogue, tcgen05.ld of the accumulator, bias, activation, stores
+// Stages hand over through mbarriers (TMA -> MMA by transaction bytes, MMA -> TMA and
+// MMA -> epilogue by tcgen05.commit).  Every wait is bounded: when one runs out the block raises
+// an abort flag, lets outstanding copies land, frees its tensor memory and reports
+// SLONN_ERR_TIMEOUT through the status word.  No cluster launch, no multicast.
+//
+// Sums are not bit-compatible with the fixed-order fp32 kernels (the tensor core's accumulation
+// order is not specified), so this path is only used where the caller asked for it.
+#include <cuda.h>
+
+#include <cstring>
+#include <mutex>
+
+#include "slonn_common.cuh"
+#include "slonn_dense_tc.cuh"
+
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr uint32_t TMEM_COLS = 128;
+constexpr uint32_t STAGE_A_BYTES = BM * BK * 2, STAGE_B_BYTES = BN * BK * 2;
+constexpr uint32_t RING_BYTES = STAGES * (STAGE_A_BYTES + STAGE_B_BYTES);
+constexpr uint32_t SMEM_BYTES = RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+// instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = 128
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+// Bounded wait; false when it gave up or another role already raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+{
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1u;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap *map, int32_t c0, int32_t c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst_smem), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+// shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
+{
+    const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    return ((uint64_t)hi << 32) | lo;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(IDESC), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u); // NaN stays NaN
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+__global__ void __launch_bounds__(128, 1)
+dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const slonn_dense_epilogue E, uint32_t N, uint32_t K)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    const uint32_t m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    // rows this launch must produce (a device-side count when the rows were compacted on the device)
+    const uint32_t m_valid = E.row_count ? min(*E.row_count, E.M) : E.M;
+    if (m0 >= m_valid) return; // uniform for the block: nothing allocated yet
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u; // swizzle atoms need 1024-byte alignment
+    const uint32_t bars = base + RING_BYTES;
+    const uint32_t full0 = bars, empty0 = bars + 8 * STAGES, tmem_full = bars + 16 * STAGES;
+    const uint32_t tmem_slot_addr = bars + 16 * STAGES + 8;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot_addr - smem_u32(smem_raw)));
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        mbar_init(tmem_full, 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) { // one warp allocates the accumulator columns and gives the permit back
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot_addr), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t num_kb = (K + BK - 1) / BK;
+
+    if (warp == 0 && lane == 0) {
+        // ---- TMA producer ----
+        for (uint32_t kb = 0; kb < num_kb; ++kb) {
+            const uint32_t s = kb % STAGES, ph = (kb / STAGES) & 1u;
+            if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
+            mbar_expect_tx(full0 + 8 * s, STAGE_A_BYTES + STAGE_B_BYTES);
+            tma_load_2d(base + s * STAGE_A_BYTES, &map_a, (int32_t)(kb * BK), (int32_t)m0, full0 + 8 * s);
+            tma_load_2d(base + STAGES * STAGE_A_BYTES + s * STAGE_B_BYTES, &map_b, (int32_t)(kb * BK), (int32_t)n0,
+                        full0 + 8 * s);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---- MMA issuer ----
+        bool ok = true;
+        for (uint32_t kb = 0; kb < num_kb && ok; ++kb) {
+            const uint32_t s = kb % STAGES, ph = (kb / STAGES) & 1u;
+            ok = mbar_wait(full0 + 8 * s, ph, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t da = umma_desc(base + s * STAGE_A_BYTES);
+            const uint64_t db = umma_desc(base + STAGES * STAGE_A_BYTES + s * STAGE_B_BYTES);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k) // 32 bytes further along K inside the swizzle atom
+                umma_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), (kb | (uint32_t)k) != 0u);
+            umma_commit(empty0 + 8 * s); // frees the stage once these MMAs have read it
+        }
+        if (ok) umma_commit(tmem_full); // accumulator complete
+    }
+    __syncwarp();
+
+    // ---- epilogue: TMEM lane = row of the tile, TMEM column = column of the tile ----
+    const bool acc_ready = __all_sync(SLONN_FULL_MASK, mbar_wait(tmem_full, 0u, abort_flag)); // warp-uniform
+    tc_fence_after();
+    if (acc_ready) {
+        const uint32_t m = m0 + warp * 32 + lane;
+        const bool row_ok = m < m_valid;
+        uint64_t f32_off = 0;
+        if (row_ok && (E.out_f32 || E.out_ids)) {
+            const uint32_t src = E.row_map ? E.row_map[m] : m;
+            f32_off = E.indptr ? E.indptr[(uint64_t)src * E.ip_mul + E.ip_add] : (uint64_t)src * E.f32_stride;
+        }
+        for (uint32_t c = 0; c < (uint32_t)BN; c += 32) {
+            uint32_t r[32];
+            tmem_load32(tmem_base + ((warp * 32u) << 16) + c, r); // whole warp takes part
+            if (!row_ok) continue;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const uint32_t n = n0 + c + j;
+                if (n < N) {
+                    float v = __uint_as_float(r[j]) + (E.bias ? __ldg(E.bias + n) : 0.0f);
+                    if (E.relu) v = v > 0.0f ? v : 0.0f;
+                    if (E.out_f32) E.out_f32[f32_off + n] = v;
+                    if (E.out_ids) E.out_ids[f32_off + n] = n;
+                    if (E.out_bf16) E.out_bf16[(uint64_t)m * E.ld_bf16 + n] = f32_to_bf16_rne(v);
+                }
+            }
+        }
+    }
+    if (*abort_flag) {
+        // a wait ran out: give copies that may still be in flight time to land before the block leaves
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        if (threadIdx.x == 0 && E.status) slonn_report(E.status, SLONN_ERR_TIMEOUT, blockIdx.y, blockIdx.x);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side ----------------------------------------------------------------
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode()
+{
+    static std::mutex mu;
+    static encode_tiled_fn fn = nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (encode_tiled_fn)p;
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][cols] row-major, tiles of 128 rows x 64 columns, 128-byte swizzle, zero fill outside
+int make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols)
+{
+    encode_tiled_fn enc = get_encode();
+    if (!enc) return SLONN_ERR_CUDA;
+    if (((uintptr_t)ptr & 15u) || ((cols * 2) & 15u)) return SLONN_ERR_ALIGN;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+} // namespace
+
+int slonn_dense_tc_launch(const void *A, const void *W, uint32_t N, uint32_t K, const slonn_dense_epilogue &E,
+                          cudaStream_t st)
+{
+    if (!A || !W || E.M == 0 || N == 0 || K == 0) return SLONN_ERR_ARG;
+    CUtensorMap ma, mb;
+    int rc;
+    if ((rc = make_map(&ma, A, E.M, K))) return rc;
+    if ((rc = make_map(&mb, W, N, K))) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(dense_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
+            return SLONN_ERR_CUDA;
+        attr_set = true;
+    }
+    const dim3 grid((N + BN - 1) / BN, (E.M + BM - 1) / BM);
+    dense_tc_kernel<<<grid, 128, SMEM_BYTES, st>>>(ma, mb, E, N, K);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+extern "C" int slonn_dense_layer(const void *x_bf16, const void *w_bf16, const float *bias, uint32_t M, uint32_t N,
+                                 uint32_t D, uint32_t relu, float *out_f32, void *out_bf16, uint32_t *status,
+                                 void *stream)
+{
+    if (!x_bf16 || !w_bf16 || (!out_f32 && !out_bf16)) return SLONN_ERR_ARG;
+    if (M == 0 || N == 0 || D == 0) return SLONN_ERR_DIM;
+    slonn_dense_epilogue E;
+    memset(&E, 0, sizeof(E));
+    E.M = M; E.bias = bias; E.relu = relu;
+    E.out_f32 = out_f32; E.f32_stride = N;
+    E.out_bf16 = (uint16_t *)out_bf16; E.ld_bf16 = N;
+    E.status = status;
+    if (status && cudaMemsetAsync(status, 0, 4 * sizeof(uint32_t), (cudaStream_t)stream) != cudaSuccess) return SLONN_ERR_CUDA;
+    return slonn_dense_tc_launch(x_bf16, w_bf16, N, D, E, (cudaStream_t)stream);
+}
