@@ -173,6 +173,8 @@ def main():
                     help="budget of every query in basis points; 0 = the workload's mixed per-query budgets (c5)")
     ap.add_argument("--queries", type=int, default=None, help="override the workload's query count")
     ap.add_argument("--n-cal", type=int, default=None)
+    ap.add_argument("--dense-tc", action="store_true",
+                    help="route 100 %% budget queries to the tensor-core dense path (not bit-exact for them)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -227,7 +229,8 @@ def main():
         return replicas.slowest_rank_ms(e0.elapsed_time(e1), dev) / steps
 
     # ---- headline: device-resident inputs ----
-    batch = harness.DeviceBatch(dm, wl.x, wl.budget_bp, max_budget_bp=max_bp, full_outputs=False)
+    flags = sl.FLAG_DENSE_TC if args.dense_tc else 0
+    batch = harness.DeviceBatch(dm, wl.x, wl.budget_bp, max_budget_bp=max_bp, full_outputs=False, flags=flags)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -276,7 +279,7 @@ def main():
     if not args.no_sweep and world == 1:
         for bp in wl.budgets_named:
             bps = np.full(n, bp, np.uint16)
-            b2 = harness.DeviceBatch(dm, wl.x, bps, max_budget_bp=bp, full_outputs=False)
+            b2 = harness.DeviceBatch(dm, wl.x, bps, max_budget_bp=bp, full_outputs=False, flags=flags)
             ms2 = timed(b2, max(3, args.steps // 4), 3)
             st_ms, st_cnt = sl.slonn_run_timed(dm.model, b2.batch, b2.ws, b2.ws_bytes, stream)
             k2, _, _, _, ach2 = stage_roofline(st_ms, st_cnt, bps, 1)
@@ -341,7 +344,8 @@ def main():
                        "queries_per_step_per_gpu": n, "budget_bp": args.budget_bp,
                        "l2": "inputs_larger_than_l2" if (wl.x.nbytes if not wl.first_sparse else 0) > L2_BYTES
                              else "weights_and_inputs_l2_resident",
-                       "table_bytes": dm.table_bytes(), "parallelism": f"replicas x{world}"},
+                       "table_bytes": dm.table_bytes(), "parallelism": f"replicas x{world}",
+                       "full_budget_route": "tensor cores (bf16 activations)" if args.dense_tc else "fixed-order fp32 kernels"},
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": (sum(stage_cnt.values()) // prof_steps + (1 if stage_cnt["plan"] else 0)) * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "budget_sweep": sweep,

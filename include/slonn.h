@@ -165,11 +165,25 @@ typedef struct {
     uint32_t *status;              /* required. [4] words: [0] first error code seen on the   */
                                    /* device (0 = ok, else -SLONN_ERR_*), [1] query index,    */
                                    /* [2] layer index, [3] reserved.  Cleared by slonn_run    */
+    uint32_t flags;                /* HOST value: 0 or SLONN_FLAG_* below                     */
     uint32_t kernel_path;          /* HOST value: SLONN_PATH_AUTO, or force one of the two    */
                                    /* kernel families (results are identical; for testing and */
                                    /* tuning).  _FUSED on a network it cannot take returns    */
                                    /* SLONN_ERR_DIM                                           */
 } slonn_batch;
+
+/*
+ * SLONN_FLAG_DENSE_TC: queries whose budget is 10000 bp compute every node of every layer, i.e.
+ * the plain dense network (Sec. 3.4).  With this flag they are taken out of the per-query
+ * kernels, compacted, and run layer by layer as bf16 matrix products on the tensor cores
+ * (activations rounded to bf16 between layers, fp32 accumulation).  Their active sets are still
+ * "all nodes" and their logits stay within the bf16-weight tolerance (2e-2 of the largest
+ * logit), but nothing about them is bit-compatible with the fixed-order kernels: values differ
+ * in the last bits, and a hash code or an argmax decided by a near-tie can differ.  Other
+ * queries are unaffected.  Honoured when weights are bf16, the first layer is dense, the last
+ * layer has no activator and max_budget_bp is 10000 (or 0); otherwise ignored.
+ */
+#define SLONN_FLAG_DENSE_TC 1u
 
 #define SLONN_PATH_AUTO 0    /* library chooses                                               */
 #define SLONN_PATH_STAGED 1  /* one block per query and stage: any width, any batch size      */
@@ -181,9 +195,10 @@ int slonn_active_capacity(const slonn_model *m, uint32_t n_queries, uint32_t max
                           uint64_t *entries);
 /* logit_stride for this model at max_budget_bp (see slonn_batch.logits). */
 int slonn_logit_stride(const slonn_model *m, uint32_t max_budget_bp, uint32_t *stride);
-/* Bytes of device workspace slonn_run needs (256-byte aligned buffer). */
+/* Bytes of device workspace slonn_run needs (256-byte aligned buffer) for a batch with these
+ * n_queries, max_budget_bp and flags. */
 int slonn_workspace_bytes(const slonn_model *m, uint32_t n_queries, uint32_t max_budget_bp,
-                          uint64_t *bytes);
+                          uint32_t flags, uint64_t *bytes);
 
 /*
  * Runs the batch on `stream`: asynchronous, no allocation, no host
@@ -228,7 +243,7 @@ int slonn_dense_layer(const void *x_bf16, const void *w_bf16, const float *bias,
  * ends).  The call performs no cudaMalloc / cudaFree and uses no allocating
  * library routine.
  *
- *   - The batch must fit: if slonn_workspace_bytes(m, n_queries, max_budget_bp)
+ *   - The batch must fit: if slonn_workspace_bytes(m, n_queries, max_budget_bp, flags)
  *     exceeds SLONN_STATIC_WORKSPACE_BYTES the call returns SLONN_ERR_WORKSPACE
  *     and launches nothing.  Use smaller batches or slonn_run.
  *   - The model's device must be the current device (else SLONN_ERR_ARG).
@@ -260,7 +275,8 @@ int slonn_run_static(const slonn_model *m, const slonn_batch *batch, void *strea
 #define SLONN_STAGE_SPARSE_FIRST 3  /* first layer fed by CSR rows                   */
 #define SLONN_STAGE_ARGMAX 4        /* prediction                                    */
 #define SLONN_STAGE_FUSED 5         /* all of 1, 2, 4 in the one-warp-per-query kernel */
-#define SLONN_N_STAGES 6
+#define SLONN_STAGE_DENSE_TC 6      /* 100 % budget queries on the tensor cores        */
+#define SLONN_N_STAGES 7
 int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *workspace,
                     uint64_t workspace_bytes, void *stream, float *stage_ms,
                     uint32_t *stage_launches);
@@ -274,7 +290,7 @@ int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *worksp
  * h2d_bytes / d2h_bytes (host, nullable) receive the bytes copied each way.
  */
 int slonn_host_workspace_bytes(const slonn_model *m, uint32_t n_queries, uint32_t max_budget_bp,
-                               uint64_t x_nnz, uint64_t *bytes);
+                               uint32_t flags, uint64_t x_nnz, uint64_t *bytes);
 int slonn_run_host(const slonn_model *m, const slonn_batch *host_batch, void *workspace,
                    uint64_t workspace_bytes, void *stream, uint64_t *h2d_bytes,
                    uint64_t *d2h_bytes);

@@ -49,7 +49,7 @@ class _Batch(C.Structure):
                 ("max_budget_bp", C.c_uint32), ("logits", C.c_void_p), ("logit_ids", C.c_void_p),
                 ("pred", C.c_void_p), ("codes", C.c_void_p), ("active_indptr", C.c_void_p),
                 ("active_ids", C.c_void_p), ("active_vals", C.c_void_p), ("status", C.c_void_p),
-                ("kernel_path", C.c_uint32)]
+                ("flags", C.c_uint32), ("kernel_path", C.c_uint32)]
 
 
 _lib = None
@@ -81,7 +81,7 @@ def lib():
         L.slonn_logit_stride.restype = C.c_int
         L.slonn_logit_stride.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
         L.slonn_workspace_bytes.restype = C.c_int
-        L.slonn_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint64)]
+        L.slonn_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint64)]
         L.slonn_run.restype = C.c_int
         L.slonn_run.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p]
         L.slonn_run_static.restype = C.c_int
@@ -93,7 +93,7 @@ def lib():
         L.slonn_run_timed.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p,
                                       C.c_void_p, C.c_void_p]
         L.slonn_host_workspace_bytes.restype = C.c_int
-        L.slonn_host_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64,
+        L.slonn_host_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64,
                                                  C.POINTER(C.c_uint64)]
         L.slonn_run_host.restype = C.c_int
         L.slonn_run_host.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p,
@@ -238,17 +238,18 @@ def slonn_logit_stride(model: Model, max_budget_bp: int = 0) -> int:
     return v.value
 
 
-def slonn_workspace_bytes(model: Model, n_queries: int, max_budget_bp: int = 0) -> int:
+def slonn_workspace_bytes(model: Model, n_queries: int, max_budget_bp: int = 0, flags: int = 0) -> int:
     v = C.c_uint64()
-    rc = lib().slonn_workspace_bytes(model.handle, n_queries, max_budget_bp, C.byref(v))
+    rc = lib().slonn_workspace_bytes(model.handle, n_queries, max_budget_bp, flags, C.byref(v))
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_workspace_bytes")
     return v.value
 
 
-def slonn_host_workspace_bytes(model: Model, n_queries: int, max_budget_bp: int = 0, x_nnz: int = 0) -> int:
+def slonn_host_workspace_bytes(model: Model, n_queries: int, max_budget_bp: int = 0, x_nnz: int = 0,
+                               flags: int = 0) -> int:
     v = C.c_uint64()
-    rc = lib().slonn_host_workspace_bytes(model.handle, n_queries, max_budget_bp, x_nnz, C.byref(v))
+    rc = lib().slonn_host_workspace_bytes(model.handle, n_queries, max_budget_bp, flags, x_nnz, C.byref(v))
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_host_workspace_bytes")
     return v.value
@@ -256,7 +257,7 @@ def slonn_host_workspace_bytes(model: Model, n_queries: int, max_budget_bp: int 
 
 def make_batch(n_queries: int, budget_bp, logits, status, x_dense=None, x_csr=None, max_budget_bp: int = 0,
                logit_ids=None, pred=None, codes=None, active_indptr=None, active_ids=None,
-               active_vals=None, kernel_path: int = 0) -> _Batch:
+               active_vals=None, kernel_path: int = 0, flags: int = 0) -> _Batch:
     """Fills a slonn_batch from tensors/arrays (device for slonn_run, host for slonn_run_host)."""
     b = _Batch()
     b.n_queries = n_queries
@@ -269,6 +270,7 @@ def make_batch(n_queries: int, budget_bp, logits, status, x_dense=None, x_csr=No
     b.active_indptr, b.active_ids, b.active_vals = _ptr(active_indptr), _ptr(active_ids), _ptr(active_vals)
     b.status = _ptr(status)
     b.kernel_path = kernel_path
+    b.flags = flags
     return b
 
 
@@ -301,7 +303,8 @@ def slonn_run_static(model: Model, batch: _Batch, stream=None) -> None:
         raise SlonnError(rc, "slonn_run_static")
 
 
-STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused")
+STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused", "dense_tc")
+FLAG_DENSE_TC = 1
 PATH_AUTO, PATH_STAGED, PATH_FUSED = 0, 1, 2
 
 

@@ -35,6 +35,7 @@ struct slonn_fused_layer {
 struct slonn_fused_params {
     slonn_fused_layer layer[SLONN_MAX_LAYERS];
     uint32_t n_layers, n, n_act, K, L;
+    const uint16_t *skip_bp; // nullable: queries with this budget == 10000 are handled elsewhere
     const float *x;          // [n][D0]
     const uint64_t *indptr;  // [n * n_act + 1]
     uint32_t *out_ids;       // CSR payload, nullable
@@ -193,6 +194,7 @@ __global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, SLONN_FUSED_MIN_BLOCKS
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const uint32_t q = blockIdx.x * SLONN_FUSED_WARPS + warp;
     if (q >= P.n) return;
+    if (P.skip_bp && P.skip_bp[q] == 10000u) return;
     unsigned char *wbase = reinterpret_cast<unsigned char *>(smem4) + (size_t)warp * P.warp_bytes;
     float4 *xbuf4 = reinterpret_cast<float4 *>(wbase);
     float *xbuf = reinterpret_cast<float *>(wbase);

@@ -5,6 +5,7 @@
 #include <cstring>
 #include <mutex>
 
+#include "slonn_dense_tc.cuh"
 #include "slonn_fused_kernel.cuh"
 #include "slonn_run_kernels.cuh"
 
@@ -56,10 +57,25 @@ uint32_t dense_width(const slonn_model *m)
 }
 
 struct ws_layout {
-    uint64_t indptr, plan_sums, ids, vals, dense0, dense1, total;
+    uint64_t indptr, plan_sums, ids, vals, dense0, dense1, tc_list, tc_count, tc_a0, tc_a1, total;
 };
 
-ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp)
+// widest bf16 activation matrix row the tensor-core route needs
+uint32_t tc_width(const slonn_model *m)
+{
+    uint32_t w = 0;
+    for (uint32_t l = 0; l < m->n_layers; ++l) w = std::max(w, m->layer[l].D);
+    return w;
+}
+
+// whether the batch's 100 % budget queries take the tensor-core route
+bool tc_route(const slonn_model *m, uint32_t max_bp, uint32_t flags)
+{
+    return (flags & SLONN_FLAG_DENSE_TC) && max_bp == 10000u && m->dtype == SLONN_BF16 && !m->first_sparse &&
+           !m->layer[m->n_layers - 1].has_act;
+}
+
+ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp, uint32_t flags)
 {
     ws_layout w;
     const uint64_t ent = active_entries(m, n, max_bp);
@@ -72,6 +88,14 @@ ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp)
     const uint64_t db = align_up((uint64_t)n * dense_width(m) * sizeof(float), 256);
     w.dense0 = o; o += db;
     w.dense1 = o; o += db;
+    w.tc_list = w.tc_count = w.tc_a0 = w.tc_a1 = 0;
+    if (tc_route(m, max_bp, flags)) {
+        w.tc_list = o; o = align_up(o + (uint64_t)n * sizeof(uint32_t), 256);
+        w.tc_count = o; o += 256;
+        const uint64_t ab = align_up((uint64_t)n * tc_width(m) * sizeof(uint16_t), 256);
+        w.tc_a0 = o; o += ab;
+        w.tc_a1 = o; o += ab;
+    }
     w.total = std::max<uint64_t>(o, 256);
     return w;
 }
@@ -155,7 +179,8 @@ int launch_fused_t(const slonn_fused_params &P, cudaStream_t st)
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
-int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *indptr, uint32_t stride, cudaStream_t st)
+int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *indptr, uint32_t stride,
+                 const uint16_t *skip_bp, cudaStream_t st)
 {
     slonn_fused_params P;
     memset(&P, 0, sizeof(P));
@@ -176,7 +201,7 @@ int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *ind
         }
     }
     P.n_layers = m->n_layers; P.n = b->n_queries; P.n_act = m->n_act; P.K = m->K; P.L = m->L;
-    P.x = b->x_dense; P.indptr = indptr;
+    P.x = b->x_dense; P.indptr = indptr; P.skip_bp = skip_bp;
     P.out_ids = b->active_ids; P.out_vals = b->active_vals; P.codes = b->codes;
     P.logits = b->logits; P.logit_stride = stride; P.logit_ids = b->logit_ids; P.pred = b->pred;
     P.status = b->status;
@@ -249,10 +274,11 @@ extern "C" int slonn_logit_stride(const slonn_model *m, uint32_t max_bp, uint32_
     return SLONN_OK;
 }
 
-extern "C" int slonn_workspace_bytes(const slonn_model *m, uint32_t n, uint32_t max_bp, uint64_t *bytes)
+extern "C" int slonn_workspace_bytes(const slonn_model *m, uint32_t n, uint32_t max_bp, uint32_t flags,
+                                     uint64_t *bytes)
 {
     if (!model_ok(m) || !bytes) return SLONN_ERR_ARG;
-    *bytes = carve(m, n, eff_max_bp(max_bp)).total;
+    *bytes = carve(m, n, eff_max_bp(max_bp), flags).total;
     return SLONN_OK;
 }
 
@@ -271,7 +297,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     if (last.has_act && !b->logit_ids) return SLONN_ERR_ARG;
     if (b->x_dense && ((uintptr_t)b->x_dense & 15u)) return SLONN_ERR_ALIGN;
 
-    const ws_layout wl = carve(m, n, max_bp);
+    const ws_layout wl = carve(m, n, max_bp, b->flags);
     if (!workspace || ((uintptr_t)workspace & 255u) || ws_bytes < wl.total) return SLONN_ERR_WORKSPACE;
     char *ws = (char *)workspace;
     uint64_t *indptr = b->active_indptr ? b->active_indptr : (uint64_t *)(ws + wl.indptr);
@@ -302,15 +328,66 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
     }
 
+    // queries at a 100 % budget on the tensor cores (on request): they compute every node of every
+    // layer, so they are a dense matrix product over the compacted set of such queries
+    const uint16_t *skip_bp = nullptr;
+    if (b->flags & ~SLONN_FLAG_DENSE_TC) return SLONN_ERR_ARG;
+    if (tc_route(m, max_bp, b->flags)) {
+        uint32_t *tc_list = (uint32_t *)(ws + wl.tc_list), *tc_count = (uint32_t *)(ws + wl.tc_count);
+        uint16_t *A[2] = {(uint16_t *)(ws + wl.tc_a0), (uint16_t *)(ws + wl.tc_a1)};
+        TIC(SLONN_STAGE_DENSE_TC);
+        int rc = SLONN_OK;
+        if (cudaMemsetAsync(tc_count, 0, sizeof(uint32_t), st) != cudaSuccess) rc = SLONN_ERR_CUDA;
+        if (!rc) {
+            dense_compact_kernel<<<(n + 255) / 256, 256, 0, st>>>(b->budget_bp, n, tc_list, tc_count);
+            dense_gather_x_kernel<<<n, 128, 0, st>>>(b->x_dense, m->layer[0].D, tc_list, tc_count, A[0]);
+            if (cudaGetLastError() != cudaSuccess) rc = SLONN_ERR_CUDA;
+        }
+        for (uint32_t l = 0; l < m->n_layers && !rc; ++l) {
+            const slonn_layer &ly = m->layer[l];
+            const bool is_last = (l + 1 == m->n_layers);
+            slonn_dense_epilogue E;
+            memset(&E, 0, sizeof(E));
+            E.M = n; E.row_count = tc_count; E.row_map = tc_list; E.bias = ly.bias; E.relu = is_last ? 0u : 1u;
+            E.status = b->status;
+            if (is_last) {
+                E.out_f32 = b->logits; E.f32_stride = stride;
+            } else {
+                E.out_bf16 = A[(l + 1) & 1]; E.ld_bf16 = ly.N;
+                if (ly.has_act) {
+                    E.out_f32 = vals; E.out_ids = ids; E.indptr = indptr; E.ip_mul = m->n_act; E.ip_add = m->act_index[l];
+                }
+            }
+            rc = slonn_dense_tc_launch(A[l & 1], ly.W, ly.N, ly.D, E, st);
+            if (!rc && ly.has_act && b->codes) {
+                const uint32_t t = n * m->L;
+                dense_codes_kernel<<<(t + 127) / 128, 128, 0, st>>>(tc_list, tc_count, vals, indptr, m->n_act,
+                                                                   m->act_index[l], ly.hash_nodes, m->K, m->L, b->codes);
+                if (cudaGetLastError() != cudaSuccess) rc = SLONN_ERR_CUDA;
+            }
+        }
+        TOC();
+        if (rc) return rc;
+        skip_bp = b->budget_bp;
+    }
+
     // narrow networks with enough queries to fill the GPU: one warp per query, every layer in one launch
     if (b->kernel_path > SLONN_PATH_FUSED) return SLONN_ERR_ARG;
     if (b->kernel_path == SLONN_PATH_FUSED && !fused_eligible(m)) return SLONN_ERR_DIM;
     if (b->kernel_path == SLONN_PATH_FUSED ||
         (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n >= 512)) {
         TIC(SLONN_STAGE_FUSED);
-        const int rc = launch_fused(m, b, indptr, stride, st);
+        const int rc = launch_fused(m, b, indptr, stride, skip_bp, st);
         TOC();
-        return rc;
+        if (rc || !skip_bp || !b->pred) return rc;
+        // predictions of the tensor-core queries (the fused kernel wrote the others; same rule)
+        slonn_argmax_params ap;
+        memset(&ap, 0, sizeof(ap));
+        ap.logits = b->logits; ap.stride = stride; ap.n = n; ap.pred = b->pred; ap.fixed_len = last.N;
+        TIC(SLONN_STAGE_ARGMAX);
+        argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
+        TOC();
+        return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
     }
 
     // input := x
@@ -340,6 +417,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         slonn_gather_params gp;
         memset(&gp, 0, sizeof(gp));
         gp.in = in; gp.W = ly.W; gp.bias = ly.bias; gp.D = ly.D; gp.N = ly.N; gp.nchunks = nchunks;
+        gp.skip_bp = skip_bp;
         gp.n_act = m->n_act; gp.indptr = indptr; gp.ids = ids;
         gp.relu = is_last ? 0u : 1u;
         uint32_t max_rows = ly.N;
@@ -348,6 +426,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             slonn_select_params sp;
             memset(&sp, 0, sizeof(sp));
             sp.in = in; sp.W = ly.W; sp.bias = ly.bias; sp.D = ly.D; sp.N = ly.N; sp.nchunks = nchunks;
+            sp.skip_bp = skip_bp;
             sp.hash_nodes = ly.hash_nodes; sp.tables = ly.tables; sp.cap = ly.cap; sp.K = m->K; sp.L = m->L;
             sp.n_act = m->n_act; sp.a = a; sp.layer = l; sp.indptr = indptr; sp.out_ids = ids;
             sp.codes = b->codes; sp.status = b->status;
@@ -442,7 +521,7 @@ extern "C" int slonn_run_static(const slonn_model *m, const slonn_batch *b, void
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return SLONN_ERR_CUDA;
     if (dev != m->device || dev < 0 || dev >= 64) return SLONN_ERR_ARG; // the model's device must be current
-    const uint64_t need = carve(m, b->n_queries, eff_max_bp(b->max_budget_bp)).total;
+    const uint64_t need = carve(m, b->n_queries, eff_max_bp(b->max_budget_bp), b->flags).total;
     if (need > SLONN_STATIC_WORKSPACE_BYTES) return SLONN_ERR_WORKSPACE;
     void *ws = nullptr;
     {
@@ -464,7 +543,7 @@ struct host_layout {
         inner, total;
 };
 
-host_layout carve_host(const slonn_model *m, uint32_t n, uint32_t max_bp, uint64_t x_nnz)
+host_layout carve_host(const slonn_model *m, uint32_t n, uint32_t max_bp, uint32_t flags, uint64_t x_nnz)
 {
     host_layout h;
     memset(&h, 0, sizeof(h));
@@ -490,16 +569,16 @@ host_layout carve_host(const slonn_model *m, uint32_t n, uint32_t max_bp, uint64
     h.a_vals = take(ent * 4);
     h.status = take(16);
     h.inner = o;
-    h.total = o + carve(m, n, max_bp).total;
+    h.total = o + carve(m, n, max_bp, flags).total;
     return h;
 }
 } // namespace
 
-extern "C" int slonn_host_workspace_bytes(const slonn_model *m, uint32_t n, uint32_t max_bp, uint64_t x_nnz,
-                                          uint64_t *bytes)
+extern "C" int slonn_host_workspace_bytes(const slonn_model *m, uint32_t n, uint32_t max_bp, uint32_t flags,
+                                          uint64_t x_nnz, uint64_t *bytes)
 {
     if (!model_ok(m) || !bytes) return SLONN_ERR_ARG;
-    *bytes = carve_host(m, n, eff_max_bp(max_bp), x_nnz).total;
+    *bytes = carve_host(m, n, eff_max_bp(max_bp), flags, x_nnz).total;
     return SLONN_OK;
 }
 
@@ -515,7 +594,7 @@ extern "C" int slonn_run_host(const slonn_model *m, const slonn_batch *hb, void 
     const uint32_t max_bp = eff_max_bp(hb->max_budget_bp);
     cudaStream_t st = (cudaStream_t)stream;
     const uint64_t x_nnz = m->first_sparse ? hb->x_indptr[n] : 0; // host array: readable here
-    const host_layout hl = carve_host(m, n, max_bp, x_nnz);
+    const host_layout hl = carve_host(m, n, max_bp, hb->flags, x_nnz);
     if (!workspace || ((uintptr_t)workspace & 255u) || ws_bytes < hl.total) return SLONN_ERR_WORKSPACE;
     char *ws = (char *)workspace;
     uint32_t stride = 0;

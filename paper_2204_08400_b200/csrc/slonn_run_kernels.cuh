@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(SLONN_PLAN_THREADS) plan_final_kernel(slonn_pl
 // hash + select: one block per query
 // ---------------------------------------------------------------------------
 struct slonn_select_params {
+    const uint16_t *skip_bp;    // nullable: queries with this budget == 10000 are handled elsewhere
     slonn_input in;
     const void *W;
     const float *bias;
@@ -154,6 +155,7 @@ __global__ void __launch_bounds__(SLONN_THREADS) hash_select_kernel(slonn_select
     __shared__ uint32_t s_total;
 
     const uint32_t q = blockIdx.x;
+    if (P.skip_bp && P.skip_bp[q] == 10000u) return;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t H = P.K * P.L;
     const uint64_t off = P.indptr[(uint64_t)q * P.n_act + P.a];
@@ -281,6 +283,7 @@ __global__ void __launch_bounds__(SLONN_THREADS) hash_select_kernel(slonn_select
 // gather-dot: the selected rows of one layer
 // ---------------------------------------------------------------------------
 struct slonn_gather_params {
+    const uint16_t *skip_bp;  // nullable: queries with this budget == 10000 are handled elsewhere
     slonn_input in;
     const void *W;
     const float *bias;
@@ -303,6 +306,7 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_
     extern __shared__ float4 smem4[];
     const uint32_t q = blockIdx.x / P.ctas_per_query;
     const uint32_t chunk = blockIdx.x - q * P.ctas_per_query;
+    if (P.skip_bp && P.skip_bp[q] == 10000u) return;
     uint64_t off = 0;
     uint32_t B = P.N;
     if (P.use_list) {
@@ -453,4 +457,60 @@ __global__ void __launch_bounds__(256) argmax_kernel(slonn_argmax_params P)
     }
     if (lane == 0 && bi != 0xffffffffu)
         P.pred[q] = P.logit_ids ? P.logit_ids[(uint64_t)q * P.stride + bi] : bi;
+}
+
+
+// ---------------------------------------------------------------------------
+// tensor-core route for 100 % budgets: which queries, their inputs as bf16 rows, their codes
+// ---------------------------------------------------------------------------
+__global__ void dense_compact_kernel(const uint16_t *bp, uint32_t n, uint32_t *list, uint32_t *count)
+{
+    const uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t lane = threadIdx.x & 31u;
+    const bool full = q < n && bp[q] == 10000u;
+    const uint32_t mask = __ballot_sync(SLONN_FULL_MASK, full);
+    if (mask == 0u) return;
+    uint32_t base = 0;
+    if (lane == (uint32_t)(__ffs(mask) - 1)) base = atomicAdd(count, (uint32_t)__popc(mask));
+    base = __shfl_sync(SLONN_FULL_MASK, base, __ffs(mask) - 1);
+    if (full) list[base + __popc(mask & ((1u << lane) - 1u))] = q;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2_rne(float a, float b)
+{
+    uint32_t ua = __float_as_uint(a), ub = __float_as_uint(b);
+    ua = (ua & 0x7fffffffu) > 0x7f800000u ? (ua >> 16) | 0x40u : (ua + 0x7fffu + ((ua >> 16) & 1u)) >> 16;
+    ub = (ub & 0x7fffffffu) > 0x7f800000u ? (ub >> 16) | 0x40u : (ub + 0x7fffu + ((ub >> 16) & 1u)) >> 16;
+    return (ua & 0xffffu) | (ub << 16);
+}
+
+// A[m][:] = bf16(x[list[m]][:]) for m < *count; D a multiple of 4
+__global__ void dense_gather_x_kernel(const float *x, uint32_t D, const uint32_t *list, const uint32_t *count,
+                                      uint16_t *A)
+{
+    const uint32_t m = blockIdx.x;
+    if (m >= *count) return;
+    const float4 *src = reinterpret_cast<const float4 *>(x + (uint64_t)list[m] * D);
+    uint2 *dst = reinterpret_cast<uint2 *>(A + (uint64_t)m * D);
+    for (uint32_t i = threadIdx.x; i < (D >> 2); i += blockDim.x) {
+        const float4 v = __ldg(src + i);
+        dst[i] = make_uint2(pack_bf16x2_rne(v.x, v.y), pack_bf16x2_rne(v.z, v.w));
+    }
+}
+
+// codes of the tensor-core queries: bit j of key_b = [activation of hash node (b, j) > 0]
+// (hidden layers are ReLU, so the activation is positive exactly when the pre-activation is)
+__global__ void dense_codes_kernel(const uint32_t *list, const uint32_t *count, const float *vals,
+                                   const uint64_t *indptr, uint32_t n_act, uint32_t a, const uint32_t *hash_nodes,
+                                   uint32_t K, uint32_t L, uint16_t *codes)
+{
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t m = t / L, b = t - m * L;
+    if (m >= *count) return;
+    const uint32_t q = list[m];
+    const float *v = vals + indptr[(uint64_t)q * n_act + a]; // all nodes are active: position = node id
+    uint32_t key = 0;
+    for (uint32_t j = 0; j < K; ++j)
+        if (v[hash_nodes[b * K + j]] > 0.0f) key |= (1u << j);
+    codes[((uint64_t)q * n_act + a) * L + b] = (uint16_t)key;
 }

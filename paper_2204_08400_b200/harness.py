@@ -63,7 +63,7 @@ class DeviceBatch:
     """Device buffers of one batch: inputs uploaded once, outputs preallocated."""
 
     def __init__(self, dm: DeviceModel, x, budget_bp: np.ndarray, max_budget_bp: int = 0, full_outputs=True,
-                 kernel_path: int = 0):
+                 kernel_path: int = 0, flags: int = 0):
         dev = dm.device
         self.dm = dm
         m = dm.model
@@ -89,12 +89,12 @@ class DeviceBatch:
             self.indptr = torch.zeros(n * m.n_act + 1, dtype=torch.int64, device=dev)
             self.ids = torch.zeros(max(self.cap, 1), dtype=torch.int32, device=dev)
             self.vals = torch.zeros(max(self.cap, 1), dtype=torch.float32, device=dev)
-        self.ws_bytes = sl.slonn_workspace_bytes(m, self.n, self.max_bp)
+        self.ws_bytes = sl.slonn_workspace_bytes(m, self.n, self.max_bp, flags)
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
         self.batch = sl.make_batch(self.n, self.bp, self.logits, self.status, x_dense=self.x_dense,
                                    x_csr=self.x_csr, max_budget_bp=self.max_bp, logit_ids=self.logit_ids,
                                    pred=self.pred, codes=self.codes, active_indptr=self.indptr,
-                                   active_ids=self.ids, active_vals=self.vals, kernel_path=kernel_path)
+                                   active_ids=self.ids, active_vals=self.vals, kernel_path=kernel_path, flags=flags)
 
     def run(self, stream=None):
         sl.slonn_run(self.dm.model, self.batch, self.ws, self.ws_bytes, stream)
@@ -119,7 +119,8 @@ class DeviceBatch:
         return out
 
 
-def run_once(dm: DeviceModel, x, budget_bp: np.ndarray, max_budget_bp: int = 0, kernel_path: int = 0) -> dict:
-    b = DeviceBatch(dm, x, budget_bp, max_budget_bp, kernel_path=kernel_path)
+def run_once(dm: DeviceModel, x, budget_bp: np.ndarray, max_budget_bp: int = 0, kernel_path: int = 0,
+             flags: int = 0) -> dict:
+    b = DeviceBatch(dm, x, budget_bp, max_budget_bp, kernel_path=kernel_path, flags=flags)
     b.run()
     return b.results()

@@ -44,3 +44,60 @@ def run_dense(M, N, D, relu, seed):
 ])
 def test_dense_layer_matches_float64_matmul(M, N, D, relu):
     run_dense(M, N, D, relu, seed=M + N + D)
+
+
+# ---- 100 % budget queries routed to the tensor cores inside slonn_run --------------------------
+
+def check_tc_route(wl, kernel_path):
+    import sys, os
+    sys.path.insert(0, os.path.dirname(__file__))
+    from oracle import oracle as orc
+    from paper_2204_08400_b200 import binding as sl, harness
+    from parity_util import oracle_model, oracle_run
+    dm = harness.DeviceModel(wl)
+    om = oracle_model(wl)
+    g = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=kernel_path, flags=sl.FLAG_DENSE_TC)
+    ref = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=kernel_path)          # canonical kernels only
+    o64 = oracle_run(om, wl, wl.x, wl.budget_bp, orc.REF64)
+    assert g["status"][0] == 0
+    full = wl.budget_bp == 10000
+    assert 0 < full.sum() < full.size
+    n_act = sum(wl.has_act)
+    ip = g["active_indptr"].astype(np.int64)
+    assert np.array_equal(g["active_indptr"], ref["active_indptr"])
+    # queries below 100 %: untouched by the flag, bit for bit
+    for q in np.nonzero(~full)[0]:
+        s, e = ip[q * n_act], ip[q * n_act + n_act]
+        assert np.array_equal(g["active_ids"][s:e], ref["active_ids"][s:e])
+        assert np.array_equal(g["active_vals"][s:e], ref["active_vals"][s:e])
+        assert np.array_equal(g["logits"][q], ref["logits"][q]) and g["pred"][q] == ref["pred"][q]
+        assert np.array_equal(g["codes"][q], ref["codes"][q])
+    # queries at 100 %: every node active, values and logits within the bf16 tolerance of the fp64 oracle
+    worst = 0.0
+    code_same = 0
+    for q in np.nonzero(full)[0]:
+        s, e = ip[q * n_act], ip[q * n_act + n_act]
+        assert np.array_equal(g["active_ids"][s:e], ref["active_ids"][s:e])            # all nodes, ascending
+        want = o64["logits"][q]
+        err = np.max(np.abs(g["logits"][q].astype(np.float64) - want)) / np.max(np.abs(want))
+        worst = max(worst, float(err))
+        margin = np.sort(want)[-1] - np.sort(want)[-2]
+        if margin > 0.05 * np.max(np.abs(want)):
+            assert g["pred"][q] == o64["pred"][q]
+        v64 = o64["active_vals"][s:e]
+        assert np.max(np.abs(g["active_vals"][s:e] - v64)) <= 2e-2 * max(np.max(np.abs(v64)), 1e-30)
+        code_same += int(np.array_equal(g["codes"][q], o64["codes"][q]))
+    assert worst <= 2e-2, worst
+    assert code_same >= 0.9 * full.sum()     # a code bit decided by a near-zero sum may differ
+    dm.free()
+
+
+@pytest.mark.parametrize("kernel_path", [1, 2])
+def test_full_budget_queries_on_tensor_cores_narrow(kernel_path):
+    wl = wl_mod.load("c5", n_queries=700, n_cal=512, dims=[512, 1024, 1024, 200])
+    check_tc_route(wl, kernel_path)
+
+
+def test_full_budget_queries_on_tensor_cores_wide():
+    wl = wl_mod.load("c5", n_queries=300, n_cal=256, dims=[2048, 4096, 4096, 1000])
+    check_tc_route(wl, 0)
