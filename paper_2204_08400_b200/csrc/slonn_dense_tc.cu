@@ -28,7 +28,8 @@ constexpr int BM = 128, BN = 128, BK = 64, STAGES = 4, UMMA_K = 16;
 constexpr uint32_t TMEM_COLS = 128;
 constexpr uint32_t STAGE_A_BYTES = BM * BK * 2, STAGE_B_BYTES = BN * BK * 2;
 constexpr uint32_t RING_BYTES = STAGES * (STAGE_A_BYTES + STAGE_B_BYTES);
-constexpr uint32_t SMEM_BYTES = RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr uint32_t EPI_BYTES = 4 * (32 * 33) * 4 + 4 * 32 * 8; // per-warp 32x33 fp32 tile + 32 row offsets
+constexpr uint32_t SMEM_BYTES = RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ + EPI_BYTES;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 // instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = 128
@@ -137,6 +138,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const uint32_t bars = base + RING_BYTES;
     const uint32_t full0 = bars, empty0 = bars + 8 * STAGES, tmem_full = bars + 16 * STAGES;
     const uint32_t tmem_slot_addr = bars + 16 * STAGES + 8;
+    const uint32_t epi_addr = bars + 256;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot_addr - smem_u32(smem_raw)));
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -189,28 +191,39 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const bool acc_ready = __all_sync(SLONN_FULL_MASK, mbar_wait(tmem_full, 0u, abort_flag)); // warp-uniform
     tc_fence_after();
     if (acc_ready) {
+        // Each lane reads one accumulator row (32 columns at a time); the warp then turns the 32x32
+        // block around in shared memory so that a store instruction covers 32 consecutive columns
+        // of one output row.
+        float *tile = reinterpret_cast<float *>(smem_raw + (epi_addr - smem_u32(smem_raw))) + warp * (32 * 33);
+        unsigned long long *row_off = reinterpret_cast<unsigned long long *>(
+            smem_raw + (epi_addr - smem_u32(smem_raw)) + 4 * (32 * 33) * sizeof(float)) + warp * 32;
         const uint32_t m = m0 + warp * 32 + lane;
-        const bool row_ok = m < m_valid;
-        uint64_t f32_off = 0;
-        if (row_ok && (E.out_f32 || E.out_ids)) {
+        unsigned long long off = ~0ull; // ~0: row not present
+        if (m < m_valid) {
             const uint32_t src = E.row_map ? E.row_map[m] : m;
-            f32_off = E.indptr ? E.indptr[(uint64_t)src * E.ip_mul + E.ip_add] : (uint64_t)src * E.f32_stride;
+            off = E.indptr ? E.indptr[(uint64_t)src * E.ip_mul + E.ip_add] : (uint64_t)src * E.f32_stride;
         }
+        row_off[lane] = off;
+        __syncwarp();
         for (uint32_t c = 0; c < (uint32_t)BN; c += 32) {
             uint32_t r[32];
             tmem_load32(tmem_base + ((warp * 32u) << 16) + c, r); // whole warp takes part
-            if (!row_ok) continue;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const uint32_t n = n0 + c + j;
-                if (n < N) {
-                    float v = __uint_as_float(r[j]) + (E.bias ? __ldg(E.bias + n) : 0.0f);
-                    if (E.relu) v = v > 0.0f ? v : 0.0f;
-                    if (E.out_f32) E.out_f32[f32_off + n] = v;
-                    if (E.out_ids) E.out_ids[f32_off + n] = n;
-                    if (E.out_bf16) E.out_bf16[(uint64_t)m * E.ld_bf16 + n] = f32_to_bf16_rne(v);
-                }
+            for (int j = 0; j < 32; ++j) tile[lane * 33 + j] = __uint_as_float(r[j]);
+            __syncwarp();
+            const uint32_t n = n0 + c + lane;
+            const float bias = (E.bias && n < N) ? __ldg(E.bias + n) : 0.0f;
+#pragma unroll 4
+            for (int rr = 0; rr < 32; ++rr) {
+                const unsigned long long ro = row_off[rr];
+                if (ro == ~0ull || n >= N) continue;
+                float v = tile[rr * 33 + lane] + bias;
+                if (E.relu) v = v > 0.0f ? v : 0.0f;
+                if (E.out_f32) E.out_f32[ro + n] = v;
+                if (E.out_ids) E.out_ids[ro + n] = n;
+                if (E.out_bf16) E.out_bf16[(uint64_t)(m0 + warp * 32 + rr) * E.ld_bf16 + n] = f32_to_bf16_rne(v);
             }
+            __syncwarp();
         }
     }
     if (*abort_flag) {

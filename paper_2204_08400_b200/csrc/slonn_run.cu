@@ -354,8 +354,10 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
                 E.out_f32 = b->logits; E.f32_stride = stride;
             } else {
                 E.out_bf16 = A[(l + 1) & 1]; E.ld_bf16 = ly.N;
-                if (ly.has_act) {
-                    E.out_f32 = vals; E.out_ids = ids; E.indptr = indptr; E.ip_mul = m->n_act; E.ip_add = m->act_index[l];
+                if (ly.has_act) { // the lists are written only for a caller that reads them (or their codes)
+                    E.out_f32 = (b->active_vals || b->codes) ? vals : nullptr;
+                    E.out_ids = b->active_ids ? ids : nullptr;
+                    E.indptr = indptr; E.ip_mul = m->n_act; E.ip_add = m->act_index[l];
                 }
             }
             rc = slonn_dense_tc_launch(A[l & 1], ly.W, ly.N, ly.D, E, st);
