@@ -571,7 +571,7 @@ host_layout carve_host(const slonn_model *m, uint32_t n, uint32_t max_bp, uint32
     h.a_vals = take(ent * 4);
     h.status = take(16);
     h.inner = o;
-    h.total = o + carve(m, n, max_bp, flags).total;
+    h.total = o + carve(m, n, max_bp, flags).total + 512; // + status words of a batch run in pieces
     return h;
 }
 } // namespace
@@ -581,6 +581,81 @@ extern "C" int slonn_host_workspace_bytes(const slonn_model *m, uint32_t n, uint
 {
     if (!model_ok(m) || !bytes) return SLONN_ERR_ARG;
     *bytes = carve_host(m, n, eff_max_bp(max_bp), flags, x_nnz).total;
+    return SLONN_OK;
+}
+
+// Copies in, runs and copies out the queries [q0, q0 + cnt) of a host batch on one stream, using
+// `ws` (device) for staging and workspace.  The status words go to status_host (copied back) or,
+// when status_dev is given, stay on the device there.
+static int run_host_range(const slonn_model *m, const slonn_batch *hb, uint32_t q0, uint32_t cnt, char *ws,
+                          uint64_t ws_bytes, cudaStream_t st, uint32_t *status_host, uint32_t *status_dev,
+                          uint64_t *up_out, uint64_t *down_out)
+{
+    const slonn_layer &last = m->layer[m->n_layers - 1];
+    const uint32_t max_bp = eff_max_bp(hb->max_budget_bp);
+    const uint64_t nnz0 = m->first_sparse ? hb->x_indptr[q0] : 0;
+    const uint64_t x_nnz = m->first_sparse ? hb->x_indptr[q0 + cnt] - nnz0 : 0;
+    if (m->first_sparse && q0 != 0) return SLONN_ERR_ARG; // CSR rows are only run in one piece
+    const host_layout hl = carve_host(m, cnt, max_bp, hb->flags, x_nnz);
+    if (ws_bytes < hl.total) return SLONN_ERR_WORKSPACE;
+    uint32_t stride = 0;
+    slonn_logit_stride(m, max_bp, &stride);
+    const uint64_t ent = active_entries(m, cnt, max_bp);
+    uint64_t up = 0, down = 0;
+#define H2D(dst, src, bytes)                                                                      \
+    do {                                                                                          \
+        if ((bytes) && cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyHostToDevice, st) != cudaSuccess) \
+            return SLONN_ERR_CUDA;                                                                \
+        up += (bytes);                                                                            \
+    } while (0)
+#define D2H(dst, src, bytes)                                                                      \
+    do {                                                                                          \
+        if ((bytes) && cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToHost, st) != cudaSuccess) \
+            return SLONN_ERR_CUDA;                                                                \
+        down += (bytes);                                                                          \
+    } while (0)
+
+    slonn_batch db = *hb;
+    db.n_queries = cnt;
+    if (m->first_sparse) {
+        H2D(ws + hl.indptr_in, hb->x_indptr, ((uint64_t)cnt + 1) * 8);
+        H2D(ws + hl.ids_in, hb->x_ids, x_nnz * 4);
+        H2D(ws + hl.vals_in, hb->x_vals, x_nnz * 4);
+        db.x_dense = nullptr;
+        db.x_indptr = (const uint64_t *)(ws + hl.indptr_in);
+        db.x_ids = (const uint32_t *)(ws + hl.ids_in);
+        db.x_vals = (const float *)(ws + hl.vals_in);
+    } else {
+        const uint64_t D0 = m->dims[0];
+        H2D(ws + hl.x, hb->x_dense + (uint64_t)q0 * D0, (uint64_t)cnt * D0 * 4);
+        db.x_dense = (const float *)(ws + hl.x);
+    }
+    H2D(ws + hl.bp, hb->budget_bp + q0, (uint64_t)cnt * 2);
+    db.budget_bp = (const uint16_t *)(ws + hl.bp);
+    db.logits = (float *)(ws + hl.logits);
+    db.logit_ids = last.has_act ? (uint32_t *)(ws + hl.logit_ids) : nullptr;
+    db.pred = hb->pred ? (uint32_t *)(ws + hl.pred) : nullptr;
+    db.codes = hb->codes ? (uint16_t *)(ws + hl.codes) : nullptr;
+    db.active_indptr = (uint64_t *)(ws + hl.a_indptr);
+    db.active_ids = (uint32_t *)(ws + hl.a_ids);
+    db.active_vals = (float *)(ws + hl.a_vals);
+    db.status = status_dev ? status_dev : (uint32_t *)(ws + hl.status);
+
+    const int rc = slonn_run(m, &db, ws + hl.inner, ws_bytes - hl.inner, st);
+    if (rc) return rc;
+
+    D2H(hb->logits + (uint64_t)q0 * stride, db.logits, (uint64_t)cnt * stride * 4);
+    if (last.has_act) D2H(hb->logit_ids + (uint64_t)q0 * stride, db.logit_ids, (uint64_t)cnt * stride * 4);
+    if (hb->pred) D2H(hb->pred + q0, db.pred, (uint64_t)cnt * 4);
+    if (hb->codes) D2H(hb->codes + (uint64_t)q0 * m->n_act * m->L, db.codes, (uint64_t)cnt * m->n_act * m->L * 2);
+    if (hb->active_indptr) D2H(hb->active_indptr, db.active_indptr, ((uint64_t)cnt * m->n_act + 1) * 8);
+    if (hb->active_ids) D2H(hb->active_ids, db.active_ids, ent * 4);
+    if (hb->active_vals) D2H(hb->active_vals, db.active_vals, ent * 4);
+    if (!status_dev) D2H(status_host, db.status, 16);
+#undef H2D
+#undef D2H
+    *up_out += up;
+    *down_out += down;
     return SLONN_OK;
 }
 
@@ -599,61 +674,69 @@ extern "C" int slonn_run_host(const slonn_model *m, const slonn_batch *hb, void 
     const host_layout hl = carve_host(m, n, max_bp, hb->flags, x_nnz);
     if (!workspace || ((uintptr_t)workspace & 255u) || ws_bytes < hl.total) return SLONN_ERR_WORKSPACE;
     char *ws = (char *)workspace;
-    uint32_t stride = 0;
-    slonn_logit_stride(m, max_bp, &stride);
-    const uint64_t ent = active_entries(m, n, max_bp);
     uint64_t up = 0, down = 0;
-#define H2D(dst, src, bytes)                                                                      \
-    do {                                                                                          \
-        if ((bytes) && cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyHostToDevice, st) != cudaSuccess) \
-            return SLONN_ERR_CUDA;                                                                \
-        up += (bytes);                                                                            \
-    } while (0)
-#define D2H(dst, src, bytes)                                                                      \
-    do {                                                                                          \
-        if ((bytes) && cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToHost, st) != cudaSuccess) \
-            return SLONN_ERR_CUDA;                                                                \
-        down += (bytes);                                                                          \
-    } while (0)
 
-    slonn_batch db = *hb;
-    if (m->first_sparse) {
-        H2D(ws + hl.indptr_in, hb->x_indptr, ((uint64_t)n + 1) * 8);
-        H2D(ws + hl.ids_in, hb->x_ids, x_nnz * 4);
-        H2D(ws + hl.vals_in, hb->x_vals, x_nnz * 4);
-        db.x_dense = nullptr;
-        db.x_indptr = (const uint64_t *)(ws + hl.indptr_in);
-        db.x_ids = (const uint32_t *)(ws + hl.ids_in);
-        db.x_vals = (const float *)(ws + hl.vals_in);
+    // Large dense batches go through in pieces on two internal streams, so that the copy of one
+    // piece overlaps the kernels of the other.  The per-(query, layer) lists are indexed from the
+    // start of the batch, so a caller that wants them back gets the batch in one piece.
+    const uint32_t pieces = 8;
+    const bool wants_lists = hb->active_indptr || hb->active_ids || hb->active_vals;
+    uint32_t piece = (n + pieces - 1) / pieces;
+    piece = (piece + 255u) / 256u * 256u;
+    const uint64_t half = ((ws_bytes - 256) / 2) & ~(uint64_t)255; // two piece areas, then the pieces' status words
+    bool piecewise = !m->first_sparse && !wants_lists && n >= 8192 && !(hb->flags & SLONN_FLAG_DENSE_TC);
+    if (piecewise && carve_host(m, piece, max_bp, hb->flags, 0).total > half) piecewise = false;
+
+    if (!piecewise) {
+        const int rc = run_host_range(m, hb, 0, n, ws, ws_bytes, st, hb->status, nullptr, &up, &down);
+        if (rc) return rc;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return SLONN_ERR_CUDA;
     } else {
-        H2D(ws + hl.x, hb->x_dense, (uint64_t)n * m->dims[0] * 4);
-        db.x_dense = (const float *)(ws + hl.x);
+        cudaStream_t s2[2] = {nullptr, nullptr};
+        cudaEvent_t ev_start = nullptr, ev_done[2] = {nullptr, nullptr};
+        uint32_t status[pieces + 1][4];
+        memset(status, 0, sizeof(status));
+        int rc = SLONN_OK;
+        bool ok = cudaStreamCreateWithFlags(&s2[0], cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&s2[1], cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&ev_done[0], cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&ev_done[1], cudaEventDisableTiming) == cudaSuccess;
+        if (ok) { // the internal streams start after whatever the caller queued on `stream`
+            ok = cudaEventRecord(ev_start, st) == cudaSuccess && cudaStreamWaitEvent(s2[0], ev_start, 0) == cudaSuccess &&
+                 cudaStreamWaitEvent(s2[1], ev_start, 0) == cudaSuccess;
+        }
+        uint32_t k = 0;
+        for (uint32_t q0 = 0; ok && rc == SLONN_OK && q0 < n; q0 += piece, ++k) {
+            const uint32_t cnt = std::min(piece, n - q0);
+            rc = run_host_range(m, hb, q0, cnt, ws + (k & 1u) * half, half, s2[k & 1u], nullptr,
+                                (uint32_t *)(ws + 2 * half) + 4 * k, &up, &down);
+        }
+        if (ok && rc == SLONN_OK) {
+            ok = cudaEventRecord(ev_done[0], s2[0]) == cudaSuccess && cudaEventRecord(ev_done[1], s2[1]) == cudaSuccess &&
+                 cudaStreamWaitEvent(st, ev_done[0], 0) == cudaSuccess && cudaStreamWaitEvent(st, ev_done[1], 0) == cudaSuccess &&
+                 cudaMemcpyAsync(status, ws + 2 * half, (size_t)k * 16, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+            down += (uint64_t)k * 16;
+        }
+        // nothing below may return before the internal streams are idle and destroyed
+        const bool synced = cudaStreamSynchronize(s2[0]) == cudaSuccess && cudaStreamSynchronize(s2[1]) == cudaSuccess &&
+                            cudaStreamSynchronize(st) == cudaSuccess;
+        if (s2[0]) cudaStreamDestroy(s2[0]);
+        if (s2[1]) cudaStreamDestroy(s2[1]);
+        if (ev_start) cudaEventDestroy(ev_start);
+        if (ev_done[0]) cudaEventDestroy(ev_done[0]);
+        if (ev_done[1]) cudaEventDestroy(ev_done[1]);
+        if (rc) return rc;
+        if (!ok || !synced) return SLONN_ERR_CUDA;
+        // first error of any piece, query index made batch-relative
+        memset(hb->status, 0, 16);
+        for (uint32_t i = 0; i < k; ++i)
+            if (status[i][0]) {
+                hb->status[0] = status[i][0]; hb->status[1] = status[i][1] + i * piece;
+                hb->status[2] = status[i][2]; hb->status[3] = status[i][3];
+                break;
+            }
     }
-    H2D(ws + hl.bp, hb->budget_bp, (uint64_t)n * 2);
-    db.budget_bp = (const uint16_t *)(ws + hl.bp);
-    db.logits = (float *)(ws + hl.logits);
-    db.logit_ids = last.has_act ? (uint32_t *)(ws + hl.logit_ids) : nullptr;
-    db.pred = hb->pred ? (uint32_t *)(ws + hl.pred) : nullptr;
-    db.codes = hb->codes ? (uint16_t *)(ws + hl.codes) : nullptr;
-    db.active_indptr = (uint64_t *)(ws + hl.a_indptr);
-    db.active_ids = (uint32_t *)(ws + hl.a_ids);
-    db.active_vals = (float *)(ws + hl.a_vals);
-    db.status = (uint32_t *)(ws + hl.status);
-
-    const int rc = slonn_run(m, &db, ws + hl.inner, ws_bytes - hl.inner, st);
-    if (rc) return rc;
-
-    D2H(hb->logits, db.logits, (uint64_t)n * stride * 4);
-    if (last.has_act) D2H(hb->logit_ids, db.logit_ids, (uint64_t)n * stride * 4);
-    if (hb->pred) D2H(hb->pred, db.pred, (uint64_t)n * 4);
-    if (hb->codes) D2H(hb->codes, db.codes, (uint64_t)n * m->n_act * m->L * 2);
-    if (hb->active_indptr) D2H(hb->active_indptr, db.active_indptr, ((uint64_t)n * m->n_act + 1) * 8);
-    if (hb->active_ids) D2H(hb->active_ids, db.active_ids, ent * 4);
-    if (hb->active_vals) D2H(hb->active_vals, db.active_vals, ent * 4);
-    D2H(hb->status, db.status, 16);
-#undef H2D
-#undef D2H
-    if (cudaStreamSynchronize(st) != cudaSuccess) return SLONN_ERR_CUDA;
     if (h2d_bytes) *h2d_bytes = up;
     if (d2h_bytes) *d2h_bytes = down;
     return SLONN_OK;

@@ -251,3 +251,36 @@ def test_plan_offsets_span_many_tiles():
     # more (query, layer) entries than one plan tile, mixed budgets: offsets must equal the oracle's
     wl = custom_workload(61, [32, 64, 40, 8], [1, 1, 0], "f32", n=5000, n_cal=100, K=2, L=2)
     check(wl)
+
+
+def test_host_buffer_entry_point_in_pieces_matches_device_entry_point():
+    # 10,000 queries: large enough for the two-stream piecewise route of slonn_run_host
+    import torch
+    from paper_2204_08400_b200 import binding as sl, harness
+    wl = custom_workload(62, [64, 128, 24], [1, 0], "bf16", n=10000, n_cal=200, K=3, L=2)
+    dm = harness.DeviceModel(wl)
+    want = harness.run_once(dm, wl.x, wl.budget_bp)
+    n, max_bp = wl.n_queries, int(wl.budget_bp.max())
+    stride = sl.slonn_logit_stride(dm.model, max_bp)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    logits = torch.zeros((n, stride), dtype=torch.float32).pin_memory()
+    pred = torch.zeros(n, dtype=torch.int32).pin_memory()
+    codes = torch.zeros((n, 1, 2), dtype=torch.int16).pin_memory()
+    status = torch.ones(4, dtype=torch.int32).pin_memory()
+    nb = sl.slonn_host_workspace_bytes(dm.model, n, max_bp)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dm.device)
+    bp = wl.budget_bp.copy()
+    hb = sl.make_batch(n, pin(bp.view(np.int16)), logits, status, x_dense=pin(wl.x), max_budget_bp=max_bp,
+                       pred=pred, codes=codes)
+    up, down = sl.slonn_run_host(dm.model, hb, ws, nb)
+    assert int(status[0]) == 0
+    assert up == wl.x.nbytes + bp.nbytes
+    assert np.array_equal(logits.numpy(), want["logits"])
+    assert np.array_equal(pred.numpy().view(np.uint32), want["pred"])
+    assert np.array_equal(codes.numpy().view(np.uint16), want["codes"])
+    # an invalid budget in a later piece is reported with its batch-relative query index
+    bp[7777] = 0
+    hb = sl.make_batch(n, pin(bp.view(np.int16)), logits, status, x_dense=pin(wl.x), max_budget_bp=max_bp, pred=pred)
+    sl.slonn_run_host(dm.model, hb, ws, nb)
+    assert int(status[0]) == 5 and int(status[1]) == 7777
+    dm.free()
