@@ -28,6 +28,13 @@ from paper_2204_08400_b200 import workloads  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu captures
+# summarised under profiles/ (same workload, same launch shape).  Keyed by (kernel, workload, queries, budget);
+# anything else reports null.  Set an entry to None when its kernel changes until the capture is redone.
+NCU_TRAFFIC = {
+    ("fused_network_kernel", "c2", 65536, 1000): 216.8e6,   # profiles/fused_network_c2_65536q_10pct.md
+}
+
 
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -269,7 +276,9 @@ def main():
     peak, peak_kind = measured_peaks()
     kernel, k_ms, k_launches, k_bytes, achieved = stage_roofline(stage_ms, stage_cnt, wl.budget_bp, prof_steps)
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                "frac": achieved / peak, "peak_kind": peak_kind,
+                "traffic": NCU_TRAFFIC.get((kernel, args.workload, n, args.budget_bp)) if not args.dense_tc else None,
+                "frac_of_nominal_8TBps": achieved / 8000.0,
                 "bytes_per_step": int(k_bytes), "launches_per_step": k_launches,
                 "avg_launch_ms": k_ms / max(k_launches, 1),
                 "stage_ms_per_step": {s: stage_ms[s] / prof_steps for s in sl.STAGES}}
