@@ -166,7 +166,7 @@ typedef struct {
                                    /* device (0 = ok, else -SLONN_ERR_*), [1] query index,    */
                                    /* [2] layer index, [3] reserved.  Cleared by slonn_run    */
     uint32_t flags;                /* HOST value: 0 or SLONN_FLAG_* below                     */
-    uint32_t kernel_path;          /* HOST value: SLONN_PATH_AUTO, or force one of the two    */
+    uint32_t kernel_path;          /* HOST value: SLONN_PATH_AUTO, or force one of the        */
                                    /* kernel families (results are identical; for testing and */
                                    /* tuning).  _FUSED on a network it cannot take returns    */
                                    /* SLONN_ERR_DIM                                           */
@@ -187,6 +187,9 @@ typedef struct {
 
 #define SLONN_PATH_AUTO 0    /* library chooses                                               */
 #define SLONN_PATH_STAGED 1  /* one block per query and stage: any width, any batch size      */
+#define SLONN_PATH_CLUSTER 3 /* one thread-block cluster per query through all layers, for a      */
+                             /* handful of queries (latency): widths and layers <= 8192, dense  */
+                             /* first layer, no SLONN_FLAG_DENSE_TC                             */
 #define SLONN_PATH_FUSED 2   /* one warp per query through all layers: widths <= 1024 inputs, */
                              /* <= 4096 nodes per layer, dense first layer                    */
 
@@ -276,7 +279,8 @@ int slonn_run_static(const slonn_model *m, const slonn_batch *batch, void *strea
 #define SLONN_STAGE_ARGMAX 4        /* prediction                                    */
 #define SLONN_STAGE_FUSED 5         /* all of 1, 2, 4 in the one-warp-per-query kernel */
 #define SLONN_STAGE_DENSE_TC 6      /* 100 % budget queries on the tensor cores        */
-#define SLONN_N_STAGES 7
+#define SLONN_STAGE_CLUSTER 7       /* all of 1, 2, 4 in the one-cluster-per-query kernel */
+#define SLONN_N_STAGES 8
 int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *workspace,
                     uint64_t workspace_bytes, void *stream, float *stage_ms,
                     uint32_t *stage_launches);

@@ -303,9 +303,9 @@ def slonn_run_static(model: Model, batch: _Batch, stream=None) -> None:
         raise SlonnError(rc, "slonn_run_static")
 
 
-STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused", "dense_tc")
+STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused", "dense_tc", "cluster")
 FLAG_DENSE_TC = 1
-PATH_AUTO, PATH_STAGED, PATH_FUSED = 0, 1, 2
+PATH_AUTO, PATH_STAGED, PATH_FUSED, PATH_CLUSTER = 0, 1, 2, 3
 
 
 def slonn_run_timed(model: Model, batch: _Batch, workspace, workspace_bytes: int, stream=None):

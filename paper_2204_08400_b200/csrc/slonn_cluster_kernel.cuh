@@ -1,0 +1,212 @@
+// Latency path for a handful of queries (the paper's setting: batch size 1, Sec. 4): one
+// thread-block CLUSTER carries one query through every layer in a single launch.
+//
+// Each block of the cluster keeps a full copy of the current layer input in its shared memory.
+// Per layer:
+//   1. the K*L hash rows are split over all warps of the cluster; every sum is written to every
+//      block's shared memory (distributed shared memory stores);        cluster barrier
+//   2. every block forms the keys and runs the same first-B-distinct selection redundantly, so
+//      each holds the same ascending id list without a broadcast;
+//   3. the selected rows are split over all warps of the cluster (one row per warp, deep load
+//      prefetch); each activation is scattered into every block's copy of the next layer's
+//      input;                                                           cluster barrier
+// Two hardware cluster barriers per layer replace two kernel launches per layer.  Every block
+// executes the same number of barriers whatever the data (no early exit).  Arithmetic is the
+// library's fixed-order dot product (warp_dot_row1), so results are identical to the other paths.
+#pragma once
+#include <cooperative_groups.h>
+
+#include "slonn_run_kernels.cuh"
+
+#define SLONN_CLUSTER_MAX_D 8192
+#define SLONN_CLUSTER_MAX_N 8192
+#ifndef SLONN_CLUSTER_THREADS
+#define SLONN_CLUSTER_THREADS 512
+#endif
+#ifndef SLONN_CLUSTER_SIZE
+#define SLONN_CLUSTER_SIZE 16 // blocks (SMs) per query; above 8 needs the non-portable cluster size opt-in
+#endif
+
+struct slonn_cluster_layer {
+    const void *W;
+    const float *bias;
+    const uint32_t *hash_nodes;
+    const void *tables;
+    uint32_t D, N, nchunks, cap;
+    uint32_t has_act, a, relu, id_bytes;
+};
+
+struct slonn_cluster_params {
+    slonn_cluster_layer layer[SLONN_MAX_LAYERS];
+    uint32_t n_layers, n, n_act, K, L, cluster;
+    const float *x;          // [n][D0]
+    const uint64_t *indptr;  // [n * n_act + 1]
+    uint32_t *out_ids;       // CSR payload, nullable
+    float *out_vals;         // CSR payload, nullable
+    uint16_t *codes;         // nullable
+    float *logits;
+    uint32_t logit_stride;
+    uint32_t *logit_ids;     // budgeted last layer only
+    uint32_t *pred;          // nullable
+    uint32_t *status;
+    uint32_t xbuf_floats;    // floats per input buffer (two buffers)
+    uint32_t ids_cap;        // entries of the id list
+    uint32_t bitmap_words;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(SLONN_CLUSTER_THREADS, 1)
+cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ float4 smem4[];
+    __shared__ float zh[128];
+    __shared__ uint32_t keys[8];
+    __shared__ uint32_t scan_ws[32];
+    __shared__ uint32_t scan_total;
+    __shared__ uint32_t s_total;
+
+    const uint32_t C = P.cluster;
+    const uint32_t rank = cluster.block_rank();
+    const uint32_t q = blockIdx.x / C;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const uint32_t gwarp = rank * nwarps + warp, gwarps = C * nwarps; // warp index within the cluster
+
+    float *xbuf[2] = {reinterpret_cast<float *>(smem4), reinterpret_cast<float *>(smem4) + P.xbuf_floats};
+    uint32_t *ids_s = reinterpret_cast<uint32_t *>(reinterpret_cast<float *>(smem4) + 2 * P.xbuf_floats);
+    uint32_t *bitmap = ids_s + P.ids_cap;
+
+    // input := x (every block its own copy, in the staging order of layer 0)
+    uint32_t cur = 0;
+    {
+        const slonn_cluster_layer &l0 = P.layer[0];
+        const float4 *src = reinterpret_cast<const float4 *>(P.x + (uint64_t)q * l0.D);
+        float4 *dst = reinterpret_cast<float4 *>(xbuf[0]);
+        for (uint32_t i = threadIdx.x; i < (l0.D >> 2); i += blockDim.x) {
+            const float4 v = __ldg(src + i);
+            if (BF16) dst[(i & 1u) * l0.nchunks + (i >> 1)] = v;
+            else dst[i] = v;
+        }
+    }
+    __syncthreads();
+
+    for (uint32_t l = 0; l < P.n_layers; ++l) {
+        const slonn_cluster_layer &ly = P.layer[l];
+        const bool is_last = (l + 1 == P.n_layers);
+        const uint32_t nxt = cur ^ 1u;
+        const float4 *xs4 = reinterpret_cast<const float4 *>(xbuf[cur]);
+        const uint32_t next_chunks = is_last ? 0u : P.layer[l + 1].nchunks;
+
+        // the buffer the activations of this layer are scattered into starts at zero
+        {
+            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            float4 *dst = reinterpret_cast<float4 *>(xbuf[nxt]);
+            for (uint32_t i = threadIdx.x; i < ((ly.N + 3u) >> 2); i += blockDim.x) dst[i] = z;
+        }
+        uint64_t off = 0;
+        uint32_t B = ly.N;
+        if (ly.has_act) {
+            off = P.indptr[(uint64_t)q * P.n_act + ly.a];
+            B = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + ly.a + 1] - off);
+            // 1. FreeHash rows, spread over the cluster; each sum goes to every block
+            const uint32_t H = P.K * P.L;
+            for (uint32_t h = gwarp; h < H; h += gwarps) {
+                const uint32_t nd = __ldg(ly.hash_nodes + h);
+                const float sum = warp_dot_row1<BF16>(reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)nd * ly.nchunks,
+                                                      xs4, ly.nchunks, lane);
+                const float z = sum + __ldg(ly.bias + nd);
+                if (lane < C) *cluster.map_shared_rank(&zh[h], lane) = z;
+            }
+            for (uint32_t i = threadIdx.x; i < ((ly.N + 31u) >> 5); i += blockDim.x) bitmap[i] = 0u;
+            if (threadIdx.x == 0) s_total = 0;
+        }
+        cluster.sync(); // hash sums delivered, every block's next buffer zeroed
+
+        bool implicit_ids = true;
+        if (ly.has_act) {
+            // 2. keys and selection, redundantly in every block
+            if (threadIdx.x < P.L) {
+                uint32_t key = 0;
+                for (uint32_t j = 0; j < P.K; ++j)
+                    if (zh[threadIdx.x * P.K + j] > 0.0f) key |= (1u << j);
+                keys[threadIdx.x] = key;
+                if (rank == 0 && P.codes) P.codes[((uint64_t)q * P.n_act + ly.a) * P.L + threadIdx.x] = (uint16_t)key;
+            }
+            __syncthreads();
+            bool ok;
+            if (ly.id_bytes == 2)
+                ok = block_select<uint16_t>(ly.tables, ly.cap, P.K, P.L, ly.N, B, keys, bitmap, ids_s, scan_ws,
+                                            &scan_total, &s_total);
+            else
+                ok = block_select<uint32_t>(ly.tables, ly.cap, P.K, P.L, ly.N, B, keys, bitmap, ids_s, scan_ws,
+                                            &scan_total, &s_total);
+            if (!ok && rank == 0 && threadIdx.x == 0) slonn_report(P.status, SLONN_ERR_ARG, q, l);
+            __syncthreads();
+            implicit_ids = false;
+            if (rank == 0 && P.out_ids)
+                for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) P.out_ids[off + i] = ids_s[i];
+        }
+
+        // 3. the selected rows, one per warp, spread over the cluster
+        for (uint32_t r = gwarp; r < B; r += gwarps) {
+            const uint32_t nd = implicit_ids ? r : ids_s[r];
+            const float sum = warp_dot_row1<BF16>(reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)nd * ly.nchunks, xs4,
+                                                  ly.nchunks, lane);
+            float z = sum + __ldg(ly.bias + nd);
+            if (ly.relu) z = z > 0.0f ? z : 0.0f;
+            if (lane == 0) {
+                if (ly.has_act && P.out_vals) P.out_vals[off + r] = z;
+                if (is_last) {
+                    if (ly.has_act) {
+                        P.logits[(uint64_t)q * P.logit_stride + r] = z;
+                        P.logit_ids[(uint64_t)q * P.logit_stride + r] = nd;
+                    } else {
+                        P.logits[(uint64_t)q * P.logit_stride + nd] = z;
+                    }
+                }
+            }
+            // next layer's input (or, after the last layer, the logits by position for the argmax)
+            if (!is_last) {
+                if (lane < C) *cluster.map_shared_rank(&xbuf[nxt][xs_index<BF16>(nd, next_chunks)], lane) = z;
+            } else if (lane == 0) {
+                *cluster.map_shared_rank(&xbuf[nxt][r], 0) = z;
+            }
+        }
+        cluster.sync(); // every activation of this layer delivered
+        cur = nxt;
+
+        if (is_last && rank == 0 && P.pred) {
+            // prediction: lowest node id among the largest computed logits (block 0 holds them by position)
+            const float *lg = xbuf[cur];
+            float best = 0.0f;
+            uint32_t bi = 0xffffffffu;
+            for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) {
+                const float v = lg[i];
+                if (bi == 0xffffffffu || v > best) { best = v; bi = i; }
+            }
+            // positions ascend with node ids, so the lowest position is the lowest id
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) {
+                const float ob = __shfl_xor_sync(SLONN_FULL_MASK, best, o);
+                const uint32_t oi = __shfl_xor_sync(SLONN_FULL_MASK, bi, o);
+                if (oi != 0xffffffffu && (bi == 0xffffffffu || ob > best || (ob == best && oi < bi))) { best = ob; bi = oi; }
+            }
+            __shared__ float wbest[32];
+            __shared__ uint32_t wbi[32];
+            if (lane == 0) { wbest[warp] = best; wbi[warp] = bi; }
+            __syncthreads();
+            if (warp == 0) {
+                best = lane < nwarps ? wbest[lane] : 0.0f;
+                bi = lane < nwarps ? wbi[lane] : 0xffffffffu;
+#pragma unroll
+                for (int o = 16; o >= 1; o >>= 1) {
+                    const float ob = __shfl_xor_sync(SLONN_FULL_MASK, best, o);
+                    const uint32_t oi = __shfl_xor_sync(SLONN_FULL_MASK, bi, o);
+                    if (oi != 0xffffffffu && (bi == 0xffffffffu || ob > best || (ob == best && oi < bi))) { best = ob; bi = oi; }
+                }
+                if (lane == 0 && bi != 0xffffffffu) P.pred[q] = implicit_ids ? bi : ids_s[bi];
+            }
+        }
+    }
+}

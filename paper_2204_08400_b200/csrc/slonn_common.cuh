@@ -150,6 +150,45 @@ __device__ __forceinline__ void warp_dot_rows(const uint4 *const (&rows)[R], con
     }
 }
 
+// Fixed-order dot product of ONE weight row, for launches where latency matters more than
+// throughput (a handful of queries): up to 8 of the lane's 16-byte chunks are in flight at once.
+// Same chunk-to-lane assignment, same order within a lane, xor butterfly 16, 8, 4, 2, 1; every
+// lane returns the sum (bias not included).
+template <bool BF16>
+__device__ __forceinline__ float warp_dot_row1(const uint4 *row, const float4 *xs4, uint32_t nchunks, uint32_t lane)
+{
+    constexpr int VPC = BF16 ? 8 : 4;
+#ifndef SLONN_ROW1_DEPTH
+#define SLONN_ROW1_DEPTH 8
+#endif
+    constexpr int DEPTH = SLONN_ROW1_DEPTH; // chunks of this lane loaded before the first one is used
+    float acc[1] = {0.0f};
+    for (uint32_t c0 = lane; c0 < nchunks; c0 += 32 * DEPTH) {
+        uint4 w[DEPTH][1];
+#pragma unroll
+        for (int i = 0; i < DEPTH; ++i)
+            if (c0 + 32 * i < nchunks) w[i][0] = __ldg(row + c0 + 32 * i);
+#pragma unroll
+        for (int i = 0; i < DEPTH; ++i) {
+            const uint32_t c = c0 + 32 * i;
+            if (c < nchunks) {
+                float x[VPC];
+                const float4 xa = xs4[c];
+                x[0] = xa.x; x[1] = xa.y; x[2] = xa.z; x[3] = xa.w;
+                if (BF16) {
+                    const float4 xb = xs4[nchunks + c];
+                    x[VPC - 4] = xb.x; x[VPC - 3] = xb.y; x[VPC - 2] = xb.z; x[VPC - 1] = xb.w;
+                }
+                chunk_fma<BF16, 1, 0, VPC>::run(w[i], x, acc);
+            }
+        }
+    }
+    float a = acc[0];
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) a = a + __shfl_xor_sync(SLONN_FULL_MASK, a, off);
+    return a;
+}
+
 // ---- layer input descriptor --------------------------------------------------
 
 enum { SLONN_IN_DENSE = 0, SLONN_IN_LIST = 1 };

@@ -8,6 +8,7 @@
 #include "slonn_dense_tc.cuh"
 #include "slonn_fused_kernel.cuh"
 #include "slonn_run_kernels.cuh"
+#include "slonn_cluster_kernel.cuh"
 
 namespace {
 
@@ -111,21 +112,33 @@ int set_smem(K kernel, size_t bytes)
     return SLONN_OK;
 }
 
+template <bool BF16, typename IDT, bool LAT>
+int launch_select_t(const slonn_select_params &P, uint32_t n, uint32_t threads, size_t smem, cudaStream_t st)
+{
+    const int rc = set_smem(hash_select_kernel<BF16, IDT, LAT>, smem);
+    if (rc) return rc;
+    hash_select_kernel<BF16, IDT, LAT><<<n, threads, smem, st>>>(P);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+// Fewer queries than SMs: latency variant, one warp per hash row (at least 8, at most 32 warps).
 int launch_select(const slonn_model *m, const slonn_select_params &P, uint32_t n, cudaStream_t st)
 {
     const size_t smem = (size_t)P.D * 4 + (size_t)((P.N + 31) / 32) * 4;
     const bool bf = m->dtype == SLONN_BF16;
     const bool id16 = m->layer[P.layer].id_bytes == 2;
-    int rc;
-    if (bf && id16) { if ((rc = set_smem(hash_select_kernel<true, uint16_t>, smem))) return rc;
-        hash_select_kernel<true, uint16_t><<<n, SLONN_THREADS, smem, st>>>(P); }
-    else if (bf) { if ((rc = set_smem(hash_select_kernel<true, uint32_t>, smem))) return rc;
-        hash_select_kernel<true, uint32_t><<<n, SLONN_THREADS, smem, st>>>(P); }
-    else if (id16) { if ((rc = set_smem(hash_select_kernel<false, uint16_t>, smem))) return rc;
-        hash_select_kernel<false, uint16_t><<<n, SLONN_THREADS, smem, st>>>(P); }
-    else { if ((rc = set_smem(hash_select_kernel<false, uint32_t>, smem))) return rc;
-        hash_select_kernel<false, uint32_t><<<n, SLONN_THREADS, smem, st>>>(P); }
-    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+    const bool lat = n <= 148;
+    const uint32_t threads = lat ? 32u * std::min(32u, std::max(8u, m->H)) : (uint32_t)SLONN_THREADS;
+    if (lat) {
+        if (bf && id16) return launch_select_t<true, uint16_t, true>(P, n, threads, smem, st);
+        if (bf) return launch_select_t<true, uint32_t, true>(P, n, threads, smem, st);
+        if (id16) return launch_select_t<false, uint16_t, true>(P, n, threads, smem, st);
+        return launch_select_t<false, uint32_t, true>(P, n, threads, smem, st);
+    }
+    if (bf && id16) return launch_select_t<true, uint16_t, false>(P, n, threads, smem, st);
+    if (bf) return launch_select_t<true, uint32_t, false>(P, n, threads, smem, st);
+    if (id16) return launch_select_t<false, uint16_t, false>(P, n, threads, smem, st);
+    return launch_select_t<false, uint32_t, false>(P, n, threads, smem, st);
 }
 
 // Rows per block: whole queries per block once the batch alone fills the GPU,
@@ -142,18 +155,33 @@ void gather_shape(uint32_t n, uint32_t max_rows, uint32_t *rows_per_cta, uint32_
     *ctas_per_query = (uint32_t)((max_rows + rpc - 1) / rpc);
 }
 
+template <bool BF16, bool LAT>
+int launch_gather_t(const slonn_gather_params &P, uint64_t grid, uint32_t threads, size_t smem, cudaStream_t st)
+{
+    const int rc = set_smem(gather_dot_kernel<BF16, LAT>, smem);
+    if (rc) return rc;
+    gather_dot_kernel<BF16, LAT><<<(uint32_t)grid, threads, smem, st>>>(P);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
 int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint32_t max_rows, cudaStream_t st)
 {
-    gather_shape(n, max_rows, &P.rows_per_cta, &P.ctas_per_query);
+    // so few rows that the GPU cannot be filled: latency variant, 4 warps per block, one row per warp
+    const bool lat = (uint64_t)n * max_rows <= 148ull * 64;
+    uint32_t threads = SLONN_THREADS;
+    if (lat) {
+        threads = 128;
+        P.rows_per_cta = 4;
+        P.ctas_per_query = (max_rows + 3) / 4;
+    } else {
+        gather_shape(n, max_rows, &P.rows_per_cta, &P.ctas_per_query);
+    }
     const size_t smem = (size_t)P.D * 4;
     const uint64_t grid = (uint64_t)n * P.ctas_per_query;
     if (grid == 0 || grid > 0x7fffffffull) return SLONN_ERR_DIM;
-    int rc;
-    if (m->dtype == SLONN_BF16) { if ((rc = set_smem(gather_dot_kernel<true>, smem))) return rc;
-        gather_dot_kernel<true><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(P); }
-    else { if ((rc = set_smem(gather_dot_kernel<false>, smem))) return rc;
-        gather_dot_kernel<false><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(P); }
-    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+    const bool bf = m->dtype == SLONN_BF16;
+    if (lat) return bf ? launch_gather_t<true, true>(P, grid, threads, smem, st) : launch_gather_t<false, true>(P, grid, threads, smem, st);
+    return bf ? launch_gather_t<true, false>(P, grid, threads, smem, st) : launch_gather_t<false, false>(P, grid, threads, smem, st);
 }
 
 // ---- whole-network kernel for narrow layers -----------------------------------
@@ -219,6 +247,85 @@ int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *ind
         if (max_rounds <= 8) return launch_fused_t<false, 8>(P, st);
     }
     return SLONN_ERR_DIM;
+}
+
+// ---- one cluster per query: latency path for a handful of queries ---------------
+
+bool cluster_eligible(const slonn_model *m)
+{
+    if (m->first_sparse) return false;
+    for (uint32_t l = 0; l < m->n_layers; ++l)
+        if (m->layer[l].D > SLONN_CLUSTER_MAX_D || m->layer[l].N > SLONN_CLUSTER_MAX_N) return false;
+    return true;
+}
+
+// most rows any layer computes for one query at this budget
+uint32_t cluster_max_rows(const slonn_model *m, uint32_t max_bp)
+{
+    uint32_t r = 0;
+    for (uint32_t l = 0; l < m->n_layers; ++l)
+        r = std::max(r, m->layer[l].has_act ? slonn_budget_nodes(max_bp, m->layer[l].N) : m->layer[l].N);
+    return r;
+}
+
+template <bool BF16>
+int launch_cluster_t(const slonn_cluster_params &P, size_t smem, cudaStream_t st)
+{
+    if (cudaFuncSetAttribute(cluster_network_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+        return SLONN_ERR_CUDA;
+    if (P.cluster > 8 && cudaFuncSetAttribute(cluster_network_kernel<BF16>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) !=
+                             cudaSuccess)
+        return SLONN_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(P.n * P.cluster, 1, 1);
+    cfg.blockDim = dim3(SLONN_CLUSTER_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = P.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0; // the device must be able to co-schedule at least one such cluster
+    if (cudaOccupancyMaxActiveClusters(&clusters, cluster_network_kernel<BF16>, &cfg) != cudaSuccess || clusters < 1) {
+        cudaGetLastError();
+        return SLONN_ERR_DIM;
+    }
+    return cudaLaunchKernelEx(&cfg, cluster_network_kernel<BF16>, P) == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+int launch_cluster(const slonn_model *m, const slonn_batch *b, const uint64_t *indptr, uint32_t stride, cudaStream_t st)
+{
+    slonn_cluster_params P;
+    memset(&P, 0, sizeof(P));
+    const uint32_t esz = m->dtype == SLONN_BF16 ? 2u : 4u;
+    uint32_t xbuf = 4, ids_cap = 4, words = 1;
+    for (uint32_t l = 0; l < m->n_layers; ++l) {
+        const slonn_layer &ly = m->layer[l];
+        slonn_cluster_layer &f = P.layer[l];
+        f.W = ly.W; f.bias = ly.bias; f.hash_nodes = ly.hash_nodes; f.tables = ly.tables;
+        f.D = ly.D; f.N = ly.N; f.nchunks = ly.D * esz / 16u; f.cap = ly.cap;
+        f.has_act = ly.has_act; f.a = m->act_index[l]; f.relu = (l + 1 == m->n_layers) ? 0u : 1u;
+        f.id_bytes = ly.id_bytes;
+        xbuf = std::max(xbuf, std::max((ly.D + 3u) / 4u * 4u, (ly.N + 3u) / 4u * 4u));
+        if (ly.has_act) {
+            ids_cap = std::max(ids_cap, (ly.N + 3u) / 4u * 4u);
+            words = std::max(words, (ly.N + 31u) / 32u);
+        }
+    }
+    P.n_layers = m->n_layers; P.n = b->n_queries; P.n_act = m->n_act; P.K = m->K; P.L = m->L; P.cluster = SLONN_CLUSTER_SIZE;
+    P.x = b->x_dense; P.indptr = indptr;
+    P.out_ids = b->active_ids; P.out_vals = b->active_vals; P.codes = b->codes;
+    P.logits = b->logits; P.logit_stride = stride; P.logit_ids = b->logit_ids; P.pred = b->pred;
+    P.status = b->status;
+    P.xbuf_floats = xbuf; P.ids_cap = ids_cap; P.bitmap_words = words;
+    const size_t smem = (size_t)xbuf * 8 + (size_t)ids_cap * 4 + (size_t)words * 4;
+    if (smem > 200 * 1024) return SLONN_ERR_DIM;
+    return m->dtype == SLONN_BF16 ? launch_cluster_t<true>(P, smem, st) : launch_cluster_t<false>(P, smem, st);
 }
 
 } // namespace
@@ -373,8 +480,19 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         skip_bp = b->budget_bp;
     }
 
+    // a handful of queries: one thread-block cluster per query, every layer in one launch
+    if (b->kernel_path > SLONN_PATH_CLUSTER) return SLONN_ERR_ARG;
+    if (b->kernel_path == SLONN_PATH_CLUSTER && (!cluster_eligible(m) || skip_bp)) return SLONN_ERR_DIM;
+    if (b->kernel_path == SLONN_PATH_CLUSTER || (b->kernel_path == SLONN_PATH_AUTO && cluster_eligible(m) && n <= 4 && !skip_bp &&
+         cluster_max_rows(m, max_bp) <= 1024)) {
+        TIC(SLONN_STAGE_CLUSTER);
+        const int rc = launch_cluster(m, b, indptr, stride, st);
+        TOC();
+        if (rc != SLONN_ERR_DIM || b->kernel_path == SLONN_PATH_CLUSTER) return rc;
+        // the device cannot co-schedule such a cluster: fall through to the other kernels
+    }
+
     // narrow networks with enough queries to fill the GPU: one warp per query, every layer in one launch
-    if (b->kernel_path > SLONN_PATH_FUSED) return SLONN_ERR_ARG;
     if (b->kernel_path == SLONN_PATH_FUSED && !fused_eligible(m)) return SLONN_ERR_DIM;
     if (b->kernel_path == SLONN_PATH_FUSED ||
         (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n >= 512)) {

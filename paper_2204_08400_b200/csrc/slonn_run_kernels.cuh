@@ -142,8 +142,107 @@ __device__ __forceinline__ uint32_t table_entry(const void *tables, uint32_t cap
     return (uint32_t)__ldg(t + (((uint64_t)b << K) + key) * cap + r);
 }
 
-template <bool BF16, typename IDT>
-__global__ void __launch_bounds__(SLONN_THREADS) hash_select_kernel(slonn_select_params P)
+// First B distinct ids of the rank-interleaved bucket lists, written ascending to out[0..B)
+// (global or shared memory).  Called by every thread of the block; bitmap ((N+31)/32 words) must
+// be zero, *s_total zero, keys[L] set, all behind a barrier.  B == N gives every node.  Returns
+// false when the lists did not hold B distinct ids (malformed tables); out is then 0..B-1.
+template <typename IDT>
+__device__ __forceinline__ bool block_select(const void *tables, uint32_t cap, uint32_t K, uint32_t L, uint32_t N,
+                                             uint32_t B, const uint32_t *keys, uint32_t *bitmap, uint32_t *out,
+                                             uint32_t *scan_ws, uint32_t *scan_total, uint32_t *s_total)
+{
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t nwords = (N + 31u) >> 5;
+    if (B == N) { // every node
+        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
+        return true;
+    }
+    if (B > cap) { // reported by the plan; keep the output in range
+        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
+        return true;
+    }
+
+    // (3)+(4) read the L lists rank by rank; the first B distinct ids are the active set.
+    // Position pos = rank * L + table.  A block-wide step marks blockDim.x positions
+    // at once; the step that would pass B is undone and replayed 32 positions at a
+    // time by warp 0, which cuts exactly at B.
+    const uint32_t npos = B * L; // B distinct ids are always found within rank < B
+    uint32_t total = 0;
+    for (uint32_t base = 0; base < npos; base += blockDim.x) {
+        const uint32_t pos = base + threadIdx.x;
+        const bool valid = pos < npos;
+        uint32_t id = 0;
+        bool won = false;
+        if (valid) {
+            const uint32_t r = pos / L, b = pos - r * L;
+            id = table_entry<IDT>(tables, cap, K, b, keys[b], r);
+            if (id < N) {
+                const uint32_t bit = 1u << (id & 31u);
+                won = (atomicOr(&bitmap[id >> 5], bit) & bit) == 0u;
+            }
+        }
+        const uint32_t cnt = (uint32_t)__syncthreads_count(won);
+        if (total + cnt < B) { total += cnt; continue; }
+        if (total + cnt == B) { total = B; break; }
+        // crossing step: undo, then replay in order
+        if (won) atomicAnd(&bitmap[id >> 5], ~(1u << (id & 31u)));
+        __syncthreads();
+        if (warp == 0) {
+            for (uint32_t sub = 0; sub < blockDim.x && total < B; sub += 32) {
+                const uint32_t p2 = base + sub + lane;
+                const bool v2 = p2 < npos;
+                uint32_t id2 = 0xffffffffu - lane; // distinct dummies
+                bool fresh = false;
+                if (v2) {
+                    const uint32_t r = p2 / L, b = p2 - r * L;
+                    id2 = table_entry<IDT>(tables, cap, K, b, keys[b], r);
+                    if (id2 < N) fresh = ((bitmap[id2 >> 5] >> (id2 & 31u)) & 1u) == 0u;
+                }
+                const uint32_t same = __match_any_sync(SLONN_FULL_MASK, id2);
+                const bool first = (uint32_t)(__ffs(same) - 1) == lane;
+                const bool take = fresh && first;
+                const uint32_t bal = __ballot_sync(SLONN_FULL_MASK, take);
+                const uint32_t need = B - total;
+                const uint32_t rank = __popc(bal & ((1u << lane) - 1u));
+                if (take && rank < need) atomicOr(&bitmap[id2 >> 5], 1u << (id2 & 31u));
+                const uint32_t c = (uint32_t)__popc(bal);
+                total += c < need ? c : need;
+                __syncwarp();
+            }
+            if (lane == 0) *s_total = total;
+        }
+        __syncthreads();
+        total = *s_total;
+        break;
+    }
+    __syncthreads();
+    if (total != B) { // cannot happen with well-formed tables; keep the output in range
+        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
+        return false;
+    }
+
+    // emit ascending ids: popcount prefix over the bitmap words
+    const uint32_t wpt = (nwords + blockDim.x - 1) / blockDim.x;
+    const uint32_t w0 = threadIdx.x * wpt;
+    const uint32_t w1 = min(w0 + wpt, nwords);
+    uint32_t cnt = 0;
+    for (uint32_t w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+    uint32_t o = block_exclusive_scan<uint32_t>(cnt, scan_ws, scan_total);
+    for (uint32_t w = w0; w < w1; ++w) {
+        uint32_t bits = bitmap[w];
+        while (bits) {
+            const uint32_t t = __ffs(bits) - 1;
+            bits &= bits - 1;
+            out[o++] = (w << 5) + t;
+        }
+    }
+    return true;
+}
+
+// LAT: latency variant for a handful of queries -- up to 32 warps per block, one hash row per warp
+// with deep load prefetch, instead of 4 rows per warp pass.
+template <bool BF16, typename IDT, bool LAT>
+__global__ void __launch_bounds__(LAT ? 1024 : SLONN_THREADS) hash_select_kernel(slonn_select_params P)
 {
     extern __shared__ float4 smem4[];
     float4 *xs4 = smem4;
@@ -165,6 +264,14 @@ __global__ void __launch_bounds__(SLONN_THREADS) hash_select_kernel(slonn_select
     // (1) FreeHash: z_h = w_h . x + b_h for the layer's K*L hash nodes
     stage_input<BF16>(P.in, q, P.D, P.nchunks, xs4);
     const uint32_t row_u4 = P.nchunks; // uint4 per weight row
+    if (LAT) {
+        for (uint32_t h = warp; h < H; h += nwarps) {
+            const uint32_t nd = __ldg(P.hash_nodes + h);
+            const float sum = warp_dot_row1<BF16>(reinterpret_cast<const uint4 *>(P.W) + (uint64_t)nd * row_u4, xs4,
+                                                  P.nchunks, lane);
+            if (lane == 0) zh[h] = sum + __ldg(P.bias + nd);
+        }
+    } else
     for (uint32_t h0 = warp * SLONN_ROWS_PER_WARP; h0 < H; h0 += nwarps * SLONN_ROWS_PER_WARP) {
         const uint4 *rows[SLONN_ROWS_PER_WARP];
 #pragma unroll
@@ -192,91 +299,10 @@ __global__ void __launch_bounds__(SLONN_THREADS) hash_select_kernel(slonn_select
     if (threadIdx.x == 0) s_total = 0;
     __syncthreads();
 
-    uint32_t *out = P.out_ids + off;
-    if (B == P.N) { // every node
-        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
-        return;
-    }
-    if (B > P.cap) { // reported by the plan; keep the output in range
-        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
-        return;
-    }
-
-    // (3)+(4) read the L lists rank by rank; the first B distinct ids are the active set.
-    // Position pos = rank * L + table.  A block-wide step marks blockDim.x positions
-    // at once; the step that would pass B is undone and replayed 32 positions at a
-    // time by warp 0, which cuts exactly at B.
-    const uint32_t npos = B * P.L; // B distinct ids are always found within rank < B
-    uint32_t total = 0;
-    for (uint32_t base = 0; base < npos; base += blockDim.x) {
-        const uint32_t pos = base + threadIdx.x;
-        const bool valid = pos < npos;
-        uint32_t id = 0;
-        bool won = false;
-        if (valid) {
-            const uint32_t r = pos / P.L, b = pos - r * P.L;
-            id = table_entry<IDT>(P.tables, P.cap, P.K, b, keys[b], r);
-            if (id < P.N) {
-                const uint32_t bit = 1u << (id & 31u);
-                won = (atomicOr(&bitmap[id >> 5], bit) & bit) == 0u;
-            }
-        }
-        const uint32_t cnt = (uint32_t)__syncthreads_count(won);
-        if (total + cnt < B) { total += cnt; continue; }
-        if (total + cnt == B) { total = B; break; }
-        // crossing step: undo, then replay in order
-        if (won) atomicAnd(&bitmap[id >> 5], ~(1u << (id & 31u)));
-        __syncthreads();
-        if (warp == 0) {
-            for (uint32_t sub = 0; sub < blockDim.x && total < B; sub += 32) {
-                const uint32_t p2 = base + sub + lane;
-                const bool v2 = p2 < npos;
-                uint32_t id2 = 0xffffffffu - lane; // distinct dummies
-                bool fresh = false;
-                if (v2) {
-                    const uint32_t r = p2 / P.L, b = p2 - r * P.L;
-                    id2 = table_entry<IDT>(P.tables, P.cap, P.K, b, keys[b], r);
-                    if (id2 < P.N) fresh = ((bitmap[id2 >> 5] >> (id2 & 31u)) & 1u) == 0u;
-                }
-                const uint32_t same = __match_any_sync(SLONN_FULL_MASK, id2);
-                const bool first = (uint32_t)(__ffs(same) - 1) == lane;
-                const bool take = fresh && first;
-                const uint32_t bal = __ballot_sync(SLONN_FULL_MASK, take);
-                const uint32_t need = B - total;
-                const uint32_t rank = __popc(bal & ((1u << lane) - 1u));
-                if (take && rank < need) atomicOr(&bitmap[id2 >> 5], 1u << (id2 & 31u));
-                const uint32_t c = (uint32_t)__popc(bal);
-                total += c < need ? c : need;
-                __syncwarp();
-            }
-            if (lane == 0) s_total = total;
-        }
-        __syncthreads();
-        total = s_total;
-        break;
-    }
-    __syncthreads();
-    if (total != B) { // cannot happen with well-formed tables; keep the output in range
-        if (threadIdx.x == 0) slonn_report(P.status, SLONN_ERR_ARG, q, P.layer);
-        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
-        return;
-    }
-
-    // emit ascending ids: popcount prefix over the bitmap words
-    const uint32_t wpt = (nwords + blockDim.x - 1) / blockDim.x;
-    const uint32_t w0 = threadIdx.x * wpt;
-    const uint32_t w1 = min(w0 + wpt, nwords);
-    uint32_t cnt = 0;
-    for (uint32_t w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
-    uint32_t o = block_exclusive_scan<uint32_t>(cnt, scan_ws, &scan_total);
-    for (uint32_t w = w0; w < w1; ++w) {
-        uint32_t bits = bitmap[w];
-        while (bits) {
-            const uint32_t t = __ffs(bits) - 1;
-            bits &= bits - 1;
-            out[o++] = (w << 5) + t;
-        }
-    }
+    if (!block_select<IDT>(P.tables, P.cap, P.K, P.L, P.N, B, keys, bitmap, P.out_ids + off, scan_ws, &scan_total,
+                           &s_total) &&
+        threadIdx.x == 0)
+        slonn_report(P.status, SLONN_ERR_ARG, q, P.layer);
 }
 
 // ---------------------------------------------------------------------------
@@ -300,7 +326,7 @@ struct slonn_gather_params {
     uint32_t rows_per_cta, ctas_per_query;
 };
 
-template <bool BF16>
+template <bool BF16, bool LAT>
 __global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_params P)
 {
     extern __shared__ float4 smem4[];
@@ -320,6 +346,26 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_
     stage_input<BF16>(P.in, q, P.D, P.nchunks, smem4);
 
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    if (LAT) { // one row per warp, deep load prefetch
+        for (uint32_t r = r0 + warp; r < r1; r += nwarps) {
+            const uint32_t nd = P.use_list ? __ldg(P.ids + off + r) : r;
+            const float sum = warp_dot_row1<BF16>(reinterpret_cast<const uint4 *>(P.W) + (uint64_t)nd * P.nchunks, smem4,
+                                                  P.nchunks, lane);
+            if (lane == 0) {
+                float z = sum + __ldg(P.bias + nd);
+                if (P.relu) z = z > 0.0f ? z : 0.0f;
+                if (P.use_list) {
+                    if (P.out_vals) P.out_vals[off + r] = z;
+                    if (P.out_dense) {
+                        P.out_dense[(uint64_t)q * P.out_stride + r] = z;
+                        if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q * P.out_stride + r] = nd;
+                    }
+                } else {
+                    P.out_dense[(uint64_t)q * P.out_stride + nd] = z;
+                }
+            }
+        }
+    } else
     for (uint32_t r = r0 + warp * SLONN_ROWS_PER_WARP; r < r1; r += nwarps * SLONN_ROWS_PER_WARP) {
         const uint4 *rows[SLONN_ROWS_PER_WARP];
 #pragma unroll
