@@ -253,6 +253,20 @@ def main():
     value = n_all / (ms_step / 1e3)
     launches_per_step = None  # counted below from the per-stage launch counters
 
+    # ---- per-query latency for small batches (the paper serves at batch size 1): one event pair per step ----
+    latency = None
+    if n <= 64:
+        reps = max(args.steps, 1000)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b_ in evs:
+            a.record(stream)
+            batch.run(stream)
+            b_.record(stream)
+            torch.cuda.synchronize(dev)      # a server answers one request before it takes the next
+        t = np.array([a.elapsed_time(b_) for a, b_ in evs]) * 1e3
+        latency = {"unit": "us per batch", "launches": reps, "p50": float(np.percentile(t, 50)),
+                   "p90": float(np.percentile(t, 90)), "p99": float(np.percentile(t, 99)), "min": float(t.min())}
+
     # ---- per-stage device time of the same step (event pair around every launch) ----
     stage_ms = {s: 0.0 for s in sl.STAGES}
     stage_cnt = {s: 0 for s in sl.STAGES}
@@ -266,6 +280,8 @@ def main():
         gb = sum(gathered_bytes(wl, bps))
         if ms_by_stage["fused"] > 0:     # one launch does hash + select + gather for every layer
             kernel, ms, launches, nbytes = "fused_network_kernel", ms_by_stage["fused"], cnt_by_stage["fused"], gb + hash_bytes(wl, bps.size)
+        elif ms_by_stage["cluster"] > 0:
+            kernel, ms, launches, nbytes = "cluster_network_kernel", ms_by_stage["cluster"], cnt_by_stage["cluster"], gb + hash_bytes(wl, bps.size)
         else:
             kernel, ms, launches, nbytes = "gather_dot_kernel", ms_by_stage["gather_dot"], cnt_by_stage["gather_dot"], gb
         ms /= steps
@@ -357,7 +373,7 @@ def main():
                        "full_budget_route": "tensor cores (bf16 activations)" if args.dense_tc else "fixed-order fp32 kernels"},
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": (sum(stage_cnt.values()) // prof_steps + (1 if stage_cnt["plan"] else 0)) * args.steps,
-            "roofline": roofline, "cpu_baseline": cpu, "budget_sweep": sweep,
+            "roofline": roofline, "cpu_baseline": cpu, "budget_sweep": sweep, "latency": latency,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
