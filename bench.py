@@ -266,6 +266,22 @@ def main():
         t = np.array([a.elapsed_time(b_) for a, b_ in evs]) * 1e3
         latency = {"unit": "us per batch", "launches": reps, "p50": float(np.percentile(t, 50)),
                    "p90": float(np.percentile(t, 90)), "p99": float(np.percentile(t, 99)), "min": float(t.min())}
+        # the same step captured once in a CUDA graph and replayed per request
+        gs = torch.cuda.Stream(dev)
+        with torch.cuda.stream(gs):
+            batch.run(gs)
+            gs.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=gs):
+                batch.run(torch.cuda.current_stream(dev))
+            tg = []
+            for _ in range(reps):
+                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); graph.replay(); b_.record()
+                torch.cuda.synchronize(dev)
+                tg.append(a.elapsed_time(b_) * 1e3)
+        latency["graph_replay_p50"] = float(np.percentile(tg, 50))
+        latency["graph_replay_p99"] = float(np.percentile(tg, 99))
 
     # ---- per-stage device time of the same step (event pair around every launch) ----
     stage_ms = {s: 0.0 for s in sl.STAGES}

@@ -285,3 +285,29 @@ def test_host_buffer_entry_point_in_pieces_matches_device_entry_point():
     sl.slonn_run_host(dm.model, hb, ws, nb)
     assert int(status[0]) == 5 and int(status[1]) == 7777
     dm.free()
+
+
+def test_slonn_run_replays_from_a_cuda_graph():
+    # slonn_run only enqueues work on the caller's stream (no allocation, no host synchronisation),
+    # so a serving loop can capture it once and replay it per request
+    import torch
+    from paper_2204_08400_b200 import harness
+    wl = custom_workload(63, [136, 200, 96, 24], [1, 1, 0], "bf16", n=3, n_cal=300, K=4, L=2)
+    dm = harness.DeviceModel(wl)
+    for path in (1, 2, 3):
+        want = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=path)
+        b = harness.DeviceBatch(dm, wl.x, wl.budget_bp, kernel_path=path)
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            b.run(s)                      # first call outside the capture (sets kernel attributes)
+            s.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                b.run(torch.cuda.current_stream())
+            for t in (b.logits, b.pred, b.ids, b.vals):
+                t.zero_()
+            g.replay()
+        got = b.results()
+        for k in ("logits", "pred", "codes", "active_ids", "active_vals"):
+            assert np.array_equal(got[k], want[k]), (path, k)
+    dm.free()
