@@ -390,6 +390,8 @@ def main():
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": (sum(stage_cnt.values()) // prof_steps + (1 if stage_cnt["plan"] else 0)) * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "budget_sweep": sweep, "latency": latency,
+            "table_build": {"ms": dm.build_ms, "calibration_rows": dm.n_cal,
+                            "rows_per_s": dm.n_cal / (dm.build_ms / 1e3), "timing": "host wall clock around slonn_build"},
         }
         print(json.dumps(line), flush=True)
     if world > 1:

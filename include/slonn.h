@@ -129,6 +129,21 @@ int slonn_model_info(const slonn_model *m, uint32_t layer, uint32_t *hash_nodes,
  */
 int slonn_model_tables_to_host(const slonn_model *m, uint32_t layer, void *dst_host, uint64_t dst_bytes);
 
+/*
+ * Persisting a trained Node Activator (the paper trains it "pre- or post-deployment",
+ * Sec. 3.2: the tables outlive the process that made them).  slonn_serialize writes the
+ * model's configuration, hash nodes and tables into a HOST buffer of at least
+ * slonn_serialized_bytes(); slonn_deserialize rebuilds a model from such a blob without any
+ * calibration pass.  Weights and biases are not stored: pass the same device arrays again
+ * (same rules as slonn_build: referenced, must outlive the model).  A blob that is truncated,
+ * damaged (checksum) or inconsistent with itself is refused with SLONN_ERR_ARG before
+ * anything is allocated.  Both calls are synchronous.
+ */
+int slonn_serialized_bytes(const slonn_model *m, uint64_t *bytes);
+int slonn_serialize(const slonn_model *m, void *dst_host, uint64_t dst_bytes);
+int slonn_deserialize(const void *src_host, uint64_t src_bytes, const void *const *W,
+                      const float *const *bias, void *stream, slonn_model **out);
+
 /* Frees the model and everything it owns.  NULL is accepted. */
 void slonn_free(slonn_model *m);
 

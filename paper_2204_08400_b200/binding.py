@@ -20,7 +20,8 @@ LIB_PATH = os.environ.get("SLONN_LIB", os.path.join(_HERE, "libslonn.so"))  # SL
 EXPORTS = [
     "slonn_version", "slonn_strerror", "slonn_build", "slonn_model_info", "slonn_model_tables_to_host",
     "slonn_free", "slonn_active_capacity", "slonn_logit_stride", "slonn_workspace_bytes", "slonn_run",
-    "slonn_run_timed", "slonn_run_static", "slonn_dense_layer",
+    "slonn_run_timed", "slonn_run_static", "slonn_dense_layer", "slonn_serialized_bytes", "slonn_serialize",
+    "slonn_deserialize",
     "slonn_host_workspace_bytes", "slonn_run_host",
 ]
 
@@ -74,6 +75,13 @@ def lib():
                                        C.POINTER(C.c_uint64), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
         L.slonn_model_tables_to_host.restype = C.c_int
         L.slonn_model_tables_to_host.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64]
+        L.slonn_serialized_bytes.restype = C.c_int
+        L.slonn_serialized_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
+        L.slonn_serialize.restype = C.c_int
+        L.slonn_serialize.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
+        L.slonn_deserialize.restype = C.c_int
+        L.slonn_deserialize.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.POINTER(C.c_void_p)]
         L.slonn_free.restype = None
         L.slonn_free.argtypes = [C.c_void_p]
         L.slonn_active_capacity.restype = C.c_int
@@ -192,6 +200,37 @@ def slonn_build(dims: Sequence[int], has_activator: Sequence[int], dtype: int, W
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_build")
     return Model(out.value, keep, dims, has_activator, dtype, K, L, bool(first_layer_sparse))
+
+
+def slonn_serialize(model: Model) -> np.ndarray:
+    """The trained activator (configuration, hash nodes, tables) as a byte array; weights not included."""
+    nb = C.c_uint64()
+    rc = lib().slonn_serialized_bytes(model.handle, C.byref(nb))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_serialized_bytes")
+    buf = np.empty(nb.value, dtype=np.uint8)
+    rc = lib().slonn_serialize(model.handle, buf.ctypes.data, buf.nbytes)
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_serialize")
+    return buf
+
+
+def slonn_deserialize(blob: np.ndarray, W: List, bias: List, stream=None) -> Model:
+    """Rebuilds a model from slonn_serialize's bytes and the (device) weights it was trained on."""
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    n_layers = len(W)
+    Wp = (C.c_void_p * n_layers)(*[_ptr(w) for w in W])
+    bp = (C.c_void_p * n_layers)(*[_ptr(b) for b in bias])
+    out = C.c_void_p()
+    rc = lib().slonn_deserialize(blob.ctypes.data, blob.nbytes, C.cast(Wp, C.c_void_p), C.cast(bp, C.c_void_p),
+                                 _stream_ptr(stream), C.byref(out))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_deserialize")
+    hdr = np.frombuffer(blob[:32].tobytes(), dtype=np.uint32)
+    n_l, dtype, K, L, first_sparse = int(hdr[2]), int(hdr[3]), int(hdr[4]), int(hdr[5]), int(hdr[7])
+    dims = np.frombuffer(blob[32:32 + 4 * 17].tobytes(), dtype=np.uint32)[: n_l + 1].tolist()
+    has_act = blob[32 + 4 * 17: 32 + 4 * 17 + n_l].tolist()
+    return Model(out.value, [list(W), list(bias)], dims, has_act, dtype, K, L, bool(first_sparse))
 
 
 def slonn_free(model: Model) -> None:

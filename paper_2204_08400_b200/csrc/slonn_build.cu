@@ -567,3 +567,156 @@ fail:
     slonn_free(m);
     return rc;
 }
+
+// ---------------------------------------------------------------------------
+// Persisting a trained Node Activator.  The paper trains it "pre- or post-deployment"
+// (Sec. 3.2), i.e. the tables are an artefact that outlives the process that made them.
+// Blob (little endian): header, then per activator layer { L*K hash nodes, cap, id_bytes,
+// table bytes }, then a 64-bit FNV-1a checksum of everything before it.  Weights are not part
+// of the blob: the caller passes them again when loading, as for slonn_build.
+// ---------------------------------------------------------------------------
+namespace {
+
+struct blob_header {
+    uint32_t magic, version, n_layers, dtype, K, L, list_cap, first_sparse;
+    uint32_t dims[SLONN_MAX_LAYERS + 1];
+    uint8_t has_act[SLONN_MAX_LAYERS];
+};
+constexpr uint32_t BLOB_MAGIC = 0x4e4e4c53u; // "SLNN"
+constexpr uint32_t BLOB_VERSION = 1;
+
+uint64_t fnv1a(const unsigned char *p, uint64_t n)
+{
+    uint64_t h = 0xcbf29ce484222325ull;
+    for (uint64_t i = 0; i < n; ++i) { h ^= p[i]; h *= 0x100000001b3ull; }
+    return h;
+}
+
+uint64_t blob_bytes(const slonn_model *m)
+{
+    uint64_t b = sizeof(blob_header);
+    for (uint32_t l = 0; l < m->n_layers; ++l)
+        if (m->layer[l].has_act) b += sizeof(uint32_t) * m->H + 2 * sizeof(uint32_t) + m->layer[l].table_bytes;
+    return b + sizeof(uint64_t);
+}
+
+} // namespace
+
+extern "C" int slonn_serialized_bytes(const slonn_model *m, uint64_t *bytes)
+{
+    if (!m || m->magic != SLONN_MAGIC || !bytes) return SLONN_ERR_ARG;
+    *bytes = blob_bytes(m);
+    return SLONN_OK;
+}
+
+extern "C" int slonn_serialize(const slonn_model *m, void *dst_host, uint64_t dst_bytes)
+{
+    if (!m || m->magic != SLONN_MAGIC || !dst_host) return SLONN_ERR_ARG;
+    const uint64_t need = blob_bytes(m);
+    if (dst_bytes < need) return SLONN_ERR_WORKSPACE;
+    unsigned char *p = (unsigned char *)dst_host;
+    blob_header h;
+    memset(&h, 0, sizeof(h));
+    h.magic = BLOB_MAGIC; h.version = BLOB_VERSION; h.n_layers = m->n_layers; h.dtype = (uint32_t)m->dtype;
+    h.K = m->K; h.L = m->L; h.list_cap = m->list_cap; h.first_sparse = m->first_sparse;
+    for (uint32_t l = 0; l <= m->n_layers; ++l) h.dims[l] = m->dims[l];
+    for (uint32_t l = 0; l < m->n_layers; ++l) h.has_act[l] = (uint8_t)m->layer[l].has_act;
+    memcpy(p, &h, sizeof(h));
+    uint64_t o = sizeof(h);
+    for (uint32_t l = 0; l < m->n_layers; ++l) {
+        const slonn_layer &ly = m->layer[l];
+        if (!ly.has_act) continue;
+        memcpy(p + o, m->hash_nodes_host[l], sizeof(uint32_t) * m->H); o += sizeof(uint32_t) * m->H;
+        memcpy(p + o, &ly.cap, 4); o += 4;
+        memcpy(p + o, &ly.id_bytes, 4); o += 4;
+        if (cudaMemcpy(p + o, ly.tables, ly.table_bytes, cudaMemcpyDeviceToHost) != cudaSuccess) return SLONN_ERR_CUDA;
+        o += ly.table_bytes;
+    }
+    const uint64_t sum = fnv1a(p, o);
+    memcpy(p + o, &sum, 8);
+    return SLONN_OK;
+}
+
+extern "C" int slonn_deserialize(const void *src_host, uint64_t src_bytes, const void *const *W,
+                                 const float *const *bias, void *stream, slonn_model **out)
+{
+    if (!src_host || !W || !bias || !out) return SLONN_ERR_ARG;
+    if (src_bytes < sizeof(blob_header) + 8) return SLONN_ERR_ARG;
+    const unsigned char *p = (const unsigned char *)src_host;
+    blob_header h;
+    memcpy(&h, p, sizeof(h));
+    if (h.magic != BLOB_MAGIC || h.version != BLOB_VERSION) return SLONN_ERR_ARG;
+    if (h.n_layers < 1 || h.n_layers > SLONN_MAX_LAYERS) return SLONN_ERR_DIM;
+    if (h.dtype != SLONN_F32 && h.dtype != SLONN_BF16) return SLONN_ERR_DTYPE;
+    if (h.K < 1 || h.K > 16 || h.L < 1 || h.L > 8) return SLONN_ERR_DIM;
+    uint64_t sum_stored;
+    memcpy(&sum_stored, p + src_bytes - 8, 8);
+    if (fnv1a(p, src_bytes - 8) != sum_stored) return SLONN_ERR_ARG; // damaged or truncated blob
+    const uint32_t esz = h.dtype == SLONN_BF16 ? 2u : 4u, H = h.K * h.L, nb = 1u << h.K;
+    // walk the layer records once to validate sizes before anything is allocated
+    {
+        uint64_t o = sizeof(h);
+        for (uint32_t l = 0; l < h.n_layers; ++l) {
+            const uint32_t D = h.dims[l], N = h.dims[l + 1];
+            if (D == 0 || N == 0) return SLONN_ERR_DIM;
+            if (!W[l] || !bias[l]) return SLONN_ERR_ARG;
+            if ((uintptr_t)W[l] & 15u) return SLONN_ERR_ALIGN;
+            if (!(l == 0 && h.first_sparse) && (((uint64_t)D * esz) & 15u)) return SLONN_ERR_ALIGN;
+            if (!h.has_act[l]) continue;
+            if (H > N || (l == 0 && h.first_sparse)) return SLONN_ERR_DIM;
+            if (o + sizeof(uint32_t) * H + 8 > src_bytes - 8) return SLONN_ERR_ARG;
+            for (uint32_t k = 0; k < H; ++k) {
+                uint32_t nd;
+                memcpy(&nd, p + o + 4 * k, 4);
+                if (nd >= N) return SLONN_ERR_ARG;
+            }
+            o += sizeof(uint32_t) * H;
+            uint32_t cap, idb;
+            memcpy(&cap, p + o, 4); memcpy(&idb, p + o + 4, 4); o += 8;
+            if (cap < 1 || cap > N || idb != (N <= 65536u ? 2u : 4u)) return SLONN_ERR_ARG;
+            const uint64_t tb = (uint64_t)h.L * nb * cap * idb;
+            if (o + tb > src_bytes - 8) return SLONN_ERR_ARG;
+            o += tb;
+        }
+        if (o != src_bytes - 8) return SLONN_ERR_ARG;
+    }
+
+    slonn_model *m = new (std::nothrow) slonn_model;
+    if (!m) return SLONN_ERR_NOMEM;
+    memset(m, 0, sizeof(*m));
+    m->magic = SLONN_MAGIC;
+    cudaGetDevice(&m->device);
+    m->n_layers = h.n_layers; m->dtype = (int32_t)h.dtype; m->K = h.K; m->L = h.L; m->H = H;
+    m->list_cap = h.list_cap; m->first_sparse = h.first_sparse ? 1u : 0u;
+    for (uint32_t l = 0; l <= h.n_layers; ++l) m->dims[l] = h.dims[l];
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = SLONN_OK;
+    uint64_t o = sizeof(h);
+    for (uint32_t l = 0; l < h.n_layers; ++l) {
+        slonn_layer &ly = m->layer[l];
+        ly.W = W[l]; ly.bias = bias[l]; ly.D = h.dims[l]; ly.N = h.dims[l + 1];
+        ly.has_act = h.has_act[l] ? 1u : 0u;
+        if (!ly.has_act) continue;
+        m->act_index[l] = m->n_act++;
+        memcpy(m->hash_nodes_host[l], p + o, sizeof(uint32_t) * H); o += sizeof(uint32_t) * H;
+        memcpy(&ly.cap, p + o, 4); memcpy(&ly.id_bytes, p + o + 4, 4); o += 8;
+        ly.table_bytes = (uint64_t)h.L * nb * ly.cap * ly.id_bytes;
+        CK(cudaMalloc(&ly.hash_nodes, sizeof(uint32_t) * H));
+        CK(cudaMemcpyAsync(ly.hash_nodes, m->hash_nodes_host[l], sizeof(uint32_t) * H, cudaMemcpyHostToDevice, st));
+        CK(cudaMalloc(&ly.tables, ly.table_bytes));
+        CK(cudaMemcpyAsync(ly.tables, p + o, ly.table_bytes, cudaMemcpyHostToDevice, st));
+        o += ly.table_bytes;
+    }
+    if (m->first_sparse) {
+        slonn_layer &l0 = m->layer[0];
+        CK(cudaMalloc(&l0.WT, (uint64_t)l0.N * l0.D * esz));
+        transpose_kernel<<<dim3((l0.D + 31) / 32, (l0.N + 31) / 32), dim3(32, 8), 0, st>>>(l0.W, l0.WT, l0.N, l0.D, esz);
+        CK(cudaGetLastError());
+    }
+    CK(cudaStreamSynchronize(st));
+    *out = m;
+    return SLONN_OK;
+fail:
+    slonn_free(m);
+    return rc;
+}

@@ -1,6 +1,7 @@
 """Device-side plumbing shared by the tests, the benchmark and the smoke check:
 uploads a workload with torch, calls the binding, brings results back as numpy.
 torch is used for device memory and streams only."""
+import time
 from typing import Optional
 
 import numpy as np
@@ -41,10 +42,14 @@ class DeviceModel:
         else:
             c = wl.calib if n_cal is None else wl.calib[:n_cal]
             calib_dense = _dev(c, self.device)
+        torch.cuda.synchronize(self.device)
+        t0 = time.perf_counter()
         self.model = sl.slonn_build(wl.dims, wl.has_act, dtype, self.W, self.bias, calib_dense=calib_dense,
                                     calib_csr=calib_csr, K=wl.K, L=wl.L, list_cap=wl.list_cap, seed=wl.seed,
                                     first_layer_sparse=wl.first_sparse, hash_nodes_override=hash_nodes_override)
         torch.cuda.synchronize(self.device)
+        self.build_ms = (time.perf_counter() - t0) * 1e3   # slonn_build synchronises before it returns
+        self.n_cal = int(calib_csr[0].numel() - 1) if calib_csr is not None else int(calib_dense.shape[0])
 
     def hash_nodes(self, layer: int) -> np.ndarray:
         return sl.slonn_model_info(self.model, layer)["hash_nodes"]
