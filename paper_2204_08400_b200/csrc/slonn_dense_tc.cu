@@ -3,19 +3,23 @@
 // (Sec. 3.4: at a 100 % budget an SLO-NN is the full network), the one stage of the path that
 // is a dense contraction.
 //
-// One 128x128 output tile per block, K in steps of 64 (one 128-byte swizzle atom):
+// Persistent kernel, one block per SM, 128 x 256 output tiles, K in steps of 64 (one 128-byte
+// swizzle atom), six warps with fixed roles:
 //   warp 0 / one lane : TMA producer, cp.async.bulk.tensor 2-D tile loads into a 4-stage ring
-//   warp 1 / one lane : tcgen05.mma issuer, accumulator in tensor memory (128 lanes x 128 columns)
-//   warps 0-3         : epilogue, tcgen05.ld of the accumulator, bias, activation, stores
-// Stages hand over through mbarriers (TMA -> MMA by transaction bytes, MMA -> TMA and
-// MMA -> epilogue by tcgen05.commit).  Every wait is bounded: when one runs out the block raises
-// an abort flag, lets outstanding copies land, frees its tensor memory and reports
+//   warp 1 / one lane : tcgen05.mma issuer; two accumulators of 256 columns in tensor memory,
+//                       so the MMAs of tile i+1 run while tile i is drained
+//   warps 2-5         : epilogue, tcgen05.ld of one accumulator (32 rows per warp), bias,
+//                       activation, shared-memory transpose, coalesced stores
+// Hand-over through mbarriers: TMA -> MMA by transaction bytes, MMA -> TMA and MMA -> epilogue by
+// tcgen05.commit, epilogue -> MMA by plain arrivals.  Every wait is bounded: when one runs out the
+// block raises an abort flag, lets outstanding copies land, frees its tensor memory and reports
 // SLONN_ERR_TIMEOUT through the status word.  No cluster launch, no multicast.
 //
 // Sums are not bit-compatible with the fixed-order fp32 kernels (the tensor core's accumulation
 // order is not specified), so this path is only used where the caller asked for it.
 #include <cuda.h>
 
+#include <algorithm>
 #include <cstring>
 #include <mutex>
 
@@ -24,15 +28,16 @@
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 4, UMMA_K = 16;
-constexpr uint32_t TMEM_COLS = 128;
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int THREADS = 192, EPI_WARPS = 4;
+constexpr uint32_t TMEM_COLS = 2 * BN; // two accumulators
 constexpr uint32_t STAGE_A_BYTES = BM * BK * 2, STAGE_B_BYTES = BN * BK * 2;
 constexpr uint32_t RING_BYTES = STAGES * (STAGE_A_BYTES + STAGE_B_BYTES);
-constexpr uint32_t EPI_BYTES = 4 * (32 * 33) * 4 + 4 * 32 * 8; // per-warp 32x33 fp32 tile + 32 row offsets
+constexpr uint32_t EPI_BYTES = EPI_WARPS * (32 * 33) * 4 + EPI_WARPS * 32 * 8; // per-warp 32x33 fp32 tile + 32 row offsets
 constexpr uint32_t SMEM_BYTES = RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ + EPI_BYTES;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
-// instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = 128
+// instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = 256
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -44,6 +49,10 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 {
@@ -123,28 +132,30 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float f)
     return (uint16_t)(u >> 16);
 }
 
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(THREADS, 1)
 dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const slonn_dense_epilogue E, uint32_t N, uint32_t K)
 {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
-    const uint32_t m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     // rows this launch must produce (a device-side count when the rows were compacted on the device)
     const uint32_t m_valid = E.row_count ? min(*E.row_count, E.M) : E.M;
-    if (m0 >= m_valid) return; // uniform for the block: nothing allocated yet
+    const uint32_t m_tiles = (m_valid + BM - 1) / BM, n_tiles = (N + BN - 1) / BN;
+    const uint32_t tiles = m_tiles * n_tiles;
+    if (blockIdx.x >= tiles) return; // uniform for the block: nothing allocated yet
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u; // swizzle atoms need 1024-byte alignment
     const uint32_t bars = base + RING_BYTES;
-    const uint32_t full0 = bars, empty0 = bars + 8 * STAGES, tmem_full = bars + 16 * STAGES;
-    const uint32_t tmem_slot_addr = bars + 16 * STAGES + 8;
+    const uint32_t full0 = bars, empty0 = bars + 8 * STAGES;
+    const uint32_t tfull0 = bars + 16 * STAGES, tempty0 = tfull0 + 16;
+    const uint32_t tmem_slot_addr = tempty0 + 16;
     const uint32_t epi_addr = bars + 256;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot_addr - smem_u32(smem_raw)));
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        mbar_init(tmem_full, 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, EPI_WARPS); }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -158,78 +169,101 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t num_kb = (K + BK - 1) / BK;
 
-    if (warp == 0 && lane == 0) {
-        // ---- TMA producer ----
-        for (uint32_t kb = 0; kb < num_kb; ++kb) {
-            const uint32_t s = kb % STAGES, ph = (kb / STAGES) & 1u;
-            if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
-            mbar_expect_tx(full0 + 8 * s, STAGE_A_BYTES + STAGE_B_BYTES);
-            tma_load_2d(base + s * STAGE_A_BYTES, &map_a, (int32_t)(kb * BK), (int32_t)m0, full0 + 8 * s);
-            tma_load_2d(base + STAGES * STAGE_A_BYTES + s * STAGE_B_BYTES, &map_b, (int32_t)(kb * BK), (int32_t)n0,
-                        full0 + 8 * s);
+    if (warp == 0) {
+        // ---- TMA producer: runs ahead over this block's tiles ----
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (uint32_t t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+                const uint32_t m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
+                for (uint32_t kb = 0; kb < num_kb; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+                    if (!(ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag))) break;
+                    mbar_expect_tx(full0 + 8 * s, STAGE_A_BYTES + STAGE_B_BYTES);
+                    tma_load_2d(base + s * STAGE_A_BYTES, &map_a, (int32_t)(kb * BK), (int32_t)m0, full0 + 8 * s);
+                    tma_load_2d(base + STAGES * STAGE_A_BYTES + s * STAGE_B_BYTES, &map_b, (int32_t)(kb * BK),
+                                (int32_t)n0, full0 + 8 * s);
+                }
+            }
         }
-    } else if (warp == 1 && lane == 0) {
-        // ---- MMA issuer ----
-        bool ok = true;
-        for (uint32_t kb = 0; kb < num_kb && ok; ++kb) {
-            const uint32_t s = kb % STAGES, ph = (kb / STAGES) & 1u;
-            ok = mbar_wait(full0 + 8 * s, ph, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            const uint64_t da = umma_desc(base + s * STAGE_A_BYTES);
-            const uint64_t db = umma_desc(base + STAGES * STAGE_A_BYTES + s * STAGE_B_BYTES);
+    } else if (warp == 1) {
+        // ---- MMA issuer: alternates between the two accumulators ----
+        if (lane == 0) {
+            uint32_t it = 0, ti = 0;
+            bool ok = true;
+            for (uint32_t t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++ti) {
+                const uint32_t acc = ti & 1u, aph = (ti >> 1) & 1u;
+                if (!(ok = mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag))) break; // drained by the epilogue
+                tc_fence_after();
+                const uint32_t d = tmem_base + acc * BN;
+                for (uint32_t kb = 0; kb < num_kb; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+                    if (!(ok = mbar_wait(full0 + 8 * s, ph, abort_flag))) break;
+                    tc_fence_after();
+                    const uint64_t da = umma_desc(base + s * STAGE_A_BYTES);
+                    const uint64_t db = umma_desc(base + STAGES * STAGE_A_BYTES + s * STAGE_B_BYTES);
 #pragma unroll
-            for (int k = 0; k < BK / UMMA_K; ++k) // 32 bytes further along K inside the swizzle atom
-                umma_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), (kb | (uint32_t)k) != 0u);
-            umma_commit(empty0 + 8 * s); // frees the stage once these MMAs have read it
+                    for (int k = 0; k < BK / UMMA_K; ++k) // 32 bytes further along K inside the swizzle atom
+                        umma_bf16(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), (kb | (uint32_t)k) != 0u);
+                    umma_commit(empty0 + 8 * s); // frees the stage once these MMAs have read it
+                }
+                if (ok) umma_commit(tfull0 + 8 * acc); // accumulator complete
+            }
         }
-        if (ok) umma_commit(tmem_full); // accumulator complete
+    } else {
+        // ---- epilogue warps: TMEM lane = row of the tile, TMEM column = column of the tile ----
+        const uint32_t ew = warp - 2;        // slice of the staging area
+        const uint32_t quarter = warp & 3u;  // the TMEM lanes 32*quarter .. +31 this warp may read
+        float *tile = reinterpret_cast<float *>(smem_raw + (epi_addr - smem_u32(smem_raw))) + ew * (32 * 33);
+        unsigned long long *row_off = reinterpret_cast<unsigned long long *>(
+            smem_raw + (epi_addr - smem_u32(smem_raw)) + EPI_WARPS * (32 * 33) * sizeof(float)) + ew * 32;
+        uint32_t ti = 0;
+        for (uint32_t t = blockIdx.x; t < tiles; t += gridDim.x, ++ti) {
+            const uint32_t m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
+            const uint32_t acc = ti & 1u, aph = (ti >> 1) & 1u;
+            // warp-uniform outcome of the wait
+            if (!__all_sync(SLONN_FULL_MASK, mbar_wait(tfull0 + 8 * acc, aph, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t mrow0 = m0 + quarter * 32;
+            unsigned long long off = ~0ull; // ~0: row not present
+            if (mrow0 + lane < m_valid) {
+                const uint32_t src = E.row_map ? E.row_map[mrow0 + lane] : mrow0 + lane;
+                off = E.indptr ? E.indptr[(uint64_t)src * E.ip_mul + E.ip_add] : (uint64_t)src * E.f32_stride;
+            }
+            row_off[lane] = off;
+            __syncwarp();
+            for (uint32_t c = 0; c < (uint32_t)BN; c += 32) {
+                if (n0 + c >= N) break; // columns past the layer width (uniform)
+                uint32_t r[32];
+                tmem_load32(tmem_base + ((quarter * 32u) << 16) + acc * BN + c, r); // whole warp takes part
+#pragma unroll
+                for (int j = 0; j < 32; ++j) tile[lane * 33 + j] = __uint_as_float(r[j]);
+                __syncwarp();
+                const uint32_t n = n0 + c + lane;
+                const float bias = (E.bias && n < N) ? __ldg(E.bias + n) : 0.0f;
+#pragma unroll 4
+                for (int rr = 0; rr < 32; ++rr) {
+                    const unsigned long long ro = row_off[rr];
+                    if (ro == ~0ull || n >= N) continue;
+                    float v = tile[rr * 33 + lane] + bias;
+                    if (E.relu) v = v > 0.0f ? v : 0.0f;
+                    if (E.out_f32) E.out_f32[ro + n] = v;
+                    if (E.out_ids) E.out_ids[ro + n] = n;
+                    if (E.out_bf16) E.out_bf16[(uint64_t)(mrow0 + rr) * E.ld_bf16 + n] = f32_to_bf16_rne(v);
+                }
+                __syncwarp();
+            }
+            // this warp has read its part of the accumulator: hand it back to the MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+        }
     }
     __syncwarp();
-
-    // ---- epilogue: TMEM lane = row of the tile, TMEM column = column of the tile ----
-    const bool acc_ready = __all_sync(SLONN_FULL_MASK, mbar_wait(tmem_full, 0u, abort_flag)); // warp-uniform
-    tc_fence_after();
-    if (acc_ready) {
-        // Each lane reads one accumulator row (32 columns at a time); the warp then turns the 32x32
-        // block around in shared memory so that a store instruction covers 32 consecutive columns
-        // of one output row.
-        float *tile = reinterpret_cast<float *>(smem_raw + (epi_addr - smem_u32(smem_raw))) + warp * (32 * 33);
-        unsigned long long *row_off = reinterpret_cast<unsigned long long *>(
-            smem_raw + (epi_addr - smem_u32(smem_raw)) + 4 * (32 * 33) * sizeof(float)) + warp * 32;
-        const uint32_t m = m0 + warp * 32 + lane;
-        unsigned long long off = ~0ull; // ~0: row not present
-        if (m < m_valid) {
-            const uint32_t src = E.row_map ? E.row_map[m] : m;
-            off = E.indptr ? E.indptr[(uint64_t)src * E.ip_mul + E.ip_add] : (uint64_t)src * E.f32_stride;
-        }
-        row_off[lane] = off;
-        __syncwarp();
-        for (uint32_t c = 0; c < (uint32_t)BN; c += 32) {
-            uint32_t r[32];
-            tmem_load32(tmem_base + ((warp * 32u) << 16) + c, r); // whole warp takes part
-#pragma unroll
-            for (int j = 0; j < 32; ++j) tile[lane * 33 + j] = __uint_as_float(r[j]);
-            __syncwarp();
-            const uint32_t n = n0 + c + lane;
-            const float bias = (E.bias && n < N) ? __ldg(E.bias + n) : 0.0f;
-#pragma unroll 4
-            for (int rr = 0; rr < 32; ++rr) {
-                const unsigned long long ro = row_off[rr];
-                if (ro == ~0ull || n >= N) continue;
-                float v = tile[rr * 33 + lane] + bias;
-                if (E.relu) v = v > 0.0f ? v : 0.0f;
-                if (E.out_f32) E.out_f32[ro + n] = v;
-                if (E.out_ids) E.out_ids[ro + n] = n;
-                if (E.out_bf16) E.out_bf16[(uint64_t)(m0 + warp * 32 + rr) * E.ld_bf16 + n] = f32_to_bf16_rne(v);
-            }
-            __syncwarp();
-        }
-    }
     if (*abort_flag) {
         // a wait ran out: give copies that may still be in flight time to land before the block leaves
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-        if (threadIdx.x == 0 && E.status) slonn_report(E.status, SLONN_ERR_TIMEOUT, blockIdx.y, blockIdx.x);
+        if (threadIdx.x == 0 && E.status) slonn_report(E.status, SLONN_ERR_TIMEOUT, blockIdx.x, 0);
     }
     tc_fence_before();
     __syncthreads();
@@ -260,15 +294,15 @@ encode_tiled_fn get_encode()
     return fn;
 }
 
-// bf16 matrix [rows][cols] row-major, tiles of 128 rows x 64 columns, 128-byte swizzle, zero fill outside
-int make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols)
+// bf16 matrix [rows][cols] row-major, tiles of box_rows rows x 64 columns, 128-byte swizzle, zero fill outside
+int make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols, uint32_t box_rows)
 {
     encode_tiled_fn enc = get_encode();
     if (!enc) return SLONN_ERR_CUDA;
     if (((uintptr_t)ptr & 15u) || ((cols * 2) & 15u)) return SLONN_ERR_ALIGN;
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -284,16 +318,24 @@ int slonn_dense_tc_launch(const void *A, const void *W, uint32_t N, uint32_t K, 
     if (!A || !W || E.M == 0 || N == 0 || K == 0) return SLONN_ERR_ARG;
     CUtensorMap ma, mb;
     int rc;
-    if ((rc = make_map(&ma, A, E.M, K))) return rc;
-    if ((rc = make_map(&mb, W, N, K))) return rc;
+    if ((rc = make_map(&ma, A, E.M, K, BM))) return rc;
+    if ((rc = make_map(&mb, W, N, K, BN))) return rc;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(dense_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
             return SLONN_ERR_CUDA;
         attr_set = true;
     }
-    const dim3 grid((N + BN - 1) / BN, (E.M + BM - 1) / BM);
-    dense_tc_kernel<<<grid, 128, SMEM_BYTES, st>>>(ma, mb, E, N, K);
+    static int sm_count = 0;
+    if (sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 1)
+            return SLONN_ERR_CUDA;
+    }
+    const uint64_t tiles = (uint64_t)((N + BN - 1) / BN) * ((E.M + BM - 1) / BM);
+    const uint32_t grid = (uint32_t)std::min<uint64_t>(tiles, (uint64_t)sm_count); // one persistent block per SM
+    dense_tc_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, E, N, K);
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
