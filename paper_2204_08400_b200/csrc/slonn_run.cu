@@ -122,13 +122,16 @@ int launch_select_t(const slonn_select_params &P, uint32_t n, uint32_t threads, 
 }
 
 // Fewer queries than SMs: latency variant, one warp per hash row (at least 8, at most 32 warps).
-int launch_select(const slonn_model *m, const slonn_select_params &P, uint32_t n, cudaStream_t st)
+// Very long lists (thousands of positions to walk per query): the same variant with 1024 threads,
+// so that a selection step covers 1024 list positions.
+int launch_select(const slonn_model *m, const slonn_select_params &P, uint32_t n, uint32_t max_rows, cudaStream_t st)
 {
     const size_t smem = (size_t)P.D * 4 + (size_t)((P.N + 31) / 32) * 4;
     const bool bf = m->dtype == SLONN_BF16;
     const bool id16 = m->layer[P.layer].id_bytes == 2;
-    const bool lat = n <= 148;
-    const uint32_t threads = lat ? 32u * std::min(32u, std::max(8u, m->H)) : (uint32_t)SLONN_THREADS;
+    const bool few = n <= 148, long_lists = (uint64_t)max_rows * m->L >= 8192;
+    const bool lat = few || long_lists;
+    const uint32_t threads = long_lists ? 1024u : few ? 32u * std::min(32u, std::max(8u, m->H)) : (uint32_t)SLONN_THREADS;
     if (lat) {
         if (bf && id16) return launch_select_t<true, uint16_t, true>(P, n, threads, smem, st);
         if (bf) return launch_select_t<true, uint32_t, true>(P, n, threads, smem, st);
@@ -550,13 +553,13 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             sp.hash_nodes = ly.hash_nodes; sp.tables = ly.tables; sp.cap = ly.cap; sp.K = m->K; sp.L = m->L;
             sp.n_act = m->n_act; sp.a = a; sp.layer = l; sp.indptr = indptr; sp.out_ids = ids;
             sp.codes = b->codes; sp.status = b->status;
+            max_rows = slonn_budget_nodes(max_bp, ly.N);
             TIC(SLONN_STAGE_HASH_SELECT);
-            rc = launch_select(m, sp, n, st);
+            rc = launch_select(m, sp, n, max_rows, st);
             TOC();
             if (rc) return rc;
             gp.use_list = 1; gp.a = a; gp.out_vals = vals;
             if (is_last) { gp.out_dense = b->logits; gp.out_dense_ids = b->logit_ids; gp.out_stride = stride; }
-            max_rows = slonn_budget_nodes(max_bp, ly.N);
             TIC(SLONN_STAGE_GATHER_DOT);
             rc = launch_gather(m, gp, n, max_rows, st);
             TOC();

@@ -168,14 +168,25 @@ __device__ __forceinline__ bool block_select(const void *tables, uint32_t cap, u
     // time by warp 0, which cuts exactly at B.
     const uint32_t npos = B * L; // B distinct ids are always found within rank < B
     uint32_t total = 0;
-    for (uint32_t base = 0; base < npos; base += blockDim.x) {
+    uint32_t ahead[4] = {0, 0, 0, 0}; // list entries of this thread for the next four steps (one round trip)
+    uint32_t step = 0;
+    for (uint32_t base = 0; base < npos; base += blockDim.x, ++step) {
+        if ((step & 3u) == 0u) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t p = base + u * blockDim.x + threadIdx.x;
+                if (p < npos) {
+                    const uint32_t r = p / L, b = p - r * L;
+                    ahead[u] = table_entry<IDT>(tables, cap, K, b, keys[b], r);
+                }
+            }
+        }
         const uint32_t pos = base + threadIdx.x;
         const bool valid = pos < npos;
-        uint32_t id = 0;
+        const uint32_t id = ahead[0];
+        ahead[0] = ahead[1]; ahead[1] = ahead[2]; ahead[2] = ahead[3];
         bool won = false;
         if (valid) {
-            const uint32_t r = pos / L, b = pos - r * L;
-            id = table_entry<IDT>(tables, cap, K, b, keys[b], r);
             if (id < N) {
                 const uint32_t bit = 1u << (id & 31u);
                 won = (atomicOr(&bitmap[id >> 5], bit) & bit) == 0u;

@@ -311,3 +311,53 @@ def test_slonn_run_replays_from_a_cuda_graph():
         for k in ("logits", "pred", "codes", "active_ids", "active_vals"):
             assert np.array_equal(got[k], want[k]), (path, k)
     dm.free()
+
+
+def test_api_misuse_is_reported_by_error_codes():
+    import torch
+    from paper_2204_08400_b200 import binding as sl, harness
+    dev = torch.device("cuda:0")
+    W = [torch.zeros((16, 8), dtype=torch.float32, device=dev), torch.zeros((4, 16), dtype=torch.float32, device=dev)]
+    b = [torch.zeros(16, device=dev), torch.zeros(4, device=dev)]
+    calib = torch.zeros((10, 8), device=dev)
+
+    def build(**kw):
+        args = dict(dims=[8, 16, 4], has_activator=[1, 0], dtype=sl.SLONN_F32, W=W, bias=b, calib_dense=calib, K=2, L=2)
+        args.update(kw)
+        return sl.slonn_build(**args)
+
+    for kw, code in (
+        (dict(dtype=7), "DTYPE"),
+        (dict(K=0), "DIM"),
+        (dict(K=5, L=4), "DIM"),                                     # K*L = 20 hash nodes > 16 nodes
+        (dict(dims=[6, 16, 4]), "ALIGN"),                            # 6 floats = 24 bytes per row: not 16-byte rows
+        (dict(calib_dense=None), "ARG"),
+        (dict(first_layer_sparse=True), "ARG"),                      # a CSR first layer may not carry an activator
+        (dict(hash_nodes_override=[np.array([0, 1, 2, 2]), None]), "ARG"),   # repeated hash node
+        (dict(hash_nodes_override=[np.array([0, 1, 2, 99]), None]), "ARG"),  # node id out of range
+    ):
+        with pytest.raises(sl.SlonnError) as e:
+            build(**kw)
+        assert e.value.code == sl.ERR[code], (kw, e.value.code)
+
+    wl = custom_workload(64, [32, 64, 8], [1, 0], "f32", n=8, n_cal=80, K=2, L=2, budgets=(2500,))
+    dm = harness.DeviceModel(wl)
+    batch = harness.DeviceBatch(dm, wl.x, wl.budget_bp)
+    with pytest.raises(sl.SlonnError) as e:                          # workspace too small
+        sl.slonn_run(dm.model, batch.batch, batch.ws, batch.ws_bytes - 256)
+    assert e.value.code == sl.ERR["WORKSPACE"]
+    with pytest.raises(sl.SlonnError) as e:                          # misaligned workspace
+        sl.slonn_run(dm.model, batch.batch, batch.ws.data_ptr() + 16, batch.ws_bytes)
+    assert e.value.code == sl.ERR["WORKSPACE"]
+    bad = sl.make_batch(8, batch.bp, None, batch.status, x_dense=batch.x_dense, max_budget_bp=batch.max_bp)   # no logits
+    with pytest.raises(sl.SlonnError) as e:
+        sl.slonn_run(dm.model, bad, batch.ws, batch.ws_bytes)
+    assert e.value.code == sl.ERR["ARG"]
+    bad = sl.make_batch(8, batch.bp, batch.logits, batch.status, x_dense=batch.x_dense, max_budget_bp=batch.max_bp,
+                        kernel_path=9)
+    with pytest.raises(sl.SlonnError) as e:
+        sl.slonn_run(dm.model, bad, batch.ws, batch.ws_bytes)
+    assert e.value.code == sl.ERR["ARG"]
+    batch.run()                                                      # the model is still usable afterwards
+    assert batch.results()["status"][0] == 0
+    dm.free()
