@@ -109,6 +109,36 @@ __device__ __forceinline__ float reduce_rows4(const float (&a)[4], uint32_t lane
     return k;
 }
 
+// The same for 8 rows with 9 shuffles: after stride 16 a lane carries four of the rows, after
+// stride 8 two, after stride 4 one.  Returns the sum of row (lane >> 2); the 4 lanes of a group
+// hold the same value.
+__device__ __forceinline__ float reduce_rows8(const float (&a)[8], uint32_t lane)
+{
+    const bool hi16 = (lane & 16u) != 0u;
+    float k[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float keep = hi16 ? a[4 + i] : a[i];
+        const float send = hi16 ? a[i] : a[4 + i];
+        k[i] = keep + __shfl_xor_sync(SLONN_FULL_MASK, send, 16);
+    }
+    const bool hi8 = (lane & 8u) != 0u;
+    float m[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const float keep = hi8 ? k[2 + i] : k[i];
+        const float send = hi8 ? k[i] : k[2 + i];
+        m[i] = keep + __shfl_xor_sync(SLONN_FULL_MASK, send, 8);
+    }
+    const bool hi4 = (lane & 4u) != 0u;
+    float v = hi4 ? m[1] : m[0];
+    const float s4 = hi4 ? m[0] : m[1];
+    v = v + __shfl_xor_sync(SLONN_FULL_MASK, s4, 4);
+    v = v + __shfl_xor_sync(SLONN_FULL_MASK, v, 2);
+    v = v + __shfl_xor_sync(SLONN_FULL_MASK, v, 1);
+    return v;
+}
+
 // Where input element j lives in the staged copy of a query's input vector.
 // fp32 weights: plain order.  bf16 weights: a 16-byte weight chunk holds 8
 // elements, so the 8 matching inputs are split into two float4 planes (first

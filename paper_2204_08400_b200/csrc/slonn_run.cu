@@ -146,10 +146,10 @@ int launch_select(const slonn_model *m, const slonn_select_params &P, uint32_t n
 
 // Rows per block: whole queries per block once the batch alone fills the GPU,
 // smaller row chunks for small batches so that every SM gets work.
-void gather_shape(uint32_t n, uint32_t max_rows, uint32_t *rows_per_cta, uint32_t *ctas_per_query)
+void gather_shape(uint32_t n, uint32_t max_rows, uint32_t rows_per_pass, uint32_t *rows_per_cta, uint32_t *ctas_per_query)
 {
-    const uint32_t unit = (SLONN_THREADS / 32) * SLONN_ROWS_PER_WARP; // rows one block pass covers
-    const uint64_t want_ctas = 148ull * 16;                            // a few waves of resident blocks
+    const uint32_t unit = (SLONN_THREADS / 32) * rows_per_pass; // rows one block pass covers
+    const uint64_t want_ctas = 148ull * 16;                     // a few waves of resident blocks
     uint64_t total_rows = (uint64_t)n * max_rows;
     uint64_t rpc = (total_rows + want_ctas - 1) / want_ctas;
     rpc = std::max<uint64_t>(unit, (rpc + unit - 1) / unit * unit);
@@ -158,12 +158,12 @@ void gather_shape(uint32_t n, uint32_t max_rows, uint32_t *rows_per_cta, uint32_
     *ctas_per_query = (uint32_t)((max_rows + rpc - 1) / rpc);
 }
 
-template <bool BF16, bool LAT>
+template <bool BF16, bool LAT, int R>
 int launch_gather_t(const slonn_gather_params &P, uint64_t grid, uint32_t threads, size_t smem, cudaStream_t st)
 {
-    const int rc = set_smem(gather_dot_kernel<BF16, LAT>, smem);
+    const int rc = set_smem(gather_dot_kernel<BF16, LAT, R>, smem);
     if (rc) return rc;
-    gather_dot_kernel<BF16, LAT><<<(uint32_t)grid, threads, smem, st>>>(P);
+    gather_dot_kernel<BF16, LAT, R><<<(uint32_t)grid, threads, smem, st>>>(P);
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
@@ -171,20 +171,22 @@ int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint
 {
     // so few rows that the GPU cannot be filled: latency variant, 4 warps per block, one row per warp
     const bool lat = (uint64_t)n * max_rows <= 148ull * 64;
+    const bool short_rows = P.nchunks <= 32; // a row is one 512-byte round: 8 rows per warp pass
     uint32_t threads = SLONN_THREADS;
     if (lat) {
         threads = 128;
         P.rows_per_cta = 4;
         P.ctas_per_query = (max_rows + 3) / 4;
     } else {
-        gather_shape(n, max_rows, &P.rows_per_cta, &P.ctas_per_query);
+        gather_shape(n, max_rows, short_rows ? 8u : 4u, &P.rows_per_cta, &P.ctas_per_query);
     }
     const size_t smem = (size_t)P.D * 4;
     const uint64_t grid = (uint64_t)n * P.ctas_per_query;
     if (grid == 0 || grid > 0x7fffffffull) return SLONN_ERR_DIM;
     const bool bf = m->dtype == SLONN_BF16;
-    if (lat) return bf ? launch_gather_t<true, true>(P, grid, threads, smem, st) : launch_gather_t<false, true>(P, grid, threads, smem, st);
-    return bf ? launch_gather_t<true, false>(P, grid, threads, smem, st) : launch_gather_t<false, false>(P, grid, threads, smem, st);
+    if (lat) return bf ? launch_gather_t<true, true, 4>(P, grid, threads, smem, st) : launch_gather_t<false, true, 4>(P, grid, threads, smem, st);
+    if (short_rows) return bf ? launch_gather_t<true, false, 8>(P, grid, threads, smem, st) : launch_gather_t<false, false, 8>(P, grid, threads, smem, st);
+    return bf ? launch_gather_t<true, false, 4>(P, grid, threads, smem, st) : launch_gather_t<false, false, 4>(P, grid, threads, smem, st);
 }
 
 // ---- whole-network kernel for narrow layers -----------------------------------

@@ -8,7 +8,8 @@
 #include "slonn_common.cuh"
 
 #define SLONN_THREADS 256
-#define SLONN_ROWS_PER_WARP 4 // the 6-shuffle reduction (reduce_rows4) is written for 4 rows
+#define SLONN_ROWS_PER_WARP 4 // hash rows per warp pass (reduce_rows4)
+
 
 // ---------------------------------------------------------------------------
 // block-wide exclusive scan of one value per thread (blockDim.x <= 1024)
@@ -337,7 +338,9 @@ struct slonn_gather_params {
     uint32_t rows_per_cta, ctas_per_query;
 };
 
-template <bool BF16, bool LAT>
+// R: rows per warp pass, 4 (6-shuffle reduction) or 8 (9 shuffles; pays off for rows of one
+// 512-byte round, where the reduction is most of the work).
+template <bool BF16, bool LAT, int R>
 __global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_params P)
 {
     extern __shared__ float4 smem4[];
@@ -377,19 +380,29 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_
             }
         }
     } else
-    for (uint32_t r = r0 + warp * SLONN_ROWS_PER_WARP; r < r1; r += nwarps * SLONN_ROWS_PER_WARP) {
-        const uint4 *rows[SLONN_ROWS_PER_WARP];
+    for (uint32_t r = r0 + warp * R; r < r1; r += nwarps * R) {
+        const uint4 *rows[R];
 #pragma unroll
-        for (int k = 0; k < SLONN_ROWS_PER_WARP; ++k) {
+        for (int k = 0; k < R; ++k) {
             const uint32_t rr = min(r + k, r1 - 1);
             const uint32_t nd = P.use_list ? __ldg(P.ids + off + rr) : rr;
             rows[k] = reinterpret_cast<const uint4 *>(P.W) + (uint64_t)nd * P.nchunks;
         }
-        float acc[SLONN_ROWS_PER_WARP];
-        warp_dot_rows<BF16, SLONN_ROWS_PER_WARP>(rows, smem4, P.nchunks, lane, acc);
-        const float sum = reduce_rows4(acc, lane); // row r + (lane >> 3)
-        const uint32_t mr = r + (lane >> 3);
-        if ((lane & 7u) == 0u && mr < r1) {
+        float acc[R];
+        warp_dot_rows<BF16, R>(rows, smem4, P.nchunks, lane, acc);
+        float sum;
+        uint32_t mr;
+        bool writer;
+        if constexpr (R == 8) {
+            sum = reduce_rows8(acc, lane); // row r + (lane >> 2)
+            mr = r + (lane >> 2);
+            writer = (lane & 3u) == 0u;
+        } else {
+            sum = reduce_rows4(acc, lane); // row r + (lane >> 3)
+            mr = r + (lane >> 3);
+            writer = (lane & 7u) == 0u;
+        }
+        if (writer && mr < r1) {
             const uint32_t nd = P.use_list ? __ldg(P.ids + off + mr) : mr;
             float z = sum + __ldg(P.bias + nd);
             if (P.relu) z = z > 0.0f ? z : 0.0f;
