@@ -361,3 +361,45 @@ def test_api_misuse_is_reported_by_error_codes():
     batch.run()                                                      # the model is still usable afterwards
     assert batch.results()["status"][0] == 0
     dm.free()
+
+
+def test_many_tables_and_long_keys():
+    # K*L = 96 hash functions, 8 tables of 4096 buckets: most buckets are never reached and fall
+    # back to the global ranking
+    wl = custom_workload(65, [64, 128, 16], [1, 0], "f32", n=150, n_cal=300, K=12, L=8,
+                         budgets=(300, 2500, 10000))
+    check(wl)
+
+
+def test_node_id_width_switches_above_65536_nodes():
+    # 65,568 output nodes: the tables hold 32-bit ids (16-bit up to 65,536 nodes)
+    from paper_2204_08400_b200 import harness, binding as sl
+    wl = custom_workload(66, [32, 64, 65568], [0, 1], "f32", n=6, n_cal=48, K=2, L=2, budgets=(10, 100))
+    dm = harness.DeviceModel(wl)
+    assert sl.slonn_model_info(dm.model, 1)["id_bytes"] == 4
+    dm.free()
+    check(wl)
+    wl16 = custom_workload(67, [32, 64, 65536], [0, 1], "f32", n=4, n_cal=32, K=2, L=1, budgets=(10,))
+    dm = harness.DeviceModel(wl16)
+    assert sl.slonn_model_info(dm.model, 1)["id_bytes"] == 2
+    dm.free()
+    check(wl16)
+
+
+def test_csr_rows_empty_and_longer_than_one_tile():
+    # first layer fed by CSR rows: a query without any nonzero, and rows with 300 nonzeros
+    # (more than the 128 the kernel stages at a time)
+    import dataclasses
+    rng = np.random.default_rng(68)
+    base = wl_mod.load("c3", n_queries=8, n_cal=128, budget_bp=1000, dims=[4000, 64, 2000])
+
+    def rows(lengths):
+        ids, vals, ip = [], [], [0]
+        for n in lengths:
+            ids.append(np.sort(rng.choice(4000, n, replace=False)).astype(np.uint32))
+            vals.append(np.exp(rng.standard_normal(n)).astype(np.float32))
+            ip.append(ip[-1] + n)
+        return np.asarray(ip, np.uint64), np.concatenate(ids), np.concatenate(vals)
+
+    wl = dataclasses.replace(base, x=rows([300, 0, 75, 129, 128, 1, 257, 0]), calib=rows([75] * 100 + [300] * 28))
+    check(wl)
