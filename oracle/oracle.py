@@ -40,7 +40,8 @@ class _Batch(C.Structure):
 def lib():
     global _lib
     if _lib is None:
-        path = build_oracle.build()
+        # SLONN_ORACLE_LIB: another build of the oracle (the mutation tests point it at broken copies)
+        path = os.environ.get("SLONN_ORACLE_LIB") or build_oracle.build()
         L = C.CDLL(path)
         L.orc_dot_canon32.restype = C.c_float
         L.orc_dot_canon32.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_float]

@@ -403,3 +403,16 @@ def test_csr_rows_empty_and_longer_than_one_tile():
 
     wl = dataclasses.replace(base, x=rows([300, 0, 75, 129, 128, 1, 257, 0]), calib=rows([75] * 100 + [300] * 28))
     check(wl)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_zero_inputs_and_tied_logits(dtype):
+    # pre-activations of exactly 0 (hash bit 0, ReLU 0) and exactly equal logits (lowest id wins)
+    import dataclasses
+    wl = custom_workload(69, [64, 96, 16], [1, 0], dtype, n=48, n_cal=200, K=3, L=2, bias_scale=0.0)
+    for w in (wl.W_f32[1], wl.W_store[1]):
+        w[9] = w[2]; w[13] = w[2]                 # three identical output nodes
+    x = wl.x.copy()
+    x[::3] = 0.0                                  # every third query is all zeros
+    wl = dataclasses.replace(wl, x=x)
+    check(wl)

@@ -364,3 +364,36 @@ def test_canon32_and_ref64_decisions_agree_on_c1_like_workload():
     rel = np.max(np.abs(la - lb), axis=1) / np.maximum(np.max(np.abs(lb), axis=1), 1e-30)
     assert rel.max() < 1e-5
     assert np.array_equal(a["pred"][agree], b["pred"][agree])
+
+
+def test_zero_preactivation_gives_a_zero_hash_bit():
+    # FreeHash (Def. 2) is a sign; a pre-activation of exactly 0 is "not active", as for ReLU
+    rng = np.random.default_rng(50)
+    m = tiny_model(rng, [12, 24, 4], [1, 0], K=3, L=2, bias_scale=0.0)
+    m.build(calib_dense=relu_inputs(rng, 80, 12), seed=6)
+    x = np.zeros((3, 12), np.float32)                      # every pre-activation is exactly 0
+    for mode in (orc.CANON32, orc.REF64):
+        r = m.run(np.full(3, 2500, np.uint16), x_dense=x, mode=mode)
+        assert np.all(r["codes"] == 0)
+    # and a strictly positive one sets it
+    hn = m.hash_nodes(0)
+    x1 = np.zeros((1, 12), np.float32)
+    x1[0] = m.W[0][hn[0, 1]]                               # x parallel to hash function 1 of table 0
+    r = m.run(np.full(1, 2500, np.uint16), x_dense=x1)
+    assert (int(r["codes"][0, 0, 0]) >> 1) & 1 == 1
+
+
+def test_prediction_takes_the_lowest_id_among_equal_logits():
+    rng = np.random.default_rng(51)
+    m = tiny_model(rng, [10, 14, 6], [0, 0], K=2, L=1)
+    m.W[1][4] = m.W[1][1]; m.bias[1][4] = m.bias[1][1]      # outputs 1 and 4 are the same function
+    m.W[1][5] = m.W[1][1]; m.bias[1][5] = m.bias[1][1]
+    x = relu_inputs(rng, 40, 10)
+    for mode in (orc.CANON32, orc.REF64):
+        r = m.run(np.full(40, 10000, np.uint16), x_dense=x, mode=mode)
+        lg = r["logits"]
+        assert np.array_equal(lg[:, 1], lg[:, 4])
+        top_is_tied = np.argmax(lg, axis=1) == 1
+        assert top_is_tied.sum() >= 3                       # the tie decides the prediction for some inputs
+        assert np.array_equal(r["pred"], np.argmax(lg, axis=1).astype(np.uint32))   # numpy: first maximum
+        assert not np.any(np.isin(r["pred"], [4, 5]))
