@@ -119,6 +119,10 @@ _SPECS = {
                c_seed=102, law="u01_half_zero", n=65536, n_cal=16384, budgets=(500, 1000, 2500, 5000, 10000)),
     "c3": dict(dims=[100000, 128, 200000], has_act=[0, 1], dtype="f32", w_seed=20, x_seed=21,
                c_seed=103, law="sparse75", n=256, n_cal=16384, budgets=(100, 500, 1000)),
+    # like c3 with a 1,000,000-node output layer (512 MB of fp32 rows, four times the L2): the gathered rows
+    # come from HBM, not from cache.  Lists are capped at 10,000 entries (1 % of the layer).
+    "c3xl": dict(dims=[100000, 128, 1000000], has_act=[0, 1], dtype="f32", w_seed=22, x_seed=23,
+                 c_seed=106, law="sparse75", n=256, n_cal=2048, budgets=(10, 50, 100), list_cap=10000),
     "c4": dict(dims=[4096] + [4096] * 8 + [1000], has_act=[1] * 8 + [0], dtype="bf16", w_seed=3,
                x_seed=31, c_seed=104, law="relu_normal", n=4096, n_cal=8192, budgets=(1000, 2500, 5000)),
     "c5": dict(dims=[2048, 4096, 4096, 1000], has_act=[1, 1, 0], dtype="bf16", w_seed=40, x_seed=41,
@@ -154,5 +158,5 @@ def load(name: str, n_queries: Optional[int] = None, n_cal: Optional[int] = None
         bp = np.full(n, s["budgets"][0], dtype=np.uint16)
     return Workload(name=name, dims=dims_, has_act=has_act, dtype=s["dtype"], W_f32=W_f32,
                     W_store=W_store, bias=bias, first_sparse=first_sparse, calib=calib, x=x,
-                    budget_bp=bp, seed=s["w_seed"] + 1000, list_cap=list_cap,
+                    budget_bp=bp, seed=s["w_seed"] + 1000, list_cap=list_cap or s.get("list_cap", 0),
                     budgets_named=tuple(s["budgets"]))
