@@ -208,6 +208,24 @@ typedef struct {
 #define SLONN_PATH_FUSED 2   /* one warp per query through all layers: widths <= 1024 inputs, */
                              /* <= 4096 nodes per layer, dense first layer                    */
 
+/*
+ * Latency-Constrained Accuracy-Optimized budgets (Sec. 2.3, Eq. 3): for each query the largest
+ * profiled k whose predicted total time t0 + T(k, beta) meets the query's latency target tau.
+ *   profile_bp, profile_ms : [n_k] the latency profile T(k, beta) of the current co-location
+ *                            scenario: budgets in basis points and the measured latency of a
+ *                            batch at that budget (n_k <= 4096, any order)
+ *   t0, tau                : [n] time already spent on the query outside inference, and its
+ *                            latency target (same unit as profile_ms)
+ *   budget_bp              : [n] out: ready to be used as slonn_batch.budget_bp
+ *   feasible               : [n] out, nullable: 0 where no profiled k meets the target (Def. 1:
+ *                            the SLO cannot be fulfilled); such queries get the smallest profiled k
+ * All pointers are device pointers; asynchronous on `stream`.  The accuracy-constrained policy
+ * (ACLO, Eq. 2) needs Confidence tables trained on labelled data and is not part of this library.
+ */
+int slonn_lcao_budgets(const uint16_t *profile_bp, const float *profile_ms, uint32_t n_k,
+                       const float *t0, const float *tau, uint32_t n, uint16_t *budget_bp,
+                       uint8_t *feasible, void *stream);
+
 /* Number of entries active_ids / active_vals need for n queries at max_budget_bp. */
 int slonn_active_capacity(const slonn_model *m, uint32_t n_queries, uint32_t max_budget_bp,
                           uint64_t *entries);

@@ -72,6 +72,8 @@ def lib():
                                 C.c_uint32, C.c_uint64, C.c_void_p]
         L.orc_run.restype = C.c_int
         L.orc_run.argtypes = [C.c_void_p, C.POINTER(_Batch)]
+        L.orc_lcao_budgets.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32,
+                                       C.c_void_p, C.c_void_p]
         L.orc_threads.restype = C.c_int
         _lib = L
     return _lib
@@ -111,6 +113,15 @@ def sample_hash_nodes(var, H, seed, layer):
     out = np.empty(H, dtype=np.uint32)
     lib().orc_sample_hash_nodes(_p(var), var.size, H, seed, layer, _p(out))
     return out
+
+
+def lcao_budgets(profile_bp, profile_ms, t0, tau):
+    """Eq. 3: per query the largest profiled k with t0 + T(k) <= tau; returns (budget_bp, feasible)."""
+    pb = _arr(profile_bp, np.uint16); pm = _arr(profile_ms, np.float32)
+    t0 = _arr(t0, np.float32); tau = _arr(tau, np.float32)
+    out = np.zeros(t0.size, np.uint16); ok = np.zeros(t0.size, np.uint8)
+    lib().orc_lcao_budgets(_p(pb), _p(pm), pb.size, _p(t0), _p(tau), t0.size, _p(out), _p(ok))
+    return out, ok
 
 
 def threads():

@@ -621,3 +621,30 @@ int orc_threads(void) { return omp_get_max_threads(); }
 #else
 int orc_threads(void) { return 1; }
 #endif
+
+/* ------------------------------------------------------------------ */
+/* LCAO budget choice (Sec. 2.3, Eq. 3)                                */
+/* ------------------------------------------------------------------ */
+
+/* Latency-Constrained Accuracy-Optimized: the largest profiled k whose predicted total time
+ * t0 + T(k, beta) still meets the latency target tau.  profile_bp / profile_ms: the latency
+ * profile T(k, beta) of one co-location scenario at n_k settings of k.  When no setting meets
+ * the target the query cannot be served within its SLO (Def. 1): feasible = 0 and the smallest
+ * profiled k is returned. */
+void orc_lcao_budgets(const uint16_t *profile_bp, const float *profile_ms, uint32_t n_k, const float *t0,
+                      const float *tau, uint32_t n, uint16_t *budget_bp, uint8_t *feasible)
+{
+    for (uint32_t q = 0; q < n; ++q) {
+        int found = 0;
+        uint16_t best = 0, smallest = profile_bp[0];
+        for (uint32_t i = 0; i < n_k; ++i) {
+            if (profile_bp[i] < smallest) smallest = profile_bp[i];
+            if (t0[q] + profile_ms[i] <= tau[q] && (!found || profile_bp[i] > best)) {
+                best = profile_bp[i];
+                found = 1;
+            }
+        }
+        budget_bp[q] = found ? best : smallest;
+        feasible[q] = (uint8_t)found;
+    }
+}

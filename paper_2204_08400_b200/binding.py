@@ -21,7 +21,7 @@ EXPORTS = [
     "slonn_version", "slonn_strerror", "slonn_build", "slonn_model_info", "slonn_model_tables_to_host",
     "slonn_free", "slonn_active_capacity", "slonn_logit_stride", "slonn_workspace_bytes", "slonn_run",
     "slonn_run_timed", "slonn_run_static", "slonn_dense_layer", "slonn_serialized_bytes", "slonn_serialize",
-    "slonn_deserialize",
+    "slonn_deserialize", "slonn_lcao_budgets",
     "slonn_host_workspace_bytes", "slonn_run_host",
 ]
 
@@ -82,6 +82,9 @@ def lib():
         L.slonn_deserialize.restype = C.c_int
         L.slonn_deserialize.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.POINTER(C.c_void_p)]
+        L.slonn_lcao_budgets.restype = C.c_int
+        L.slonn_lcao_budgets.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32,
+                                         C.c_void_p, C.c_void_p, C.c_void_p]
         L.slonn_free.restype = None
         L.slonn_free.argtypes = [C.c_void_p]
         L.slonn_active_capacity.restype = C.c_int
@@ -231,6 +234,14 @@ def slonn_deserialize(blob: np.ndarray, W: List, bias: List, stream=None) -> Mod
     dims = np.frombuffer(blob[32:32 + 4 * 17].tobytes(), dtype=np.uint32)[: n_l + 1].tolist()
     has_act = blob[32 + 4 * 17: 32 + 4 * 17 + n_l].tolist()
     return Model(out.value, [list(W), list(bias)], dims, has_act, dtype, K, L, bool(first_sparse))
+
+
+def slonn_lcao_budgets(profile_bp, profile_ms, t0, tau, budget_bp, feasible=None, stream=None) -> None:
+    """Eq. 3 on the device: budget_bp[q] = largest profiled k with t0[q] + T(k) <= tau[q]."""
+    rc = lib().slonn_lcao_budgets(_ptr(profile_bp), _ptr(profile_ms), int(profile_bp.numel()), _ptr(t0), _ptr(tau),
+                                  int(t0.numel()), _ptr(budget_bp), _ptr(feasible), _stream_ptr(stream))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_lcao_budgets")
 
 
 def slonn_free(model: Model) -> None:

@@ -660,6 +660,19 @@ extern "C" int slonn_run_static(const slonn_model *m, const slonn_batch *b, void
     return run_impl(m, b, ws, SLONN_STATIC_WORKSPACE_BYTES, stream, nullptr);
 }
 
+// ---- budget policy ---------------------------------------------------------------
+
+extern "C" int slonn_lcao_budgets(const uint16_t *profile_bp, const float *profile_ms, uint32_t n_k, const float *t0,
+                                  const float *tau, uint32_t n, uint16_t *budget_bp, uint8_t *feasible, void *stream)
+{
+    if (!profile_bp || !profile_ms || !t0 || !tau || !budget_bp) return SLONN_ERR_ARG;
+    if (n_k == 0 || n_k > 4096) return SLONN_ERR_DIM;
+    if (n == 0) return SLONN_OK;
+    lcao_budget_kernel<<<(n + 255) / 256, 256, n_k * 6 + 8, (cudaStream_t)stream>>>(profile_bp, profile_ms, n_k, t0, tau, n,
+                                                                                    budget_bp, feasible);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
 // ---- host-buffer variant -----------------------------------------------------
 
 namespace {

@@ -584,3 +584,28 @@ __global__ void dense_codes_kernel(const uint32_t *list, const uint32_t *count, 
         if (v[hash_nodes[b * K + j]] > 0.0f) key |= (1u << j);
     codes[((uint64_t)q * n_act + a) * L + b] = (uint16_t)key;
 }
+
+
+// ---------------------------------------------------------------------------
+// LCAO (Eq. 3 of the paper): per query the largest profiled k with t0 + T(k) <= tau
+// ---------------------------------------------------------------------------
+__global__ void lcao_budget_kernel(const uint16_t *profile_bp, const float *profile_ms, uint32_t n_k, const float *t0,
+                                   const float *tau, uint32_t n, uint16_t *budget_bp, uint8_t *feasible)
+{
+    extern __shared__ float s_prof[]; // n_k latencies, then n_k budgets (as uint16)
+    uint16_t *s_bp = reinterpret_cast<uint16_t *>(s_prof + n_k);
+    for (uint32_t i = threadIdx.x; i < n_k; i += blockDim.x) { s_prof[i] = profile_ms[i]; s_bp[i] = profile_bp[i]; }
+    __syncthreads();
+    const uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= n) return;
+    const float base = t0[q], limit = tau[q];
+    bool found = false;
+    uint32_t best = 0, smallest = 0xffffu;
+    for (uint32_t i = 0; i < n_k; ++i) {
+        const uint32_t bp = s_bp[i];
+        smallest = min(smallest, bp);
+        if (__fadd_rn(base, s_prof[i]) <= limit && (!found || bp > best)) { best = bp; found = true; }
+    }
+    budget_bp[q] = (uint16_t)(found ? best : smallest);
+    if (feasible) feasible[q] = found ? 1 : 0;
+}

@@ -30,6 +30,8 @@ MUTANTS = {
     "generator constant mistyped": ("0xBF58476D1CE4E5B9ull", "0xBF58476D1CE4E5B1ull"),
     "hash bit of zero counts as set": ("node_z32_dense(m, l, h, in32)) > 0.0f;", "node_z32_dense(m, l, h, in32)) >= 0.0f;"),
     "scores summed in fp32": ("for (uint32_t i = 0; i < N; ++i) s[i] += (double)a[i];", "for (uint32_t i = 0; i < N; ++i) s[i] = (double)((float)s[i] + a[i]);"),
+    "LCAO takes the smallest feasible budget": ("(!found || profile_bp[i] > best)", "(!found || profile_bp[i] < best)"),
+    "LCAO ignores the time already spent": ("if (t0[q] + profile_ms[i] <= tau[q]", "if (profile_ms[i] <= tau[q]"),
     "argmax keeps the last maximum": ("if (ref ? (out64[n] > out64[best]) : (out32[n] > out32[best])) best = n;",
                                       "if (ref ? (out64[n] >= out64[best]) : (out32[n] >= out32[best])) best = n;"),
 }
@@ -47,6 +49,7 @@ def test_pins_catch_planted_mistake(name, tmp_path):
                     "-o", str(lib), str(src), "-lm"], check=True)
     env = dict(os.environ, SLONN_ORACLE_LIB=str(lib), OMP_NUM_THREADS="2")
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
-                        os.path.join(ROOT, "tests", "test_oracle_pins.py"), os.path.join(ROOT, "tests", "test_oracle_method.py")],
+                        os.path.join(ROOT, "tests", "test_oracle_pins.py"), os.path.join(ROOT, "tests", "test_oracle_method.py"),
+                        os.path.join(ROOT, "tests", "test_lcao.py"), "-m", "not gpu"],
                        env=env, cwd=ROOT, capture_output=True, text=True)
     assert r.returncode == 1, f"the pins did not notice: {name}\n{r.stdout[-600:]}"
