@@ -184,6 +184,7 @@ def main():
                     help="route 100 %% budget queries to the tensor-core dense path (not bit-exact for them)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-baseline", action="store_true", help="time the oracle also for workloads other than c1/c2")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -368,7 +369,10 @@ def main():
 
     # ---- the CPU oracle beside it (rank 0, single-GPU runs only) ----
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    # the oracle builds its own tables from the same calibration rows: seconds for c1/c2, many minutes for
+    # the wide networks, so those need --cpu-baseline (and usually --n-cal) to be asked for explicitly
+    want_cpu = args.cpu_baseline or (args.workload in ("c1", "c2") and not args.no_cpu_baseline)
+    if rank == 0 and world == 1 and want_cpu:
         qps, cores, n1, dt, _ = oracle_queries_per_sec(wl, None if not args.budget_bp else args.budget_bp)
         cpu = {"value": qps, "unit": "queries/s", "cores": cores, "kind": "oracle",
                "sample": f"first {n1} of {n} queries, {dt:.1f} s"}

@@ -122,14 +122,14 @@ int launch_select_t(const slonn_select_params &P, uint32_t n, uint32_t threads, 
 }
 
 // Fewer queries than SMs: latency variant, one warp per hash row (at least 8, at most 32 warps).
-// Very long lists (thousands of positions to walk per query): the same variant with 1024 threads,
+// Very long lists (tens of thousands of positions to walk per query): the same variant with 1024 threads,
 // so that a selection step covers 1024 list positions.
 int launch_select(const slonn_model *m, const slonn_select_params &P, uint32_t n, uint32_t max_rows, cudaStream_t st)
 {
     const size_t smem = (size_t)P.D * 4 + (size_t)((P.N + 31) / 32) * 4;
     const bool bf = m->dtype == SLONN_BF16;
     const bool id16 = m->layer[P.layer].id_bytes == 2;
-    const bool few = n <= 148, long_lists = (uint64_t)max_rows * m->L >= 8192;
+    const bool few = n <= 148, long_lists = (uint64_t)max_rows * m->L >= 32768;
     const bool lat = few || long_lists;
     const uint32_t threads = long_lists ? 1024u : few ? 32u * std::min(32u, std::max(8u, m->H)) : (uint32_t)SLONN_THREADS;
     if (lat) {
