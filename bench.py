@@ -136,6 +136,11 @@ def oracle_queries_per_sec(wl, budget_bp, target_seconds=12.0):
     return n1 / dt, orc.threads(), n1, dt, (om, xs, bp)
 
 
+def workload_label(args, wl):
+    return (f"{args.workload}: " + "-".join(map(str, wl.dims)) + f" {wl.dtype} weights, {wl.n_queries} queries/GPU, budget " +
+            (f"{args.budget_bp} bp" if args.budget_bp else "mixed 5/10/25/50/100 %") + f", K={wl.K} L={wl.L}")
+
+
 def run_reference(args, rank, world):
     if rank != 0:
         return
@@ -159,8 +164,8 @@ def run_reference(args, rank, world):
         "impl": "reference", "metric": "queries_per_sec_at_budget", "value": value, "unit": "queries/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: " + "-".join(map(str, wl.dims)) + f" {wl.dtype}, budget {args.budget_bp} bp",
-                   "queries_per_step": n1},
+        "config": {"workload": workload_label(args, wl), "queries_per_step_per_gpu": wl.n_queries,
+                   "budget_bp": args.budget_bp, "queries_timed_per_step": n1},
         "cpu_baseline": {"value": value, "unit": "queries/s", "cores": cores, "kind": "oracle",
                          "sample": f"first {n1} of {wl.n_queries} queries per step"},
         "e2e": {"value": value, "unit": "queries/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -383,9 +388,7 @@ def main():
             "metric": "queries_per_sec_at_budget", "value": value, "unit": "queries/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": esz_name, "data": "synthetic",
-            "config": {"workload": f"{args.workload}: " + "-".join(map(str, wl.dims)) +
-                                   f" {wl.dtype} weights, {n} queries/GPU, budget " +
-                                   (f"{args.budget_bp} bp" if args.budget_bp else "mixed 5/10/25/50/100 %") + f", K={wl.K} L={wl.L}",
+            "config": {"workload": workload_label(args, wl),
                        "queries_per_step_per_gpu": n, "budget_bp": args.budget_bp,
                        "l2": "inputs_larger_than_l2" if (wl.x.nbytes if not wl.first_sparse else 0) > L2_BYTES
                              else "weights_and_inputs_l2_resident",
