@@ -510,7 +510,8 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         memset(&ap, 0, sizeof(ap));
         ap.logits = b->logits; ap.stride = stride; ap.n = n; ap.pred = b->pred; ap.fixed_len = last.N;
         TIC(SLONN_STAGE_ARGMAX);
-        argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
+        if (stride >= 2048) argmax_block_kernel<<<n, 256, 0, st>>>(ap);
+        else argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
         TOC();
         return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
     }
@@ -592,7 +593,8 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             ap.fixed_len = last.N;
         }
         TIC(SLONN_STAGE_ARGMAX);
-        argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
+        if (stride >= 2048) argmax_block_kernel<<<n, 256, 0, st>>>(ap);
+        else argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
         TOC();
         if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
     }

@@ -462,18 +462,18 @@ __global__ void __launch_bounds__(128) sparse_first_layer_kernel(slonn_sparse_pa
         __syncthreads();
         if (n < P.N) {
             const uint32_t m = min(128u, nnz - base);
-#pragma unroll
-            for (uint32_t jb = 0; jb < 128; jb += 32) {
+            for (uint32_t jb = 0; jb < m; jb += 32) {
+                // 32 loads in flight (entries past the end re-read the last one and are not used)
+                float w[32];
 #pragma unroll
                 for (uint32_t p = 0; p < 32; ++p) {
-                    if (jb + p < m) {
-                        const uint64_t idx = (uint64_t)s_ids[jb + p] * P.N + n;
-                        float w;
-                        if (BF16) w = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(P.WT) + idx) << 16);
-                        else w = __ldg(reinterpret_cast<const float *>(P.WT) + idx);
-                        acc[p] = fmaf(w, s_vals[jb + p], acc[p]);
-                    }
+                    const uint64_t idx = (uint64_t)s_ids[min(jb + p, m - 1)] * P.N + n;
+                    if (BF16) w[p] = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(P.WT) + idx) << 16);
+                    else w[p] = __ldg(reinterpret_cast<const float *>(P.WT) + idx);
                 }
+#pragma unroll
+                for (uint32_t p = 0; p < 32; ++p)
+                    if (jb + p < m) acc[p] = fmaf(w[p], s_vals[jb + p], acc[p]);
             }
         }
     }
@@ -529,6 +529,49 @@ __global__ void __launch_bounds__(256) argmax_kernel(slonn_argmax_params P)
         P.pred[q] = P.logit_ids ? P.logit_ids[(uint64_t)q * P.stride + bi] : bi;
 }
 
+
+// The same with one block per query, for logit rows of thousands of entries.
+__global__ void __launch_bounds__(256) argmax_block_kernel(slonn_argmax_params P)
+{
+    __shared__ float wbest[8];
+    __shared__ uint32_t wbi[8];
+    const uint32_t q = blockIdx.x;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    uint32_t len = P.fixed_len;
+    if (P.indptr)
+        len = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - P.indptr[(uint64_t)q * P.n_act + P.a]);
+    const float *lg = P.logits + (uint64_t)q * P.stride;
+    float best = 0.0f;
+    uint32_t bi = 0xffffffffu;
+    for (uint32_t i0 = threadIdx.x; i0 < len; i0 += 8 * blockDim.x) {
+        float v[8]; // eight loads in flight per thread
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t i = i0 + u * blockDim.x;
+            v[u] = i < len ? lg[i] : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t i = i0 + u * blockDim.x;
+            if (i < len && (bi == 0xffffffffu || v[u] > best)) { best = v[u]; bi = i; }
+        }
+    }
+    for (int round = 0; round < 2; ++round) {
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            const float ob = __shfl_xor_sync(SLONN_FULL_MASK, best, off);
+            const uint32_t oi = __shfl_xor_sync(SLONN_FULL_MASK, bi, off);
+            if (oi != 0xffffffffu && (bi == 0xffffffffu || ob > best || (ob == best && oi < bi))) { best = ob; bi = oi; }
+        }
+        if (round == 1) break;
+        if (lane == 0) { wbest[warp] = best; wbi[warp] = bi; }
+        __syncthreads();
+        best = lane < (blockDim.x >> 5) ? wbest[lane] : 0.0f;
+        bi = lane < (blockDim.x >> 5) ? wbi[lane] : 0xffffffffu;
+    }
+    if (threadIdx.x == 0 && bi != 0xffffffffu)
+        P.pred[q] = P.logit_ids ? P.logit_ids[(uint64_t)q * P.stride + bi] : bi;
+}
 
 // ---------------------------------------------------------------------------
 // tensor-core route for 100 % budgets: which queries, their inputs as bf16 rows, their codes
