@@ -83,6 +83,7 @@ cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
         const slonn_cluster_layer &l0 = P.layer[0];
         const float4 *src = reinterpret_cast<const float4 *>(P.x + (uint64_t)q * l0.D);
         float4 *dst = reinterpret_cast<float4 *>(xbuf[0]);
+#pragma unroll 4
         for (uint32_t i = threadIdx.x; i < (l0.D >> 2); i += blockDim.x) {
             const float4 v = __ldg(src + i);
             if (BF16) dst[(i & 1u) * l0.nchunks + (i >> 1)] = v;

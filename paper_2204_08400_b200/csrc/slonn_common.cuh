@@ -241,6 +241,7 @@ __device__ __forceinline__ void stage_input(const slonn_input &in, uint32_t q, u
     const uint32_t nvec = D >> 2;
     if (in.kind == SLONN_IN_DENSE) {
         const float4 *src = reinterpret_cast<const float4 *>(in.dense + (uint64_t)q * D);
+#pragma unroll 4
         for (uint32_t i = threadIdx.x; i < nvec; i += blockDim.x) {
             const float4 v = __ldg(src + i);
             if (BF16) xs4[(i & 1u) * nchunks + (i >> 1)] = v;
@@ -253,6 +254,7 @@ __device__ __forceinline__ void stage_input(const slonn_input &in, uint32_t q, u
         const uint64_t s0 = in.indptr[(uint64_t)q * in.ip_mul + in.ip_add];
         const uint32_t len = (uint32_t)(in.indptr[(uint64_t)q * in.ip_mul + in.ip_add + 1] - s0);
         float *xs = reinterpret_cast<float *>(xs4);
+#pragma unroll 4
         for (uint32_t i = threadIdx.x; i < len; i += blockDim.x) {
             const uint32_t j = in.ids[s0 + i];
             if (j < D) xs[xs_index<BF16>(j, nchunks)] = in.vals[s0 + i];
