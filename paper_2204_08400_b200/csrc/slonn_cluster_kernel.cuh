@@ -40,7 +40,9 @@ struct slonn_cluster_params {
     slonn_cluster_layer layer[SLONN_MAX_LAYERS];
     uint32_t n_layers, n, n_act, K, L, cluster;
     const float *x;          // [n][D0]
-    const uint64_t *indptr;  // [n * n_act + 1]
+    const uint16_t *budget_bp; // [n]
+    uint32_t max_bp;
+    uint64_t *indptr_out;    // [n * n_act + 1], nullable: written for the caller (the kernel derives its own offsets)
     uint32_t *out_ids;       // CSR payload, nullable
     float *out_vals;         // CSR payload, nullable
     uint16_t *codes;         // nullable
@@ -53,6 +55,18 @@ struct slonn_cluster_params {
     uint32_t ids_cap;        // entries of the id list
     uint32_t bitmap_words;
 };
+
+// Node count of activator layer l for query q (same rule and the same clamping as the plan kernels).
+__device__ __forceinline__ uint32_t cluster_count(const slonn_cluster_params &P, uint32_t q, uint32_t l, bool *bad)
+{
+    uint32_t bp = P.budget_bp[q];
+    *bad = (bp < 1u) || (bp > 10000u) || (bp > P.max_bp);
+    if (bp < 1u) bp = 1u;
+    if (bp > P.max_bp) bp = P.max_bp;
+    const uint32_t B = slonn_budget_nodes(bp, P.layer[l].N);
+    if (B > P.layer[l].cap && B != P.layer[l].N) *bad = true;
+    return B;
+}
 
 template <bool BF16>
 __global__ void __launch_bounds__(SLONN_CLUSTER_THREADS, 1)
@@ -76,6 +90,27 @@ cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
     float *xbuf[2] = {reinterpret_cast<float *>(smem4), reinterpret_cast<float *>(smem4) + P.xbuf_floats};
     uint32_t *ids_s = reinterpret_cast<uint32_t *>(reinterpret_cast<float *>(smem4) + 2 * P.xbuf_floats);
     uint32_t *bitmap = ids_s + P.ids_cap;
+
+    // List offsets: with a handful of queries every block simply adds up the counts of the (query,
+    // layer) entries before its own instead of waiting for a separate planning launch.
+    __shared__ uint64_t s_off[SLONN_MAX_LAYERS];
+    __shared__ uint32_t s_cnt[SLONN_MAX_LAYERS];
+    if (threadIdx.x == 0) {
+        uint64_t run = 0;
+        bool bad;
+        for (uint32_t qq = 0; qq <= q; ++qq)
+            for (uint32_t l = 0; l < P.n_layers; ++l) {
+                if (!P.layer[l].has_act) continue;
+                const uint32_t B = cluster_count(P, qq, l, &bad);
+                if (qq == q) {
+                    s_off[l] = run; s_cnt[l] = B;
+                    if (bad && rank == 0) slonn_report(P.status, SLONN_ERR_BUDGET, q, l);
+                }
+                if (rank == 0 && q + 1 == P.n && P.indptr_out) P.indptr_out[(uint64_t)qq * P.n_act + P.layer[l].a] = run;
+                run += B;
+            }
+        if (rank == 0 && q + 1 == P.n && P.indptr_out) P.indptr_out[(uint64_t)P.n * P.n_act] = run;
+    }
 
     // input := x (every block its own copy, in the staging order of layer 0)
     uint32_t cur = 0;
@@ -108,8 +143,8 @@ cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
         uint64_t off = 0;
         uint32_t B = ly.N;
         if (ly.has_act) {
-            off = P.indptr[(uint64_t)q * P.n_act + ly.a];
-            B = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + ly.a + 1] - off);
+            off = s_off[l];
+            B = s_cnt[l];
             // 1. FreeHash rows, spread over the cluster; each sum goes to every block
             const uint32_t H = P.K * P.L;
             for (uint32_t h = gwarp; h < H; h += gwarps) {

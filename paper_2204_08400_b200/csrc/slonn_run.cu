@@ -303,7 +303,7 @@ int launch_cluster_t(const slonn_cluster_params &P, size_t smem, cudaStream_t st
     return cudaLaunchKernelEx(&cfg, cluster_network_kernel<BF16>, P) == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
-int launch_cluster(const slonn_model *m, const slonn_batch *b, const uint64_t *indptr, uint32_t stride, cudaStream_t st)
+int launch_cluster(const slonn_model *m, const slonn_batch *b, uint32_t max_bp, uint32_t stride, cudaStream_t st)
 {
     slonn_cluster_params P;
     memset(&P, 0, sizeof(P));
@@ -323,7 +323,7 @@ int launch_cluster(const slonn_model *m, const slonn_batch *b, const uint64_t *i
         }
     }
     P.n_layers = m->n_layers; P.n = b->n_queries; P.n_act = m->n_act; P.K = m->K; P.L = m->L; P.cluster = SLONN_CLUSTER_SIZE;
-    P.x = b->x_dense; P.indptr = indptr;
+    P.x = b->x_dense; P.budget_bp = b->budget_bp; P.max_bp = max_bp; P.indptr_out = b->active_indptr;
     P.out_ids = b->active_ids; P.out_vals = b->active_vals; P.codes = b->codes;
     P.logits = b->logits; P.logit_stride = stride; P.logit_ids = b->logit_ids; P.pred = b->pred;
     P.status = b->status;
@@ -420,6 +420,20 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     uint32_t stride = 0;
     slonn_logit_stride(m, max_bp, &stride);
 
+    // a handful of queries: one thread-block cluster per query, every layer in one launch (it derives the
+    // list offsets itself, so no planning launch either)
+    if (b->flags & ~SLONN_FLAG_DENSE_TC) return SLONN_ERR_ARG;
+    if (b->kernel_path > SLONN_PATH_CLUSTER) return SLONN_ERR_ARG;
+    if (b->kernel_path == SLONN_PATH_CLUSTER && (!cluster_eligible(m) || tc_route(m, max_bp, b->flags))) return SLONN_ERR_DIM;
+    if (b->kernel_path == SLONN_PATH_CLUSTER || (b->kernel_path == SLONN_PATH_AUTO && cluster_eligible(m) && n <= 4 && !tc_route(m, max_bp, b->flags) &&
+         cluster_max_rows(m, max_bp) <= 1024)) {
+        TIC(SLONN_STAGE_CLUSTER);
+        const int rc = launch_cluster(m, b, max_bp, stride, st);
+        TOC();
+        if (rc != SLONN_ERR_DIM || b->kernel_path == SLONN_PATH_CLUSTER) return rc;
+        // the device cannot co-schedule such a cluster: fall through to the other kernels
+    }
+
     // offsets of every (query, activator layer) list
     if (m->n_act) {
         slonn_plan_params pp;
@@ -483,18 +497,6 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         TOC();
         if (rc) return rc;
         skip_bp = b->budget_bp;
-    }
-
-    // a handful of queries: one thread-block cluster per query, every layer in one launch
-    if (b->kernel_path > SLONN_PATH_CLUSTER) return SLONN_ERR_ARG;
-    if (b->kernel_path == SLONN_PATH_CLUSTER && (!cluster_eligible(m) || skip_bp)) return SLONN_ERR_DIM;
-    if (b->kernel_path == SLONN_PATH_CLUSTER || (b->kernel_path == SLONN_PATH_AUTO && cluster_eligible(m) && n <= 4 && !skip_bp &&
-         cluster_max_rows(m, max_bp) <= 1024)) {
-        TIC(SLONN_STAGE_CLUSTER);
-        const int rc = launch_cluster(m, b, indptr, stride, st);
-        TOC();
-        if (rc != SLONN_ERR_DIM || b->kernel_path == SLONN_PATH_CLUSTER) return rc;
-        // the device cannot co-schedule such a cluster: fall through to the other kernels
     }
 
     // narrow networks with enough queries to fill the GPU: one warp per query, every layer in one launch
