@@ -164,68 +164,43 @@ __device__ __forceinline__ bool block_select(const void *tables, uint32_t cap, u
     }
 
     // (3)+(4) read the L lists rank by rank; the first B distinct ids are the active set.
-    // Position pos = rank * L + table.  A block-wide step marks blockDim.x positions
-    // at once; the step that would pass B is undone and replayed 32 positions at a
-    // time by warp 0, which cuts exactly at B.
+    // Position pos = rank * L + table.  Positions are taken strictly in order, in steps that
+    // never hold more positions than ids still missing (need = B - total): a step can then add at
+    // most `need` new ids, so the count never passes B, and when it reaches B the marked ids are
+    // exactly the distinct ids of a prefix of the position sequence -- the first B distinct ones.
+    // (Which of two equal ids inside a step wins the atomic does not matter: one does.)
+    // Each thread fetches its entries of the next four rows of blockDim.x positions in one go.
     const uint32_t npos = B * L; // B distinct ids are always found within rank < B
+    const uint32_t T = blockDim.x;
     uint32_t total = 0;
-    uint32_t ahead[4] = {0, 0, 0, 0}; // list entries of this thread for the next four steps (one round trip)
-    uint32_t step = 0;
-    for (uint32_t base = 0; base < npos; base += blockDim.x, ++step) {
-        if ((step & 3u) == 0u) {
+    (void)lane; (void)warp; (void)s_total;
+    for (uint32_t w0 = 0; w0 < npos && total < B; w0 += 4 * T) {
+        uint32_t ahead[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t p = base + u * blockDim.x + threadIdx.x;
-                if (p < npos) {
-                    const uint32_t r = p / L, b = p - r * L;
-                    ahead[u] = table_entry<IDT>(tables, cap, K, b, keys[b], r);
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t p = w0 + u * T + threadIdx.x;
+            if (p < npos) {
+                const uint32_t r = p / L, b = p - r * L;
+                ahead[u] = table_entry<IDT>(tables, cap, K, b, keys[b], r);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t row0 = w0 + u * T;              // this row holds positions row0 .. row0 + T - 1
+            const uint32_t row1 = min(row0 + T, npos);
+            const uint32_t mine = row0 + threadIdx.x;
+            uint32_t p = row0;
+            while (p < row1 && total < B) {                // uniform for the block
+                const uint32_t s = min(B - total, row1 - p);
+                bool won = false;
+                if (mine >= p && mine < p + s && ahead[u] < N) {
+                    const uint32_t bit = 1u << (ahead[u] & 31u);
+                    won = (atomicOr(&bitmap[ahead[u] >> 5], bit) & bit) == 0u;
                 }
+                total += (uint32_t)__syncthreads_count(won);
+                p += s;
             }
         }
-        const uint32_t pos = base + threadIdx.x;
-        const bool valid = pos < npos;
-        const uint32_t id = ahead[0];
-        ahead[0] = ahead[1]; ahead[1] = ahead[2]; ahead[2] = ahead[3];
-        bool won = false;
-        if (valid) {
-            if (id < N) {
-                const uint32_t bit = 1u << (id & 31u);
-                won = (atomicOr(&bitmap[id >> 5], bit) & bit) == 0u;
-            }
-        }
-        const uint32_t cnt = (uint32_t)__syncthreads_count(won);
-        if (total + cnt < B) { total += cnt; continue; }
-        if (total + cnt == B) { total = B; break; }
-        // crossing step: undo, then replay in order
-        if (won) atomicAnd(&bitmap[id >> 5], ~(1u << (id & 31u)));
-        __syncthreads();
-        if (warp == 0) {
-            for (uint32_t sub = 0; sub < blockDim.x && total < B; sub += 32) {
-                const uint32_t p2 = base + sub + lane;
-                const bool v2 = p2 < npos;
-                uint32_t id2 = 0xffffffffu - lane; // distinct dummies
-                bool fresh = false;
-                if (v2) {
-                    const uint32_t r = p2 / L, b = p2 - r * L;
-                    id2 = table_entry<IDT>(tables, cap, K, b, keys[b], r);
-                    if (id2 < N) fresh = ((bitmap[id2 >> 5] >> (id2 & 31u)) & 1u) == 0u;
-                }
-                const uint32_t same = __match_any_sync(SLONN_FULL_MASK, id2);
-                const bool first = (uint32_t)(__ffs(same) - 1) == lane;
-                const bool take = fresh && first;
-                const uint32_t bal = __ballot_sync(SLONN_FULL_MASK, take);
-                const uint32_t need = B - total;
-                const uint32_t rank = __popc(bal & ((1u << lane) - 1u));
-                if (take && rank < need) atomicOr(&bitmap[id2 >> 5], 1u << (id2 & 31u));
-                const uint32_t c = (uint32_t)__popc(bal);
-                total += c < need ? c : need;
-                __syncwarp();
-            }
-            if (lane == 0) *s_total = total;
-        }
-        __syncthreads();
-        total = *s_total;
-        break;
     }
     __syncthreads();
     if (total != B) { // cannot happen with well-formed tables; keep the output in range
