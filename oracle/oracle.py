@@ -56,6 +56,9 @@ def lib():
                                     C.c_uint32, C.c_uint32, C.c_int]
         L.orc_model_set_layer.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
         L.orc_model_keep_scores.argtypes = [C.c_void_p, C.c_int]
+        L.orc_model_set_free_hash_nodes.argtypes = [C.c_void_p, C.c_int]
+        L.orc_layer_nodes.restype = C.c_uint32
+        L.orc_layer_nodes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32]
         L.orc_model_free.argtypes = [C.c_void_p]
         for name, rt in (("orc_model_hash_nodes", C.c_void_p), ("orc_model_rank", C.c_void_p),
                          ("orc_model_var", C.c_void_p), ("orc_model_score", C.c_void_p),
@@ -130,15 +133,18 @@ def threads():
 
 class OracleModel:
     """dims = [D0, N1, ..., N_out]; W[l] float32 [N_l, D_l] (bf16 weights widened
-    exactly); V = 4 for fp32 storage, 8 for bf16 storage."""
+    exactly); V = 4 for fp32 storage, 8 for bf16 storage.  free_hash_nodes: the variant in which
+    a layer's K*L hash nodes are always active and are left out of its ranked lists."""
 
-    def __init__(self, dims, has_act, W, bias, V, K=10, L=2, list_cap=0, first_sparse=False):
+    def __init__(self, dims, has_act, W, bias, V, K=10, L=2, list_cap=0, first_sparse=False,
+                 free_hash_nodes=False):
         self.dims = [int(d) for d in dims]
         self.n_layers = len(self.dims) - 1
         self.has_act = [int(bool(h)) for h in has_act]
         self.n_act = sum(self.has_act)
         self.K, self.L, self.V = int(K), int(L), int(V)
         self.first_sparse = bool(first_sparse)
+        self.free_hash_nodes = bool(free_hash_nodes)
         self.W = [_arr(w, np.float32) for w in W]
         self.bias = [_arr(b, np.float32) for b in bias]
         for l in range(self.n_layers):
@@ -152,6 +158,7 @@ class OracleModel:
             raise ValueError("orc_model_new rejected the arguments")
         for l in range(self.n_layers):
             lib().orc_model_set_layer(self._m, l, _p(self.W[l]), _p(self.bias[l]))
+        lib().orc_model_set_free_hash_nodes(self._m, int(self.free_hash_nodes))
 
     def __del__(self):
         if getattr(self, "_m", None):
@@ -223,7 +230,7 @@ class OracleModel:
     def budgets(self, budget_bp):
         """[n, n_act] node counts per query and activator layer."""
         act_N = [self.dims[l + 1] for l in range(self.n_layers) if self.has_act[l]]
-        return np.array([[budget_nodes(bp, N) for N in act_N] for bp in np.asarray(budget_bp)],
+        return np.array([[int(lib().orc_layer_nodes(self._m, int(bp), N)) for N in act_N] for bp in np.asarray(budget_bp)],
                         dtype=np.int64).reshape(len(budget_bp), len(act_N))
 
     def run(self, budget_bp, x_dense=None, x_csr=None, mode=CANON32):

@@ -112,6 +112,9 @@ typedef struct orc_model {
     uint32_t K, L;         /* key bits per table, number of tables */
     uint32_t list_cap;     /* 0 => full permutation */
     int first_sparse;      /* layer 0 takes a sparse operand (id-ascending list) */
+    int free_hash_nodes;   /* variant of Sec. 3.4: the K*L hash nodes of a layer are always part of
+                            * its active set (their pre-activations are computed for the keys anyway)
+                            * and never appear in its ranked lists; the budget counts list nodes only */
     const float *W[ORC_MAX_LAYERS];    /* row-major [N_l][D_l], referenced */
     const float *bias[ORC_MAX_LAYERS]; /* [N_l], referenced */
     uint32_t *hash_nodes[ORC_MAX_LAYERS]; /* [L*K]; draw b*K+j = function j of table b */
@@ -143,6 +146,19 @@ void orc_model_set_layer(orc_model *m, uint32_t l, const float *W, const float *
 }
 
 void orc_model_keep_scores(orc_model *m, int keep) { m->keep_scores = keep; }
+void orc_model_set_free_hash_nodes(orc_model *m, int on) { m->free_hash_nodes = on; }
+
+/* Nodes computed in a layer of N nodes at budget bp: the budget's node count, and in the
+ * free-hash-node variant that many list nodes (at most the N - K*L non-hash nodes) plus the
+ * K*L hash nodes. */
+uint32_t orc_layer_nodes(const orc_model *m, uint32_t bp, uint32_t N)
+{
+    const uint32_t B = orc_budget_nodes(bp, N);
+    if (!m->free_hash_nodes) return B;
+    const uint32_t H = m->K * m->L;
+    const uint32_t rest = N - H;
+    return (B < rest ? B : rest) + H;
+}
 
 void orc_model_free(orc_model *m)
 {
@@ -292,7 +308,9 @@ static int train_layer_tables(orc_model *m, uint32_t l, const float *A, uint32_t
     const uint32_t N = m->dims[l + 1], K = m->K, L = m->L, H = K * L;
     const uint32_t nb = 1u << K;
     if (H > N) return ORC_ERR_ARG;
-    const uint32_t cap = (m->list_cap == 0 || m->list_cap > N) ? N : m->list_cap;
+    /* lists hold every node, or in the free-hash-node variant every node that is not a hash node */
+    const uint32_t listable = m->free_hash_nodes ? N - H : N;
+    const uint32_t cap = (m->list_cap == 0 || m->list_cap > listable) ? listable : m->list_cap;
 
     /* variance of each node's activation over the calibration set (population,
      * two-pass, fp64, sample order) */
@@ -345,21 +363,32 @@ static int train_layer_tables(orc_model *m, uint32_t l, const float *A, uint32_t
     m->rank[l] = (uint32_t *)malloc(sizeof(uint32_t) * (uint64_t)L * nb * cap);
     uint32_t *glist = (uint32_t *)malloc(sizeof(uint32_t) * N);
     if (!m->rank[l] || !glist) return ORC_ERR_NOMEM;
+    uint8_t *is_hash = (uint8_t *)calloc(N, 1);
+    if (!is_hash) return ORC_ERR_NOMEM;
+    if (m->free_hash_nodes) for (uint32_t h = 0; h < H; ++h) is_hash[hn[h]] = 1;
     for (uint32_t i = 0; i < N; ++i) glist[i] = i;
     { sort_ctx c = { global }; qsort_r(glist, N, sizeof(uint32_t), cmp_rank, &c); }
     int err = ORC_OK;
 #pragma omp parallel for schedule(dynamic)
     for (uint32_t bk = 0; bk < L * nb; ++bk) {
         uint32_t *dst = m->rank[l] + (uint64_t)bk * cap;
-        if (count[bk] == 0) { memcpy(dst, glist, sizeof(uint32_t) * cap); continue; }
-        uint32_t *perm = (uint32_t *)malloc(sizeof(uint32_t) * N);
-        if (!perm) { err = ORC_ERR_NOMEM; continue; }
-        for (uint32_t i = 0; i < N; ++i) perm[i] = i;
-        sort_ctx c = { score + (uint64_t)bk * N };
-        qsort_r(perm, N, sizeof(uint32_t), cmp_rank, &c);
-        memcpy(dst, perm, sizeof(uint32_t) * cap);
+        const uint32_t *src = glist;
+        uint32_t *perm = NULL;
+        if (count[bk] != 0) {
+            perm = (uint32_t *)malloc(sizeof(uint32_t) * N);
+            if (!perm) { err = ORC_ERR_NOMEM; continue; }
+            for (uint32_t i = 0; i < N; ++i) perm[i] = i;
+            sort_ctx c = { score + (uint64_t)bk * N };
+            qsort_r(perm, N, sizeof(uint32_t), cmp_rank, &c);
+            src = perm;
+        }
+        /* the first cap listable nodes of the ranking, in ranking order */
+        uint32_t o = 0;
+        for (uint32_t i = 0; i < N && o < cap; ++i)
+            if (!is_hash[src[i]]) dst[o++] = src[i];
         free(perm);
     }
+    free(is_hash);
     free(glist); free(global);
     m->cap[l] = cap;
     free(m->bucket_count[l]); m->bucket_count[l] = count;
@@ -444,6 +473,33 @@ static int select_active(const orc_model *m, uint32_t l, const uint32_t *keys, u
     uint32_t o = 0;
     for (uint32_t i = 0; i < N; ++i) if (seen[i]) out_ids[o++] = i;
     return (int)B;
+}
+
+/* The same in the free-hash-node variant: the layer's K*L hash nodes, plus the first
+ * min(B, N - K*L) distinct ids of the rank-interleaved lists (which hold no hash node), ascending.
+ * Returns the number of ids, or a negative error. */
+static int select_active_free(const orc_model *m, uint32_t l, const uint32_t *keys, uint32_t B,
+                              uint32_t *out_ids, uint8_t *seen /* [N] scratch */)
+{
+    const uint32_t N = m->dims[l + 1], L = m->L, nb = 1u << m->K, cap = m->cap[l], H = m->K * m->L;
+    const uint32_t want = B < N - H ? B : N - H;
+    memset(seen, 0, N);
+    for (uint32_t h = 0; h < H; ++h) seen[m->hash_nodes[l][h]] = 1;
+    if (want == N - H) {
+        for (uint32_t i = 0; i < N; ++i) out_ids[i] = i;
+        return (int)N;
+    }
+    if (want > cap) return ORC_ERR_BUDGET;
+    uint32_t got = 0;
+    for (uint32_t r = 0; r < cap && got < want; ++r)
+        for (uint32_t b = 0; b < L && got < want; ++b) {
+            uint32_t id = m->rank[l][((uint64_t)b * nb + keys[b]) * cap + r];
+            if (!seen[id]) { seen[id] = 1; ++got; }
+        }
+    if (got < want) return ORC_ERR_BUDGET;
+    uint32_t o = 0;
+    for (uint32_t i = 0; i < N; ++i) if (seen[i]) out_ids[o++] = i;
+    return (int)o;
 }
 
 typedef struct {
@@ -532,8 +588,10 @@ static int run_query(const orc_model *m, const orc_batch *bt, uint32_t q)
             }
             /* (3) ranked lists -> top-k% */
             B = orc_budget_nodes(bp, N);
-            int s = select_active(m, l, keys, B, ids, seen);
+            int s = m->free_hash_nodes ? select_active_free(m, l, keys, B, ids, seen)
+                                       : select_active(m, l, keys, B, ids, seen);
             if (s < 0) { rc = s; goto done; }
+            B = (uint32_t)s; /* nodes to compute */
         } else {
             for (uint32_t i = 0; i < N; ++i) ids[i] = i;
         }
@@ -596,7 +654,7 @@ int orc_run(const orc_model *m, const orc_batch *bt)
             for (uint32_t l = 0; l < m->n_layers; ++l) {
                 if (!m->has_act[l]) continue;
                 bt->active_indptr[(uint64_t)q * n_act + a] = off;
-                off += orc_budget_nodes(bt->budget_bp[q], m->dims[l + 1]);
+                off += orc_layer_nodes(m, bt->budget_bp[q], m->dims[l + 1]);
                 ++a;
             }
         }

@@ -25,8 +25,10 @@ MUTANTS = {
     "hidden activation not rectified": ("return z > 0.0f ? z : 0.0f;", "return z;"),
     "sample variance instead of population variance": ("for (uint32_t i = 0; i < N; ++i) var[i] = var[i] / (double)n_cal;",
                                                        "for (uint32_t i = 0; i < N; ++i) var[i] = var[i] / (double)(n_cal - 1);"),
-    "empty buckets get the identity order": ("if (count[bk] == 0) { memcpy(dst, glist, sizeof(uint32_t) * cap); continue; }",
-                                             "if (count[bk] == 0) { for (uint32_t i = 0; i < cap; ++i) dst[i] = i; continue; }"),
+    "empty buckets get the identity order": ("{ sort_ctx c = { global }; qsort_r(glist, N, sizeof(uint32_t), cmp_rank, &c); }", "{ }"),
+    "free variant: hash nodes stay in the lists": ("if (!is_hash[src[i]]) dst[o++] = src[i];", "dst[o++] = src[i];"),
+    "free variant: hash nodes missing from the active set": ("for (uint32_t h = 0; h < H; ++h) seen[m->hash_nodes[l][h]] = 1;\n    if (want", "if (want"),
+    "free variant: the budget counts the hash nodes": ("const uint32_t want = B < N - H ? B : N - H;", "const uint32_t want = B > H ? (B - H < N - H ? B - H : N - H) : 0;"),
     "generator constant mistyped": ("0xBF58476D1CE4E5B9ull", "0xBF58476D1CE4E5B1ull"),
     "hash bit of zero counts as set": ("node_z32_dense(m, l, h, in32)) > 0.0f;", "node_z32_dense(m, l, h, in32)) >= 0.0f;"),
     "scores summed in fp32": ("for (uint32_t i = 0; i < N; ++i) s[i] += (double)a[i];", "for (uint32_t i = 0; i < N; ++i) s[i] = (double)((float)s[i] + a[i]);"),
@@ -50,6 +52,7 @@ def test_pins_catch_planted_mistake(name, tmp_path):
     env = dict(os.environ, SLONN_ORACLE_LIB=str(lib), OMP_NUM_THREADS="2")
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
                         os.path.join(ROOT, "tests", "test_oracle_pins.py"), os.path.join(ROOT, "tests", "test_oracle_method.py"),
-                        os.path.join(ROOT, "tests", "test_lcao.py"), "-m", "not gpu"],
+                        os.path.join(ROOT, "tests", "test_lcao.py"), os.path.join(ROOT, "tests", "test_oracle_free_hash.py"),
+                        "-m", "not gpu"],
                        env=env, cwd=ROOT, capture_output=True, text=True)
     assert r.returncode == 1, f"the pins did not notice: {name}\n{r.stdout[-600:]}"
