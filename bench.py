@@ -138,14 +138,15 @@ def oracle_queries_per_sec(wl, budget_bp, target_seconds=12.0):
 
 def workload_label(args, wl):
     return (f"{args.workload}: " + "-".join(map(str, wl.dims)) + f" {wl.dtype} weights, {wl.n_queries} queries/GPU, budget " +
-            (f"{args.budget_bp} bp" if args.budget_bp else "mixed 5/10/25/50/100 %") + f", K={wl.K} L={wl.L}")
+            (f"{args.budget_bp} bp" if args.budget_bp else "mixed 5/10/25/50/100 %") + f", K={wl.K} L={wl.L}" +
+            (", hash nodes always active" if wl.free_hash_nodes else ""))
 
 
 def run_reference(args, rank, world):
     if rank != 0:
         return
     wl = workloads.load(args.workload, n_queries=args.queries, n_cal=args.n_cal,
-                        budget_bp=args.budget_bp if args.budget_bp else None)
+                        budget_bp=args.budget_bp if args.budget_bp else None, free_hash_nodes=args.free_hash_nodes)
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     from oracle import oracle as orc
     from parity_util import oracle_run
@@ -187,6 +188,8 @@ def main():
     ap.add_argument("--n-cal", type=int, default=None)
     ap.add_argument("--dense-tc", action="store_true",
                     help="route 100 %% budget queries to the tensor-core dense path (not bit-exact for them)")
+    ap.add_argument("--free-hash-nodes", action="store_true",
+                    help="the variant in which a layer's K*L hash nodes are always active and absent from its lists")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline", action="store_true", help="time the oracle also for workloads other than c1/c2")
@@ -217,7 +220,7 @@ def main():
     # every rank is a replica with its own batch (same law, rank-specific seed is not needed:
     # throughput does not depend on the draw; parity tests cover the values)
     wl = workloads.load(args.workload, n_queries=args.queries, n_cal=args.n_cal,
-                        budget_bp=args.budget_bp if args.budget_bp else None)
+                        budget_bp=args.budget_bp if args.budget_bp else None, free_hash_nodes=args.free_hash_nodes)
     max_bp = int(wl.budget_bp.max())
     n = wl.n_queries
     dm = harness.DeviceModel(wl, device=dev)

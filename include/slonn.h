@@ -83,6 +83,12 @@ typedef struct {
                                    /*    then carry no activator; calibration is CSR as well  */
     const uint32_t *const *hash_nodes_override; /* host, nullable; per layer nullable: L*K    */
                                    /* distinct node ids to use instead of sampling            */
+    uint32_t free_hash_nodes;      /* 1: the variant of Sec. 3.4 in which a hash function's   */
+                                   /*    dot product doubles as its node's output: a layer's  */
+                                   /*    K*L hash nodes are always in its active set and are  */
+                                   /*    left out of its ranked lists; the budget then counts */
+                                   /*    list nodes only, so a layer computes                 */
+                                   /*    min(B, N - K*L) + K*L nodes.  Needs K*L < N_l.       */
 } slonn_build_desc;
 
 typedef struct {
@@ -158,8 +164,9 @@ typedef struct {
     const uint32_t *x_ids;
     const float *x_vals;
     const uint16_t *budget_bp;     /* [n] per-query budget k in basis points, 1..10000;       */
-                                   /* node count per activator layer = max(1, round half up   */
-                                   /* of bp * N_l / 10000)                                    */
+                                   /* node count per activator layer B = max(1, round half up */
+                                   /* of bp * N_l / 10000); free_hash_nodes models compute    */
+                                   /* min(B, N_l - K*L) listed nodes plus the K*L hash nodes  */
     uint32_t max_budget_bp;        /* HOST value: upper bound of budget_bp[] (0 = 10000);     */
                                    /* sizes the launch grids, the workspace and logit_stride  */
     /* outputs (nullable unless stated) */

@@ -36,7 +36,7 @@ class _BuildDesc(C.Structure):
     _fields_ = [("n_layers", C.c_uint32), ("dims", C.c_void_p), ("has_activator", C.c_void_p),
                 ("dtype", C.c_int32), ("K", C.c_uint32), ("L", C.c_uint32), ("list_cap", C.c_uint32),
                 ("seed", C.c_uint64), ("first_layer_sparse", C.c_uint32),
-                ("hash_nodes_override", C.c_void_p)]
+                ("hash_nodes_override", C.c_void_p), ("free_hash_nodes", C.c_uint32)]
 
 
 class _Rows(C.Structure):
@@ -141,7 +141,7 @@ def strerror(code: int) -> str:
 class Model:
     """Handle of a built model; keeps the referenced weight tensors alive."""
 
-    def __init__(self, handle, keep, dims, has_activator, dtype, K, L, first_layer_sparse):
+    def __init__(self, handle, keep, dims, has_activator, dtype, K, L, first_layer_sparse, free_hash_nodes=False):
         self.handle = handle
         self._keep = keep
         self.dims = list(dims)
@@ -149,6 +149,7 @@ class Model:
         self.n_act = sum(1 for h in has_activator if h)
         self.dtype, self.K, self.L = dtype, K, L
         self.first_layer_sparse = first_layer_sparse
+        self.free_hash_nodes = free_hash_nodes
 
     def free(self):
         if self.handle:
@@ -164,7 +165,8 @@ class Model:
 
 def slonn_build(dims: Sequence[int], has_activator: Sequence[int], dtype: int, W: List, bias: List,
                 calib_dense=None, calib_csr=None, K: int = 10, L: int = 2, list_cap: int = 0, seed: int = 0,
-                first_layer_sparse: bool = False, hash_nodes_override=None, stream=None) -> Model:
+                first_layer_sparse: bool = False, hash_nodes_override=None, stream=None,
+                free_hash_nodes: bool = False) -> Model:
     """W[l], bias[l], calib_*: device tensors (W as float32 or as uint16/bfloat16 bit patterns)."""
     n_layers = len(dims) - 1
     d = np.asarray(dims, dtype=np.uint32)
@@ -179,6 +181,7 @@ def slonn_build(dims: Sequence[int], has_activator: Sequence[int], dtype: int, W
     desc.dtype = dtype
     desc.K, desc.L, desc.list_cap, desc.seed = K, L, list_cap, seed
     desc.first_layer_sparse = int(bool(first_layer_sparse))
+    desc.free_hash_nodes = int(bool(free_hash_nodes))
     ov_keep = []
     if hash_nodes_override is not None:
         ov = (C.c_void_p * n_layers)()
@@ -202,7 +205,7 @@ def slonn_build(dims: Sequence[int], has_activator: Sequence[int], dtype: int, W
                            _stream_ptr(stream), C.byref(out))
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_build")
-    return Model(out.value, keep, dims, has_activator, dtype, K, L, bool(first_layer_sparse))
+    return Model(out.value, keep, dims, has_activator, dtype, K, L, bool(first_layer_sparse), bool(free_hash_nodes))
 
 
 def slonn_serialize(model: Model) -> np.ndarray:
@@ -229,11 +232,12 @@ def slonn_deserialize(blob: np.ndarray, W: List, bias: List, stream=None) -> Mod
                                  _stream_ptr(stream), C.byref(out))
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_deserialize")
-    hdr = np.frombuffer(blob[:32].tobytes(), dtype=np.uint32)
-    n_l, dtype, K, L, first_sparse = int(hdr[2]), int(hdr[3]), int(hdr[4]), int(hdr[5]), int(hdr[7])
-    dims = np.frombuffer(blob[32:32 + 4 * 17].tobytes(), dtype=np.uint32)[: n_l + 1].tolist()
-    has_act = blob[32 + 4 * 17: 32 + 4 * 17 + n_l].tolist()
-    return Model(out.value, [list(W), list(bias)], dims, has_act, dtype, K, L, bool(first_sparse))
+    hdr = np.frombuffer(blob[:36].tobytes(), dtype=np.uint32)
+    n_l, dtype, K, L, first_sparse, free_hash = (int(hdr[2]), int(hdr[3]), int(hdr[4]), int(hdr[5]), int(hdr[7]),
+                                                 int(hdr[8]))
+    dims = np.frombuffer(blob[36:36 + 4 * 17].tobytes(), dtype=np.uint32)[: n_l + 1].tolist()
+    has_act = blob[36 + 4 * 17: 36 + 4 * 17 + n_l].tolist()
+    return Model(out.value, [list(W), list(bias)], dims, has_act, dtype, K, L, bool(first_sparse), bool(free_hash))
 
 
 def slonn_lcao_budgets(profile_bp, profile_ms, t0, tau, budget_bp, feasible=None, stream=None) -> None:

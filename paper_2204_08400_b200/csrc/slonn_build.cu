@@ -155,10 +155,12 @@ __device__ __forceinline__ uint64_t score_sort_key(double s)
 // One block per segment: stable LSD radix sort (8 bits per pass) of the segment's
 // N (key, id) pairs; ids start ascending, so equal scores keep the lower id first.
 // seg_active[s] == 0 skips the segment.  The sorted ids end in ids_out[s][0..N).
+// The n_last ids in `last` (nullable) get the largest key, which no score maps to, so they end
+// behind every other id without changing the order of the others.
 #define SORT_THREADS 256
 __global__ void __launch_bounds__(SORT_THREADS)
 segment_sort_kernel(const double *score, uint32_t N, const uint32_t *seg_active, uint64_t *keyA, uint64_t *keyB,
-                    uint32_t *idA, uint32_t *idB, uint32_t *ids_out)
+                    uint32_t *idA, uint32_t *idB, uint32_t *ids_out, const uint32_t *last, uint32_t n_last)
 {
     __shared__ uint32_t hist[256];
     __shared__ uint32_t bin_base[256];
@@ -178,6 +180,10 @@ segment_sort_kernel(const double *score, uint32_t N, const uint32_t *seg_active,
     for (uint32_t d = threadIdx.x; d < 256; d += blockDim.x)
         for (uint32_t w = 0; w < SORT_THREADS / 32; ++w) warp_cnt[w][d] = 0;
     __syncthreads();
+    if (last) {
+        for (uint32_t h = threadIdx.x; h < n_last; h += blockDim.x) ka[last[h]] = ~0ull;
+        __syncthreads();
+    }
     for (uint32_t pass = 0; pass < 8; ++pass) {
         const uint32_t shift = pass * 8;
         for (uint32_t d = threadIdx.x; d < 256; d += blockDim.x) hist[d] = 0;
@@ -354,7 +360,12 @@ int train_layer(slonn_model *m, uint32_t l, const float *A, uint32_t n_cal, uint
     }
 
     // table storage
-    ly.cap = (m->list_cap == 0 || m->list_cap > N) ? N : m->list_cap;
+    // lists hold every node, or (hash nodes always active) every node that is not a hash node:
+    // those are sorted behind all others below and fall off the end of the list
+    {
+        const uint32_t listable = m->free_hash ? N - H : N;
+        ly.cap = (m->list_cap == 0 || m->list_cap > listable) ? listable : m->list_cap;
+    }
     ly.id_bytes = N <= 65536u ? 2u : 4u;
     ly.table_bytes = (uint64_t)nseg * ly.cap * ly.id_bytes;
     CK(cudaMalloc(&ly.tables, ly.table_bytes));
@@ -367,7 +378,8 @@ int train_layer(slonn_model *m, uint32_t l, const float *A, uint32_t n_cal, uint
         bool ok = cudaMalloc(&gkA, 8ull * N) == cudaSuccess && cudaMalloc(&gkB, 8ull * N) == cudaSuccess &&
                   cudaMalloc(&giA, 4ull * N) == cudaSuccess && cudaMalloc(&giB, 4ull * N) == cudaSuccess;
         if (ok) {
-            segment_sort_kernel<<<1, SORT_THREADS, 0, st>>>(d_sum, N, nullptr, gkA, gkB, giA, giB, d_gsorted);
+            segment_sort_kernel<<<1, SORT_THREADS, 0, st>>>(d_sum, N, nullptr, gkA, gkB, giA, giB, d_gsorted,
+                                                            m->free_hash ? ly.hash_nodes : nullptr, H);
             ok = cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(st) == cudaSuccess;
         }
         cudaFree(gkA); cudaFree(gkB); cudaFree(giA); cudaFree(giB);
@@ -391,7 +403,7 @@ int train_layer(slonn_model *m, uint32_t l, const float *A, uint32_t n_cal, uint
                                                                             d_members, bk0, d_score);
             CK(cudaGetLastError());
             segment_sort_kernel<<<cnt, SORT_THREADS, 0, st>>>(d_score, N, d_count + bk0, d_keyA, d_keyB, d_idA,
-                                                              d_idB, d_sorted);
+                                                              d_idB, d_sorted, m->free_hash ? ly.hash_nodes : nullptr, H);
             CK(cudaGetLastError());
             const dim3 g((ly.cap + 255) / 256, cnt);
             if (ly.id_bytes == 2)
@@ -489,6 +501,7 @@ extern "C" int slonn_build(const slonn_build_desc *desc, const void *const *W, c
         if (desc->has_activator[l]) {
             if (sparse0) return SLONN_ERR_ARG;
             if (desc->K * desc->L > N) return SLONN_ERR_DIM;
+            if (desc->free_hash_nodes && desc->K * desc->L >= N) return SLONN_ERR_DIM;
             ++n_act;
         }
     }
@@ -509,6 +522,7 @@ extern "C" int slonn_build(const slonn_build_desc *desc, const void *const *W, c
     m->K = desc->K; m->L = desc->L; m->H = desc->K * desc->L;
     m->list_cap = desc->list_cap;
     m->first_sparse = desc->first_layer_sparse ? 1u : 0u;
+    m->free_hash = desc->free_hash_nodes ? 1u : 0u;
     for (uint32_t l = 0; l <= desc->n_layers; ++l) m->dims[l] = desc->dims[l];
     for (uint32_t l = 0; l < desc->n_layers; ++l) {
         slonn_layer &ly = m->layer[l];
@@ -578,12 +592,12 @@ fail:
 namespace {
 
 struct blob_header {
-    uint32_t magic, version, n_layers, dtype, K, L, list_cap, first_sparse;
+    uint32_t magic, version, n_layers, dtype, K, L, list_cap, first_sparse, free_hash;
     uint32_t dims[SLONN_MAX_LAYERS + 1];
     uint8_t has_act[SLONN_MAX_LAYERS];
 };
 constexpr uint32_t BLOB_MAGIC = 0x4e4e4c53u; // "SLNN"
-constexpr uint32_t BLOB_VERSION = 1;
+constexpr uint32_t BLOB_VERSION = 2;
 
 uint64_t fnv1a(const unsigned char *p, uint64_t n)
 {
@@ -618,7 +632,7 @@ extern "C" int slonn_serialize(const slonn_model *m, void *dst_host, uint64_t ds
     blob_header h;
     memset(&h, 0, sizeof(h));
     h.magic = BLOB_MAGIC; h.version = BLOB_VERSION; h.n_layers = m->n_layers; h.dtype = (uint32_t)m->dtype;
-    h.K = m->K; h.L = m->L; h.list_cap = m->list_cap; h.first_sparse = m->first_sparse;
+    h.K = m->K; h.L = m->L; h.list_cap = m->list_cap; h.first_sparse = m->first_sparse; h.free_hash = m->free_hash;
     for (uint32_t l = 0; l <= m->n_layers; ++l) h.dims[l] = m->dims[l];
     for (uint32_t l = 0; l < m->n_layers; ++l) h.has_act[l] = (uint8_t)m->layer[l].has_act;
     memcpy(p, &h, sizeof(h));
@@ -665,15 +679,21 @@ extern "C" int slonn_deserialize(const void *src_host, uint64_t src_bytes, const
             if (!h.has_act[l]) continue;
             if (H > N || (l == 0 && h.first_sparse)) return SLONN_ERR_DIM;
             if (o + sizeof(uint32_t) * H + 8 > src_bytes - 8) return SLONN_ERR_ARG;
+            if (h.free_hash && H >= N) return SLONN_ERR_DIM;
             for (uint32_t k = 0; k < H; ++k) {
                 uint32_t nd;
                 memcpy(&nd, p + o + 4 * k, 4);
                 if (nd >= N) return SLONN_ERR_ARG;
+                for (uint32_t g = 0; g < k; ++g) { // hash nodes are distinct
+                    uint32_t other;
+                    memcpy(&other, p + o + 4 * g, 4);
+                    if (other == nd) return SLONN_ERR_ARG;
+                }
             }
             o += sizeof(uint32_t) * H;
             uint32_t cap, idb;
             memcpy(&cap, p + o, 4); memcpy(&idb, p + o + 4, 4); o += 8;
-            if (cap < 1 || cap > N || idb != (N <= 65536u ? 2u : 4u)) return SLONN_ERR_ARG;
+            if (cap < 1 || cap > (h.free_hash ? N - H : N) || idb != (N <= 65536u ? 2u : 4u)) return SLONN_ERR_ARG;
             const uint64_t tb = (uint64_t)h.L * nb * cap * idb;
             if (o + tb > src_bytes - 8) return SLONN_ERR_ARG;
             o += tb;
@@ -687,7 +707,7 @@ extern "C" int slonn_deserialize(const void *src_host, uint64_t src_bytes, const
     m->magic = SLONN_MAGIC;
     cudaGetDevice(&m->device);
     m->n_layers = h.n_layers; m->dtype = (int32_t)h.dtype; m->K = h.K; m->L = h.L; m->H = H;
-    m->list_cap = h.list_cap; m->first_sparse = h.first_sparse ? 1u : 0u;
+    m->list_cap = h.list_cap; m->first_sparse = h.first_sparse ? 1u : 0u; m->free_hash = h.free_hash ? 1u : 0u;
     for (uint32_t l = 0; l <= h.n_layers; ++l) m->dims[l] = h.dims[l];
     cudaStream_t st = (cudaStream_t)stream;
     int rc = SLONN_OK;

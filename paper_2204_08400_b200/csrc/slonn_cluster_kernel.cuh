@@ -39,6 +39,7 @@ struct slonn_cluster_layer {
 struct slonn_cluster_params {
     slonn_cluster_layer layer[SLONN_MAX_LAYERS];
     uint32_t n_layers, n, n_act, K, L, cluster;
+    uint32_t pre;            // hash nodes that are always active (0 or K*L)
     const float *x;          // [n][D0]
     const uint16_t *budget_bp; // [n]
     uint32_t max_bp;
@@ -63,8 +64,8 @@ __device__ __forceinline__ uint32_t cluster_count(const slonn_cluster_params &P,
     *bad = (bp < 1u) || (bp > 10000u) || (bp > P.max_bp);
     if (bp < 1u) bp = 1u;
     if (bp > P.max_bp) bp = P.max_bp;
-    const uint32_t B = slonn_budget_nodes(bp, P.layer[l].N);
-    if (B > P.layer[l].cap && B != P.layer[l].N) *bad = true;
+    const uint32_t B = slonn_layer_nodes(bp, P.layer[l].N, P.pre);
+    if (B - P.pre > P.layer[l].cap && B != P.layer[l].N) *bad = true;
     return B;
 }
 
@@ -79,7 +80,6 @@ cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
     __shared__ uint32_t keys[8];
     __shared__ uint32_t scan_ws[32];
     __shared__ uint32_t scan_total;
-    __shared__ uint32_t s_total;
 
     const uint32_t C = P.cluster;
     const uint32_t rank = cluster.block_rank();
@@ -155,7 +155,6 @@ cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
                 if (lane < C) *cluster.map_shared_rank(&zh[h], lane) = z;
             }
             for (uint32_t i = threadIdx.x; i < ((ly.N + 31u) >> 5); i += blockDim.x) bitmap[i] = 0u;
-            if (threadIdx.x == 0) s_total = 0;
         }
         cluster.sync(); // hash sums delivered, every block's next buffer zeroed
 
@@ -173,10 +172,10 @@ cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
             bool ok;
             if (ly.id_bytes == 2)
                 ok = block_select<uint16_t>(ly.tables, ly.cap, P.K, P.L, ly.N, B, keys, bitmap, ids_s, scan_ws,
-                                            &scan_total, &s_total);
+                                            &scan_total, ly.hash_nodes, P.pre);
             else
                 ok = block_select<uint32_t>(ly.tables, ly.cap, P.K, P.L, ly.N, B, keys, bitmap, ids_s, scan_ws,
-                                            &scan_total, &s_total);
+                                            &scan_total, ly.hash_nodes, P.pre);
             if (!ok && rank == 0 && threadIdx.x == 0) slonn_report(P.status, SLONN_ERR_ARG, q, l);
             __syncthreads();
             implicit_ids = false;

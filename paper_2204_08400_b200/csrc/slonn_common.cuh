@@ -33,6 +33,7 @@ struct slonn_model {
     uint32_t K, L, H;
     uint32_t list_cap;
     uint32_t first_sparse;
+    uint32_t free_hash;   // 1: hash nodes always active and absent from the lists
     uint32_t n_act;
     uint32_t act_index[SLONN_MAX_LAYERS]; // index of the layer among activator layers
     slonn_layer layer[SLONN_MAX_LAYERS];
@@ -48,6 +49,17 @@ __host__ __device__ __forceinline__ uint32_t slonn_budget_nodes(uint32_t bp, uin
     if (b < 1) b = 1;
     if (b > N) b = N;
     return (uint32_t)b;
+}
+
+// Nodes a layer of N nodes computes at budget bp.  pre = 0: the budget's node count.  pre = K*L
+// (models whose hash nodes are always active): that many nodes from the lists, of which there are
+// N - pre, plus the pre hash nodes.
+__host__ __device__ __forceinline__ uint32_t slonn_layer_nodes(uint32_t bp, uint32_t N, uint32_t pre)
+{
+    const uint32_t B = slonn_budget_nodes(bp, N);
+    if (pre == 0) return B;
+    const uint32_t rest = N - pre;
+    return (B < rest ? B : rest) + pre;
 }
 
 __device__ __forceinline__ void slonn_report(uint32_t *status, int code, uint32_t q, uint32_t layer)
@@ -262,6 +274,9 @@ __device__ __forceinline__ void stage_input(const slonn_input &in, uint32_t q, u
     }
     __syncthreads();
 }
+
+// hash nodes that are active whatever the budget (0 unless the model was built that way)
+inline uint32_t slonn_model_pre(const slonn_model *m) { return m->free_hash ? m->H : 0u; }
 
 // ---- internal host entry points shared between translation units ---------------
 int slonn_forward_all_rows(const slonn_model *m, uint32_t l, const float *in_dense, uint32_t n, float *out,

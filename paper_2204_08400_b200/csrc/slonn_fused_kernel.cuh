@@ -35,6 +35,7 @@ struct slonn_fused_layer {
 struct slonn_fused_params {
     slonn_fused_layer layer[SLONN_MAX_LAYERS];
     uint32_t n_layers, n, n_act, K, L;
+    uint32_t pre;            // hash nodes that are always active (0 or K*L)
     const uint16_t *skip_bp; // nullable: queries with this budget == 10000 are handled elsewhere
     const float *x;          // [n][D0]
     const uint64_t *indptr;  // [n * n_act + 1]
@@ -131,17 +132,25 @@ __device__ __forceinline__ uint32_t fused_table_entry(const void *tables, uint32
     return (uint32_t)__ldg(t + (((uint64_t)b << K) + key) * cap + r);
 }
 
-// First B distinct ids of the rank-interleaved bucket lists -> ids_s[0..B) ascending.
-// mykey: lane b holds the key of table b.  One warp, no block barrier.
+// The first `pre` hash nodes and the first B - pre distinct ids of the rank-interleaved bucket
+// lists -> ids_s[0..B) ascending.  mykey: lane b holds the key of table b.  One warp, no block barrier.
 __device__ __forceinline__ void fused_select(const slonn_fused_layer &ly, uint32_t K, uint32_t L, uint32_t mykey,
-                                             uint32_t B, uint32_t *bitmap, uint16_t *ids_s, uint32_t lane)
+                                             uint32_t B, uint32_t pre, uint32_t *bitmap, uint16_t *ids_s, uint32_t lane)
 {
     const uint32_t nwords = (ly.N + 31u) >> 5;
     for (uint32_t w = lane; w < nwords; w += 32) bitmap[w] = 0u;
     __syncwarp();
-    const uint32_t npos = B * L;
+    if (pre) {
+        for (uint32_t h = lane; h < pre; h += 32) {
+            const uint32_t nd = __ldg(ly.hash_nodes + h);
+            atomicOr(&bitmap[nd >> 5], 1u << (nd & 31u));
+        }
+        __syncwarp();
+    }
+    const uint32_t want = B - pre;
+    const uint32_t npos = want * L;
     uint32_t total = 0;
-    for (uint32_t base = 0; base < npos && total < B; base += 32) {
+    for (uint32_t base = 0; base < npos && total < want; base += 32) {
         const uint32_t pos = base + lane;
         uint32_t id = 0xffffffffu - lane; // distinct dummies for lanes past the end
         bool fresh = false;
@@ -155,7 +164,7 @@ __device__ __forceinline__ void fused_select(const slonn_fused_layer &ly, uint32
         const uint32_t same = __match_any_sync(SLONN_FULL_MASK, id);
         const bool take = fresh && ((uint32_t)(__ffs(same) - 1) == lane);
         const uint32_t bal = __ballot_sync(SLONN_FULL_MASK, take);
-        const uint32_t need = B - total;
+        const uint32_t need = want - total;
         const uint32_t rank = __popc(bal & ((1u << lane) - 1u));
         if (take && rank < need) atomicOr(&bitmap[id >> 5], 1u << (id & 31u));
         const uint32_t c = (uint32_t)__popc(bal);
@@ -252,8 +261,8 @@ __global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, SLONN_FUSED_MIN_BLOCKS
                 }
             }
             if (P.codes && lane < P.L) P.codes[((uint64_t)q * P.n_act + ly.a) * P.L + lane] = (uint16_t)mykey;
-            if (B != ly.N && B <= ly.cap) {
-                fused_select(ly, P.K, P.L, mykey, B, bitmap, ids_s, lane);
+            if (B != ly.N && B - P.pre <= ly.cap) {
+                fused_select(ly, P.K, P.L, mykey, B, P.pre, bitmap, ids_s, lane);
                 implicit_ids = false;
             }
             if (P.out_ids) {

@@ -44,7 +44,7 @@ uint64_t active_entries(const slonn_model *m, uint32_t n, uint32_t max_bp)
 {
     uint64_t per = 0;
     for (uint32_t l = 0; l < m->n_layers; ++l)
-        if (m->layer[l].has_act) per += slonn_budget_nodes(max_bp, m->layer[l].N);
+        if (m->layer[l].has_act) per += slonn_layer_nodes(max_bp, m->layer[l].N, slonn_model_pre(m));
     return per * n;
 }
 
@@ -234,6 +234,7 @@ int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *ind
         }
     }
     P.n_layers = m->n_layers; P.n = b->n_queries; P.n_act = m->n_act; P.K = m->K; P.L = m->L;
+    P.pre = slonn_model_pre(m);
     P.x = b->x_dense; P.indptr = indptr; P.skip_bp = skip_bp;
     P.out_ids = b->active_ids; P.out_vals = b->active_vals; P.codes = b->codes;
     P.logits = b->logits; P.logit_stride = stride; P.logit_ids = b->logit_ids; P.pred = b->pred;
@@ -269,7 +270,7 @@ uint32_t cluster_max_rows(const slonn_model *m, uint32_t max_bp)
 {
     uint32_t r = 0;
     for (uint32_t l = 0; l < m->n_layers; ++l)
-        r = std::max(r, m->layer[l].has_act ? slonn_budget_nodes(max_bp, m->layer[l].N) : m->layer[l].N);
+        r = std::max(r, m->layer[l].has_act ? slonn_layer_nodes(max_bp, m->layer[l].N, slonn_model_pre(m)) : m->layer[l].N);
     return r;
 }
 
@@ -323,6 +324,7 @@ int launch_cluster(const slonn_model *m, const slonn_batch *b, uint32_t max_bp, 
         }
     }
     P.n_layers = m->n_layers; P.n = b->n_queries; P.n_act = m->n_act; P.K = m->K; P.L = m->L; P.cluster = SLONN_CLUSTER_SIZE;
+    P.pre = slonn_model_pre(m);
     P.x = b->x_dense; P.budget_bp = b->budget_bp; P.max_bp = max_bp; P.indptr_out = b->active_indptr;
     P.out_ids = b->active_ids; P.out_vals = b->active_vals; P.codes = b->codes;
     P.logits = b->logits; P.logit_stride = stride; P.logit_ids = b->logit_ids; P.pred = b->pred;
@@ -382,7 +384,7 @@ extern "C" int slonn_logit_stride(const slonn_model *m, uint32_t max_bp, uint32_
 {
     if (!model_ok(m) || !stride) return SLONN_ERR_ARG;
     const slonn_layer &last = m->layer[m->n_layers - 1];
-    *stride = last.has_act ? slonn_budget_nodes(eff_max_bp(max_bp), last.N) : last.N;
+    *stride = last.has_act ? slonn_layer_nodes(eff_max_bp(max_bp), last.N, slonn_model_pre(m)) : last.N;
     return SLONN_OK;
 }
 
@@ -439,6 +441,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         slonn_plan_params pp;
         memset(&pp, 0, sizeof(pp));
         pp.budget_bp = b->budget_bp; pp.n = n; pp.n_act = m->n_act; pp.max_bp = max_bp;
+        pp.pre = slonn_model_pre(m);
         for (uint32_t l = 0; l < m->n_layers; ++l)
             if (m->layer[l].has_act) {
                 const uint32_t a = m->act_index[l];
@@ -556,9 +559,10 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             sp.in = in; sp.W = ly.W; sp.bias = ly.bias; sp.D = ly.D; sp.N = ly.N; sp.nchunks = nchunks;
             sp.skip_bp = skip_bp;
             sp.hash_nodes = ly.hash_nodes; sp.tables = ly.tables; sp.cap = ly.cap; sp.K = m->K; sp.L = m->L;
+            sp.pre = slonn_model_pre(m);
             sp.n_act = m->n_act; sp.a = a; sp.layer = l; sp.indptr = indptr; sp.out_ids = ids;
             sp.codes = b->codes; sp.status = b->status;
-            max_rows = slonn_budget_nodes(max_bp, ly.N);
+            max_rows = slonn_layer_nodes(max_bp, ly.N, slonn_model_pre(m));
             TIC(SLONN_STAGE_HASH_SELECT);
             rc = launch_select(m, sp, n, max_rows, st);
             TOC();

@@ -50,6 +50,7 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T *warp_sums /* [32] shar
 struct slonn_plan_params {
     const uint16_t *budget_bp;
     uint32_t n, n_act, max_bp;
+    uint32_t pre; // hash nodes that are always active (0 or K*L)
     uint32_t act_N[SLONN_MAX_LAYERS];
     uint32_t act_cap[SLONN_MAX_LAYERS];
     uint32_t act_layer[SLONN_MAX_LAYERS];
@@ -64,8 +65,8 @@ __device__ __forceinline__ uint32_t plan_count(const slonn_plan_params &P, uint6
     bool bad = (bp < 1u) || (bp > 10000u) || (bp > P.max_bp);
     if (bp < 1u) bp = 1u;
     if (bp > P.max_bp) bp = P.max_bp;
-    const uint32_t B = slonn_budget_nodes(bp, P.act_N[a]);
-    if (B > P.act_cap[a] && B != P.act_N[a]) bad = true;
+    const uint32_t B = slonn_layer_nodes(bp, P.act_N[a], P.pre);
+    if (B - P.pre > P.act_cap[a] && B != P.act_N[a]) bad = true;
     if (bad && check) slonn_report(P.status, SLONN_ERR_BUDGET, q, P.act_layer[a]);
     return B;
 }
@@ -128,6 +129,7 @@ struct slonn_select_params {
     const uint32_t *hash_nodes; // device [L*K]
     const void *tables;         // [L][2^K][cap]
     uint32_t cap, K, L;
+    uint32_t pre;               // hash nodes that are always active (0 or K*L)
     uint32_t n_act, a, layer;
     const uint64_t *indptr;     // offsets of (q, a)
     uint32_t *out_ids;          // CSR payload
@@ -143,38 +145,47 @@ __device__ __forceinline__ uint32_t table_entry(const void *tables, uint32_t cap
     return (uint32_t)__ldg(t + (((uint64_t)b << K) + key) * cap + r);
 }
 
-// First B distinct ids of the rank-interleaved bucket lists, written ascending to out[0..B)
-// (global or shared memory).  Called by every thread of the block; bitmap ((N+31)/32 words) must
-// be zero, *s_total zero, keys[L] set, all behind a barrier.  B == N gives every node.  Returns
-// false when the lists did not hold B distinct ids (malformed tables); out is then 0..B-1.
+// The layer's active set, written ascending to out[0..B) (global or shared memory): the first
+// B - pre distinct ids of the rank-interleaved bucket lists, and the first `pre` entries of
+// hash_nodes (pre = 0, or K*L for models whose hash nodes are always active and never listed).
+// Called by every thread of the block; bitmap ((N+31)/32 words) must be zero and keys[L] set, all
+// behind a barrier.  B == N gives every node.  Returns false when the lists did not hold enough
+// distinct ids (malformed tables); out is then 0..B-1.
 template <typename IDT>
 __device__ __forceinline__ bool block_select(const void *tables, uint32_t cap, uint32_t K, uint32_t L, uint32_t N,
                                              uint32_t B, const uint32_t *keys, uint32_t *bitmap, uint32_t *out,
-                                             uint32_t *scan_ws, uint32_t *scan_total, uint32_t *s_total)
+                                             uint32_t *scan_ws, uint32_t *scan_total, const uint32_t *hash_nodes,
+                                             uint32_t pre)
 {
-    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const uint32_t nwords = (N + 31u) >> 5;
     if (B == N) { // every node
         for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
         return true;
     }
-    if (B > cap) { // reported by the plan; keep the output in range
+    const uint32_t want = B - pre; // ids to take from the lists
+    if (want > cap) { // reported by the plan; keep the output in range
         for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
         return true;
+    }
+    if (pre) {
+        for (uint32_t h = threadIdx.x; h < pre; h += blockDim.x) {
+            const uint32_t nd = __ldg(hash_nodes + h);
+            atomicOr(&bitmap[nd >> 5], 1u << (nd & 31u));
+        }
+        __syncthreads();
     }
 
     // (3)+(4) read the L lists rank by rank; the first B distinct ids are the active set.
     // Position pos = rank * L + table.  Positions are taken strictly in order, in steps that
-    // never hold more positions than ids still missing (need = B - total): a step can then add at
-    // most `need` new ids, so the count never passes B, and when it reaches B the marked ids are
-    // exactly the distinct ids of a prefix of the position sequence -- the first B distinct ones.
+    // never hold more positions than ids still missing (want - total): a step can then add at most
+    // that many new ids, so the count never passes `want`, and when it reaches it the marked ids are
+    // exactly the distinct ids of a prefix of the position sequence -- the first `want` distinct ones.
     // (Which of two equal ids inside a step wins the atomic does not matter: one does.)
     // Each thread fetches its entries of the next four rows of blockDim.x positions in one go.
-    const uint32_t npos = B * L; // B distinct ids are always found within rank < B
+    const uint32_t npos = want * L; // `want` distinct ids are always found within rank < want
     const uint32_t T = blockDim.x;
     uint32_t total = 0;
-    (void)lane; (void)warp; (void)s_total;
-    for (uint32_t w0 = 0; w0 < npos && total < B; w0 += 4 * T) {
+    for (uint32_t w0 = 0; w0 < npos && total < want; w0 += 4 * T) {
         uint32_t ahead[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -190,8 +201,8 @@ __device__ __forceinline__ bool block_select(const void *tables, uint32_t cap, u
             const uint32_t row1 = min(row0 + T, npos);
             const uint32_t mine = row0 + threadIdx.x;
             uint32_t p = row0;
-            while (p < row1 && total < B) {                // uniform for the block
-                const uint32_t s = min(B - total, row1 - p);
+            while (p < row1 && total < want) {             // uniform for the block
+                const uint32_t s = min(want - total, row1 - p);
                 bool won = false;
                 if (mine >= p && mine < p + s && ahead[u] < N) {
                     const uint32_t bit = 1u << (ahead[u] & 31u);
@@ -203,7 +214,7 @@ __device__ __forceinline__ bool block_select(const void *tables, uint32_t cap, u
         }
     }
     __syncthreads();
-    if (total != B) { // cannot happen with well-formed tables; keep the output in range
+    if (total != want) { // cannot happen with well-formed tables; keep the output in range
         for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) out[i] = i;
         return false;
     }
@@ -238,7 +249,6 @@ __global__ void __launch_bounds__(LAT ? 1024 : SLONN_THREADS) hash_select_kernel
     __shared__ uint32_t keys[8];
     __shared__ uint32_t scan_ws[32];
     __shared__ uint32_t scan_total;
-    __shared__ uint32_t s_total;
 
     const uint32_t q = blockIdx.x;
     if (P.skip_bp && P.skip_bp[q] == 10000u) return;
@@ -283,11 +293,10 @@ __global__ void __launch_bounds__(LAT ? 1024 : SLONN_THREADS) hash_select_kernel
         keys[threadIdx.x] = key;
         if (P.codes) P.codes[((uint64_t)q * P.n_act + P.a) * P.L + threadIdx.x] = (uint16_t)key;
     }
-    if (threadIdx.x == 0) s_total = 0;
     __syncthreads();
 
     if (!block_select<IDT>(P.tables, P.cap, P.K, P.L, P.N, B, keys, bitmap, P.out_ids + off, scan_ws, &scan_total,
-                           &s_total) &&
+                           P.hash_nodes, P.pre) &&
         threadIdx.x == 0)
         slonn_report(P.status, SLONN_ERR_ARG, q, P.layer);
 }

@@ -46,7 +46,8 @@ class DeviceModel:
         t0 = time.perf_counter()
         self.model = sl.slonn_build(wl.dims, wl.has_act, dtype, self.W, self.bias, calib_dense=calib_dense,
                                     calib_csr=calib_csr, K=wl.K, L=wl.L, list_cap=wl.list_cap, seed=wl.seed,
-                                    first_layer_sparse=wl.first_sparse, hash_nodes_override=hash_nodes_override)
+                                    first_layer_sparse=wl.first_sparse, hash_nodes_override=hash_nodes_override,
+                                    free_hash_nodes=wl.free_hash_nodes)
         torch.cuda.synchronize(self.device)
         self.build_ms = (time.perf_counter() - t0) * 1e3   # slonn_build synchronises before it returns
         self.n_cal = int(calib_csr[0].numel() - 1) if calib_csr is not None else int(calib_dense.shape[0])

@@ -101,6 +101,7 @@ class Workload:
     seed: int = 0                   # hash-node sampling seed
     list_cap: int = 0
     budgets_named: Tuple[int, ...] = field(default_factory=tuple)
+    free_hash_nodes: bool = False   # hash nodes always active and absent from the lists (Sec. 3.4 variant)
 
     @property
     def n_queries(self) -> int:
@@ -131,7 +132,8 @@ _SPECS = {
 
 
 def load(name: str, n_queries: Optional[int] = None, n_cal: Optional[int] = None,
-         budget_bp: Optional[int] = None, list_cap: int = 0, dims: Optional[List[int]] = None) -> Workload:
+         budget_bp: Optional[int] = None, list_cap: int = 0, dims: Optional[List[int]] = None,
+         free_hash_nodes: bool = False) -> Workload:
     """Draw a named workload.  n_queries / n_cal shrink the query and calibration
     sets (same laws, same seeds); budget_bp gives every query one budget, else
     c5 draws a mixed stream (seed 4) and the others use their first named budget.
@@ -159,4 +161,4 @@ def load(name: str, n_queries: Optional[int] = None, n_cal: Optional[int] = None
     return Workload(name=name, dims=dims_, has_act=has_act, dtype=s["dtype"], W_f32=W_f32,
                     W_store=W_store, bias=bias, first_sparse=first_sparse, calib=calib, x=x,
                     budget_bp=bp, seed=s["w_seed"] + 1000, list_cap=list_cap or s.get("list_cap", 0),
-                    budgets_named=tuple(s["budgets"]))
+                    budgets_named=tuple(s["budgets"]), free_hash_nodes=bool(free_hash_nodes))

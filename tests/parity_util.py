@@ -11,7 +11,7 @@ TOL = {"f32": 1e-5, "bf16": 2e-2}   # max relative logit error against the fp64 
 
 def oracle_model(wl: Workload, n_cal=None, hash_nodes_override=None) -> orc.OracleModel:
     m = orc.OracleModel(wl.dims, wl.has_act, wl.W_f32, wl.bias, V=wl.V, K=wl.K, L=wl.L,
-                        list_cap=wl.list_cap, first_sparse=wl.first_sparse)
+                        list_cap=wl.list_cap, first_sparse=wl.first_sparse, free_hash_nodes=wl.free_hash_nodes)
     if wl.first_sparse:
         ip, ids, vals = wl.calib
         if n_cal is not None:

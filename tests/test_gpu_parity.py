@@ -416,3 +416,43 @@ def test_zero_inputs_and_tied_logits(dtype):
     x[::3] = 0.0                                  # every third query is all zeros
     wl = dataclasses.replace(wl, x=x)
     check(wl)
+
+
+# ---- hash nodes always active and absent from the lists (Sec. 3.4 variant) ---------
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_free_hash_nodes_small_mlp(dtype):
+    wl = custom_workload(90, [136, 200, 96, 24], [1, 1, 0], dtype, n=300, n_cal=700, K=4, L=2,
+                         budgets=(100, 1000, 2500, 5000, 9300, 10000))   # 9300: B above the 88 non-hash nodes of layer 2
+    wl.free_hash_nodes = True
+    check(wl)
+
+
+def test_free_hash_nodes_output_activator_three_tables_and_list_cap():
+    wl = custom_workload(91, [72, 160, 328], [1, 1], "f32", n=120, n_cal=500, K=3, L=3, list_cap=120,
+                         budgets=(100, 700, 3300, 10000))
+    wl.free_hash_nodes = True
+    check(wl)
+
+
+def test_free_hash_nodes_c2_reduced():
+    for bp in (500, 2500, 10000):
+        wl = wl_mod.load("c2", n_queries=600, n_cal=2048, budget_bp=bp, free_hash_nodes=True)
+        check(wl, expect_build=(bp == 500))
+
+
+def test_free_hash_nodes_c4_reduced_and_serialization_round_trip():
+    from paper_2204_08400_b200 import binding as sl, harness
+    wl = wl_mod.load("c4", n_queries=3, n_cal=512, budget_bp=1000, dims=[512, 1024, 1024, 1024, 1024, 1024, 1024, 1024, 1024, 200],
+                     free_hash_nodes=True)
+    check(wl)
+    dm = harness.DeviceModel(wl, n_cal=512)
+    want = harness.run_once(dm, wl.x, wl.budget_bp)
+    blob = sl.slonn_serialize(dm.model)
+    built, dm.model = dm.model, sl.slonn_deserialize(blob, dm.W, dm.bias)
+    assert dm.model.free_hash_nodes
+    got = harness.run_once(dm, wl.x, wl.budget_bp)
+    for k in ("logits", "pred", "codes", "active_indptr", "active_ids", "active_vals"):
+        assert np.array_equal(got[k], want[k]), k
+    sl.slonn_free(built)
+    dm.free()
