@@ -78,6 +78,14 @@ def lib():
         L.orc_lcao_budgets.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32,
                                        C.c_void_p, C.c_void_p]
         L.orc_threads.restype = C.c_int
+        L.orc_confidence.restype = C.c_double
+        L.orc_confidence.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32]
+        L.orc_confidence_build.restype = C.c_int
+        L.orc_confidence_build.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_void_p,
+                                           C.c_void_p]
+        L.orc_aclo_budgets.restype = C.c_int
+        L.orc_aclo_budgets.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p,
+                                       C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -129,6 +137,13 @@ def lcao_budgets(profile_bp, profile_ms, t0, tau):
 
 def threads():
     return int(lib().orc_threads())
+
+
+def confidence(z_full, z_k):
+    """Eq. 1 with the cross-entropy as distance: c = sum_j softmax(z_full)_j * log softmax(z_k)_j."""
+    a = _arr(z_full, np.float32); b = _arr(z_k, np.float32)
+    assert a.shape == b.shape and a.ndim == 1
+    return float(lib().orc_confidence(_p(a), _p(b), a.size))
 
 
 class OracleModel:
@@ -225,6 +240,31 @@ class OracleModel:
         rc = lib().orc_model_set_tables(self._m, l, _p(hn), _p(rk), rk.shape[2])
         if rc != 0:
             raise RuntimeError(f"orc_model_set_tables failed: {rc}")
+
+    # ---- confidence tables, ACLO -------------------------------------------
+    def confidence_build(self, calib_dense, profile_bp):
+        """Confidence LSH tables: (sum [L, 2^K, n_k] float64, count [L, 2^K] uint32)."""
+        cd = _arr(calib_dense, np.float32); pb = _arr(profile_bp, np.uint16)
+        s = np.zeros((self.L, 1 << self.K, pb.size), np.float64)
+        c = np.zeros((self.L, 1 << self.K), np.uint32)
+        rc = lib().orc_confidence_build(self._m, _p(cd), cd.shape[0], _p(pb), pb.size, _p(s), _p(c))
+        if rc != 0:
+            raise RuntimeError(f"orc_confidence_build failed: {rc}")
+        return s, c
+
+    def aclo_budgets(self, conf_sum, conf_count, profile_bp, x_dense, threshold, target=None):
+        """Eq. 2: (budget_bp [n] uint16, met [n] uint8, estimate [n, n_k] float64)."""
+        s = _arr(conf_sum, np.float64); c = _arr(conf_count, np.uint32); pb = _arr(profile_bp, np.uint16)
+        xd = _arr(x_dense, np.float32); th = _arr(np.atleast_2d(threshold), np.float32)
+        tg = _arr(target, np.uint32)
+        n = xd.shape[0]
+        assert th.shape[1] == pb.size and s.shape == (self.L, 1 << self.K, pb.size)
+        out = np.zeros(n, np.uint16); met = np.zeros(n, np.uint8); est = np.zeros((n, pb.size), np.float64)
+        rc = lib().orc_aclo_budgets(self._m, _p(s), _p(c), _p(pb), pb.size, _p(xd), n, _p(th), _p(tg), _p(out),
+                                    _p(met), _p(est))
+        if rc != 0:
+            raise RuntimeError(f"orc_aclo_budgets failed: {rc}")
+        return out, met, est
 
     # ---- run -------------------------------------------------------------
     def budgets(self, budget_bp):

@@ -4,7 +4,9 @@
  * A plain, slow, CPU-only statement of the SLO-NN inference path of
  * "Dynamic Network Adaptation at Inference" (arxiv 2204.08400): Node-Activator
  * training (Algorithm 1 with the variance-proportional FreeHash sampling of
- * Sec. 3.4) and the SLO-aware forward pass (Fig. 2 steps 1,3,4; Sec. 3.3).
+ * Sec. 3.4) and the SLO-aware forward pass (Fig. 2 steps 1,3,4; Sec. 3.3),
+ * plus the two budget rules that feed it (LCAO, Eq. 3; ACLO, Eq. 2 with the
+ * Confidence tables of Sec. 3.2).
  * Only tests, the smoke check and the CPU-baseline leg of the benchmark may
  * call it.  It shares no code with the CUDA library and includes none of its
  * headers.
@@ -33,7 +35,10 @@
  * against hand-worked orderings and exact small-integer sums; the selection
  * against its closed form and brute force; Algorithm 1 against a
  * dict-of-lists restatement on tiny layers; the budget rounding against hand
- * computed counts; sampling against frequencies.  Parity unpinned: nothing in
+ * computed counts; sampling against frequencies; the free-hash-node variant
+ * against list filtering and the closed-form selection; the confidence measure
+ * against scipy's entropy kernels and closed forms, the Confidence tables and
+ * the ACLO rule against brute force.  Parity unpinned: nothing in
  * this file; the paper's accuracy and speed-up claims are not reproduced here
  * at all (they need its datasets and trained weights).
  *
@@ -705,4 +710,126 @@ void orc_lcao_budgets(const uint16_t *profile_bp, const float *profile_ms, uint3
         budget_bp[q] = found ? best : smallest;
         feasible[q] = (uint8_t)found;
     }
+}
+
+/* ------------------------------------------------------------------ */
+/* Confidence (Sec. 2.1, Eq. 1), Confidence LSH tables (Sec. 3.2,      */
+/* Eq. 4) and the ACLO budget choice (Sec. 2.2, Eq. 2)                 */
+/* ------------------------------------------------------------------ */
+
+/* c(k, x) = -distance(y, y_k) with the cross-entropy as distance (the paper's choice for
+ * classification): y = softmax of the full network's logits is the target distribution,
+ * y_k = softmax of the logits with the top k% of nodes computed.
+ *   c = sum_j y_j * log y_k,j        (fp64; both softmaxes shifted by their maximum) */
+double orc_confidence(const float *z_full, const float *z_k, uint32_t n)
+{
+    double mf = (double)z_full[0], mk = (double)z_k[0];
+    for (uint32_t j = 1; j < n; ++j) {
+        if ((double)z_full[j] > mf) mf = (double)z_full[j];
+        if ((double)z_k[j] > mk) mk = (double)z_k[j];
+    }
+    double sf = 0.0, sk = 0.0;
+    for (uint32_t j = 0; j < n; ++j) {
+        sf += exp((double)z_full[j] - mf);
+        sk += exp((double)z_k[j] - mk);
+    }
+    const double lse_k = mk + log(sk);
+    double c = 0.0;
+    for (uint32_t j = 0; j < n; ++j) {
+        const double y = exp((double)z_full[j] - mf) / sf;
+        c += y * ((double)z_k[j] - lse_k);
+    }
+    return c;
+}
+
+/* Confidence LSH tables: one set of L tables for the whole network, keyed by the hash functions
+ * of the first layer's Node Activator.  For every profiled k_i and every training row x':
+ * c(k_i, x') from a k_i% run and a 100 % run (CANON32 logits); the row's value is added to the
+ * bucket it hashes to in each table.
+ *   sum   [L][2^K][n_k]  fp64, rows added in row order
+ *   count [L][2^K]       rows per bucket
+ * Needs: layer 0 carries an activator and takes a dense input; the last layer carries none (the
+ * distance is taken over the complete logit vector). */
+int orc_confidence_build(const orc_model *m, const float *calib_dense, uint32_t n_cal,
+                         const uint16_t *profile_bp, uint32_t n_k, double *sum, uint32_t *count)
+{
+    if (!m->has_act[0] || m->first_sparse || m->has_act[m->n_layers - 1] || n_cal == 0 || n_k == 0)
+        return ORC_ERR_ARG;
+    const uint32_t n_out = m->dims[m->n_layers], L = m->L, nb = 1u << m->K;
+    const uint32_t n_act = count_act_layers(m);
+    float *zf = (float *)malloc(sizeof(float) * (uint64_t)n_cal * n_out);
+    float *zk = (float *)malloc(sizeof(float) * (uint64_t)n_cal * n_out);
+    uint16_t *codes = (uint16_t *)malloc(sizeof(uint16_t) * (uint64_t)n_cal * n_act * L);
+    uint16_t *bp = (uint16_t *)malloc(sizeof(uint16_t) * n_cal);
+    if (!zf || !zk || !codes || !bp) return ORC_ERR_NOMEM;
+    orc_batch bt;
+    memset(&bt, 0, sizeof(bt));
+    bt.n_queries = n_cal; bt.x_dense = calib_dense; bt.budget_bp = bp; bt.mode = ORC_CANON32;
+    bt.logit_stride = n_out;
+    for (uint32_t x = 0; x < n_cal; ++x) bp[x] = 10000;
+    bt.logits32 = zf; bt.codes = codes;
+    int rc = orc_run(m, &bt);
+    memset(sum, 0, sizeof(double) * (uint64_t)L * nb * n_k);
+    memset(count, 0, sizeof(uint32_t) * (uint64_t)L * nb);
+    for (uint32_t x = 0; x < n_cal && rc == ORC_OK; ++x)
+        for (uint32_t b = 0; b < L; ++b) count[b * nb + codes[((uint64_t)x * n_act + 0) * L + b]] += 1;
+    bt.logits32 = zk; bt.codes = NULL;
+    for (uint32_t i = 0; i < n_k && rc == ORC_OK; ++i) {
+        for (uint32_t x = 0; x < n_cal; ++x) bp[x] = profile_bp[i];
+        rc = orc_run(m, &bt);
+        if (rc != ORC_OK) break;
+        for (uint32_t x = 0; x < n_cal; ++x) {
+            const double c = orc_confidence(zf + (uint64_t)x * n_out, zk + (uint64_t)x * n_out, n_out);
+            for (uint32_t b = 0; b < L; ++b) {
+                const uint32_t key = codes[((uint64_t)x * n_act + 0) * L + b];
+                sum[((uint64_t)b * nb + key) * n_k + i] += c;
+            }
+        }
+    }
+    free(zf); free(zk); free(codes); free(bp);
+    return rc;
+}
+
+/* Accuracy-Constrained Latency-Optimized (Eq. 2): the smallest profiled k whose estimated
+ * confidence reaches the threshold that the accuracy target maps to.
+ *   estimate (Eq. 4, aggregation = arithmetic mean): over the training rows that share a bucket
+ *   with x in any of the L tables (a row counted once per table it shares):
+ *       c^(k_i, x) = sum_b sum[b][key_b(x)][i] / sum_b count[b][key_b(x)]
+ *   keys: the first layer's FreeHash keys of x (CANON32);
+ *   threshold [n_targets][n_k]: t_i of each accuracy target (found on held-out data by the
+ *   caller), target[q] picks the row;
+ *   profile_bp ascending.  No training row in any of x's buckets, or no k_i reaching its
+ *   threshold: the full network (10000 bp), met = 0. */
+int orc_aclo_budgets(const orc_model *m, const double *sum, const uint32_t *count,
+                     const uint16_t *profile_bp, uint32_t n_k, const float *x_dense, uint32_t n,
+                     const float *threshold, const uint32_t *target, uint16_t *budget_bp,
+                     uint8_t *met, double *estimate /* [n][n_k], nullable */)
+{
+    if (!m->has_act[0] || m->first_sparse) return ORC_ERR_ARG;
+    const uint32_t D = m->dims[0], L = m->L, K = m->K, nb = 1u << K;
+    for (uint32_t q = 0; q < n; ++q) {
+        const float *in = x_dense + (uint64_t)q * D;
+        uint32_t keys[8];
+        for (uint32_t b = 0; b < L; ++b) {
+            uint32_t key = 0;
+            for (uint32_t j = 0; j < K; ++j)
+                if (node_z32_dense(m, 0, m->hash_nodes[0][b * K + j], in) > 0.0f) key |= (1u << j);
+            keys[b] = key;
+        }
+        uint64_t rows = 0;
+        for (uint32_t b = 0; b < L; ++b) rows += count[b * nb + keys[b]];
+        const float *thr = threshold + (uint64_t)(target ? target[q] : 0) * n_k;
+        uint16_t pick = 10000;
+        uint8_t ok = 0;
+        for (uint32_t i = 0; i < n_k; ++i) {
+            double s = 0.0;
+            for (uint32_t b = 0; b < L; ++b) s += sum[((uint64_t)b * nb + keys[b]) * n_k + i];
+            const double est = rows ? s / (double)rows : 0.0;
+            if (estimate) estimate[(uint64_t)q * n_k + i] = est;
+            if (!ok && rows && est >= (double)thr[i]) { pick = profile_bp[i]; ok = 1; }
+        }
+        budget_bp[q] = pick;
+        if (met) met[q] = ok;
+    }
+    return ORC_OK;
 }

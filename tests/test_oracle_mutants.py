@@ -34,6 +34,15 @@ MUTANTS = {
     "scores summed in fp32": ("for (uint32_t i = 0; i < N; ++i) s[i] += (double)a[i];", "for (uint32_t i = 0; i < N; ++i) s[i] = (double)((float)s[i] + a[i]);"),
     "LCAO takes the smallest feasible budget": ("(!found || profile_bp[i] > best)", "(!found || profile_bp[i] < best)"),
     "LCAO ignores the time already spent": ("if (t0[q] + profile_ms[i] <= tau[q]", "if (profile_ms[i] <= tau[q]"),
+    "confidence: log-sum-exp forgets the shift": ("const double lse_k = mk + log(sk);", "const double lse_k = log(sk);"),
+    "confidence: the k% prediction is the target": ("const double y = exp((double)z_full[j] - mf) / sf;\n        c += y * ((double)z_k[j] - lse_k);",
+                                                    "const double y = exp((double)z_k[j] - mk) / sk;\n        c += y * ((double)z_full[j] - mf - log(sf));"),
+    "confidence tables: counts keyed by the last activator": ("count[b * nb + codes[((uint64_t)x * n_act + 0) * L + b]] += 1;",
+                                                              "count[b * nb + codes[((uint64_t)x * n_act + n_act - 1) * L + b]] += 1;"),
+    "ACLO takes the largest k that meets its threshold": ("if (!ok && rows && est >= (double)thr[i])", "if (rows && est >= (double)thr[i])"),
+    "ACLO threshold strict": ("est >= (double)thr[i]", "est > (double)thr[i]"),
+    "ACLO estimate averages per-table means": ("const double est = rows ? s / (double)rows : 0.0;",
+                                               "double est = 0.0; for (uint32_t b = 0; b < L; ++b) if (count[b * nb + keys[b]]) est += sum[((uint64_t)b * nb + keys[b]) * n_k + i] / count[b * nb + keys[b]] / L; (void)s;"),
     "argmax keeps the last maximum": ("if (ref ? (out64[n] > out64[best]) : (out32[n] > out32[best])) best = n;",
                                       "if (ref ? (out64[n] >= out64[best]) : (out32[n] >= out32[best])) best = n;"),
 }
@@ -53,6 +62,7 @@ def test_pins_catch_planted_mistake(name, tmp_path):
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
                         os.path.join(ROOT, "tests", "test_oracle_pins.py"), os.path.join(ROOT, "tests", "test_oracle_method.py"),
                         os.path.join(ROOT, "tests", "test_lcao.py"), os.path.join(ROOT, "tests", "test_oracle_free_hash.py"),
+                        os.path.join(ROOT, "tests", "test_aclo.py"),
                         "-m", "not gpu"],
                        env=env, cwd=ROOT, capture_output=True, text=True)
     assert r.returncode == 1, f"the pins did not notice: {name}\n{r.stdout[-600:]}"
