@@ -375,6 +375,32 @@ def main():
         e2e = {"value": n_all / (ms_e / 1e3), "unit": "queries/s", "h2d_bytes_per_step": int(up),
                "d2h_bytes_per_step": int(down), "ms_per_step": ms_e}
 
+    # ---- budget policies on the device (outside the timed region): Confidence tables + ACLO lookup ----
+    policy = None
+    if rank == 0 and world == 1 and not args.no_sweep and wl.has_act[0] and not wl.first_sparse and not wl.has_act[-1]:
+        prof = np.array(sorted(set(wl.budgets_named) | {10000}), np.uint16)
+        rows = harness._dev(wl.calib[: min(dm.n_cal, 4096)], dev)
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        conf = sl.slonn_confidence_build(dm.model, rows, prof, stream)
+        torch.cuda.synchronize(dev)
+        conf_ms = (time.perf_counter() - t0) * 1e3
+        thr = torch.full((1, prof.size), -1.0, dtype=torch.float32, device=dev)
+        xq = harness._dev(wl.x, dev)
+        bpo = torch.zeros(n, dtype=torch.int16, device=dev)
+        for _ in range(3):
+            sl.slonn_aclo_budgets(dm.model, conf, xq, thr, bpo, stream=stream)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for _ in range(10):
+            sl.slonn_aclo_budgets(dm.model, conf, xq, thr, bpo, stream=stream)
+        a1.record(stream)
+        torch.cuda.synchronize(dev)
+        policy = {"confidence_build_ms": conf_ms, "confidence_rows": int(rows.shape[0]), "profile_bp": prof.tolist(),
+                  "aclo_budgets_ms_per_batch": a0.elapsed_time(a1) / 10, "queries": n}
+        sl.slonn_confidence_free(conf)
+        del rows, xq, bpo
+
     # ---- the CPU oracle beside it (rank 0, single-GPU runs only) ----
     cpu = None
     # the oracle builds its own tables from the same calibration rows: seconds for c1/c2, many minutes for
@@ -400,6 +426,7 @@ def main():
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": (sum(stage_cnt.values()) // prof_steps + (1 if stage_cnt["plan"] else 0)) * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "budget_sweep": sweep, "latency": latency,
+            "policy": policy,
             "table_build": {"ms": dm.build_ms, "calibration_rows": dm.n_cal,
                             "rows_per_s": dm.n_cal / (dm.build_ms / 1e3), "timing": "host wall clock around slonn_build"},
         }

@@ -8,8 +8,8 @@
  *   run   : the SLO-aware forward pass (Fig. 2 steps 1, 3, 4; Sec. 3.3): hash the
  *           layer input, fetch one ranked node list per table, keep the top k% of
  *           the lists, compute only those nodes, pass the sparse activation on.
- * The percentage k is chosen elsewhere (the paper's ACLO / LCAO policies) and
- * arrives here as a per-query budget.
+ * The percentage k arrives as a per-query budget; the paper's two rules for
+ * choosing it (LCAO, ACLO) are provided as separate calls that write such budgets.
  *
  * Conventions
  *   - Every function returns SLONN_OK (0) or a negative SLONN_ERR_* code.  Nothing
@@ -226,12 +226,58 @@ typedef struct {
  *   budget_bp              : [n] out: ready to be used as slonn_batch.budget_bp
  *   feasible               : [n] out, nullable: 0 where no profiled k meets the target (Def. 1:
  *                            the SLO cannot be fulfilled); such queries get the smallest profiled k
- * All pointers are device pointers; asynchronous on `stream`.  The accuracy-constrained policy
- * (ACLO, Eq. 2) needs Confidence tables trained on labelled data and is not part of this library.
+ * All pointers are device pointers; asynchronous on `stream`.
  */
 int slonn_lcao_budgets(const uint16_t *profile_bp, const float *profile_ms, uint32_t n_k,
                        const float *t0, const float *tau, uint32_t n, uint16_t *budget_bp,
                        uint8_t *feasible, void *stream);
+
+/*
+ * Confidence LSH tables (Sec. 3.2, Eq. 4) for the Accuracy-Constrained Latency-Optimized policy.
+ * The confidence of the network on input x at budget k is c(k, x) = -distance(y, y_k) (Sec. 2.1,
+ * Eq. 1) with the cross-entropy as distance: y = softmax of the complete network's logits (the
+ * target distribution), y_k = softmax of the logits at budget k, c = sum_j y_j log y_k,j (fp64).
+ * The tables are one set of L tables for the whole network, keyed by the first layer's FreeHash
+ * keys.  Training needs no labels: every row is run at 100 % and at each profiled k; its c(k, x)
+ * is added to the bucket it hashes to in each table (fp64, rows in order), and the rows per
+ * bucket are counted.
+ *   rows       : dense training rows (device), as for slonn_build
+ *   profile_bp : HOST, [n_k] budgets in basis points, strictly ascending, n_k <= 64
+ * Needs a model whose layer 0 carries an activator and takes dense input and whose last layer
+ * carries none (the distance is taken over the complete logit vector); otherwise SLONN_ERR_ARG.
+ * Allocates, runs 1 + n_k forward passes over the rows and synchronises `stream`.
+ */
+typedef struct slonn_confidence slonn_confidence;
+int slonn_confidence_build(const slonn_model *m, const slonn_rows *rows, const uint16_t *profile_bp,
+                           uint32_t n_k, void *stream, slonn_confidence **out);
+/* Copies the tables to HOST arrays: sum [L][2^K][n_k] (fp64), count [L][2^K]; synchronous. */
+int slonn_confidence_to_host(const slonn_confidence *c, double *sum_host, uint64_t sum_entries,
+                             uint32_t *count_host, uint64_t count_entries);
+/* Frees the tables.  NULL is accepted. */
+void slonn_confidence_free(slonn_confidence *c);
+
+/*
+ * ACLO budgets (Sec. 2.2, Eq. 2): for each query the smallest profiled k whose estimated
+ * confidence reaches the threshold its accuracy target maps to.  The estimate (Eq. 4 with the
+ * arithmetic mean) pools the training rows that share a bucket with x in any of the L tables:
+ *     c^(k_i, x) = sum_b sum[b][key_b(x)][i] / sum_b count[b][key_b(x)]
+ *   x_dense    : [n][D0] the queries (16-byte aligned); their keys are computed here with the
+ *                same fixed-order dot products as in slonn_run
+ *   threshold  : [n_targets][n_k] confidence threshold t_i of each accuracy target at each
+ *                profiled k (the caller finds them on held-out data, Sec. 3.2)
+ *   target     : [n] row of `threshold` per query; NULL = row 0 for every query
+ *   budget_bp  : [n] out, ready to be used as slonn_batch.budget_bp
+ *   met        : [n] out, nullable: 0 where no training row shares a bucket with x or no
+ *                profiled k reaches its threshold; such queries get 10000 bp (the full network)
+ *   estimate   : [n][n_k] out, nullable: the estimates (0 where no row shares a bucket)
+ *   status     : [4] nullable, as in slonn_batch: a target index out of range is reported there
+ *                (the query then uses row 0); not cleared by this call
+ * All pointers are device pointers; asynchronous on `stream`; no allocation.
+ */
+int slonn_aclo_budgets(const slonn_model *m, const slonn_confidence *c, const float *x_dense,
+                       uint32_t n, const float *threshold, uint32_t n_targets, const uint32_t *target,
+                       uint16_t *budget_bp, uint8_t *met, double *estimate, uint32_t *status,
+                       void *stream);
 
 /* Number of entries active_ids / active_vals need for n queries at max_budget_bp. */
 int slonn_active_capacity(const slonn_model *m, uint32_t n_queries, uint32_t max_budget_bp,

@@ -21,7 +21,8 @@ EXPORTS = [
     "slonn_version", "slonn_strerror", "slonn_build", "slonn_model_info", "slonn_model_tables_to_host",
     "slonn_free", "slonn_active_capacity", "slonn_logit_stride", "slonn_workspace_bytes", "slonn_run",
     "slonn_run_timed", "slonn_run_static", "slonn_dense_layer", "slonn_serialized_bytes", "slonn_serialize",
-    "slonn_deserialize", "slonn_lcao_budgets",
+    "slonn_deserialize", "slonn_lcao_budgets", "slonn_confidence_build", "slonn_confidence_to_host",
+    "slonn_confidence_free", "slonn_aclo_budgets",
     "slonn_host_workspace_bytes", "slonn_run_host",
 ]
 
@@ -82,6 +83,15 @@ def lib():
         L.slonn_deserialize.restype = C.c_int
         L.slonn_deserialize.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.POINTER(C.c_void_p)]
+        L.slonn_confidence_build.restype = C.c_int
+        L.slonn_confidence_build.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
+        L.slonn_confidence_to_host.restype = C.c_int
+        L.slonn_confidence_to_host.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64]
+        L.slonn_confidence_free.restype = None
+        L.slonn_confidence_free.argtypes = [C.c_void_p]
+        L.slonn_aclo_budgets.restype = C.c_int
+        L.slonn_aclo_budgets.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32,
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.slonn_lcao_budgets.restype = C.c_int
         L.slonn_lcao_budgets.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32,
                                          C.c_void_p, C.c_void_p, C.c_void_p]
@@ -246,6 +256,63 @@ def slonn_lcao_budgets(profile_bp, profile_ms, t0, tau, budget_bp, feasible=None
                                   int(t0.numel()), _ptr(budget_bp), _ptr(feasible), _stream_ptr(stream))
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_lcao_budgets")
+
+
+class Confidence:
+    """Handle of trained Confidence LSH tables."""
+
+    def __init__(self, handle, K, L, profile_bp):
+        self.handle, self.K, self.L = handle, K, L
+        self.profile_bp = np.asarray(profile_bp, dtype=np.uint16).copy()
+
+    def free(self):
+        if self.handle:
+            lib().slonn_confidence_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def slonn_confidence_build(model: Model, rows_dense, profile_bp, stream=None) -> Confidence:
+    """rows_dense: device tensor [n_rows, D0]; profile_bp: host sequence, strictly ascending."""
+    pb = np.ascontiguousarray(profile_bp, dtype=np.uint16)
+    rows = _Rows()
+    rows.n_rows = rows_dense.shape[0]
+    rows.dense = _ptr(rows_dense)
+    out = C.c_void_p()
+    rc = lib().slonn_confidence_build(model.handle, C.byref(rows), pb.ctypes.data, int(pb.size), _stream_ptr(stream),
+                                      C.byref(out))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_confidence_build")
+    return Confidence(out.value, model.K, model.L, pb)
+
+
+def slonn_confidence_to_host(conf: Confidence):
+    """(sum [L, 2^K, n_k] float64, count [L, 2^K] uint32)."""
+    s = np.zeros((conf.L, 1 << conf.K, conf.profile_bp.size), np.float64)
+    c = np.zeros((conf.L, 1 << conf.K), np.uint32)
+    rc = lib().slonn_confidence_to_host(conf.handle, s.ctypes.data, s.size, c.ctypes.data, c.size)
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_confidence_to_host")
+    return s, c
+
+
+def slonn_confidence_free(conf: Confidence) -> None:
+    conf.free()
+
+
+def slonn_aclo_budgets(model: Model, conf: Confidence, x_dense, threshold, budget_bp, target=None, met=None,
+                       estimate=None, status=None, stream=None) -> None:
+    """Eq. 2 on the device; threshold: device tensor [n_targets, n_k] float32; outputs are device tensors."""
+    rc = lib().slonn_aclo_budgets(model.handle, conf.handle, _ptr(x_dense), int(x_dense.shape[0]), _ptr(threshold),
+                                  int(threshold.shape[0]), _ptr(target), _ptr(budget_bp), _ptr(met), _ptr(estimate),
+                                  _ptr(status), _stream_ptr(stream))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_aclo_budgets")
 
 
 def slonn_free(model: Model) -> None:

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libslonn.so")
-SOURCES = ["slonn_run.cu", "slonn_build.cu", "slonn_dense_tc.cu"]
+SOURCES = ["slonn_run.cu", "slonn_build.cu", "slonn_dense_tc.cu", "slonn_policy.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Wno-deprecated-gpu-targets"]
 

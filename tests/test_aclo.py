@@ -174,3 +174,95 @@ def test_aclo_threshold_is_inclusive():
     got, met, est = m.aclo_budgets(s, c, PROFILE, x, thr)
     assert np.all(est[:, 0] == -2.0) and np.all(est[:, 1] == -1.0)
     assert np.all(got == PROFILE[1]) and np.all(met == 1)
+
+
+# ---------------------------------------------------------------------------
+# device entry points against the oracle
+# ---------------------------------------------------------------------------
+
+def _device_case(wl, n_cal):
+    import torch
+    from paper_2204_08400_b200 import binding as sl, harness
+    from parity_util import oracle_model
+    dm = harness.DeviceModel(wl, n_cal=n_cal)
+    om = oracle_model(wl, n_cal=n_cal)
+    rows = wl.calib[:n_cal]
+    want_s, want_c = om.confidence_build(rows, PROFILE)
+    conf = sl.slonn_confidence_build(dm.model, harness._dev(rows, dm.device), PROFILE)
+    got_s, got_c = sl.slonn_confidence_to_host(conf)
+    assert np.array_equal(got_c, want_c), "rows per bucket"
+    # same logits bit for bit, same order of additions; exp and log come from two math libraries
+    assert np.allclose(got_s, want_s, rtol=1e-11, atol=1e-11), "bucket sums"
+    return torch, sl, harness, dm, om, conf, want_s, want_c
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_device_confidence_tables_and_aclo_budgets(dtype):
+    from test_gpu_parity import custom_workload
+    wl = custom_workload(330, [136, 200, 96, 24], [1, 1, 0], dtype, n=500, n_cal=700, K=4, L=2)
+    torch, sl, harness, dm, om, conf, s, c = _device_case(wl, 700)
+    # thresholds between observed estimates (no query sits on a threshold), three accuracy targets
+    _, seen, est = om.aclo_budgets(s, c, PROFILE, wl.x, np.full((1, PROFILE.size), -np.inf, np.float32))
+    qs = [0.25, 0.5, 0.8]
+    thr = np.stack([np.quantile(est[seen == 1], q, axis=0) for q in qs]).astype(np.float32)
+    target = np.random.default_rng(331).integers(0, 3, wl.n_queries).astype(np.uint32)
+    want_bp, want_met, want_est = om.aclo_budgets(s, c, PROFILE, wl.x, thr, target)
+    margin = np.min(np.abs(want_est - thr[target].astype(np.float64)), axis=1)
+    dev = dm.device
+    x = harness._dev(wl.x, dev)
+    bp = torch.zeros(wl.n_queries, dtype=torch.int16, device=dev)
+    met = torch.zeros(wl.n_queries, dtype=torch.uint8, device=dev)
+    estd = torch.zeros((wl.n_queries, PROFILE.size), dtype=torch.float64, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    sl.slonn_aclo_budgets(dm.model, conf, x, harness._dev(thr, dev), bp, target=harness._dev(target, dev), met=met,
+                          estimate=estd, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().numpy()[0] == 0
+    got_bp = bp.cpu().numpy().view(np.uint16)
+    assert np.allclose(estd.cpu().numpy(), want_est, rtol=1e-11, atol=1e-11)
+    clear = margin > 1e-9                                     # decisions away from a threshold are unique
+    assert clear.mean() > 0.99
+    assert np.array_equal(got_bp[clear], want_bp[clear]) and np.array_equal(met.cpu().numpy()[clear], want_met[clear])
+    assert len(set(got_bp.tolist())) >= 3
+    # the budgets feed the forward pass as they are
+    g = harness.run_once(dm, wl.x, got_bp, max_budget_bp=10000)
+    o = om.run(got_bp, x_dense=wl.x)
+    assert g["status"][0] == 0 and np.array_equal(g["pred"], o["pred"]) and np.array_equal(g["logits"], o["logits"])
+    # a target index outside the threshold table is reported, not followed
+    bad = torch.full((wl.n_queries,), 7, dtype=torch.int32, device=dev)
+    sl.slonn_aclo_budgets(dm.model, conf, x, harness._dev(thr, dev), bp, target=bad, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().numpy().view(np.uint32)[0] == 1       # -SLONN_ERR_ARG
+    sl.slonn_confidence_free(conf)
+    dm.free()
+
+
+@pytest.mark.gpu
+def test_device_confidence_tables_c2_reduced():
+    from paper_2204_08400_b200 import workloads as wl_mod
+    wl = wl_mod.load("c2", n_queries=256, n_cal=2048, budget_bp=1000)
+    torch, sl, harness, dm, om, conf, s, c = _device_case(wl, 2048)
+    sl.slonn_confidence_free(conf)
+    dm.free()
+
+
+@pytest.mark.gpu
+def test_device_confidence_refuses_unsupported_models_and_profiles():
+    from paper_2204_08400_b200 import binding as sl, harness
+    from test_gpu_parity import custom_workload
+    wl = custom_workload(332, [72, 160, 328], [1, 1], "f32", n=16, n_cal=200, K=3, L=2)   # budgeted output layer
+    dm = harness.DeviceModel(wl)
+    rows = harness._dev(wl.calib, dm.device)
+    with pytest.raises(sl.SlonnError) as e:
+        sl.slonn_confidence_build(dm.model, rows, PROFILE)
+    assert e.value.code == sl.ERR["ARG"]
+    dm.free()
+    wl = custom_workload(333, [72, 160, 24], [1, 0], "f32", n=16, n_cal=200, K=3, L=2)
+    dm = harness.DeviceModel(wl)
+    rows = harness._dev(wl.calib, dm.device)
+    for prof, code in (([1000, 500], "ARG"), ([0, 500], "BUDGET"), (list(range(1, 70)), "DIM")):
+        with pytest.raises(sl.SlonnError) as e:
+            sl.slonn_confidence_build(dm.model, rows, prof)
+        assert e.value.code == sl.ERR[code]
+    dm.free()
