@@ -167,6 +167,15 @@ int launch_gather_t(const slonn_gather_params &P, uint64_t grid, uint32_t thread
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
+template <bool BF16>
+int launch_gather_short_t(const slonn_gather_params &P, uint64_t grid, size_t smem, cudaStream_t st)
+{
+    const int rc = set_smem(gather_short_kernel<BF16>, smem);
+    if (rc) return rc;
+    gather_short_kernel<BF16><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(P);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
 int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint32_t max_rows, cudaStream_t st)
 {
     // so few rows that the GPU cannot be filled: latency variant, 4 warps per block, one row per warp
@@ -178,14 +187,14 @@ int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint
         P.rows_per_cta = 4;
         P.ctas_per_query = (max_rows + 3) / 4;
     } else {
-        gather_shape(n, max_rows, short_rows ? 8u : 4u, &P.rows_per_cta, &P.ctas_per_query);
+        gather_shape(n, max_rows, short_rows ? 32u : 4u, &P.rows_per_cta, &P.ctas_per_query);
     }
     const size_t smem = (size_t)P.D * 4;
     const uint64_t grid = (uint64_t)n * P.ctas_per_query;
     if (grid == 0 || grid > 0x7fffffffull) return SLONN_ERR_DIM;
     const bool bf = m->dtype == SLONN_BF16;
     if (lat) return bf ? launch_gather_t<true, true, 4>(P, grid, threads, smem, st) : launch_gather_t<false, true, 4>(P, grid, threads, smem, st);
-    if (short_rows) return bf ? launch_gather_t<true, false, 8>(P, grid, threads, smem, st) : launch_gather_t<false, false, 8>(P, grid, threads, smem, st);
+    if (short_rows) return bf ? launch_gather_short_t<true>(P, grid, smem, st) : launch_gather_short_t<false>(P, grid, smem, st);
     return bf ? launch_gather_t<true, false, 4>(P, grid, threads, smem, st) : launch_gather_t<false, false, 4>(P, grid, threads, smem, st);
 }
 

@@ -403,6 +403,83 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_
     }
 }
 
+// Rows of at most one 512-byte round (one 16-byte chunk per lane): the lane's piece of the input is
+// loaded once and kept in registers, a warp fetches 32 row ids with one coalesced load and works
+// through them 8 rows at a time, so that the only loads inside the loop are the weight chunks
+// themselves.  Same chunk-to-lane assignment, element order and reduction as gather_dot_kernel<.., 8>.
+template <bool BF16>
+__global__ void __launch_bounds__(SLONN_THREADS, 2) gather_short_kernel(slonn_gather_params P)
+{
+    extern __shared__ float4 smem4[];
+    constexpr int VPC = BF16 ? 8 : 4;
+    constexpr int R = 8;
+    const uint32_t q = blockIdx.x / P.ctas_per_query;
+    const uint32_t chunk = blockIdx.x - q * P.ctas_per_query;
+    if (P.skip_bp && P.skip_bp[q] == 10000u) return;
+    uint64_t off = 0;
+    uint32_t B = P.N;
+    if (P.use_list) {
+        off = P.indptr[(uint64_t)q * P.n_act + P.a];
+        B = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - off);
+    }
+    const uint32_t r0 = chunk * P.rows_per_cta;
+    if (r0 >= B) return;
+    const uint32_t r1 = min(B, r0 + P.rows_per_cta);
+
+    stage_input<BF16>(P.in, q, P.D, P.nchunks, smem4);
+
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const bool has_chunk = lane < P.nchunks;
+    float x[VPC];
+#pragma unroll
+    for (int e = 0; e < VPC; ++e) x[e] = 0.0f;
+    if (has_chunk) {
+        const float4 xa = smem4[lane];
+        x[0] = xa.x; x[1] = xa.y; x[2] = xa.z; x[3] = xa.w;
+        if (BF16) {
+            const float4 xb = smem4[P.nchunks + lane];
+            x[VPC - 4] = xb.x; x[VPC - 3] = xb.y; x[VPC - 2] = xb.z; x[VPC - 1] = xb.w;
+        }
+    }
+    const uint4 *Wl = reinterpret_cast<const uint4 *>(P.W) + lane;
+    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+    for (uint32_t base = r0 + warp * 32u; base < r1; base += nwarps * 32u) {
+        const uint32_t mine = min(base + lane, r1 - 1);
+        const uint32_t myid = P.use_list ? __ldg(P.ids + off + mine) : mine;
+#pragma unroll
+        for (uint32_t sub = 0; sub < 4; ++sub) {
+            const uint32_t r = base + sub * R;
+            if (r >= r1) break; // uniform
+            uint4 w[R];
+#pragma unroll
+            for (int k = 0; k < R; ++k) {
+                const uint32_t nd = __shfl_sync(SLONN_FULL_MASK, myid, sub * R + k); // rows past r1 repeat the last id
+                w[k] = has_chunk ? __ldg(Wl + (uint64_t)nd * P.nchunks) : zero4;
+            }
+            float acc[R];
+#pragma unroll
+            for (int k = 0; k < R; ++k) acc[k] = 0.0f;
+            chunk_fma<BF16, R, 0, VPC>::run(w, x, acc);
+            const float sum = reduce_rows8(acc, lane); // row r + (lane >> 2)
+            const uint32_t mr = r + (lane >> 2);
+            const uint32_t nd = __shfl_sync(SLONN_FULL_MASK, myid, sub * R + (lane >> 2));
+            if ((lane & 3u) == 0u && mr < r1) {
+                float z = sum + __ldg(P.bias + nd);
+                if (P.relu) z = z > 0.0f ? z : 0.0f;
+                if (P.use_list) {
+                    if (P.out_vals) P.out_vals[off + mr] = z;
+                    if (P.out_dense) {
+                        P.out_dense[(uint64_t)q * P.out_stride + mr] = z;
+                        if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q * P.out_stride + mr] = nd;
+                    }
+                } else {
+                    P.out_dense[(uint64_t)q * P.out_stride + nd] = z;
+                }
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------
 // layer 0 fed by CSR rows (sparse operand): thread n owns output node n and walks
 // the row's nonzeros in id order; nonzero number j goes to partial sum j mod 32.
