@@ -308,7 +308,11 @@ def main():
         elif ms_by_stage["cluster"] > 0:
             kernel, ms, launches, nbytes = "cluster_network_kernel", ms_by_stage["cluster"], cnt_by_stage["cluster"], gb + hash_bytes(wl, bps.size)
         else:
-            kernel, ms, launches, nbytes = "gather_dot_kernel", ms_by_stage["gather_dot"], cnt_by_stage["gather_dot"], gb
+            esz = 2 if wl.dtype == "bf16" else 4
+            gather_layers = [l for l in range(len(wl.dims) - 1) if not (l == 0 and wl.first_sparse)]
+            short = all(wl.dims[l] * esz <= 512 for l in gather_layers)   # rows of one 512-byte round
+            kernel = "gather_short_kernel" if short else "gather_dot_kernel"
+            ms, launches, nbytes = ms_by_stage["gather_dot"], cnt_by_stage["gather_dot"], gb
         ms /= steps
         launches //= steps
         ach = nbytes / (ms / 1e3) / 1e9 if ms > 0 else 0.0
