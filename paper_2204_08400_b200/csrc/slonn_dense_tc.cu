@@ -37,8 +37,11 @@ constexpr uint32_t EPI_BYTES = EPI_WARPS * (32 * 33) * 4 + EPI_WARPS * 32 * 8; /
 constexpr uint32_t SMEM_BYTES = RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ + EPI_BYTES;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
-// instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = 256
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = bn (a multiple of 16)
+__device__ __forceinline__ uint32_t umma_idesc(uint32_t bn)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -94,13 +97,14 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
     return ((uint64_t)hi << 32) | lo;
 }
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate)
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(IDESC), "r"(accumulate)
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar)
@@ -134,13 +138,14 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float f)
 
 __global__ void __launch_bounds__(THREADS, 1)
 dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const slonn_dense_epilogue E, uint32_t N, uint32_t K)
+                const slonn_dense_epilogue E, uint32_t N, uint32_t K, uint32_t bn)
 {
+    // bn: columns per tile, a multiple of 16 up to BN (narrow layers take a narrower MMA and B tile)
     extern __shared__ unsigned char smem_raw[];
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
     // rows this launch must produce (a device-side count when the rows were compacted on the device)
     const uint32_t m_valid = E.row_count ? min(*E.row_count, E.M) : E.M;
-    const uint32_t m_tiles = (m_valid + BM - 1) / BM, n_tiles = (N + BN - 1) / BN;
+    const uint32_t m_tiles = (m_valid + BM - 1) / BM, n_tiles = (N + bn - 1) / bn;
     const uint32_t tiles = m_tiles * n_tiles;
     if (blockIdx.x >= tiles) return; // uniform for the block: nothing allocated yet
 
@@ -175,11 +180,11 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             uint32_t it = 0;
             bool ok = true;
             for (uint32_t t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
-                const uint32_t m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
+                const uint32_t m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * bn;
                 for (uint32_t kb = 0; kb < num_kb; ++kb, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!(ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag))) break;
-                    mbar_expect_tx(full0 + 8 * s, STAGE_A_BYTES + STAGE_B_BYTES);
+                    mbar_expect_tx(full0 + 8 * s, STAGE_A_BYTES + bn * BK * 2);
                     tma_load_2d(base + s * STAGE_A_BYTES, &map_a, (int32_t)(kb * BK), (int32_t)m0, full0 + 8 * s);
                     tma_load_2d(base + STAGES * STAGE_A_BYTES + s * STAGE_B_BYTES, &map_b, (int32_t)(kb * BK),
                                 (int32_t)n0, full0 + 8 * s);
@@ -191,6 +196,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (lane == 0) {
             uint32_t it = 0, ti = 0;
             bool ok = true;
+            const uint32_t idesc = umma_idesc(bn);
             for (uint32_t t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++ti) {
                 const uint32_t acc = ti & 1u, aph = (ti >> 1) & 1u;
                 if (!(ok = mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag))) break; // drained by the epilogue
@@ -204,7 +210,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     const uint64_t db = umma_desc(base + STAGES * STAGE_A_BYTES + s * STAGE_B_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) // 32 bytes further along K inside the swizzle atom
-                        umma_bf16(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), (kb | (uint32_t)k) != 0u);
+                        umma_bf16(d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | (uint32_t)k) != 0u);
                     umma_commit(empty0 + 8 * s); // frees the stage once these MMAs have read it
                 }
                 if (ok) umma_commit(tfull0 + 8 * acc); // accumulator complete
@@ -217,9 +223,15 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         float *tile = reinterpret_cast<float *>(smem_raw + (epi_addr - smem_u32(smem_raw))) + ew * (32 * 33);
         unsigned long long *row_off = reinterpret_cast<unsigned long long *>(
             smem_raw + (epi_addr - smem_u32(smem_raw)) + EPI_WARPS * (32 * 33) * sizeof(float)) + ew * 32;
+        // Row-major outputs with 16-byte aligned rows (no fp32 output addressed through per-row list
+        // offsets, no id output) can be written by the lane that holds the row.
+        const bool direct = !(E.out_f32 && E.indptr) && !E.out_ids &&
+                            (!E.bias || (reinterpret_cast<uintptr_t>(E.bias) & 15u) == 0u) &&
+                            (!E.out_f32 || ((reinterpret_cast<uintptr_t>(E.out_f32) & 15u) == 0u && (E.f32_stride & 3u) == 0u)) &&
+                            (!E.out_bf16 || ((reinterpret_cast<uintptr_t>(E.out_bf16) & 15u) == 0u && (E.ld_bf16 & 7u) == 0u));
         uint32_t ti = 0;
         for (uint32_t t = blockIdx.x; t < tiles; t += gridDim.x, ++ti) {
-            const uint32_t m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
+            const uint32_t m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * bn;
             const uint32_t acc = ti & 1u, aph = (ti >> 1) & 1u;
             // warp-uniform outcome of the wait
             if (!__all_sync(SLONN_FULL_MASK, mbar_wait(tfull0 + 8 * acc, aph, abort_flag))) break;
@@ -232,10 +244,49 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
             row_off[lane] = off;
             __syncwarp();
-            for (uint32_t c = 0; c < (uint32_t)BN; c += 32) {
+            for (uint32_t c = 0; c < bn; c += 32) {
                 if (n0 + c >= N) break; // columns past the layer width (uniform)
                 uint32_t r[32];
                 tmem_load32(tmem_base + ((quarter * 32u) << 16) + acc * BN + c, r); // whole warp takes part
+                if (direct && n0 + c + 32 <= N) {
+                    // plain row-major outputs, 32 whole columns: the lane owns a row of the tile and writes
+                    // its 32 values itself with 16-byte stores, no trip through shared memory
+                    const float4 *b4 = reinterpret_cast<const float4 *>(E.bias + n0 + c);
+                    float v[32];
+#pragma unroll
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        const float4 bb = E.bias ? __ldg(b4 + j4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        v[4 * j4 + 0] = __uint_as_float(r[4 * j4 + 0]) + bb.x;
+                        v[4 * j4 + 1] = __uint_as_float(r[4 * j4 + 1]) + bb.y;
+                        v[4 * j4 + 2] = __uint_as_float(r[4 * j4 + 2]) + bb.z;
+                        v[4 * j4 + 3] = __uint_as_float(r[4 * j4 + 3]) + bb.w;
+                    }
+                    if (E.relu) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = v[j] > 0.0f ? v[j] : 0.0f;
+                    }
+                    if (off != ~0ull) {
+                        if (E.out_f32) {
+                            float4 *dst = reinterpret_cast<float4 *>(E.out_f32 + off + n0 + c);
+#pragma unroll
+                            for (int j4 = 0; j4 < 8; ++j4)
+                                dst[j4] = make_float4(v[4 * j4], v[4 * j4 + 1], v[4 * j4 + 2], v[4 * j4 + 3]);
+                        }
+                        if (E.out_bf16) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(E.out_bf16 + (uint64_t)(mrow0 + lane) * E.ld_bf16 + n0 + c);
+#pragma unroll
+                            for (int j8 = 0; j8 < 4; ++j8) {
+                                uint4 o;
+                                o.x = (uint32_t)f32_to_bf16_rne(v[8 * j8 + 0]) | ((uint32_t)f32_to_bf16_rne(v[8 * j8 + 1]) << 16);
+                                o.y = (uint32_t)f32_to_bf16_rne(v[8 * j8 + 2]) | ((uint32_t)f32_to_bf16_rne(v[8 * j8 + 3]) << 16);
+                                o.z = (uint32_t)f32_to_bf16_rne(v[8 * j8 + 4]) | ((uint32_t)f32_to_bf16_rne(v[8 * j8 + 5]) << 16);
+                                o.w = (uint32_t)f32_to_bf16_rne(v[8 * j8 + 6]) | ((uint32_t)f32_to_bf16_rne(v[8 * j8 + 7]) << 16);
+                                dst[j8] = o;
+                            }
+                        }
+                    }
+                    continue;
+                }
 #pragma unroll
                 for (int j = 0; j < 32; ++j) tile[lane * 33 + j] = __uint_as_float(r[j]);
                 __syncwarp();
@@ -319,7 +370,8 @@ int slonn_dense_tc_launch(const void *A, const void *W, uint32_t N, uint32_t K, 
     CUtensorMap ma, mb;
     int rc;
     if ((rc = make_map(&ma, A, E.M, K, BM))) return rc;
-    if ((rc = make_map(&mb, W, N, K, BN))) return rc;
+    const uint32_t bn = std::min<uint32_t>((uint32_t)BN, (N + 15u) / 16u * 16u);
+    if ((rc = make_map(&mb, W, N, K, bn))) return rc;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(dense_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
@@ -333,9 +385,9 @@ int slonn_dense_tc_launch(const void *A, const void *W, uint32_t N, uint32_t K, 
             cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 1)
             return SLONN_ERR_CUDA;
     }
-    const uint64_t tiles = (uint64_t)((N + BN - 1) / BN) * ((E.M + BM - 1) / BM);
+    const uint64_t tiles = (uint64_t)((N + bn - 1) / bn) * ((E.M + BM - 1) / BM);
     const uint32_t grid = (uint32_t)std::min<uint64_t>(tiles, (uint64_t)sm_count); // one persistent block per SM
-    dense_tc_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, E, N, K);
+    dense_tc_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, E, N, K, bn);
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
