@@ -18,6 +18,7 @@
 // Sums are not bit-compatible with the fixed-order fp32 kernels (the tensor core's accumulation
 // order is not specified), so this path is only used where the caller asked for it.
 #include <cuda.h>
+#include <cuda_bf16.h>
 
 #include <algorithm>
 #include <cstring>
@@ -134,6 +135,13 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float f)
     if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u); // NaN stays NaN
     u += 0x7fffu + ((u >> 16) & 1u);
     return (uint16_t)(u >> 16);
+}
+
+// two fp32 -> two bf16 (round to nearest even) in one 32-bit word, `lo` in the low half
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&p);
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -277,10 +285,10 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
                             for (int j8 = 0; j8 < 4; ++j8) {
                                 uint4 o;
-                                o.x = (uint32_t)f32_to_bf16_rne(v[8 * j8 + 0]) | ((uint32_t)f32_to_bf16_rne(v[8 * j8 + 1]) << 16);
-                                o.y = (uint32_t)f32_to_bf16_rne(v[8 * j8 + 2]) | ((uint32_t)f32_to_bf16_rne(v[8 * j8 + 3]) << 16);
-                                o.z = (uint32_t)f32_to_bf16_rne(v[8 * j8 + 4]) | ((uint32_t)f32_to_bf16_rne(v[8 * j8 + 5]) << 16);
-                                o.w = (uint32_t)f32_to_bf16_rne(v[8 * j8 + 6]) | ((uint32_t)f32_to_bf16_rne(v[8 * j8 + 7]) << 16);
+                                o.x = pack_bf16x2(v[8 * j8 + 0], v[8 * j8 + 1]);
+                                o.y = pack_bf16x2(v[8 * j8 + 2], v[8 * j8 + 3]);
+                                o.z = pack_bf16x2(v[8 * j8 + 4], v[8 * j8 + 5]);
+                                o.w = pack_bf16x2(v[8 * j8 + 6], v[8 * j8 + 7]);
                                 dst[j8] = o;
                             }
                         }
