@@ -34,8 +34,13 @@ constexpr int THREADS = 192, EPI_WARPS = 4;
 constexpr uint32_t TMEM_COLS = 2 * BN; // two accumulators
 constexpr uint32_t STAGE_A_BYTES = BM * BK * 2, STAGE_B_BYTES = BN * BK * 2;
 constexpr uint32_t RING_BYTES = STAGES * (STAGE_A_BYTES + STAGE_B_BYTES);
-constexpr uint32_t EPI_BYTES = EPI_WARPS * (32 * 33) * 4 + EPI_WARPS * 32 * 8; // per-warp 32x33 fp32 tile + 32 row offsets
-constexpr uint32_t SMEM_BYTES = RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ + EPI_BYTES;
+// per epilogue warp: two 32-row x 128-byte output slabs (bf16 tiles on their way to a TMA store); the
+// 32x33 fp32 transpose tile of the list-output path lives in the same bytes
+constexpr uint32_t OUT_SLAB_BYTES = 32 * 128, OUT_STAGE_BYTES = EPI_WARPS * 2 * OUT_SLAB_BYTES;
+constexpr uint32_t ROW_OFF_BYTES = EPI_WARPS * 32 * 8; // 32 row offsets per epilogue warp
+constexpr uint32_t SMEM_BYTES = RING_BYTES + OUT_STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ + ROW_OFF_BYTES;
+static_assert(2 * OUT_SLAB_BYTES >= 32 * 33 * 4, "the transpose tile must fit in a warp's slabs");
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory per block");
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 // instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = bn (a multiple of 16)
@@ -87,6 +92,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst_smem), "l"(map), "r"(bar), "r"(c0), "r"(c1)
         : "memory");
+}
+
+// one 2-D tile from shared memory to global memory (rows and columns outside the tensor are dropped)
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src_smem, int32_t c0, int32_t c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src_smem), "r"(c0), "r"(c1)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
 // shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128 bytes,
@@ -146,8 +160,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 
 __global__ void __launch_bounds__(THREADS, 1)
 dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const slonn_dense_epilogue E, uint32_t N, uint32_t K, uint32_t bn)
+                const __grid_constant__ CUtensorMap map_out, uint32_t tma_out, const slonn_dense_epilogue E, uint32_t N,
+                uint32_t K, uint32_t bn)
 {
+    // map_out / tma_out: the bf16 output matrix as a tensor of 64-column x 32-row boxes (128-byte swizzle),
+    // valid when tma_out != 0
     // bn: columns per tile, a multiple of 16 up to BN (narrow layers take a narrower MMA and B tile)
     extern __shared__ unsigned char smem_raw[];
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
@@ -158,7 +175,8 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     if (blockIdx.x >= tiles) return; // uniform for the block: nothing allocated yet
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u; // swizzle atoms need 1024-byte alignment
-    const uint32_t bars = base + RING_BYTES;
+    const uint32_t out_stage0 = base + RING_BYTES; // 1024-byte aligned
+    const uint32_t bars = out_stage0 + OUT_STAGE_BYTES;
     const uint32_t full0 = bars, empty0 = bars + 8 * STAGES;
     const uint32_t tfull0 = bars + 16 * STAGES, tempty0 = tfull0 + 16;
     const uint32_t tmem_slot_addr = tempty0 + 16;
@@ -228,9 +246,10 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // ---- epilogue warps: TMEM lane = row of the tile, TMEM column = column of the tile ----
         const uint32_t ew = warp - 2;        // slice of the staging area
         const uint32_t quarter = warp & 3u;  // the TMEM lanes 32*quarter .. +31 this warp may read
-        float *tile = reinterpret_cast<float *>(smem_raw + (epi_addr - smem_u32(smem_raw))) + ew * (32 * 33);
-        unsigned long long *row_off = reinterpret_cast<unsigned long long *>(
-            smem_raw + (epi_addr - smem_u32(smem_raw)) + EPI_WARPS * (32 * 33) * sizeof(float)) + ew * 32;
+        const uint32_t slab0 = out_stage0 + ew * 2 * OUT_SLAB_BYTES;
+        float *tile = reinterpret_cast<float *>(smem_raw + (slab0 - smem_u32(smem_raw)));
+        unsigned long long *row_off = reinterpret_cast<unsigned long long *>(smem_raw + (epi_addr - smem_u32(smem_raw))) + ew * 32;
+        uint32_t slab_turn = 0; // alternates between the warp's two output slabs
         // Row-major outputs with 16-byte aligned rows (no fp32 output addressed through per-row list
         // offsets, no id output) can be written by the lane that holds the row.
         const bool direct = !(E.out_f32 && E.indptr) && !E.out_ids &&
@@ -252,6 +271,64 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
             row_off[lane] = off;
             __syncwarp();
+            if (direct && tma_out) {
+                // bf16 outputs through shared memory and a TMA store: the lane converts its row of the
+                // tile, 64 columns (128 bytes) at a time, into a swizzled slab; one lane then sends the slab
+                // as a single tiled copy, so global memory sees whole 128-byte lines.
+                for (uint32_t c2 = 0; c2 < bn; c2 += 64) {
+                    if (n0 + c2 >= N) break; // uniform
+                    const uint32_t slab = slab0 + (slab_turn & 1u) * OUT_SLAB_BYTES;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); // the copy before last has read this slab
+                    __syncwarp();
+#pragma unroll
+                    for (uint32_t half = 0; half < 2; ++half) {
+                        const uint32_t c = c2 + 32u * half;
+                        if (c >= bn || n0 + c >= N) continue; // uniform; the copy drops these columns
+                        uint32_t r[32];
+                        tmem_load32(tmem_base + ((quarter * 32u) << 16) + acc * BN + c, r);
+                        float v[32];
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; ++j4) {
+                            float4 bb = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (E.bias && n0 + c + 4 * j4 + 3 < N) bb = __ldg(reinterpret_cast<const float4 *>(E.bias + n0 + c) + j4);
+                            v[4 * j4 + 0] = __uint_as_float(r[4 * j4 + 0]) + bb.x;
+                            v[4 * j4 + 1] = __uint_as_float(r[4 * j4 + 1]) + bb.y;
+                            v[4 * j4 + 2] = __uint_as_float(r[4 * j4 + 2]) + bb.z;
+                            v[4 * j4 + 3] = __uint_as_float(r[4 * j4 + 3]) + bb.w;
+                        }
+                        if (E.relu) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = v[j] > 0.0f ? v[j] : 0.0f;
+                        }
+                        if (E.out_f32 && off != ~0ull && n0 + c + 32 <= N) {
+                            float4 *dst = reinterpret_cast<float4 *>(E.out_f32 + off + n0 + c);
+#pragma unroll
+                            for (int j4 = 0; j4 < 8; ++j4)
+                                dst[j4] = make_float4(v[4 * j4], v[4 * j4 + 1], v[4 * j4 + 2], v[4 * j4 + 3]);
+                        } else if (E.out_f32 && off != ~0ull) {
+                            for (int j = 0; j < 32; ++j)
+                                if (n0 + c + j < N) E.out_f32[off + n0 + c + j] = v[j];
+                        }
+#pragma unroll
+                        for (uint32_t j8 = 0; j8 < 4; ++j8) {
+                            uint4 o;
+                            o.x = pack_bf16x2(v[8 * j8 + 0], v[8 * j8 + 1]);
+                            o.y = pack_bf16x2(v[8 * j8 + 2], v[8 * j8 + 3]);
+                            o.z = pack_bf16x2(v[8 * j8 + 4], v[8 * j8 + 5]);
+                            o.w = pack_bf16x2(v[8 * j8 + 6], v[8 * j8 + 7]);
+                            // 128-byte swizzle: 16-byte unit u of row `lane` sits at unit u ^ (lane & 7)
+                            const uint32_t unit = (half * 4u + j8) ^ (lane & 7u);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                         ::"r"(slab + lane * 128u + unit * 16u), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w)
+                                         : "memory");
+                        }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); // generic-proxy writes before the bulk copy reads
+                    __syncwarp();
+                    if (lane == 0 && mrow0 < E.M) tma_store_2d(&map_out, slab, (int32_t)(n0 + c2), (int32_t)mrow0);
+                    ++slab_turn;
+                }
+            } else
             for (uint32_t c = 0; c < bn; c += 32) {
                 if (n0 + c >= N) break; // columns past the layer width (uniform)
                 uint32_t r[32];
@@ -317,6 +394,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); // output copies done before the block may leave
     }
     __syncwarp();
     if (*abort_flag) {
@@ -353,14 +431,16 @@ encode_tiled_fn get_encode()
     return fn;
 }
 
-// bf16 matrix [rows][cols] row-major, tiles of box_rows rows x 64 columns, 128-byte swizzle, zero fill outside
-int make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols, uint32_t box_rows)
+// bf16 matrix [rows][cols] row-major with rows `ld` elements apart, tiles of box_rows rows x 64 columns,
+// 128-byte swizzle, zero fill outside
+int make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, uint64_t ld = 0)
 {
     encode_tiled_fn enc = get_encode();
     if (!enc) return SLONN_ERR_CUDA;
-    if (((uintptr_t)ptr & 15u) || ((cols * 2) & 15u)) return SLONN_ERR_ALIGN;
+    if (ld == 0) ld = cols;
+    if (((uintptr_t)ptr & 15u) || ((ld * 2) & 15u)) return SLONN_ERR_ALIGN;
     const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint64_t strides[1] = {ld * 2};
     const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
@@ -393,9 +473,18 @@ int slonn_dense_tc_launch(const void *A, const void *W, uint32_t N, uint32_t K, 
             cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 1)
             return SLONN_ERR_CUDA;
     }
+    // bf16 outputs leave through a TMA store when nothing needs per-row list addressing
+    CUtensorMap mo;
+    memset(&mo, 0, sizeof(mo));
+    uint32_t tma_out = 0;
+    if (E.out_bf16 && !(E.out_f32 && E.indptr) && !E.out_ids && ((uintptr_t)E.out_bf16 & 15u) == 0 && (E.ld_bf16 & 7u) == 0 &&
+        E.ld_bf16 >= N) {
+        if ((rc = make_map(&mo, E.out_bf16, E.M, N, 32, E.ld_bf16))) return rc;
+        tma_out = 1;
+    }
     const uint64_t tiles = (uint64_t)((N + bn - 1) / bn) * ((E.M + BM - 1) / BM);
     const uint32_t grid = (uint32_t)std::min<uint64_t>(tiles, (uint64_t)sm_count); // one persistent block per SM
-    dense_tc_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, E, N, K, bn);
+    dense_tc_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, mo, tma_out, E, N, K, bn);
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 

@@ -41,6 +41,8 @@ def run_dense(M, N, D, relu, seed):
     (200, 1000, 4096, False),    # ragged rows and columns (zero-filled tile edges)
     (77, 10, 784, True),         # K tail inside a 64-wide step, tiny N
     (1, 4096, 2048, True),       # a single row
+    (100, 40, 128, True),        # narrow layer: 48-column tile, output columns dropped by the tiled store
+    (300, 72, 192, False),       # 80-column tile: a second, partly filled 64-column output slab
 ])
 def test_dense_layer_matches_float64_matmul(M, N, D, relu):
     run_dense(M, N, D, relu, seed=M + N + D)
