@@ -44,6 +44,14 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def measured_tensor_peak():
+    """Dense bf16 TFLOP/s of a kernel timed alone (the burst figure)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["bf16_tflops"]), "measured"
+    return 1590.0, "fallback"
+
+
 def hash_bytes(wl, n):
     """Weight bytes of the FreeHash rows of one step: K*L rows per query and activator layer."""
     esz = 2 if wl.dtype == "bf16" else 4
@@ -302,6 +310,8 @@ def main():
             stage_ms[s] += ms[s]; stage_cnt[s] += cnt[s]
     def stage_roofline(ms_by_stage, cnt_by_stage, bps, steps):
         """Dominant kernel of the step and its achieved rate on the weight bytes it must touch."""
+        if flags & sl.FLAG_DENSE_TC:     # queries at 100 % leave the row kernels
+            bps = bps[bps != 10000]
         gb = sum(gathered_bytes(wl, bps))
         if ms_by_stage["fused"] > 0:     # one launch does hash + select + gather for every layer
             kernel, ms, launches, nbytes = "fused_network_kernel", ms_by_stage["fused"], cnt_by_stage["fused"], gb + hash_bytes(wl, bps.size)
@@ -327,6 +337,18 @@ def main():
                 "bytes_per_step": int(k_bytes), "launches_per_step": k_launches,
                 "avg_launch_ms": k_ms / max(k_launches, 1),
                 "stage_ms_per_step": {s: stage_ms[s] / prof_steps for s in sl.STAGES}}
+    if stage_ms["dense_tc"] >= max(stage_ms.values()):
+        # the step is dominated by the tensor-core route: its roofline is the tensor pipe.  The stage time
+        # covers the compaction of the routed queries and the bf16 copy of their inputs as well.
+        n_tc = int((wl.budget_bp == 10000).sum())
+        flops = sum(2.0 * n_tc * wl.dims[l] * wl.dims[l + 1] for l in range(len(wl.dims) - 1))
+        tc_ms = stage_ms["dense_tc"] / prof_steps
+        tpeak, tkind = measured_tensor_peak()
+        ach = flops / (tc_ms / 1e3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "dense_tc_kernel", "achieved": ach, "peak": tpeak, "unit": "TFLOP/s",
+                    "frac": ach / tpeak, "peak_kind": tkind, "traffic": None, "flops_per_step": flops,
+                    "launches_per_step": len(wl.dims) - 1, "avg_launch_ms": tc_ms / (len(wl.dims) - 1),
+                    "stage_ms_per_step": {s: stage_ms[s] / prof_steps for s in sl.STAGES}}
 
     # ---- budget sweep (the latency profile T(k, isolated) of the paper) ----
     sweep = {}
@@ -357,12 +379,12 @@ def main():
         if wl.first_sparse:
             h_csr = tuple(pinv(a) for a in wl.x)
             hb = sl.make_batch(n, h_bp, h_logits, h_status, x_csr=h_csr, max_budget_bp=max_bp,
-                               logit_ids=h_lids, pred=h_pred)
+                               logit_ids=h_lids, pred=h_pred, flags=flags)
         else:
             h_x = pin(wl.x)
             hb = sl.make_batch(n, h_bp, h_logits, h_status, x_dense=h_x, max_budget_bp=max_bp,
-                               logit_ids=h_lids, pred=h_pred)
-        nb = sl.slonn_host_workspace_bytes(dm.model, n, max_bp, x_nnz)
+                               logit_ids=h_lids, pred=h_pred, flags=flags)
+        nb = sl.slonn_host_workspace_bytes(dm.model, n, max_bp, x_nnz, flags)
         hws = torch.empty(nb, dtype=torch.uint8, device=dev)
         e_steps = max(3, min(args.steps, 10))
         for _ in range(3):
