@@ -193,17 +193,13 @@ __device__ __forceinline__ void warp_dot_rows(const uint4 *const (&rows)[R], con
 }
 
 // Fixed-order dot product of ONE weight row, for launches where latency matters more than
-// throughput (a handful of queries): up to 8 of the lane's 16-byte chunks are in flight at once.
-// Same chunk-to-lane assignment, same order within a lane, xor butterfly 16, 8, 4, 2, 1; every
-// lane returns the sum (bias not included).
-template <bool BF16>
+// throughput (a handful of queries): up to DEPTH of the lane's 16-byte chunks are in flight at once
+// (chunks of this lane loaded before the first one is used).  Same chunk-to-lane assignment, same
+// order within a lane, xor butterfly 16, 8, 4, 2, 1; every lane returns the sum (bias not included).
+template <bool BF16, int DEPTH = 8>
 __device__ __forceinline__ float warp_dot_row1(const uint4 *row, const float4 *xs4, uint32_t nchunks, uint32_t lane)
 {
     constexpr int VPC = BF16 ? 8 : 4;
-#ifndef SLONN_ROW1_DEPTH
-#define SLONN_ROW1_DEPTH 8
-#endif
-    constexpr int DEPTH = SLONN_ROW1_DEPTH; // chunks of this lane loaded before the first one is used
     float acc[1] = {0.0f};
     for (uint32_t c0 = lane; c0 < nchunks; c0 += 32 * DEPTH) {
         uint4 w[DEPTH][1];
