@@ -14,9 +14,6 @@
 #ifndef SLONN_FUSED_WARPS
 #define SLONN_FUSED_WARPS 4         // queries (warps) per block
 #endif
-#ifndef SLONN_FUSED_GROUP
-#define SLONN_FUSED_GROUP 1         // 32-chunk rounds whose loads are issued together
-#endif
 #ifndef SLONN_FUSED_MIN_BLOCKS
 #define SLONN_FUSED_MIN_BLOCKS 5    // resident blocks per SM the register allocation must allow
 #endif
@@ -96,13 +93,15 @@ __device__ __forceinline__ void fused_load_x_shared(float (&xr)[NC * fused_trait
 
 // Fixed-order partial sums of R rows against the register-resident input: lane p ends
 // with partial p of every row (the caller reduces them).
-template <bool BF16, int NC, int R>
+// GRP: 32-chunk rounds whose loads are issued together (1 when the batch fills the GPU and registers are
+// better spent on resident warps; all of them when a few warps have an SM to themselves).
+template <bool BF16, int NC, int R, int GRP>
 __device__ __forceinline__ void fused_dot_rows(const uint4 *const (&rows)[R],
                                                const float (&xr)[NC * fused_traits<BF16>::VPC], uint32_t nchunks,
                                                uint32_t lane, float (&acc)[R])
 {
     constexpr int VPC = fused_traits<BF16>::VPC;
-    constexpr int G = NC < SLONN_FUSED_GROUP ? NC : SLONN_FUSED_GROUP; // rounds whose loads are issued together
+    constexpr int G = NC < GRP ? NC : GRP; // rounds whose loads are issued together
 #pragma unroll
     for (int r = 0; r < R; ++r) acc[r] = 0.0f;
 #pragma unroll
@@ -194,8 +193,9 @@ __device__ __forceinline__ void fused_select(const slonn_fused_layer &ly, uint32
     __syncwarp();
 }
 
-template <bool BF16, int NC>
-__global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, SLONN_FUSED_MIN_BLOCKS) fused_network_kernel(const __grid_constant__ slonn_fused_params P)
+template <bool BF16, int NC, int GRP>
+__global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, GRP == 1 ? SLONN_FUSED_MIN_BLOCKS : 1)
+fused_network_kernel(const __grid_constant__ slonn_fused_params P)
 {
     constexpr int VPC = fused_traits<BF16>::VPC;
     constexpr int R = SLONN_FUSED_ROWS;
@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, SLONN_FUSED_MIN_BLOCKS
                     rows[k] = reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)nd * ly.nchunks;
                 }
                 float acc[R];
-                fused_dot_rows<BF16, NC, R>(rows, xr, ly.nchunks, lane, acc);
+                fused_dot_rows<BF16, NC, R, GRP>(rows, xr, ly.nchunks, lane, acc);
                 // lanes 8k..8k+7 hold the sum of row k; collect the R signs with one ballot
                 const uint32_t mynode = __ldg(ly.hash_nodes + min(h0 + (lane >> 3), H - 1));
                 const float z = reduce_rows4(acc, lane) + __ldg(ly.bias + mynode);
@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, SLONN_FUSED_MIN_BLOCKS
                 rows[k] = reinterpret_cast<const uint4 *>(ly.W) + (uint64_t)nd * ly.nchunks;
             }
             float acc[R];
-            fused_dot_rows<BF16, NC, R>(rows, xr, ly.nchunks, lane, acc);
+            fused_dot_rows<BF16, NC, R, GRP>(rows, xr, ly.nchunks, lane, acc);
             const float sum = reduce_rows4(acc, lane); // row r0 + (lane >> 3)
             const uint32_t r = r0 + (lane >> 3);
             if ((lane & 7u) == 0u && r < B) {

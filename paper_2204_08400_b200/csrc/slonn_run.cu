@@ -210,15 +210,25 @@ bool fused_eligible(const slonn_model *m)
     return true;
 }
 
+template <bool BF16, int NC, int GRP>
+int launch_fused_g(const slonn_fused_params &P, cudaStream_t st)
+{
+    const size_t smem = (size_t)P.warp_bytes * SLONN_FUSED_WARPS;
+    int rc = set_smem(fused_network_kernel<BF16, NC, GRP>, smem);
+    if (rc) return rc;
+    const uint32_t grid = (P.n + SLONN_FUSED_WARPS - 1) / SLONN_FUSED_WARPS;
+    fused_network_kernel<BF16, NC, GRP><<<grid, SLONN_FUSED_WARPS * 32, smem, st>>>(P);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+// Batches of at most two blocks per SM: up to four load rounds of a row pass in flight at once (the few
+// resident warps can have all the registers); larger batches: one round, five blocks per SM.
 template <bool BF16, int NC>
 int launch_fused_t(const slonn_fused_params &P, cudaStream_t st)
 {
-    const size_t smem = (size_t)P.warp_bytes * SLONN_FUSED_WARPS;
-    int rc = set_smem(fused_network_kernel<BF16, NC>, smem);
-    if (rc) return rc;
     const uint32_t grid = (P.n + SLONN_FUSED_WARPS - 1) / SLONN_FUSED_WARPS;
-    fused_network_kernel<BF16, NC><<<grid, SLONN_FUSED_WARPS * 32, smem, st>>>(P);
-    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+    if (NC > 1 && grid <= 2u * 148u) return launch_fused_g<BF16, NC, (NC > 4 ? 4 : NC)>(P, st);
+    return launch_fused_g<BF16, NC, 1>(P, st);
 }
 
 int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *indptr, uint32_t stride,
