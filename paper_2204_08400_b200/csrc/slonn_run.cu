@@ -131,7 +131,7 @@ int launch_select(const slonn_model *m, const slonn_select_params &P, uint32_t n
     const bool id16 = m->layer[P.layer].id_bytes == 2;
     const bool few = n <= 148, long_lists = (uint64_t)max_rows * m->L >= 32768;
     const bool lat = few || long_lists;
-    const uint32_t threads = long_lists ? 1024u : few ? 32u * std::min(32u, std::max(8u, m->H)) : (uint32_t)SLONN_THREADS;
+    const uint32_t threads = long_lists ? (n > 148u ? 512u : 1024u) : few ? 32u * std::min(32u, std::max(8u, m->H)) : (uint32_t)SLONN_THREADS;
     if (lat) {
         if (bf && id16) return launch_select_t<true, uint16_t, true>(P, n, threads, smem, st);
         if (bf) return launch_select_t<true, uint32_t, true>(P, n, threads, smem, st);

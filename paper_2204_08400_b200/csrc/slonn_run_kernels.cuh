@@ -181,22 +181,57 @@ __device__ __forceinline__ bool block_select(const void *tables, uint32_t cap, u
     // that many new ids, so the count never passes `want`, and when it reaches it the marked ids are
     // exactly the distinct ids of a prefix of the position sequence -- the first `want` distinct ones.
     // (Which of two equal ids inside a step wins the atomic does not matter: one does.)
-    // Each thread fetches its entries of the next four rows of blockDim.x positions in one go.
+    // Each thread fetches its entries of the next SEL_ROWS rows of blockDim.x positions in one go; while
+    // more ids are missing than the whole window holds, the window is one step (one block-wide sum of
+    // the new ids), afterwards the steps follow the rows and shrink with the ids still missing.
+    constexpr int SEL_ROWS = 8;
     const uint32_t npos = want * L; // `want` distinct ids are always found within rank < want
     const uint32_t T = blockDim.x;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = (T + 31u) >> 5;
     uint32_t total = 0;
-    for (uint32_t w0 = 0; w0 < npos && total < want; w0 += 4 * T) {
-        uint32_t ahead[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+    // When the block size is a multiple of L a thread always reads the same table: its list and the
+    // rank stride between its positions are fixed, and no division is left in the loop.
+    const bool fixed_table = (T % L) == 0u;
+    const uint32_t my_b = threadIdx.x % L, my_r = threadIdx.x / L, r_step = T / L;
+    const IDT *my_list = reinterpret_cast<const IDT *>(tables) + (((uint64_t)my_b << K) + keys[my_b]) * cap;
+    for (uint32_t w0 = 0; w0 < npos && total < want; w0 += SEL_ROWS * T) {
+        uint32_t ahead[SEL_ROWS];
+        if (fixed_table) {
+            const uint32_t r0 = w0 / L + my_r;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const uint32_t p = w0 + u * T + threadIdx.x;
-            if (p < npos) {
-                const uint32_t r = p / L, b = p - r * L;
-                ahead[u] = table_entry<IDT>(tables, cap, K, b, keys[b], r);
+            for (int u = 0; u < SEL_ROWS; ++u) {
+                const uint32_t p = w0 + u * T + threadIdx.x;
+                ahead[u] = p < npos ? (uint32_t)__ldg(my_list + r0 + u * r_step) : 0xffffffffu;
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < SEL_ROWS; ++u) {
+                const uint32_t p = w0 + u * T + threadIdx.x;
+                ahead[u] = 0xffffffffu;
+                if (p < npos) {
+                    const uint32_t r = p / L, b = p - r * L;
+                    ahead[u] = table_entry<IDT>(tables, cap, K, b, keys[b], r);
+                }
             }
         }
+        const uint32_t window = min((uint32_t)SEL_ROWS * T, npos - w0);
+        if (want - total >= window) { // uniform: the whole window cannot overshoot
+            uint32_t wins = 0;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < SEL_ROWS; ++u)
+                if (ahead[u] < N) {
+                    const uint32_t bit = 1u << (ahead[u] & 31u);
+                    wins += ((atomicOr(&bitmap[ahead[u] >> 5], bit) & bit) == 0u) ? 1u : 0u;
+                }
+            wins = __reduce_add_sync(SLONN_FULL_MASK, wins);
+            if (lane == 0) scan_ws[warp] = wins;
+            __syncthreads();
+            total += __reduce_add_sync(SLONN_FULL_MASK, lane < nwarps ? scan_ws[lane] : 0u);
+            __syncthreads(); // scan_ws is reused by the next window and by the emit below
+            continue;
+        }
+#pragma unroll
+        for (int u = 0; u < SEL_ROWS; ++u) {
             const uint32_t row0 = w0 + u * T;              // this row holds positions row0 .. row0 + T - 1
             const uint32_t row1 = min(row0 + T, npos);
             const uint32_t mine = row0 + threadIdx.x;
