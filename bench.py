@@ -198,6 +198,9 @@ def main():
                     help="route 100 %% budget queries to the tensor-core dense path (not bit-exact for them)")
     ap.add_argument("--free-hash-nodes", action="store_true",
                     help="the variant in which a layer's K*L hash nodes are always active and absent from its lists")
+    ap.add_argument("--row-kernels", action="store_true", help="sparse-input layers: force the row kernels")
+    ap.add_argument("--column-kernels", action="store_true", help="sparse-input layers: force the input-stationary kernels")
+    ap.add_argument("--kernel-path", type=int, default=0, help="0 auto, 1 per-stage kernels, 2 one warp per query, 3 cluster")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline", action="store_true", help="time the oracle also for workloads other than c1/c2")
@@ -254,7 +257,10 @@ def main():
 
     # ---- headline: device-resident inputs ----
     flags = sl.FLAG_DENSE_TC if args.dense_tc else 0
-    batch = harness.DeviceBatch(dm, wl.x, wl.budget_bp, max_budget_bp=max_bp, full_outputs=False, flags=flags)
+    flags |= sl.FLAG_ROW_KERNELS if args.row_kernels else 0
+    flags |= sl.FLAG_COLUMN_KERNELS if args.column_kernels else 0
+    batch = harness.DeviceBatch(dm, wl.x, wl.budget_bp, max_budget_bp=max_bp, full_outputs=False, flags=flags,
+                                kernel_path=args.kernel_path)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -355,7 +361,8 @@ def main():
     if not args.no_sweep and world == 1:
         for bp in wl.budgets_named:
             bps = np.full(n, bp, np.uint16)
-            b2 = harness.DeviceBatch(dm, wl.x, bps, max_budget_bp=bp, full_outputs=False, flags=flags)
+            b2 = harness.DeviceBatch(dm, wl.x, bps, max_budget_bp=bp, full_outputs=False, flags=flags,
+                                     kernel_path=args.kernel_path)
             ms2 = timed(b2, max(3, args.steps // 4), 3)
             st_ms, st_cnt = sl.slonn_run_timed(dm.model, b2.batch, b2.ws, b2.ws_bytes, stream)
             k2, _, _, _, ach2 = stage_roofline(st_ms, st_cnt, bps, 1)

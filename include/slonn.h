@@ -20,7 +20,9 @@
  *   - Ownership: the caller owns every buffer it passes in.  Weights and biases
  *     given to slonn_build are referenced, not copied: they must stay valid and
  *     unchanged until slonn_free.  The library owns what it allocates inside
- *     slonn_model (tables, hash-node ids, a transposed first-layer copy).
+ *     slonn_model (tables, hash-node ids, transposed copies of a CSR-fed first
+ *     layer and of every layer that follows an activator layer -- a snapshot of
+ *     those weights taken at build time).
  *   - A model is read-only after slonn_build; slonn_run may be called
  *     concurrently on different streams with different workspaces.
  *   - Arithmetic: every dot product is summed in fp32 in one fixed order (32
@@ -206,6 +208,18 @@ typedef struct {
  * layer has no activator and max_budget_bp is 10000 (or 0); otherwise ignored.
  */
 #define SLONN_FLAG_DENSE_TC 1u
+/*
+ * A layer whose input is the sparse output of an activator layer (Sec. 3.3) can be evaluated in two
+ * ways with identical results: row kernels read each selected weight row whole; input-stationary
+ * kernels walk the query's nonzero inputs and read single weights from a transposed copy the model
+ * keeps of such layers.  By default the library picks per query by budget (sparse inputs take the
+ * input-stationary kernels).  These two flags force one kind for the whole batch, for testing and
+ * tuning; setting both is an error.  They apply to the per-stage kernels (SLONN_PATH_STAGED or
+ * networks too wide for the one-warp-per-query kernel).
+ */
+#define SLONN_FLAG_ROW_KERNELS 2u
+#define SLONN_FLAG_COLUMN_KERNELS 4u
+#define SLONN_FLAG_ALL 7u
 
 #define SLONN_PATH_AUTO 0    /* library chooses                                               */
 #define SLONN_PATH_STAGED 1  /* one block per query and stage: any width, any batch size      */

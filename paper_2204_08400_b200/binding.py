@@ -426,6 +426,8 @@ def slonn_run_static(model: Model, batch: _Batch, stream=None) -> None:
 
 STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused", "dense_tc", "cluster")
 FLAG_DENSE_TC = 1
+FLAG_ROW_KERNELS = 2
+FLAG_COLUMN_KERNELS = 4
 PATH_AUTO, PATH_STAGED, PATH_FUSED, PATH_CLUSTER = 0, 1, 2, 3
 
 

@@ -51,6 +51,127 @@ __global__ void transpose_kernel(const void *W, void *WT, uint32_t N, uint32_t D
     }
 }
 
+// WT[d][colpos[n]] = W[n][d]: transposed copy with the node axis re-ordered
+__global__ void transpose_permuted_kernel(const void *W, void *WT, uint32_t N, uint32_t D, uint32_t esz,
+                                          const uint32_t *colpos)
+{
+    __shared__ uint32_t tile[32][33];
+    const uint32_t d0 = blockIdx.x * 32, n0 = blockIdx.y * 32;
+    for (uint32_t i = threadIdx.y; i < 32; i += blockDim.y) {
+        const uint32_t n = n0 + i, d = d0 + threadIdx.x;
+        uint32_t v = 0;
+        if (n < N && d < D)
+            v = esz == 2 ? (uint32_t)reinterpret_cast<const uint16_t *>(W)[(uint64_t)n * D + d]
+                         : reinterpret_cast<const uint32_t *>(W)[(uint64_t)n * D + d];
+        tile[i][threadIdx.x] = v;
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.y; i < 32; i += blockDim.y) {
+        const uint32_t d = d0 + i, n = n0 + threadIdx.x;
+        if (n < N && d < D) {
+            const uint32_t v = tile[threadIdx.x][i];
+            const uint64_t at = (uint64_t)d * N + colpos[n];
+            if (esz == 2) reinterpret_cast<uint16_t *>(WT)[at] = (uint16_t)v;
+            else reinterpret_cast<uint32_t *>(WT)[at] = v;
+        }
+    }
+}
+
+// WH[d][h] = W[hash_nodes[h]][d] for h < H, zero for H <= h < 32: the layer's hash rows side by side,
+// so that one input d needs one 64- or 128-byte line for all hash functions
+__global__ void hash_matrix_kernel(const void *W, void *WH, uint32_t D, uint32_t esz, const uint32_t *hash_nodes,
+                                   uint32_t H)
+{
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t d = t >> 5, h = t & 31u;
+    if (d >= D) return;
+    uint32_t v = 0;
+    if (h < H) {
+        const uint64_t at = (uint64_t)hash_nodes[h] * D + d;
+        v = esz == 2 ? (uint32_t)reinterpret_cast<const uint16_t *>(W)[at] : reinterpret_cast<const uint32_t *>(W)[at];
+    }
+    if (esz == 2) reinterpret_cast<uint16_t *>(WH)[t] = (uint16_t)v;
+    else reinterpret_cast<uint32_t *>(WH)[t] = v;
+}
+
+// How early each node appears in the layer's ranked lists: score[n] = sum over all lists of
+// max(0, T - rank of n in the list).  Integer sums, so the result does not depend on thread order.
+template <typename IDT>
+__global__ void popularity_kernel(const IDT *tables, uint64_t n_lists, uint32_t cap, uint32_t T, uint32_t N,
+                                  unsigned long long *score)
+{
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t list = t / T;
+    const uint32_t r = (uint32_t)(t - list * T);
+    if (list >= n_lists) return;
+    const uint32_t id = (uint32_t)tables[list * cap + r];
+    if (id < N) atomicAdd(score + id, (unsigned long long)(T - r));
+}
+
+// Library-owned copies for the input-stationary kernels (layers whose input is the (id, value) list of
+// an activator layer below them):
+//   WT      transposed weights [D][N]; on a layer that has its own activator the node axis is stored in
+//           the order of `colpos`: nodes that sit early in many ranked lists first, so that the nodes a
+//           query selects lie close together in every row of WT
+//   colpos  [N] node id -> column of WT (activator layers only; NULL = identity)
+//   WH      [D][32] the layer's hash rows side by side (activator layers with K*L <= 32)
+// and the plain transposed copy of a first layer fed by CSR rows.  phase 0: the CSR first layer (needed
+// by the calibration pass); phase 1: the rest (needs the finished tables).
+// Copies whose element index would not fit 32 bits are left out (such layers keep the row kernels).
+int make_transposed_copies(slonn_model *m, cudaStream_t st, int phase)
+{
+    const uint32_t esz = m->dtype == SLONN_BF16 ? 2u : 4u;
+    for (uint32_t l = 0; l < m->n_layers; ++l) {
+        slonn_layer &ly = m->layer[l];
+        const bool csr_first = (l == 0 && m->first_sparse);
+        const bool list_input = (l > 0 && m->layer[l - 1].has_act && (uint64_t)ly.N * ly.D < (1ull << 32));
+        if (phase == 0 ? !csr_first : !list_input) continue;
+        if (cudaMalloc(&ly.WT, (uint64_t)ly.N * ly.D * esz) != cudaSuccess) return SLONN_ERR_NOMEM;
+        const dim3 grid((ly.D + 31) / 32, (ly.N + 31) / 32), block(32, 8);
+        if (!ly.has_act || csr_first) {
+            transpose_kernel<<<grid, block, 0, st>>>(ly.W, ly.WT, ly.N, ly.D, esz);
+            if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+            continue;
+        }
+        // order of the node axis: by popularity in the lists, equal scores by lower id
+        const uint64_t n_lists = (uint64_t)m->L << m->K;
+        const uint32_t T = std::max(1u, std::min(ly.cap, (ly.N + 7u) / 8u));
+        unsigned long long *d_score = nullptr;
+        if (cudaMalloc(&d_score, sizeof(unsigned long long) * ly.N) != cudaSuccess) return SLONN_ERR_NOMEM;
+        std::vector<unsigned long long> score(ly.N);
+        std::vector<uint32_t> order(ly.N), colpos(ly.N);
+        bool ok = cudaMemsetAsync(d_score, 0, sizeof(unsigned long long) * ly.N, st) == cudaSuccess;
+        if (ok) {
+            const uint64_t threads = n_lists * T;
+            const uint32_t blocks = (uint32_t)((threads + 255) / 256);
+            if (ly.id_bytes == 2)
+                popularity_kernel<uint16_t><<<blocks, 256, 0, st>>>((const uint16_t *)ly.tables, n_lists, ly.cap, T, ly.N, d_score);
+            else
+                popularity_kernel<uint32_t><<<blocks, 256, 0, st>>>((const uint32_t *)ly.tables, n_lists, ly.cap, T, ly.N, d_score);
+            ok = cudaGetLastError() == cudaSuccess &&
+                 cudaMemcpyAsync(score.data(), d_score, sizeof(unsigned long long) * ly.N, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+                 cudaStreamSynchronize(st) == cudaSuccess;
+        }
+        cudaFree(d_score);
+        if (!ok) return SLONN_ERR_CUDA;
+        for (uint32_t i = 0; i < ly.N; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return score[a] > score[b]; });
+        for (uint32_t i = 0; i < ly.N; ++i) colpos[order[i]] = i;
+        if (cudaMalloc(&ly.colpos, sizeof(uint32_t) * ly.N) != cudaSuccess) return SLONN_ERR_NOMEM;
+        if (cudaMemcpyAsync(ly.colpos, colpos.data(), sizeof(uint32_t) * ly.N, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return SLONN_ERR_CUDA;
+        transpose_permuted_kernel<<<grid, block, 0, st>>>(ly.W, ly.WT, ly.N, ly.D, esz, ly.colpos);
+        if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+        if (m->H <= 32) {
+            if (cudaMalloc(&ly.WH, (uint64_t)ly.D * 32 * esz) != cudaSuccess) return SLONN_ERR_NOMEM;
+            hash_matrix_kernel<<<(ly.D * 32 + 255) / 256, 256, 0, st>>>(ly.W, ly.WH, ly.D, esz, ly.hash_nodes, m->H);
+            if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+        }
+        if (cudaStreamSynchronize(st) != cudaSuccess) return SLONN_ERR_CUDA; // colpos.data() is read by the copy above
+    }
+    return SLONN_OK;
+}
+
 // sum[i] = sum over rows of A[x][i]; var[i] = mean of (A[x][i] - mean_i)^2.  One thread per node.
 __global__ void column_stats_kernel(const float *A, uint32_t n_rows, uint32_t N, double *sum, double *var)
 {
@@ -454,6 +575,8 @@ extern "C" void slonn_free(slonn_model *m)
         cudaFree(m->layer[l].tables);
         cudaFree(m->layer[l].hash_nodes);
         cudaFree(m->layer[l].WT);
+        cudaFree(m->layer[l].colpos);
+        cudaFree(m->layer[l].WH);
     }
     m->magic = 0;
     delete m;
@@ -538,12 +661,8 @@ extern "C" int slonn_build(const slonn_build_desc *desc, const void *const *W, c
     uint32_t last_needed = 0;
     bool any = false;
 
-    if (m->first_sparse) {
-        slonn_layer &l0 = m->layer[0];
-        CK(cudaMalloc(&l0.WT, (uint64_t)l0.N * l0.D * esz));
-        transpose_kernel<<<dim3((l0.D + 31) / 32, (l0.N + 31) / 32), dim3(32, 8), 0, st>>>(l0.W, l0.WT, l0.N, l0.D, esz);
-        CK(cudaGetLastError());
-    }
+    rc = make_transposed_copies(m, st, 0);
+    if (rc) goto fail;
     for (uint32_t l = 0; l < m->n_layers; ++l)
         if (m->layer[l].has_act) { last_needed = l; any = true; }
     if (any) {
@@ -572,6 +691,9 @@ extern "C" int slonn_build(const slonn_build_desc *desc, const void *const *W, c
         CK(cudaMemcpy(hs, d_status, sizeof(hs), cudaMemcpyDeviceToHost));
         if (hs[0]) { rc = -(int)hs[0]; goto fail; }
     }
+    cudaFree(cur); cur = nullptr;
+    rc = make_transposed_copies(m, st, 1);
+    if (rc) goto fail;
     CK(cudaStreamSynchronize(st));
     cudaFree(cur); cudaFree(A); cudaFree(d_status);
     *out = m;
@@ -727,12 +849,10 @@ extern "C" int slonn_deserialize(const void *src_host, uint64_t src_bytes, const
         CK(cudaMemcpyAsync(ly.tables, p + o, ly.table_bytes, cudaMemcpyHostToDevice, st));
         o += ly.table_bytes;
     }
-    if (m->first_sparse) {
-        slonn_layer &l0 = m->layer[0];
-        CK(cudaMalloc(&l0.WT, (uint64_t)l0.N * l0.D * esz));
-        transpose_kernel<<<dim3((l0.D + 31) / 32, (l0.N + 31) / 32), dim3(32, 8), 0, st>>>(l0.W, l0.WT, l0.N, l0.D, esz);
-        CK(cudaGetLastError());
-    }
+    rc = make_transposed_copies(m, st, 0);
+    if (rc) goto fail;
+    rc = make_transposed_copies(m, st, 1);
+    if (rc) goto fail;
     CK(cudaStreamSynchronize(st));
     *out = m;
     return SLONN_OK;

@@ -21,7 +21,10 @@ struct slonn_layer {
     void *tables;         // library-owned [L][2^K][cap] ids
     uint64_t table_bytes;
     uint32_t *hash_nodes; // library-owned device copy, [L*K]
-    void *WT;             // library-owned transposed copy [D][N] (sparse-operand layer 0 only)
+    void *WT;             // library-owned transposed copy [D][N]: layer 0 fed by CSR rows, and layers whose
+                          // input is an activator layer's list (node axis in colpos order when colpos != NULL)
+    uint32_t *colpos;     // library-owned [N]: node id -> column of WT; NULL = identity
+    void *WH;             // library-owned [D][32]: the hash rows side by side (list-input activator layers)
 };
 
 struct slonn_model {

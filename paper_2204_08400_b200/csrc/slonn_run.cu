@@ -198,6 +198,76 @@ int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint
     return bf ? launch_gather_t<true, false, 4>(P, grid, threads, smem, st) : launch_gather_t<false, false, 4>(P, grid, threads, smem, st);
 }
 
+// Input-stationary gather for a layer fed by (id, value) lists: 32 * R nodes per warp pass, the passes of
+// a block spread evenly over at most 8 warps, a few blocks per SM.
+#ifndef SLONN_COLS_R
+#define SLONN_COLS_R 2
+#endif
+template <bool BF16, int R>
+int launch_gather_cols_t(const slonn_gather_params &P, uint64_t grid, uint32_t threads, size_t smem, cudaStream_t st)
+{
+    const int rc = set_smem(gather_cols_kernel<BF16, R>, smem);
+    if (rc) return rc;
+    gather_cols_kernel<BF16, R><<<(uint32_t)grid, threads, smem, st>>>(P);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+int launch_gather_cols(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint32_t max_rows, cudaStream_t st)
+{
+    const uint32_t R = SLONN_COLS_R;
+    const uint32_t passes = (max_rows + 32u * R - 1u) / (32u * R);
+    const uint64_t want_ctas = 148ull * 8;
+    uint64_t ppc = ((uint64_t)n * passes + want_ctas - 1) / want_ctas; // passes per block
+    ppc = std::min<uint64_t>(std::max<uint64_t>(ppc, 1), passes);
+    const uint32_t rounds = (uint32_t)((ppc + 7) / 8);
+    const uint32_t warps = std::max(4u, (uint32_t)((ppc + rounds - 1) / rounds));
+    P.rows_per_cta = (uint32_t)ppc * 32u * R;
+    P.ctas_per_query = (max_rows + P.rows_per_cta - 1) / P.rows_per_cta;
+    const bool bf = m->dtype == SLONN_BF16;
+    P.rows_cap = max_rows;
+    size_t scratch = cols_image_bytes(P.D, bf ? 8u : 4u);
+    if (P.use_list && P.colpos) scratch = std::max(scratch, ((size_t)2 * ((P.N + 31u) / 32u) + (size_t)3 * max_rows) * 4);
+    scratch = (scratch + 15) & ~(size_t)15;
+    P.scratch_bytes = (uint32_t)scratch;
+    const size_t smem = scratch + (size_t)cols_ent_cap(P.D, P.in_cap) * 8;
+    if (smem > 200 * 1024) return SLONN_ERR_DIM; // caller falls back to the row kernel
+    const uint64_t grid = (uint64_t)n * P.ctas_per_query;
+    if (grid == 0 || grid > 0x7fffffffull) return SLONN_ERR_DIM;
+    return bf ? launch_gather_cols_t<true, SLONN_COLS_R>(P, grid, warps * 32u, smem, st)
+              : launch_gather_cols_t<false, SLONN_COLS_R>(P, grid, warps * 32u, smem, st);
+}
+
+// Budgets up to this many basis points leave the next layer's input sparse enough for the
+// input-stationary kernels to win over reading whole weight rows.
+constexpr uint32_t SLONN_COLS_MAX_BP = 3500;
+
+// Rows of one layer for a batch whose layer input is `P.in`: the input-stationary kernel for the queries
+// whose input list is sparse (by budget), the row kernel for the others.  Results do not depend on the split.
+int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_params &P, const slonn_batch *b,
+                      uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st)
+{
+    uint32_t cols_bp = 0; // budgets 1..cols_bp take the input-stationary kernel
+    if (ly.WT && P.in.kind == SLONN_IN_LIST && !(b->flags & SLONN_FLAG_ROW_KERNELS)) {
+        // small batches cannot fill the GPU with 64-node warp passes: they keep the row kernels unless told otherwise
+        if (b->flags & SLONN_FLAG_COLUMN_KERNELS) cols_bp = (uint64_t)n * max_rows > 148ull * 64 ? 10000u : 0u;
+        else if ((uint64_t)n * max_rows >= 148ull * 1024) cols_bp = SLONN_COLS_MAX_BP;
+    }
+    if (cols_bp == 0) return launch_gather(m, P, n, max_rows, st);
+    const bool both = max_bp > cols_bp;
+    slonn_gather_params C = P;
+    C.WT = ly.WT; C.colpos = ly.colpos; C.in_cap = in_cap;
+    if (both) { C.range_bp = b->budget_bp; C.bp_lo = 0; C.bp_hi = cols_bp; }
+    // the blocks of a launch are sized for the largest budget it serves
+    const uint32_t cols_rows = both ? std::min(max_rows, P.use_list ? slonn_layer_nodes(cols_bp, ly.N, slonn_model_pre(m)) : ly.N)
+                                    : max_rows;
+    C.in_cap = std::min(in_cap, both ? slonn_layer_nodes(cols_bp, ly.D, slonn_model_pre(m)) : in_cap);
+    int rc = launch_gather_cols(m, C, n, cols_rows, st);
+    if (rc == SLONN_ERR_DIM) return launch_gather(m, P, n, max_rows, st); // staging does not fit shared memory
+    if (rc || !both) return rc;
+    P.range_bp = b->budget_bp; P.bp_lo = cols_bp + 1; P.bp_hi = 0xffffu;
+    return launch_gather(m, P, n, max_rows, st);
+}
+
 // ---- whole-network kernel for narrow layers -----------------------------------
 
 bool fused_eligible(const slonn_model *m)
@@ -443,7 +513,8 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
 
     // a handful of queries: one thread-block cluster per query, every layer in one launch (it derives the
     // list offsets itself, so no planning launch either)
-    if (b->flags & ~SLONN_FLAG_DENSE_TC) return SLONN_ERR_ARG;
+    if (b->flags & ~SLONN_FLAG_ALL) return SLONN_ERR_ARG;
+    if ((b->flags & SLONN_FLAG_ROW_KERNELS) && (b->flags & SLONN_FLAG_COLUMN_KERNELS)) return SLONN_ERR_ARG;
     if (b->kernel_path > SLONN_PATH_CLUSTER) return SLONN_ERR_ARG;
     if (b->kernel_path == SLONN_PATH_CLUSTER && (!cluster_eligible(m) || tc_route(m, max_bp, b->flags))) return SLONN_ERR_DIM;
     if (b->kernel_path == SLONN_PATH_CLUSTER || (b->kernel_path == SLONN_PATH_AUTO && cluster_eligible(m) && n <= 4 && !tc_route(m, max_bp, b->flags) &&
@@ -479,7 +550,6 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     // queries at a 100 % budget on the tensor cores (on request): they compute every node of every
     // layer, so they are a dense matrix product over the compacted set of such queries
     const uint16_t *skip_bp = nullptr;
-    if (b->flags & ~SLONN_FLAG_DENSE_TC) return SLONN_ERR_ARG;
     if (tc_route(m, max_bp, b->flags)) {
         uint32_t *tc_list = (uint32_t *)(ws + wl.tc_list), *tc_count = (uint32_t *)(ws + wl.tc_count);
         uint16_t *A[2] = {(uint16_t *)(ws + wl.tc_a0), (uint16_t *)(ws + wl.tc_a1)};
@@ -546,6 +616,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     in.kind = SLONN_IN_DENSE;
     in.dense = b->x_dense;
     int dense_cur = 0;
+    uint32_t in_cap = 0; // most entries the current input list holds (list inputs only)
 
     for (uint32_t l = 0; l < m->n_layers; ++l) {
         const slonn_layer &ly = m->layer[l];
@@ -589,17 +660,18 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             gp.use_list = 1; gp.a = a; gp.out_vals = vals;
             if (is_last) { gp.out_dense = b->logits; gp.out_dense_ids = b->logit_ids; gp.out_stride = stride; }
             TIC(SLONN_STAGE_GATHER_DOT);
-            rc = launch_gather(m, gp, n, max_rows, st);
+            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st);
             TOC();
             if (rc) return rc;
             in.kind = SLONN_IN_LIST; in.indptr = indptr; in.ids = ids; in.vals = vals;
             in.ip_mul = m->n_act; in.ip_add = a;
+            in_cap = max_rows;
         } else {
             gp.use_list = 0;
             gp.out_dense = is_last ? b->logits : dense[dense_cur];
             gp.out_stride = ly.N;
             TIC(SLONN_STAGE_GATHER_DOT);
-            rc = launch_gather(m, gp, n, max_rows, st);
+            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st);
             TOC();
             if (rc) return rc;
             in.kind = SLONN_IN_DENSE; in.dense = gp.out_dense;

@@ -2,10 +2,12 @@
 //   plan_*_kernel            budgets -> per (query, activator layer) list offsets
 //   hash_select_kernel       FreeHash bits -> keys -> bucket lists -> first B distinct ids
 //   gather_dot_kernel        the selected rows' dot products, bias, activation
+//   gather_cols_kernel       the same for a sparse (id, value) input: nonzero inputs x selected nodes
 //   sparse_first_layer_kernel  layer 0 fed by CSR rows (transposed weights)
 //   argmax_kernel            prediction over the computed logits
 #pragma once
 #include "slonn_common.cuh"
+#include "slonn_cols_kernels.cuh"
 
 #define SLONN_THREADS 256
 #define SLONN_ROWS_PER_WARP 4 // hash rows per warp pass (reduce_rows4)
@@ -355,7 +357,23 @@ struct slonn_gather_params {
     uint32_t out_stride;
     uint32_t relu;
     uint32_t rows_per_cta, ctas_per_query;
+    // queries served by this launch: budget in [bp_lo, bp_hi] (range_bp nullable = all)
+    const uint16_t *range_bp;
+    uint32_t bp_lo, bp_hi;
+    // gather_cols_kernel only
+    const void *WT;           // transposed copy [D][N], node axis in colpos order
+    const uint32_t *colpos;   // [N] node id -> column of WT; NULL = identity
+    uint32_t in_cap;          // most entries an input list of this launch can hold
+    uint32_t rows_cap;        // most nodes a query of this launch selects
+    uint32_t scratch_bytes;   // shared memory in front of the entries (input image, then node order)
 };
+
+__device__ __forceinline__ bool bp_in_range(const uint16_t *range_bp, uint32_t lo, uint32_t hi, uint32_t q)
+{
+    if (!range_bp) return true;
+    const uint32_t bp = range_bp[q];
+    return bp >= lo && bp <= hi;
+}
 
 // R: rows per warp pass, 4 (6-shuffle reduction) or 8 (9 shuffles; pays off for rows of one
 // 512-byte round, where the reduction is most of the work).
@@ -366,6 +384,7 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_
     const uint32_t q = blockIdx.x / P.ctas_per_query;
     const uint32_t chunk = blockIdx.x - q * P.ctas_per_query;
     if (P.skip_bp && P.skip_bp[q] == 10000u) return;
+    if (!bp_in_range(P.range_bp, P.bp_lo, P.bp_hi, q)) return;
     uint64_t off = 0;
     uint32_t B = P.N;
     if (P.use_list) {
@@ -451,6 +470,7 @@ __global__ void __launch_bounds__(SLONN_THREADS, 2) gather_short_kernel(slonn_ga
     const uint32_t q = blockIdx.x / P.ctas_per_query;
     const uint32_t chunk = blockIdx.x - q * P.ctas_per_query;
     if (P.skip_bp && P.skip_bp[q] == 10000u) return;
+    if (!bp_in_range(P.range_bp, P.bp_lo, P.bp_hi, q)) return;
     uint64_t off = 0;
     uint32_t B = P.N;
     if (P.use_list) {
@@ -509,6 +529,112 @@ __global__ void __launch_bounds__(SLONN_THREADS, 2) gather_short_kernel(slonn_ga
                     }
                 } else {
                     P.out_dense[(uint64_t)q * P.out_stride + nd] = z;
+                }
+            }
+        }
+    }
+}
+
+// Input-stationary variant for a layer whose input is query q's (id, value) list: lane = one
+// selected node (32 nodes per warp pass), loop over the query's nonzero inputs grouped by partial
+// sum, one weight WT[j][column of n] per lane and input.  The query's selected nodes are first put in
+// column order (a bitmap over the columns, popcount prefix: the position of each node among the
+// query's columns), so that the 32 lanes of a pass read neighbouring columns.  Same sums, same
+// order, same results as gather_dot_kernel; results are written at the node's place in the
+// id-ascending list.
+template <bool BF16, int R>
+__global__ void __launch_bounds__(SLONN_THREADS) gather_cols_kernel(slonn_gather_params P)
+{
+    extern __shared__ float4 smem4[];
+    constexpr int V = BF16 ? 8 : 4;
+    __shared__ uint32_t segcnt[32];
+    __shared__ uint32_t segstart[33];
+    __shared__ uint32_t scan_ws[32];
+    __shared__ uint32_t scan_total;
+    const uint32_t q = blockIdx.x / P.ctas_per_query;
+    const uint32_t chunk = blockIdx.x - q * P.ctas_per_query;
+    if (P.skip_bp && P.skip_bp[q] == 10000u) return;
+    if (!bp_in_range(P.range_bp, P.bp_lo, P.bp_hi, q)) return;
+    uint64_t off = 0;
+    uint32_t B = P.N;
+    if (P.use_list) {
+        off = P.indptr[(uint64_t)q * P.n_act + P.a];
+        B = min((uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - off), P.rows_cap);
+    }
+    const uint32_t r0 = chunk * P.rows_per_cta;
+    if (r0 >= B) return;
+    const uint32_t r1 = min(B, r0 + P.rows_per_cta);
+
+    // shared memory: [scratch: input image while staging, node order afterwards][entries]
+    cols_stage S;
+    S.xs = reinterpret_cast<float *>(smem4);
+    S.ent = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(smem4) + P.scratch_bytes);
+    S.segcnt = segcnt;
+    S.segstart = segstart;
+    const uint64_t s0 = P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add];
+    const uint32_t len = min((uint32_t)(P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add + 1] - s0), P.in_cap);
+    cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D, P.N);
+
+    // the query's nodes in column order: spos[slot] = column, sidx[slot] = place in the id-ascending list
+    const bool ordered = P.use_list && P.colpos;
+    uint32_t *bitmap = reinterpret_cast<uint32_t *>(smem4);
+    const uint32_t nwords = (P.N + 31u) >> 5;
+    uint32_t *wprefix = bitmap + nwords;
+    uint32_t *tmp = wprefix + nwords, *spos = tmp + P.rows_cap, *sidx = spos + P.rows_cap;
+    if (ordered) {
+        for (uint32_t w = threadIdx.x; w < nwords; w += blockDim.x) bitmap[w] = 0u;
+        for (uint32_t e = threadIdx.x; e < B; e += blockDim.x) { spos[e] = 0u; sidx[e] = 0u; }
+        __syncthreads();
+        for (uint32_t e = threadIdx.x; e < B; e += blockDim.x) {
+            const uint32_t nd = min(__ldg(P.ids + off + e), P.N - 1u);
+            const uint32_t pos = min(__ldg(P.colpos + nd), P.N - 1u);
+            tmp[e] = pos;
+            atomicOr(&bitmap[pos >> 5], 1u << (pos & 31u));
+        }
+        __syncthreads();
+        const uint32_t wpt = (nwords + blockDim.x - 1) / blockDim.x;
+        const uint32_t w0 = threadIdx.x * wpt, w1 = min(w0 + wpt, nwords);
+        uint32_t cnt = 0;
+        for (uint32_t w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+        uint32_t o = block_exclusive_scan<uint32_t>(cnt, scan_ws, &scan_total);
+        for (uint32_t w = w0; w < w1; ++w) { wprefix[w] = o; o += __popc(bitmap[w]); }
+        __syncthreads();
+        for (uint32_t e = threadIdx.x; e < B; e += blockDim.x) {
+            const uint32_t pos = tmp[e];
+            const uint32_t slot = wprefix[pos >> 5] + __popc(bitmap[pos >> 5] & ((1u << (pos & 31u)) - 1u));
+            if (slot < B) { spos[slot] = pos; sidx[slot] = e; }
+        }
+        __syncthreads();
+    }
+
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (uint32_t r = r0 + warp * (32u * R); r < r1; r += nwarps * (32u * R)) {
+        uint32_t e[R], nd[R], col[R]; // place in the list, node id, column of WT
+#pragma unroll
+        for (int k = 0; k < R; ++k) {
+            const uint32_t rr = min(r + k * 32u + lane, r1 - 1);
+            e[k] = rr; nd[k] = rr; col[k] = rr;
+            if (ordered) { e[k] = sidx[rr]; col[k] = spos[rr]; }
+            if (P.use_list) {
+                nd[k] = min(__ldg(P.ids + off + e[k]), P.N - 1u);
+                if (!ordered) col[k] = nd[k];
+            }
+        }
+        float sum[R];
+        cols_walk<BF16, R>(S, P.WT, col, sum);
+#pragma unroll
+        for (int k = 0; k < R; ++k) {
+            float z = sum[k] + __ldg(P.bias + nd[k]);
+            if (P.relu) z = z > 0.0f ? z : 0.0f;
+            if (r + k * 32u + lane < r1) {
+                if (P.use_list) {
+                    if (P.out_vals) P.out_vals[off + e[k]] = z;
+                    if (P.out_dense) {
+                        P.out_dense[(uint64_t)q * P.out_stride + e[k]] = z;
+                        if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q * P.out_stride + e[k]] = nd[k];
+                    }
+                } else {
+                    P.out_dense[(uint64_t)q * P.out_stride + nd[k]] = z;
                 }
             }
         }

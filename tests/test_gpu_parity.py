@@ -32,7 +32,7 @@ def kernel_paths(wl):
 
 
 def check(wl, n_cal=None, sample=None, expect_build=True):
-    from paper_2204_08400_b200 import harness
+    from paper_2204_08400_b200 import binding as sl, harness
     dm = harness.DeviceModel(wl, n_cal=n_cal)
     om = oracle_model(wl, n_cal=n_cal)
     if expect_build:
@@ -46,10 +46,13 @@ def check(wl, n_cal=None, sample=None, expect_build=True):
     o64 = oracle_run(om, wl, x, bp, orc.REF64)
     info = None
     for path in kernel_paths(wl):
-        g = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=path)
-        if sample is not None:
-            g = slice_results(g, sample, n_act)
-        info = assert_run_parity(g, o32, o64, wl, n_act, bool(wl.has_act[-1]))
+        # the per-stage kernels evaluate a sparse-input layer row-wise or input-wise: library's choice,
+        # then each kind forced for the whole batch
+        for flags in ((0, sl.FLAG_ROW_KERNELS, sl.FLAG_COLUMN_KERNELS) if path == 1 else (0,)):
+            g = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=path, flags=flags)
+            if sample is not None:
+                g = slice_results(g, sample, n_act)
+            info = assert_run_parity(g, o32, o64, wl, n_act, bool(wl.has_act[-1]))
     dm.free()
     return info
 
