@@ -58,22 +58,36 @@ def hash_bytes(wl, n):
     return sum(wl.K * wl.L * wl.dims[l] * esz * n for l in range(len(wl.dims) - 1) if wl.has_act[l])
 
 
-def gathered_bytes(wl, budget_bp):
-    """Algorithmic bytes of the gather-dot launches of one step: every selected weight row
-    once per query (row-granular), all queries."""
+def budget_nodes(bp, N):
+    return np.minimum(np.maximum((bp.astype(np.int64) * N + 5000) // 10000, 1), N)
+
+
+def gathered_bytes(wl, budget_bp, force_rows=False, force_cols=False, cols_max_bp=3500):
+    """Algorithmic weight bytes of one step's gather launches, all queries, split by kernel kind.
+    Row kernels (dense input, or a list input that is not sparse enough): every selected weight row
+    once per query, whole (row-granular).  Input-stationary kernels (a layer fed by the list of the
+    activator layer below, budgets up to cols_max_bp): selected nodes x input list entries
+    (B_out * B_in weights), the weights such a query needs at all."""
     esz = 2 if wl.dtype == "bf16" else 4
-    per_launch = []
+    bp = np.asarray(budget_bp)
+    rows = cols = 0
     for l in range(len(wl.dims) - 1):
         if l == 0 and wl.first_sparse:
             continue
         D, N = wl.dims[l], wl.dims[l + 1]
-        if wl.has_act[l]:
-            uniq, cnt = np.unique(budget_bp, return_counts=True)
-            total_rows = int(sum(max(1, (int(bp) * N + 5000) // 10000) * int(c) for bp, c in zip(uniq, cnt)))
-        else:
-            total_rows = N * budget_bp.size
-        per_launch.append(total_rows * D * esz)
-    return per_launch
+        b_out = budget_nodes(bp, N) if wl.has_act[l] else np.full(bp.size, N, np.int64)
+        list_input = l > 0 and wl.has_act[l - 1]
+        use_cols = np.zeros(bp.size, bool)
+        if list_input and not force_rows:
+            big = bp.size * int(b_out.max()) >= 148 * 1024
+            if force_cols:
+                use_cols[:] = bp.size * int(b_out.max()) > 148 * 64
+            elif big:
+                use_cols = bp <= cols_max_bp
+        b_in = budget_nodes(bp, D) if list_input else np.full(bp.size, D, np.int64)
+        cols += int((b_out[use_cols] * b_in[use_cols]).sum()) * esz
+        rows += int(b_out[~use_cols].sum()) * D * esz
+    return rows, cols
 
 
 class ClockSampler:
@@ -318,17 +332,21 @@ def main():
         """Dominant kernel of the step and its achieved rate on the weight bytes it must touch."""
         if flags & sl.FLAG_DENSE_TC:     # queries at 100 % leave the row kernels
             bps = bps[bps != 10000]
-        gb = sum(gathered_bytes(wl, bps))
+        row_b, col_b = gathered_bytes(wl, bps, args.row_kernels, args.column_kernels, sl.COLS_MAX_BP)
         if ms_by_stage["fused"] > 0:     # one launch does hash + select + gather for every layer
-            kernel, ms, launches, nbytes = "fused_network_kernel", ms_by_stage["fused"], cnt_by_stage["fused"], gb + hash_bytes(wl, bps.size)
+            row_b, _ = gathered_bytes(wl, bps, force_rows=True)
+            kernel, ms, launches, nbytes = "fused_network_kernel", ms_by_stage["fused"], cnt_by_stage["fused"], row_b + hash_bytes(wl, bps.size)
         elif ms_by_stage["cluster"] > 0:
-            kernel, ms, launches, nbytes = "cluster_network_kernel", ms_by_stage["cluster"], cnt_by_stage["cluster"], gb + hash_bytes(wl, bps.size)
+            row_b, _ = gathered_bytes(wl, bps, force_rows=True)
+            kernel, ms, launches, nbytes = "cluster_network_kernel", ms_by_stage["cluster"], cnt_by_stage["cluster"], row_b + hash_bytes(wl, bps.size)
+        elif ms_by_stage["gather_cols"] > ms_by_stage["gather_dot"]:
+            kernel, ms, launches, nbytes = "gather_cols_kernel", ms_by_stage["gather_cols"], cnt_by_stage["gather_cols"], col_b
         else:
             esz = 2 if wl.dtype == "bf16" else 4
             gather_layers = [l for l in range(len(wl.dims) - 1) if not (l == 0 and wl.first_sparse)]
             short = all(wl.dims[l] * esz <= 512 for l in gather_layers)   # rows of one 512-byte round
             kernel = "gather_short_kernel" if short else "gather_dot_kernel"
-            ms, launches, nbytes = ms_by_stage["gather_dot"], cnt_by_stage["gather_dot"], gb
+            ms, launches, nbytes = ms_by_stage["gather_dot"], cnt_by_stage["gather_dot"], row_b
         ms /= steps
         launches //= steps
         ach = nbytes / (ms / 1e3) / 1e9 if ms > 0 else 0.0

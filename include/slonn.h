@@ -212,11 +212,13 @@ typedef struct {
  * A layer whose input is the sparse output of an activator layer (Sec. 3.3) can be evaluated in two
  * ways with identical results: row kernels read each selected weight row whole; input-stationary
  * kernels walk the query's nonzero inputs and read single weights from a transposed copy the model
- * keeps of such layers.  By default the library picks per query by budget (sparse inputs take the
- * input-stationary kernels).  These two flags force one kind for the whole batch, for testing and
- * tuning; setting both is an error.  They apply to the per-stage kernels (SLONN_PATH_STAGED or
- * networks too wide for the one-warp-per-query kernel).
+ * keeps of such layers.  By default the library picks per query by budget: up to SLONN_COLS_MAX_BP
+ * the input list is sparse enough for the input-stationary kernels to win (batches too small to fill
+ * the GPU with their 64-node warp passes keep the row kernels).  These two flags force one kind for the whole batch, for testing and
+ * tuning; setting both is an error.  They apply to the per-stage kernels and to the
+ * one-warp-per-query kernel; the one-cluster-per-query kernel has row form only.
  */
+#define SLONN_COLS_MAX_BP 3500u /* default split: budgets up to this take the input-stationary kernels */
 #define SLONN_FLAG_ROW_KERNELS 2u
 #define SLONN_FLAG_COLUMN_KERNELS 4u
 #define SLONN_FLAG_ALL 7u
@@ -380,7 +382,8 @@ int slonn_run_static(const slonn_model *m, const slonn_batch *batch, void *strea
 #define SLONN_STAGE_FUSED 5         /* all of 1, 2, 4 in the one-warp-per-query kernel */
 #define SLONN_STAGE_DENSE_TC 6      /* 100 % budget queries on the tensor cores        */
 #define SLONN_STAGE_CLUSTER 7       /* all of 1, 2, 4 in the one-cluster-per-query kernel */
-#define SLONN_N_STAGES 8
+#define SLONN_STAGE_GATHER_COLS 8   /* selected nodes' dot products, input-stationary kernel */
+#define SLONN_N_STAGES 9
 int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *workspace,
                     uint64_t workspace_bytes, void *stream, float *stage_ms,
                     uint32_t *stage_launches);

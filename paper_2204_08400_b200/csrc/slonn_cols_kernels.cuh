@@ -21,7 +21,7 @@
 // Shared-memory image of one query's nonzero inputs, grouped by partial sum.
 struct cols_stage {
     float *xs;          // [32 * smax] scratch: inputs in segment-major order (zero = absent)
-    uint2 *ent;         // [cols_ent_cap] entries (j * N, bits of x_j), segment after segment
+    uint2 *ent;         // [cols_ent_cap] entries (j, bits of x_j), segment after segment
     uint32_t *segcnt;   // [32]
     uint32_t *segstart; // [33]
 };
@@ -46,10 +46,10 @@ __host__ __device__ __forceinline__ size_t cols_image_bytes(uint32_t D, uint32_t
 }
 
 // Builds the grouped nonzero list of query segment [s0, s0 + len) of (ids, vals).  Whole block; ends
-// with a barrier.  rowmul = N (entries carry j * N, the element offset of row j of WT).
+// with a barrier.
 template <int V>
 __device__ __forceinline__ void cols_stage_list(const cols_stage &S, const uint32_t *ids, const float *vals, uint64_t s0,
-                                                uint32_t len, uint32_t D, uint32_t rowmul)
+                                                uint32_t len, uint32_t D)
 {
     const uint32_t smax = cols_smax(D, V);
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -97,7 +97,7 @@ __device__ __forceinline__ void cols_stage_list(const cols_stage &S, const uint3
             if (v != 0.0f) {
                 const uint32_t blk = pos / V;
                 const uint32_t j = (blk * 32u + p) * V + (pos - blk * V);
-                S.ent[base + __popc(m & ((1u << lane) - 1u))] = make_uint2(j * rowmul, __float_as_uint(v));
+                S.ent[base + __popc(m & ((1u << lane) - 1u))] = make_uint2(j, __float_as_uint(v));
             }
             base += __popc(m);
         }
@@ -124,8 +124,10 @@ __device__ __forceinline__ float cols_weight(const void *WT, uint32_t idx)
 // after the fourth, and so on -- the same additions as "for off in 16, 8, 4, 2, 1: a[p] += a[p + off]",
 // with at most five pending partial results per node instead of 32 registers.
 // A segment holds a multiple of 4 entries; 4 entries x R loads are in flight at a time.
+// Row j of WT starts at element j * ld.
 template <bool BF16, int R>
-__device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, const uint32_t (&col)[R], float (&sum)[R])
+__device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, uint32_t ld, const uint32_t (&col)[R],
+                                          float (&sum)[R])
 {
     float p0[R], p1[R], p2[R], p3[R], p4[R];
 #ifndef SLONN_COLS_UNROLL
@@ -149,10 +151,10 @@ __device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, c
             float w[R][4];
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                w[r][0] = cols_weight<BF16>(WT, e0.x + col[r]);
-                w[r][1] = cols_weight<BF16>(WT, e0.z + col[r]);
-                w[r][2] = cols_weight<BF16>(WT, e1.x + col[r]);
-                w[r][3] = cols_weight<BF16>(WT, e1.z + col[r]);
+                w[r][0] = cols_weight<BF16>(WT, e0.x * ld + col[r]);
+                w[r][1] = cols_weight<BF16>(WT, e0.z * ld + col[r]);
+                w[r][2] = cols_weight<BF16>(WT, e1.x * ld + col[r]);
+                w[r][3] = cols_weight<BF16>(WT, e1.z * ld + col[r]);
             }
 #pragma unroll
             for (int r = 0; r < R; ++r) a[r] = fmaf(w[r][0], __uint_as_float(e0.y), a[r]);
@@ -200,4 +202,55 @@ __device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, c
 #pragma unroll
         for (int r = 0; r < R; ++r) sum[r] = p4[r] + a[r];
     }
+}
+
+// The same grouping done by ONE warp from its own staged vector: ids[0..len) ascending node ids of the
+// list, their values read from xs (the warp's dense input image, element j at xs_index<BF16>(j, nchunks)).
+// S.segcnt / S.segstart / S.ent are the warp's own.  Ends with __syncwarp().
+template <bool BF16>
+__device__ __forceinline__ void cols_stage_warp(const cols_stage &S, const uint16_t *ids, uint32_t len, const float *xs,
+                                                uint32_t nchunks, uint32_t lane)
+{
+    constexpr uint32_t V = BF16 ? 8u : 4u;
+    S.segcnt[lane] = 0u;
+    __syncwarp();
+    // entries per segment; lists are ascending, so the order inside a segment is the list's order
+    for (uint32_t i0 = 0; i0 < len; i0 += 32) {
+        const uint32_t i = i0 + lane;
+        const uint32_t id = i < len ? (uint32_t)ids[i] : 0u;
+        const float v = i < len ? xs[xs_index<BF16>(id, nchunks)] : 0.0f;
+        const uint32_t p = (id / V) & 31u;
+        const uint32_t same = __match_any_sync(SLONN_FULL_MASK, v != 0.0f ? p : 32u + lane);
+        if (v != 0.0f && (uint32_t)(__ffs(same) - 1) == lane) S.segcnt[p] += __popc(same);
+        __syncwarp();
+    }
+    {
+        const uint32_t c = (S.segcnt[lane] + 3u) & ~3u;
+        uint32_t incl = c;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t t = __shfl_up_sync(SLONN_FULL_MASK, incl, off);
+            if (lane >= (uint32_t)off) incl += t;
+        }
+        S.segstart[lane] = incl - c;
+        if (lane == 31) S.segstart[32] = incl;
+        S.segcnt[lane] = 0u; // reused as the fill level while placing
+    }
+    __syncwarp();
+    for (uint32_t i0 = 0; i0 < len; i0 += 32) {
+        const uint32_t i = i0 + lane;
+        const uint32_t id = i < len ? (uint32_t)ids[i] : 0u;
+        const float v = i < len ? xs[xs_index<BF16>(id, nchunks)] : 0.0f;
+        const uint32_t p = (id / V) & 31u;
+        const uint32_t same = __match_any_sync(SLONN_FULL_MASK, v != 0.0f ? p : 32u + lane);
+        if (v != 0.0f) S.ent[S.segstart[p] + S.segcnt[p] + __popc(same & ((1u << lane) - 1u))] = make_uint2(id, __float_as_uint(v));
+        __syncwarp();
+        if (v != 0.0f && (uint32_t)(__ffs(same) - 1) == lane) S.segcnt[p] += __popc(same);
+        __syncwarp();
+    }
+    { // fill every segment up to a multiple of 4 with copies of its last input carrying the value 0
+        const uint32_t at = S.segstart[lane] + S.segcnt[lane], end = S.segstart[lane + 1];
+        for (uint32_t k = at; k < end; ++k) S.ent[k] = make_uint2(S.ent[at - 1].x, 0u);
+    }
+    __syncwarp();
 }

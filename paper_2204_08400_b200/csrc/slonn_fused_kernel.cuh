@@ -7,8 +7,15 @@
 // Same arithmetic as everywhere else in the library: lane p owns partial sum
 // p and takes 16-byte weight chunks p, p+32, ... in ascending order; partials
 // are added pairwise with strides 16, 8, 4, 2, 1; bias last.
+//
+// A layer fed by the sparse output of the activator layer below takes, for queries whose budget leaves
+// that output sparse, the input-stationary form (slonn_cols_kernels.cuh): the warp groups the nonzero
+// inputs by partial sum in its own shared memory, then lanes own nodes -- the K*L hash nodes in one pass
+// over the layer's side-by-side hash rows, the selected nodes 64 per pass over the transposed weights.
+// Same sums in the same order, so which form a query takes does not show in its results.
 #pragma once
 #include "slonn_common.cuh"
+#include "slonn_cols_kernels.cuh"
 
 #define SLONN_FUSED_ROWS 4          // rows per pass; the 6-shuffle reduction is written for 4
 #ifndef SLONN_FUSED_WARPS
@@ -27,6 +34,9 @@ struct slonn_fused_layer {
     const void *tables;
     uint32_t D, N, nchunks, cap;
     uint32_t has_act, a, relu, id_bytes;
+    const void *WT;          // transposed copy [D][N] in colpos order, or NULL
+    const void *WH;          // hash rows side by side [D][32], or NULL
+    const uint32_t *colpos;  // node id -> column of WT
 };
 
 struct slonn_fused_params {
@@ -34,6 +44,7 @@ struct slonn_fused_params {
     uint32_t n_layers, n, n_act, K, L;
     uint32_t pre;            // hash nodes that are always active (0 or K*L)
     const uint16_t *skip_bp; // nullable: queries with this budget == 10000 are handled elsewhere
+    const uint16_t *budget_bp; // [n]
     const float *x;          // [n][D0]
     const uint64_t *indptr;  // [n * n_act + 1]
     uint32_t *out_ids;       // CSR payload, nullable
@@ -45,6 +56,8 @@ struct slonn_fused_params {
     uint32_t *pred;          // nullable
     uint32_t *status;
     uint32_t xbuf_floats, ids_cap, bitmap_words, warp_bytes; // per-warp shared memory carve
+    uint32_t cols_bp;        // budgets up to this take the input-stationary form where a layer offers it (0 = never)
+    uint32_t ent_cap;        // entries of a warp's grouped input list (0 = no room set aside)
 };
 
 template <bool BF16>
@@ -193,7 +206,9 @@ __device__ __forceinline__ void fused_select(const slonn_fused_layer &ly, uint32
     __syncwarp();
 }
 
-template <bool BF16, int NC, int GRP>
+// COLS: compiled with the input-stationary form (chosen on the host per batch; without it the kernel is
+// the plain row form and carries none of the extra state).
+template <bool BF16, int NC, int GRP, bool COLS>
 __global__ void __launch_bounds__(SLONN_FUSED_WARPS * 32, GRP == 1 ? SLONN_FUSED_MIN_BLOCKS : 1)
 fused_network_kernel(const __grid_constant__ slonn_fused_params P)
 {
@@ -210,15 +225,28 @@ fused_network_kernel(const __grid_constant__ slonn_fused_params P)
     uint16_t *ids_s = reinterpret_cast<uint16_t *>(wbase + (size_t)P.xbuf_floats * 4);
     uint32_t *bitmap = reinterpret_cast<uint32_t *>(wbase + (size_t)P.xbuf_floats * 4 + (size_t)P.ids_cap * 2);
 
+    // grouped nonzero inputs of the input-stationary form (this warp's own)
+    cols_stage S;
+    S.xs = nullptr;
+    S.ent = reinterpret_cast<uint2 *>(wbase + (((size_t)P.xbuf_floats * 4 + (size_t)P.ids_cap * 2 + (size_t)P.bitmap_words * 4 + 15) & ~(size_t)15)); // 16-byte aligned: read as uint4
+    S.segcnt = reinterpret_cast<uint32_t *>(S.ent + P.ent_cap);
+    S.segstart = S.segcnt + 32;
+
     float xr[NC * VPC];
     float best = 0.0f;          // running argmax over the last layer (per lane)
     uint32_t best_id = 0xffffffffu;
+    uint32_t prev_B = 0;        // entries of the list in ids_s left by the layer below (0 = none / every node)
+    const uint32_t my_bp = (COLS && P.cols_bp) ? (uint32_t)P.budget_bp[q] : 0u;
 
     for (uint32_t l = 0; l < P.n_layers; ++l) {
         const slonn_fused_layer &ly = P.layer[l];
         const bool is_last = (l + 1 == P.n_layers);
-        // input := previous activation (registers)
-        if (l == 0) fused_load_x_global<BF16, NC>(xr, P.x + (uint64_t)q * ly.D, ly.nchunks, lane);
+        // the input-stationary form: this layer keeps the copies it needs, the input is a list that fits
+        // the warp's entry buffer, and the query's budget leaves it sparse
+        const bool cols = COLS && P.cols_bp && ly.has_act && ly.WT && ly.WH && prev_B && prev_B + 96u <= P.ent_cap && my_bp <= P.cols_bp;
+        // input := previous activation (registers, or the grouped list of its nonzeros)
+        if (COLS && cols) cols_stage_warp<BF16>(S, ids_s, prev_B, xbuf, ly.nchunks, lane);
+        else if (l == 0) fused_load_x_global<BF16, NC>(xr, P.x + (uint64_t)q * ly.D, ly.nchunks, lane);
         else fused_load_x_shared<BF16, NC>(xr, xbuf4, ly.nchunks, lane);
         __syncwarp();
         uint32_t next_chunks = 0;
@@ -238,6 +266,14 @@ fused_network_kernel(const __grid_constant__ slonn_fused_params P)
             // FreeHash: signs of the K*L sampled nodes' pre-activations
             const uint32_t H = P.K * P.L;
             uint32_t mykey = 0;
+            if (COLS && cols) { // lane h computes hash node h from the side-by-side hash rows
+                const uint32_t col[1] = {lane};
+                float sum[1];
+                cols_walk<BF16, 1>(S, ly.WH, 32u, col, sum);
+                const float z = sum[0] + __ldg(ly.bias + __ldg(ly.hash_nodes + min(lane, H - 1)));
+                const uint32_t signs = __ballot_sync(SLONN_FULL_MASK, lane < H && z > 0.0f);
+                if (lane < P.L) mykey = (signs >> (lane * P.K)) & ((1u << P.K) - 1u);
+            } else
             for (uint32_t h0 = 0; h0 < H; h0 += R) {
                 const uint4 *rows[R];
 #pragma unroll
@@ -270,7 +306,36 @@ fused_network_kernel(const __grid_constant__ slonn_fused_params P)
             }
         }
 
-        // the selected rows
+        // the selected nodes
+        if (COLS && cols) {
+            for (uint32_t r0 = 0; r0 < B; r0 += 64) {
+                uint32_t nd[2], col[2];
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const uint32_t rr = min(r0 + k * 32u + lane, B - 1);
+                    nd[k] = implicit_ids ? rr : (uint32_t)ids_s[rr];
+                    col[k] = __ldg(ly.colpos + nd[k]);
+                }
+                float sum[2];
+                cols_walk<BF16, 2>(S, ly.WT, ly.N, col, sum);
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const uint32_t r = r0 + k * 32u + lane;
+                    if (r < B) {
+                        float z = sum[k] + __ldg(ly.bias + nd[k]);
+                        if (ly.relu) z = z > 0.0f ? z : 0.0f;
+                        if (P.out_vals) P.out_vals[off + r] = z;
+                        if (!is_last) {
+                            xbuf[xs_index<BF16>(nd[k], next_chunks)] = z;
+                        } else {
+                            P.logits[(uint64_t)q * P.logit_stride + r] = z;
+                            P.logit_ids[(uint64_t)q * P.logit_stride + r] = nd[k];
+                            if (best_id == 0xffffffffu || z > best) { best = z; best_id = nd[k]; }
+                        }
+                    }
+                }
+            }
+        } else
         for (uint32_t r0 = 0; r0 < B; r0 += R) {
             const uint4 *rows[R];
 #pragma unroll
@@ -302,6 +367,7 @@ fused_network_kernel(const __grid_constant__ slonn_fused_params P)
             }
         }
         __syncwarp();
+        if (COLS) prev_B = (ly.has_act && !implicit_ids) ? B : 0u;
     }
 
     if (P.pred) { // lowest node id among the largest logits

@@ -237,14 +237,10 @@ int launch_gather_cols(const slonn_model *m, slonn_gather_params &P, uint32_t n,
               : launch_gather_cols_t<false, SLONN_COLS_R>(P, grid, warps * 32u, smem, st);
 }
 
-// Budgets up to this many basis points leave the next layer's input sparse enough for the
-// input-stationary kernels to win over reading whole weight rows.
-constexpr uint32_t SLONN_COLS_MAX_BP = 3500;
-
 // Rows of one layer for a batch whose layer input is `P.in`: the input-stationary kernel for the queries
 // whose input list is sparse (by budget), the row kernel for the others.  Results do not depend on the split.
 int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_params &P, const slonn_batch *b,
-                      uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st)
+                      uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st, stage_timer *tm)
 {
     uint32_t cols_bp = 0; // budgets 1..cols_bp take the input-stationary kernel
     if (ly.WT && P.in.kind == SLONN_IN_LIST && !(b->flags & SLONN_FLAG_ROW_KERNELS)) {
@@ -252,23 +248,35 @@ int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_
         if (b->flags & SLONN_FLAG_COLUMN_KERNELS) cols_bp = (uint64_t)n * max_rows > 148ull * 64 ? 10000u : 0u;
         else if ((uint64_t)n * max_rows >= 148ull * 1024) cols_bp = SLONN_COLS_MAX_BP;
     }
-    if (cols_bp == 0) return launch_gather(m, P, n, max_rows, st);
-    const bool both = max_bp > cols_bp;
-    slonn_gather_params C = P;
-    C.WT = ly.WT; C.colpos = ly.colpos; C.in_cap = in_cap;
-    if (both) { C.range_bp = b->budget_bp; C.bp_lo = 0; C.bp_hi = cols_bp; }
-    // the blocks of a launch are sized for the largest budget it serves
-    const uint32_t cols_rows = both ? std::min(max_rows, P.use_list ? slonn_layer_nodes(cols_bp, ly.N, slonn_model_pre(m)) : ly.N)
-                                    : max_rows;
-    C.in_cap = std::min(in_cap, both ? slonn_layer_nodes(cols_bp, ly.D, slonn_model_pre(m)) : in_cap);
-    int rc = launch_gather_cols(m, C, n, cols_rows, st);
-    if (rc == SLONN_ERR_DIM) return launch_gather(m, P, n, max_rows, st); // staging does not fit shared memory
-    if (rc || !both) return rc;
-    P.range_bp = b->budget_bp; P.bp_lo = cols_bp + 1; P.bp_hi = 0xffffu;
-    return launch_gather(m, P, n, max_rows, st);
+    int rc;
+    if (cols_bp) {
+        const bool both = max_bp > cols_bp;
+        slonn_gather_params C = P;
+        C.WT = ly.WT; C.colpos = ly.colpos;
+        if (both) { C.range_bp = b->budget_bp; C.bp_lo = 0; C.bp_hi = cols_bp; }
+        // the blocks of a launch are sized for the largest budget it serves
+        const uint32_t pre = slonn_model_pre(m);
+        const uint32_t cols_rows = (both && P.use_list) ? std::min(max_rows, slonn_layer_nodes(cols_bp, ly.N, pre)) : max_rows;
+        C.in_cap = both ? std::min(in_cap, slonn_layer_nodes(cols_bp, ly.D, pre)) : in_cap;
+        TIC(SLONN_STAGE_GATHER_COLS);
+        rc = launch_gather_cols(m, C, n, cols_rows, st);
+        TOC();
+        if (rc != SLONN_ERR_DIM) { // SLONN_ERR_DIM: the staging does not fit shared memory, rows for everyone
+            if (rc || !both) return rc;
+            P.range_bp = b->budget_bp; P.bp_lo = cols_bp + 1; P.bp_hi = 0xffffu;
+        }
+    }
+    TIC(SLONN_STAGE_GATHER_DOT);
+    rc = launch_gather(m, P, n, max_rows, st);
+    TOC();
+    return rc;
 }
 
 // ---- whole-network kernel for narrow layers -----------------------------------
+
+#ifndef SLONN_FUSED_COLS_MAX_BP
+#define SLONN_FUSED_COLS_MAX_BP 1250u // batches whose largest budget is at most this take the input-stationary form
+#endif
 
 bool fused_eligible(const slonn_model *m)
 {
@@ -280,14 +288,14 @@ bool fused_eligible(const slonn_model *m)
     return true;
 }
 
-template <bool BF16, int NC, int GRP>
+template <bool BF16, int NC, int GRP, bool COLS>
 int launch_fused_g(const slonn_fused_params &P, cudaStream_t st)
 {
     const size_t smem = (size_t)P.warp_bytes * SLONN_FUSED_WARPS;
-    int rc = set_smem(fused_network_kernel<BF16, NC, GRP>, smem);
+    int rc = set_smem(fused_network_kernel<BF16, NC, GRP, COLS>, smem);
     if (rc) return rc;
     const uint32_t grid = (P.n + SLONN_FUSED_WARPS - 1) / SLONN_FUSED_WARPS;
-    fused_network_kernel<BF16, NC, GRP><<<grid, SLONN_FUSED_WARPS * 32, smem, st>>>(P);
+    fused_network_kernel<BF16, NC, GRP, COLS><<<grid, SLONN_FUSED_WARPS * 32, smem, st>>>(P);
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
@@ -297,17 +305,23 @@ template <bool BF16, int NC>
 int launch_fused_t(const slonn_fused_params &P, cudaStream_t st)
 {
     const uint32_t grid = (P.n + SLONN_FUSED_WARPS - 1) / SLONN_FUSED_WARPS;
-    if (NC > 1 && grid <= 2u * 148u) return launch_fused_g<BF16, NC, (NC > 4 ? 4 : NC)>(P, st);
-    return launch_fused_g<BF16, NC, 1>(P, st);
+    if (NC > 1 && grid <= 2u * 148u)
+        return P.cols_bp ? launch_fused_g<BF16, NC, (NC > 4 ? 4 : NC), true>(P, st) : launch_fused_g<BF16, NC, (NC > 4 ? 4 : NC), false>(P, st);
+    return P.cols_bp ? launch_fused_g<BF16, NC, 1, true>(P, st) : launch_fused_g<BF16, NC, 1, false>(P, st);
 }
 
 int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *indptr, uint32_t stride,
-                 const uint16_t *skip_bp, cudaStream_t st)
+                 const uint16_t *skip_bp, uint32_t max_bp, cudaStream_t st)
 {
     slonn_fused_params P;
     memset(&P, 0, sizeof(P));
     const uint32_t esz = m->dtype == SLONN_BF16 ? 2u : 4u;
-    uint32_t max_rounds = 1, xbuf = 4, ids_cap = 8, words = 1;
+    uint32_t max_rounds = 1, xbuf = 4, ids_cap = 8, words = 1, ent_cap = 0;
+    // budgets that take the input-stationary form in layers that offer it
+    // (the grouped input list lives in shared memory, which it takes from the L1 cache the row form relies on:
+    // only batches whose every budget is low carry it, unless the caller forces it)
+    const uint32_t cols_bp = (b->flags & SLONN_FLAG_ROW_KERNELS) ? 0u : (b->flags & SLONN_FLAG_COLUMN_KERNELS) ? 10000u
+                             : max_bp <= SLONN_FUSED_COLS_MAX_BP ? SLONN_FUSED_COLS_MAX_BP : 0u;
     for (uint32_t l = 0; l < m->n_layers; ++l) {
         const slonn_layer &ly = m->layer[l];
         slonn_fused_layer &f = P.layer[l];
@@ -315,6 +329,9 @@ int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *ind
         f.D = ly.D; f.N = ly.N; f.nchunks = ly.D * esz / 16u; f.cap = ly.cap;
         f.has_act = ly.has_act; f.a = m->act_index[l]; f.relu = (l + 1 == m->n_layers) ? 0u : 1u;
         f.id_bytes = ly.id_bytes;
+        f.WT = ly.WT; f.WH = ly.WH; f.colpos = ly.colpos;
+        if (cols_bp && l > 0 && ly.has_act && ly.WT && ly.WH && ly.colpos && m->layer[l - 1].has_act)
+            ent_cap = std::max(ent_cap, slonn_layer_nodes(std::min(max_bp, cols_bp), ly.D, slonn_model_pre(m)) + 96u);
         max_rounds = std::max(max_rounds, (f.nchunks + 31u) / 32u);
         if (l > 0) xbuf = std::max(xbuf, (ly.D + 3u) / 4u * 4u);
         if (ly.has_act) {
@@ -329,7 +346,9 @@ int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *ind
     P.logits = b->logits; P.logit_stride = stride; P.logit_ids = b->logit_ids; P.pred = b->pred;
     P.status = b->status;
     P.xbuf_floats = xbuf; P.ids_cap = ids_cap; P.bitmap_words = words;
-    P.warp_bytes = (uint32_t)align_up((uint64_t)xbuf * 4 + (uint64_t)ids_cap * 2 + (uint64_t)words * 4, 16);
+    P.cols_bp = ent_cap ? cols_bp : 0u; P.ent_cap = ent_cap; P.budget_bp = b->budget_bp;
+    P.warp_bytes = (uint32_t)align_up(align_up((uint64_t)xbuf * 4 + (uint64_t)ids_cap * 2 + (uint64_t)words * 4, 16) +
+                                          (ent_cap ? (uint64_t)ent_cap * 8 + 66 * 4 : 0), 16);
     const bool bf = m->dtype == SLONN_BF16;
     if (bf) {
         if (max_rounds <= 1) return launch_fused_t<true, 1>(P, st);
@@ -596,7 +615,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     if (b->kernel_path == SLONN_PATH_FUSED ||
         (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n >= 512)) {
         TIC(SLONN_STAGE_FUSED);
-        const int rc = launch_fused(m, b, indptr, stride, skip_bp, st);
+        const int rc = launch_fused(m, b, indptr, stride, skip_bp, max_bp, st);
         TOC();
         if (rc || !skip_bp || !b->pred) return rc;
         // predictions of the tensor-core queries (the fused kernel wrote the others; same rule)
@@ -659,9 +678,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             if (rc) return rc;
             gp.use_list = 1; gp.a = a; gp.out_vals = vals;
             if (is_last) { gp.out_dense = b->logits; gp.out_dense_ids = b->logit_ids; gp.out_stride = stride; }
-            TIC(SLONN_STAGE_GATHER_DOT);
-            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st);
-            TOC();
+            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st, tm);
             if (rc) return rc;
             in.kind = SLONN_IN_LIST; in.indptr = indptr; in.ids = ids; in.vals = vals;
             in.ip_mul = m->n_act; in.ip_add = a;
@@ -670,9 +687,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             gp.use_list = 0;
             gp.out_dense = is_last ? b->logits : dense[dense_cur];
             gp.out_stride = ly.N;
-            TIC(SLONN_STAGE_GATHER_DOT);
-            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st);
-            TOC();
+            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st, tm);
             if (rc) return rc;
             in.kind = SLONN_IN_DENSE; in.dense = gp.out_dense;
             dense_cur ^= 1;

@@ -573,7 +573,7 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_cols_kernel(slonn_gather
     S.segstart = segstart;
     const uint64_t s0 = P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add];
     const uint32_t len = min((uint32_t)(P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add + 1] - s0), P.in_cap);
-    cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D, P.N);
+    cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D);
 
     // the query's nodes in column order: spos[slot] = column, sidx[slot] = place in the id-ascending list
     const bool ordered = P.use_list && P.colpos;
@@ -621,7 +621,7 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_cols_kernel(slonn_gather
             }
         }
         float sum[R];
-        cols_walk<BF16, R>(S, P.WT, col, sum);
+        cols_walk<BF16, R>(S, P.WT, P.N, col, sum);
 #pragma unroll
         for (int k = 0; k < R; ++k) {
             float z = sum[k] + __ldg(P.bias + nd[k]);

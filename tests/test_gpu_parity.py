@@ -46,9 +46,9 @@ def check(wl, n_cal=None, sample=None, expect_build=True):
     o64 = oracle_run(om, wl, x, bp, orc.REF64)
     info = None
     for path in kernel_paths(wl):
-        # the per-stage kernels evaluate a sparse-input layer row-wise or input-wise: library's choice,
-        # then each kind forced for the whole batch
-        for flags in ((0, sl.FLAG_ROW_KERNELS, sl.FLAG_COLUMN_KERNELS) if path == 1 else (0,)):
+        # the per-stage and one-warp-per-query kernels evaluate a sparse-input layer row-wise or
+        # input-wise: library's choice, then each kind forced for the whole batch
+        for flags in ((0, sl.FLAG_ROW_KERNELS, sl.FLAG_COLUMN_KERNELS) if path in (1, 2) else (0,)):
             g = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=path, flags=flags)
             if sample is not None:
                 g = slice_results(g, sample, n_act)
