@@ -71,6 +71,8 @@ def gathered_bytes(wl, budget_bp, force_rows=False, force_cols=False, cols_max_b
     esz = 2 if wl.dtype == "bf16" else 4
     bp = np.asarray(budget_bp)
     rows = cols = 0
+    if bp.size == 0:
+        return 0, 0
     for l in range(len(wl.dims) - 1):
         if l == 0 and wl.first_sparse:
             continue
