@@ -11,6 +11,9 @@
 
 #define SLONN_THREADS 256
 #define SLONN_ROWS_PER_WARP 4 // hash rows per warp pass (reduce_rows4)
+#ifndef SLONN_SELECT_MIN_BLOCKS
+#define SLONN_SELECT_MIN_BLOCKS 4
+#endif
 
 
 // ---------------------------------------------------------------------------
@@ -277,7 +280,7 @@ __device__ __forceinline__ bool block_select(const void *tables, uint32_t cap, u
 // LAT: latency variant for a handful of queries -- up to 32 warps per block, one hash row per warp
 // with deep load prefetch, instead of 4 rows per warp pass.
 template <bool BF16, typename IDT, bool LAT>
-__global__ void __launch_bounds__(LAT ? 1024 : SLONN_THREADS) hash_select_kernel(slonn_select_params P)
+__global__ void __launch_bounds__(LAT ? 1024 : SLONN_THREADS, LAT ? 1 : SLONN_SELECT_MIN_BLOCKS) hash_select_kernel(slonn_select_params P)
 {
     extern __shared__ float4 smem4[];
     float4 *xs4 = smem4;

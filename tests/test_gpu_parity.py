@@ -389,6 +389,38 @@ def test_node_id_width_switches_above_65536_nodes():
     check(wl16)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_budget_split_between_row_and_input_stationary_kernels(dtype):
+    # one batch whose budgets lie on both sides of the library's split (35 %), large enough for the
+    # library to use the input-stationary kernels by itself: the two launches of a stage must serve
+    # disjoint sets of queries and together all of them
+    wl = custom_workload(71, [64, 512, 512, 16], [1, 1, 0], dtype, n=640, n_cal=512, K=4, L=2,
+                         budgets=(300, 2500, 3500, 3600, 5000, 10000))
+    check(wl)
+
+
+def test_input_stationary_kernel_on_a_wide_list_fed_layer():
+    # a 70,000-node budgeted layer fed by the list of the activator layer below: 32-bit ids, a column
+    # order over 70,000 nodes, many 64-node passes per query, widths that are no multiple of 32 chunks
+    wl = custom_workload(72, [48, 100, 70000], [1, 1], "f32", n=24, n_cal=64, K=3, L=2, budgets=(1000,))
+    check(wl)
+    # at 50 % the per-query node order no longer fits shared memory: the library must fall back to
+    # the row kernel even when the input-stationary one is asked for
+    wl = custom_workload(73, [48, 100, 70000], [1, 1], "f32", n=6, n_cal=64, K=3, L=2, budgets=(5000,))
+    check(wl)
+
+
+def test_input_stationary_kernels_with_an_all_zero_list():
+    # biases far below zero: every selected node of the first layer outputs exactly 0, so the next
+    # layer's grouped input list is empty and its pre-activations are the biases
+    import dataclasses
+    wl = custom_workload(74, [32, 96, 64, 8], [1, 1, 0], "bf16", n=300, n_cal=128, K=3, L=2, budgets=(1000, 3000))
+    bias = [b.copy() for b in wl.bias]
+    bias[0][:] = -1000.0
+    wl = dataclasses.replace(wl, bias=bias)
+    check(wl)
+
+
 def test_csr_rows_empty_and_longer_than_one_tile():
     # first layer fed by CSR rows: a query without any nonzero, and rows with 300 nonzeros
     # (more than the 128 the kernel stages at a time)
