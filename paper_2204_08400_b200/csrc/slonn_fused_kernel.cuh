@@ -46,7 +46,8 @@ struct slonn_fused_params {
     const uint16_t *skip_bp; // nullable: queries with this budget == 10000 are handled elsewhere
     const uint16_t *budget_bp; // [n]
     const float *x;          // [n][D0]
-    const uint64_t *indptr;  // [n * n_act + 1]
+    const uint64_t *indptr;  // [n * n_act + 1]; NULL when no active list is written (counts then come from the budgets)
+    uint32_t max_bp;         // the batch's stated largest budget
     uint32_t *out_ids;       // CSR payload, nullable
     float *out_vals;         // CSR payload, nullable
     uint16_t *codes;         // nullable
@@ -261,8 +262,17 @@ fused_network_kernel(const __grid_constant__ slonn_fused_params P)
         uint64_t off = 0;
         bool implicit_ids = true;
         if (ly.has_act) {
-            off = P.indptr[(uint64_t)q * P.n_act + ly.a];
-            B = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + ly.a + 1] - off);
+            if (P.indptr) {
+                off = P.indptr[(uint64_t)q * P.n_act + ly.a];
+                B = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + ly.a + 1] - off);
+            } else { // no list is written, so no offsets were planned: the count follows from the budget alone
+                uint32_t bp = P.budget_bp[q];
+                bool bad = (bp < 1u) || (bp > 10000u) || (bp > P.max_bp);
+                bp = min(max(bp, 1u), P.max_bp);
+                B = slonn_layer_nodes(bp, ly.N, P.pre);
+                if (B - P.pre > ly.cap && B != ly.N) bad = true;
+                if (bad && lane == 0) slonn_report(P.status, SLONN_ERR_BUDGET, q, l);
+            }
             // FreeHash: signs of the K*L sampled nodes' pre-activations
             const uint32_t H = P.K * P.L;
             uint32_t mykey = 0;

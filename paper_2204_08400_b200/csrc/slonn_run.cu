@@ -341,7 +341,7 @@ int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *ind
     }
     P.n_layers = m->n_layers; P.n = b->n_queries; P.n_act = m->n_act; P.K = m->K; P.L = m->L;
     P.pre = slonn_model_pre(m);
-    P.x = b->x_dense; P.indptr = indptr; P.skip_bp = skip_bp;
+    P.x = b->x_dense; P.indptr = indptr; P.skip_bp = skip_bp; P.max_bp = max_bp;
     P.out_ids = b->active_ids; P.out_vals = b->active_vals; P.codes = b->codes;
     P.logits = b->logits; P.logit_stride = stride; P.logit_ids = b->logit_ids; P.pred = b->pred;
     P.status = b->status;
@@ -545,8 +545,15 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         // the device cannot co-schedule such a cluster: fall through to the other kernels
     }
 
+    // narrow networks with enough queries to fill the GPU take the one-warp-per-query kernel; when the
+    // caller wants no active lists back it needs no list offsets either (each warp derives its node
+    // counts from the budget), which saves the two planning launches
+    if (b->kernel_path == SLONN_PATH_FUSED && !fused_eligible(m)) return SLONN_ERR_DIM;
+    const bool use_fused = b->kernel_path == SLONN_PATH_FUSED || (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n >= 512);
+    const bool no_plan = use_fused && !tc_route(m, max_bp, b->flags) && !b->active_indptr && !b->active_ids && !b->active_vals;
+
     // offsets of every (query, activator layer) list
-    if (m->n_act) {
+    if (m->n_act && !no_plan) {
         slonn_plan_params pp;
         memset(&pp, 0, sizeof(pp));
         pp.budget_bp = b->budget_bp; pp.n = n; pp.n_act = m->n_act; pp.max_bp = max_bp;
@@ -611,11 +618,9 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     }
 
     // narrow networks with enough queries to fill the GPU: one warp per query, every layer in one launch
-    if (b->kernel_path == SLONN_PATH_FUSED && !fused_eligible(m)) return SLONN_ERR_DIM;
-    if (b->kernel_path == SLONN_PATH_FUSED ||
-        (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n >= 512)) {
+    if (use_fused) {
         TIC(SLONN_STAGE_FUSED);
-        const int rc = launch_fused(m, b, indptr, stride, skip_bp, max_bp, st);
+        const int rc = launch_fused(m, b, no_plan ? nullptr : indptr, stride, skip_bp, max_bp, st);
         TOC();
         if (rc || !skip_bp || !b->pred) return rc;
         // predictions of the tensor-core queries (the fused kernel wrote the others; same rule)

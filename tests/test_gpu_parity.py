@@ -204,6 +204,39 @@ def test_invalid_budget_is_reported_not_fatal():
     dm.free()
 
 
+@pytest.mark.parametrize("last_budgeted", [False, True])
+def test_one_warp_per_query_kernel_without_active_lists(last_budgeted):
+    # a caller that asks for logits and predictions only: the one-warp-per-query kernel then runs without
+    # the planning launches and derives each layer's node count from the budget itself; results must not
+    # change, mixed budgets included, and an invalid budget must still be reported
+    from paper_2204_08400_b200 import binding as sl, harness
+    wl = custom_workload(75, [72, 160, 120, 24], [1, 1, 1 if last_budgeted else 0], "bf16", n=700, n_cal=256, K=3, L=2,
+                         budgets=(700, 1000, 4000, 10000))
+    dm = harness.DeviceModel(wl)
+    for flags in (0, sl.FLAG_ROW_KERNELS, sl.FLAG_COLUMN_KERNELS):
+        full = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=2, flags=flags)
+        b = harness.DeviceBatch(dm, wl.x, wl.budget_bp, full_outputs=False, kernel_path=2, flags=flags)
+        b.run()
+        g = b.results()
+        assert g["status"][0] == 0
+        assert np.array_equal(g["pred"], full["pred"])
+        if last_budgeted:
+            ip = full["active_indptr"].astype(np.int64)
+            for q in range(wl.n_queries):
+                B = int(ip[q * 3 + 3] - ip[q * 3 + 2])
+                assert np.array_equal(g["logits"][q, :B], full["logits"][q, :B])
+                assert np.array_equal(g["logit_ids"][q, :B], full["logit_ids"][q, :B])
+        else:
+            assert np.array_equal(g["logits"], full["logits"])
+    bp = wl.budget_bp.copy()
+    bp[11] = 0
+    b = harness.DeviceBatch(dm, wl.x, bp, max_budget_bp=10000, full_outputs=False, kernel_path=2)
+    b.run()
+    st = b.results()["status"]
+    assert st[0] == 5 and st[1] == 11     # SLONN_ERR_BUDGET at query 11
+    dm.free()
+
+
 def test_runs_are_deterministic():
     from paper_2204_08400_b200 import harness
     wl = custom_workload(58, [136, 200, 96, 24], [1, 1, 0], "bf16", n=256, n_cal=300, K=4, L=2)
