@@ -63,16 +63,18 @@ def budget_nodes(bp, N):
 
 
 def gathered_bytes(wl, budget_bp, force_rows=False, force_cols=False, cols_max_bp=3500):
-    """Algorithmic weight bytes of one step's gather launches, all queries, split by kernel kind.
+    """Algorithmic weight bytes of one step's gather launches, all queries, split by kernel kind:
+    (row kernels, gather_cols_kernel, layer_cols_kernel).
     Row kernels (dense input, or a list input that is not sparse enough): every selected weight row
     once per query, whole (row-granular).  Input-stationary kernels (a layer fed by the list of the
     activator layer below, budgets up to cols_max_bp): selected nodes x input list entries
-    (B_out * B_in weights), the weights such a query needs at all."""
+    (B_out * B_in weights), the weights such a query needs at all; the whole-layer kernel of an
+    activator layer also reads its K*L hash rows at the list entries."""
     esz = 2 if wl.dtype == "bf16" else 4
     bp = np.asarray(budget_bp)
-    rows = cols = 0
+    rows = cols = layer = 0
     if bp.size == 0:
-        return 0, 0
+        return 0, 0, 0
     for l in range(len(wl.dims) - 1):
         if l == 0 and wl.first_sparse:
             continue
@@ -87,9 +89,12 @@ def gathered_bytes(wl, budget_bp, force_rows=False, force_cols=False, cols_max_b
             elif big:
                 use_cols = bp <= cols_max_bp
         b_in = budget_nodes(bp, D) if list_input else np.full(bp.size, D, np.int64)
-        cols += int((b_out[use_cols] * b_in[use_cols]).sum()) * esz
+        if wl.has_act[l] and wl.K * wl.L <= 32:
+            layer += int(((b_out[use_cols] + wl.K * wl.L) * b_in[use_cols]).sum()) * esz
+        else:
+            cols += int((b_out[use_cols] * b_in[use_cols]).sum()) * esz
         rows += int(b_out[~use_cols].sum()) * D * esz
-    return rows, cols
+    return rows, cols, layer
 
 
 class ClockSampler:
@@ -334,15 +339,21 @@ def main():
         """Dominant kernel of the step and its achieved rate on the weight bytes it must touch."""
         if flags & sl.FLAG_DENSE_TC:     # queries at 100 % leave the row kernels
             bps = bps[bps != 10000]
-        row_b, col_b = gathered_bytes(wl, bps, args.row_kernels, args.column_kernels, sl.COLS_MAX_BP)
+        row_b, col_b, layer_b = gathered_bytes(wl, bps, args.row_kernels, args.column_kernels, sl.COLS_MAX_BP)
+        cols_ms = ms_by_stage["gather_cols"] + ms_by_stage["layer_cols"]
         if ms_by_stage["fused"] > 0:     # one launch does hash + select + gather for every layer
-            row_b, _ = gathered_bytes(wl, bps, force_rows=True)
+            row_b = gathered_bytes(wl, bps, force_rows=True)[0]
             kernel, ms, launches, nbytes = "fused_network_kernel", ms_by_stage["fused"], cnt_by_stage["fused"], row_b + hash_bytes(wl, bps.size)
         elif ms_by_stage["cluster"] > 0:
-            row_b, _ = gathered_bytes(wl, bps, force_rows=True)
+            row_b = gathered_bytes(wl, bps, force_rows=True)[0]
             kernel, ms, launches, nbytes = "cluster_network_kernel", ms_by_stage["cluster"], cnt_by_stage["cluster"], row_b + hash_bytes(wl, bps.size)
-        elif ms_by_stage["gather_cols"] > ms_by_stage["gather_dot"]:
-            kernel, ms, launches, nbytes = "gather_cols_kernel", ms_by_stage["gather_cols"], cnt_by_stage["gather_cols"], col_b
+        elif cols_ms > ms_by_stage["gather_dot"]:
+            # the input-stationary kernels: the whole-layer kernel of the activator layers (hash + selection +
+            # nodes) or, if larger, the plain gather of the layers without activator
+            if ms_by_stage["layer_cols"] >= ms_by_stage["gather_cols"]:
+                kernel, ms, launches, nbytes = "layer_cols_kernel", ms_by_stage["layer_cols"], cnt_by_stage["layer_cols"], layer_b
+            else:
+                kernel, ms, launches, nbytes = "gather_cols_kernel", ms_by_stage["gather_cols"], cnt_by_stage["gather_cols"], col_b
         else:
             esz = 2 if wl.dtype == "bf16" else 4
             gather_layers = [l for l in range(len(wl.dims) - 1) if not (l == 0 and wl.first_sparse)]

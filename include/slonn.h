@@ -383,7 +383,8 @@ int slonn_run_static(const slonn_model *m, const slonn_batch *batch, void *strea
 #define SLONN_STAGE_DENSE_TC 6      /* 100 % budget queries on the tensor cores        */
 #define SLONN_STAGE_CLUSTER 7       /* all of 1, 2, 4 in the one-cluster-per-query kernel */
 #define SLONN_STAGE_GATHER_COLS 8   /* selected nodes' dot products, input-stationary kernel */
-#define SLONN_N_STAGES 9
+#define SLONN_STAGE_LAYER_COLS 9    /* all of 1 and 8 for a list-fed activator layer in one launch */
+#define SLONN_N_STAGES 10
 int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *workspace,
                     uint64_t workspace_bytes, void *stream, float *stage_ms,
                     uint32_t *stage_launches);

@@ -117,6 +117,17 @@ __device__ __forceinline__ float cols_weight(const void *WT, uint32_t idx)
     return __ldg(reinterpret_cast<const float *>(WT) + idx);
 }
 
+// a[0] + ... + a[31] in the fixed tree: strides 16, 8, 4, 2, 1
+__device__ __forceinline__ float cols_tree(float (&acc)[32])
+{
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+#pragma unroll
+        for (int p = 0; p < off; ++p) acc[p] = acc[p] + acc[p + off];
+    }
+    return acc[0];
+}
+
 // The complete sums of R nodes (columns col[0..R)) over the staged nonzero inputs, bias not included.
 //
 // The 32 partial sums are taken in bit-reversed order (0, 16, 8, 24, 4, ...) and added as soon as both

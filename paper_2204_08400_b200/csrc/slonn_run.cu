@@ -237,17 +237,60 @@ int launch_gather_cols(const slonn_model *m, slonn_gather_params &P, uint32_t n,
               : launch_gather_cols_t<false, SLONN_COLS_R>(P, grid, warps * 32u, smem, st);
 }
 
+template <bool BF16, typename IDT>
+int launch_layer_cols_t(const slonn_layer_cols_params &Q, uint32_t n, uint32_t threads, size_t smem, cudaStream_t st)
+{
+    const int rc = set_smem(layer_cols_kernel<BF16, IDT>, smem);
+    if (rc) return rc;
+    layer_cols_kernel<BF16, IDT><<<n, threads, smem, st>>>(Q);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+// Hash, selection and input-stationary gather of a list-fed activator layer in one launch, one block per
+// query.  SLONN_ERR_DIM: not applicable here (no side-by-side hash rows, a batch so small that a query's
+// nodes should be spread over several blocks, or the staging does not fit) -- the caller takes the
+// separate kernels.
+int launch_layer_cols(const slonn_model *m, const slonn_layer &ly, uint32_t layer, slonn_gather_params G,
+                      const slonn_batch *b, uint32_t n, uint32_t max_rows, cudaStream_t st)
+{
+    if (!ly.WH || !ly.WT || !ly.colpos || !G.use_list) return SLONN_ERR_DIM;
+    const uint32_t passes = (max_rows + 63u) / 64u;
+    if ((uint64_t)n * passes < 148ull * 8) return SLONN_ERR_DIM; // whole queries per block would leave SMs idle
+    const uint32_t rounds = (passes + 7) / 8;
+    const uint32_t warps = std::max(4u, (passes + rounds - 1) / rounds);
+    const bool bf = m->dtype == SLONN_BF16;
+    G.rows_cap = max_rows;
+    G.rows_per_cta = passes * 64u; G.ctas_per_query = 1;
+    size_t scratch = cols_image_bytes(G.D, bf ? 8u : 4u);
+    scratch = std::max(scratch, ((size_t)2 * ((G.N + 31u) / 32u) + (size_t)3 * max_rows) * 4);
+    scratch = (scratch + 15) & ~(size_t)15;
+    G.scratch_bytes = (uint32_t)scratch;
+    const size_t smem = scratch + (size_t)cols_ent_cap(G.D, G.in_cap) * 8 + (size_t)((G.N + 31u) / 32u) * 4 + 32 * 32 * 4;
+    if (smem > 200 * 1024) return SLONN_ERR_DIM;
+    slonn_layer_cols_params Q;
+    memset(&Q, 0, sizeof(Q));
+    Q.G = G; Q.WH = ly.WH; Q.hash_nodes = ly.hash_nodes; Q.tables = ly.tables; Q.cap = ly.cap;
+    Q.K = m->K; Q.L = m->L; Q.pre = slonn_model_pre(m); Q.layer = layer; Q.codes = b->codes; Q.status = b->status;
+    const bool id16 = ly.id_bytes == 2;
+    if (bf) return id16 ? launch_layer_cols_t<true, uint16_t>(Q, n, warps * 32u, smem, st) : launch_layer_cols_t<true, uint32_t>(Q, n, warps * 32u, smem, st);
+    return id16 ? launch_layer_cols_t<false, uint16_t>(Q, n, warps * 32u, smem, st) : launch_layer_cols_t<false, uint32_t>(Q, n, warps * 32u, smem, st);
+}
+
+// Budgets 1..limit take the input-stationary kernels in this layer (0: none do).
+uint32_t cols_budget_limit(const slonn_layer &ly, const slonn_gather_params &P, const slonn_batch *b, uint32_t n, uint32_t max_rows)
+{
+    if (!ly.WT || P.in.kind != SLONN_IN_LIST || (b->flags & SLONN_FLAG_ROW_KERNELS)) return 0;
+    // small batches cannot fill the GPU with 64-node warp passes: they keep the row kernels unless told otherwise
+    if (b->flags & SLONN_FLAG_COLUMN_KERNELS) return (uint64_t)n * max_rows > 148ull * 64 ? 10000u : 0u;
+    return (uint64_t)n * max_rows >= 148ull * 1024 ? SLONN_COLS_MAX_BP : 0u;
+}
+
 // Rows of one layer for a batch whose layer input is `P.in`: the input-stationary kernel for the queries
 // whose input list is sparse (by budget), the row kernel for the others.  Results do not depend on the split.
 int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_params &P, const slonn_batch *b,
                       uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st, stage_timer *tm)
 {
-    uint32_t cols_bp = 0; // budgets 1..cols_bp take the input-stationary kernel
-    if (ly.WT && P.in.kind == SLONN_IN_LIST && !(b->flags & SLONN_FLAG_ROW_KERNELS)) {
-        // small batches cannot fill the GPU with 64-node warp passes: they keep the row kernels unless told otherwise
-        if (b->flags & SLONN_FLAG_COLUMN_KERNELS) cols_bp = (uint64_t)n * max_rows > 148ull * 64 ? 10000u : 0u;
-        else if ((uint64_t)n * max_rows >= 148ull * 1024) cols_bp = SLONN_COLS_MAX_BP;
-    }
+    const uint32_t cols_bp = cols_budget_limit(ly, P, b, n, max_rows);
     int rc;
     if (cols_bp) {
         const bool both = max_bp > cols_bp;
@@ -270,6 +313,49 @@ int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_
     rc = launch_gather(m, P, n, max_rows, st);
     TOC();
     return rc;
+}
+
+// An activator layer: FreeHash, selection and the selected nodes.  A list-fed layer with the copies for it
+// runs as ONE input-stationary launch for the queries whose budget leaves the list sparse; the others (and
+// every query where that launch does not apply) take the selection kernel followed by the row or
+// input-stationary gather.
+int launch_act_layer(const slonn_model *m, const slonn_layer &ly, uint32_t l, slonn_select_params &sp, slonn_gather_params &gp,
+                     const slonn_batch *b, uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st,
+                     stage_timer *tm)
+{
+    int rc;
+    const uint32_t cols_bp = cols_budget_limit(ly, gp, b, n, max_rows);
+    if (cols_bp && ly.WH) {
+        const bool both = max_bp > cols_bp;
+        const uint32_t pre = slonn_model_pre(m);
+        slonn_gather_params C = gp;
+        C.WT = ly.WT; C.colpos = ly.colpos;
+        if (both) { C.range_bp = b->budget_bp; C.bp_lo = 0; C.bp_hi = cols_bp; }
+        const uint32_t cols_rows = both ? std::min(max_rows, slonn_layer_nodes(cols_bp, ly.N, pre)) : max_rows;
+        C.in_cap = both ? std::min(in_cap, slonn_layer_nodes(cols_bp, ly.D, pre)) : in_cap;
+        TIC(SLONN_STAGE_LAYER_COLS);
+        rc = launch_layer_cols(m, ly, l, C, b, n, cols_rows, st);
+        TOC();
+        if (rc == SLONN_OK) {
+            if (!both) return SLONN_OK;
+            sp.range_bp = b->budget_bp; sp.bp_lo = cols_bp + 1; sp.bp_hi = 0xffffu;
+            TIC(SLONN_STAGE_HASH_SELECT);
+            rc = launch_select(m, sp, n, max_rows, st);
+            TOC();
+            if (rc) return rc;
+            gp.range_bp = b->budget_bp; gp.bp_lo = cols_bp + 1; gp.bp_hi = 0xffffu;
+            TIC(SLONN_STAGE_GATHER_DOT);
+            rc = launch_gather(m, gp, n, max_rows, st);
+            TOC();
+            return rc;
+        }
+        if (rc != SLONN_ERR_DIM) return rc;
+    }
+    TIC(SLONN_STAGE_HASH_SELECT);
+    rc = launch_select(m, sp, n, max_rows, st);
+    TOC();
+    if (rc) return rc;
+    return launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st, tm);
 }
 
 // ---- whole-network kernel for narrow layers -----------------------------------
@@ -677,13 +763,9 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             sp.n_act = m->n_act; sp.a = a; sp.layer = l; sp.indptr = indptr; sp.out_ids = ids;
             sp.codes = b->codes; sp.status = b->status;
             max_rows = slonn_layer_nodes(max_bp, ly.N, slonn_model_pre(m));
-            TIC(SLONN_STAGE_HASH_SELECT);
-            rc = launch_select(m, sp, n, max_rows, st);
-            TOC();
-            if (rc) return rc;
             gp.use_list = 1; gp.a = a; gp.out_vals = vals;
             if (is_last) { gp.out_dense = b->logits; gp.out_dense_ids = b->logit_ids; gp.out_stride = stride; }
-            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st, tm);
+            rc = launch_act_layer(m, ly, l, sp, gp, b, n, max_bp, max_rows, in_cap, st, tm);
             if (rc) return rc;
             in.kind = SLONN_IN_LIST; in.indptr = indptr; in.ids = ids; in.vals = vals;
             in.ip_mul = m->n_act; in.ip_add = a;

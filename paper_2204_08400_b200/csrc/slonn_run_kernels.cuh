@@ -10,6 +10,15 @@
 #include "slonn_cols_kernels.cuh"
 
 #define SLONN_THREADS 256
+
+// whether query q's budget lies in [lo, hi] (range_bp == NULL: every query)
+__device__ __forceinline__ bool bp_in_range(const uint16_t *range_bp, uint32_t lo, uint32_t hi, uint32_t q)
+{
+    if (!range_bp) return true;
+    const uint32_t bp = range_bp[q];
+    return bp >= lo && bp <= hi;
+}
+
 #define SLONN_ROWS_PER_WARP 4 // hash rows per warp pass (reduce_rows4)
 #ifndef SLONN_SELECT_MIN_BLOCKS
 #define SLONN_SELECT_MIN_BLOCKS 4
@@ -127,6 +136,8 @@ __global__ void __launch_bounds__(SLONN_PLAN_THREADS) plan_final_kernel(slonn_pl
 // ---------------------------------------------------------------------------
 struct slonn_select_params {
     const uint16_t *skip_bp;    // nullable: queries with this budget == 10000 are handled elsewhere
+    const uint16_t *range_bp;   // nullable: only queries whose budget lies in [bp_lo, bp_hi]
+    uint32_t bp_lo, bp_hi;
     slonn_input in;
     const void *W;
     const float *bias;
@@ -292,6 +303,7 @@ __global__ void __launch_bounds__(LAT ? 1024 : SLONN_THREADS, LAT ? 1 : SLONN_SE
 
     const uint32_t q = blockIdx.x;
     if (P.skip_bp && P.skip_bp[q] == 10000u) return;
+    if (!bp_in_range(P.range_bp, P.bp_lo, P.bp_hi, q)) return;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t H = P.K * P.L;
     const uint64_t off = P.indptr[(uint64_t)q * P.n_act + P.a];
@@ -371,12 +383,6 @@ struct slonn_gather_params {
     uint32_t scratch_bytes;   // shared memory in front of the entries (input image, then node order)
 };
 
-__device__ __forceinline__ bool bp_in_range(const uint16_t *range_bp, uint32_t lo, uint32_t hi, uint32_t q)
-{
-    if (!range_bp) return true;
-    const uint32_t bp = range_bp[q];
-    return bp >= lo && bp <= hi;
-}
 
 // R: rows per warp pass, 4 (6-shuffle reduction) or 8 (9 shuffles; pays off for rows of one
 // 512-byte round, where the reduction is most of the work).
@@ -538,6 +544,84 @@ __global__ void __launch_bounds__(SLONN_THREADS, 2) gather_short_kernel(slonn_ga
     }
 }
 
+// Second half of the input-stationary layer, shared by gather_cols_kernel and layer_cols_kernel: puts the
+// query's selected nodes in column order and evaluates nodes [r0, r1) of that order against the staged
+// input list S.  `order_mem` is block scratch of P.scratch_bytes (the staging image, dead by now).  NC: the
+// id list was written by an earlier launch and may be read through the read-only path.
+template <bool BF16, int R, bool NC>
+__device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params &P, const cols_stage &S, void *order_mem,
+                                                      uint32_t q, uint64_t off, uint32_t B, uint32_t r0, uint32_t r1,
+                                                      uint32_t *scan_ws, uint32_t *scan_total_p)
+{
+    auto list_id = [&](uint32_t e) -> uint32_t {
+        const uint32_t v = NC ? __ldg(P.ids + off + e) : P.ids[off + e];
+        return min(v, P.N - 1u);
+    };
+    // the query's nodes in column order: spos[slot] = column, sidx[slot] = place in the id-ascending list
+    const bool ordered = P.use_list && P.colpos;
+    uint32_t *bitmap = reinterpret_cast<uint32_t *>(order_mem);
+    const uint32_t nwords = (P.N + 31u) >> 5;
+    uint32_t *wprefix = bitmap + nwords;
+    uint32_t *tmp = wprefix + nwords, *spos = tmp + P.rows_cap, *sidx = spos + P.rows_cap;
+    if (ordered) {
+        for (uint32_t w = threadIdx.x; w < nwords; w += blockDim.x) bitmap[w] = 0u;
+        for (uint32_t e = threadIdx.x; e < B; e += blockDim.x) { spos[e] = 0u; sidx[e] = 0u; }
+        __syncthreads();
+        for (uint32_t e = threadIdx.x; e < B; e += blockDim.x) {
+            const uint32_t pos = min(__ldg(P.colpos + list_id(e)), P.N - 1u);
+            tmp[e] = pos;
+            atomicOr(&bitmap[pos >> 5], 1u << (pos & 31u));
+        }
+        __syncthreads();
+        const uint32_t wpt = (nwords + blockDim.x - 1) / blockDim.x;
+        const uint32_t w0 = threadIdx.x * wpt, w1 = min(w0 + wpt, nwords);
+        uint32_t cnt = 0;
+        for (uint32_t w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+        uint32_t o = block_exclusive_scan<uint32_t>(cnt, scan_ws, scan_total_p);
+        for (uint32_t w = w0; w < w1; ++w) { wprefix[w] = o; o += __popc(bitmap[w]); }
+        __syncthreads();
+        for (uint32_t e = threadIdx.x; e < B; e += blockDim.x) {
+            const uint32_t pos = tmp[e];
+            const uint32_t slot = wprefix[pos >> 5] + __popc(bitmap[pos >> 5] & ((1u << (pos & 31u)) - 1u));
+            if (slot < B) { spos[slot] = pos; sidx[slot] = e; }
+        }
+        __syncthreads();
+    }
+
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (uint32_t r = r0 + warp * (32u * R); r < r1; r += nwarps * (32u * R)) {
+        uint32_t e[R], nd[R], col[R]; // place in the list, node id, column of WT
+#pragma unroll
+        for (int k = 0; k < R; ++k) {
+            const uint32_t rr = min(r + k * 32u + lane, r1 - 1);
+            e[k] = rr; nd[k] = rr; col[k] = rr;
+            if (ordered) { e[k] = sidx[rr]; col[k] = spos[rr]; }
+            if (P.use_list) {
+                nd[k] = list_id(e[k]);
+                if (!ordered) col[k] = nd[k];
+            }
+        }
+        float sum[R];
+        cols_walk<BF16, R>(S, P.WT, P.N, col, sum);
+#pragma unroll
+        for (int k = 0; k < R; ++k) {
+            float z = sum[k] + __ldg(P.bias + nd[k]);
+            if (P.relu) z = z > 0.0f ? z : 0.0f;
+            if (r + k * 32u + lane < r1) {
+                if (P.use_list) {
+                    if (P.out_vals) P.out_vals[off + e[k]] = z;
+                    if (P.out_dense) {
+                        P.out_dense[(uint64_t)q * P.out_stride + e[k]] = z;
+                        if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q * P.out_stride + e[k]] = nd[k];
+                    }
+                } else {
+                    P.out_dense[(uint64_t)q * P.out_stride + nd[k]] = z;
+                }
+            }
+        }
+    }
+}
+
 // Input-stationary variant for a layer whose input is query q's (id, value) list: lane = one
 // selected node (32 nodes per warp pass), loop over the query's nonzero inputs grouped by partial
 // sum, one weight WT[j][column of n] per lane and input.  The query's selected nodes are first put in
@@ -578,70 +662,99 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_cols_kernel(slonn_gather
     const uint32_t len = min((uint32_t)(P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add + 1] - s0), P.in_cap);
     cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D);
 
-    // the query's nodes in column order: spos[slot] = column, sidx[slot] = place in the id-ascending list
-    const bool ordered = P.use_list && P.colpos;
-    uint32_t *bitmap = reinterpret_cast<uint32_t *>(smem4);
-    const uint32_t nwords = (P.N + 31u) >> 5;
-    uint32_t *wprefix = bitmap + nwords;
-    uint32_t *tmp = wprefix + nwords, *spos = tmp + P.rows_cap, *sidx = spos + P.rows_cap;
-    if (ordered) {
-        for (uint32_t w = threadIdx.x; w < nwords; w += blockDim.x) bitmap[w] = 0u;
-        for (uint32_t e = threadIdx.x; e < B; e += blockDim.x) { spos[e] = 0u; sidx[e] = 0u; }
-        __syncthreads();
-        for (uint32_t e = threadIdx.x; e < B; e += blockDim.x) {
-            const uint32_t nd = min(__ldg(P.ids + off + e), P.N - 1u);
-            const uint32_t pos = min(__ldg(P.colpos + nd), P.N - 1u);
-            tmp[e] = pos;
-            atomicOr(&bitmap[pos >> 5], 1u << (pos & 31u));
-        }
-        __syncthreads();
-        const uint32_t wpt = (nwords + blockDim.x - 1) / blockDim.x;
-        const uint32_t w0 = threadIdx.x * wpt, w1 = min(w0 + wpt, nwords);
-        uint32_t cnt = 0;
-        for (uint32_t w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
-        uint32_t o = block_exclusive_scan<uint32_t>(cnt, scan_ws, &scan_total);
-        for (uint32_t w = w0; w < w1; ++w) { wprefix[w] = o; o += __popc(bitmap[w]); }
-        __syncthreads();
-        for (uint32_t e = threadIdx.x; e < B; e += blockDim.x) {
-            const uint32_t pos = tmp[e];
-            const uint32_t slot = wprefix[pos >> 5] + __popc(bitmap[pos >> 5] & ((1u << (pos & 31u)) - 1u));
-            if (slot < B) { spos[slot] = pos; sidx[slot] = e; }
-        }
-        __syncthreads();
-    }
+    cols_order_and_gather<BF16, R, true>(P, S, smem4, q, off, B, r0, r1, scan_ws, &scan_total);
+}
 
+// A whole list-fed activator layer for one query per block, input-stationary: the input list is grouped
+// once and serves the FreeHash projection (lane = hash function, over the side-by-side hash rows WH, the 32
+// segments spread over the warps and their partial sums added by one thread per function in the fixed tree),
+// then keys, bucket lists and the top-k% cut exactly as in hash_select_kernel, then the selected nodes as in
+// gather_cols_kernel.  One launch and one staging instead of two of each.
+struct slonn_layer_cols_params {
+    slonn_gather_params G;      // use_list = 1; in, WT, colpos, bias, D, N, indptr, ids (= out of the selection), outputs, filters
+    const void *WH;             // [D][32]
+    const uint32_t *hash_nodes; // [L*K], L*K <= 32
+    const void *tables;
+    uint32_t cap, K, L, pre, layer;
+    uint16_t *codes;            // nullable
+    uint32_t *status;
+};
+
+template <bool BF16, typename IDT>
+__global__ void __launch_bounds__(SLONN_THREADS) layer_cols_kernel(slonn_layer_cols_params Q)
+{
+    extern __shared__ float4 smem4[];
+    constexpr int V = BF16 ? 8 : 4;
+    constexpr int R = 2;
+    const slonn_gather_params &P = Q.G;
+    __shared__ uint32_t segcnt[32];
+    __shared__ uint32_t segstart[33];
+    __shared__ uint32_t scan_ws[32];
+    __shared__ uint32_t scan_total;
+    __shared__ uint32_t keys[8];
+    __shared__ float zh[32];
+    const uint32_t q = blockIdx.x;
+    if (P.skip_bp && P.skip_bp[q] == 10000u) return;
+    if (!bp_in_range(P.range_bp, P.bp_lo, P.bp_hi, q)) return;
+    const uint64_t off = P.indptr[(uint64_t)q * P.n_act + P.a];
+    const uint32_t B = min((uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - off), P.rows_cap);
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    for (uint32_t r = r0 + warp * (32u * R); r < r1; r += nwarps * (32u * R)) {
-        uint32_t e[R], nd[R], col[R]; // place in the list, node id, column of WT
-#pragma unroll
-        for (int k = 0; k < R; ++k) {
-            const uint32_t rr = min(r + k * 32u + lane, r1 - 1);
-            e[k] = rr; nd[k] = rr; col[k] = rr;
-            if (ordered) { e[k] = sidx[rr]; col[k] = spos[rr]; }
-            if (P.use_list) {
-                nd[k] = min(__ldg(P.ids + off + e[k]), P.N - 1u);
-                if (!ordered) col[k] = nd[k];
-            }
+    const uint32_t H = Q.K * Q.L;
+    const uint32_t nwords = (P.N + 31u) >> 5;
+
+    // shared memory: [scratch: input image, then node order][entries][selection bitmap][hash partial sums]
+    cols_stage S;
+    S.xs = reinterpret_cast<float *>(smem4);
+    S.ent = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(smem4) + P.scratch_bytes);
+    S.segcnt = segcnt;
+    S.segstart = segstart;
+    uint32_t *idmap = reinterpret_cast<uint32_t *>(S.ent + cols_ent_cap(P.D, P.in_cap));
+    float *zpart = reinterpret_cast<float *>(idmap + nwords);
+    const uint64_t s0 = P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add];
+    const uint32_t len = min((uint32_t)(P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add + 1] - s0), P.in_cap);
+    cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D);
+
+    // (1) FreeHash: partial sum p of hash function `lane`, segments spread over the warps
+    for (uint32_t p = warp; p < 32; p += nwarps) {
+        float a = 0.0f;
+        const uint32_t e = segstart[p + 1];
+        for (uint32_t k = segstart[p]; k < e; k += 4) {
+            const uint4 e0 = *reinterpret_cast<const uint4 *>(S.ent + k), e1 = *reinterpret_cast<const uint4 *>(S.ent + k + 2);
+            const float w0 = cols_weight<BF16>(Q.WH, e0.x * 32u + lane), w1 = cols_weight<BF16>(Q.WH, e0.z * 32u + lane);
+            const float w2 = cols_weight<BF16>(Q.WH, e1.x * 32u + lane), w3 = cols_weight<BF16>(Q.WH, e1.z * 32u + lane);
+            a = fmaf(w0, __uint_as_float(e0.y), a);
+            a = fmaf(w1, __uint_as_float(e0.w), a);
+            a = fmaf(w2, __uint_as_float(e1.y), a);
+            a = fmaf(w3, __uint_as_float(e1.w), a);
         }
-        float sum[R];
-        cols_walk<BF16, R>(S, P.WT, P.N, col, sum);
-#pragma unroll
-        for (int k = 0; k < R; ++k) {
-            float z = sum[k] + __ldg(P.bias + nd[k]);
-            if (P.relu) z = z > 0.0f ? z : 0.0f;
-            if (r + k * 32u + lane < r1) {
-                if (P.use_list) {
-                    if (P.out_vals) P.out_vals[off + e[k]] = z;
-                    if (P.out_dense) {
-                        P.out_dense[(uint64_t)q * P.out_stride + e[k]] = z;
-                        if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q * P.out_stride + e[k]] = nd[k];
-                    }
-                } else {
-                    P.out_dense[(uint64_t)q * P.out_stride + nd[k]] = z;
-                }
-            }
-        }
+        zpart[p * 32u + lane] = a;
     }
+    for (uint32_t i = threadIdx.x; i < nwords; i += blockDim.x) idmap[i] = 0u;
+    __syncthreads();
+    if (threadIdx.x < H) {
+        float acc[32];
+#pragma unroll
+        for (int p = 0; p < 32; ++p) acc[p] = zpart[p * 32 + threadIdx.x];
+        zh[threadIdx.x] = cols_tree(acc) + __ldg(P.bias + __ldg(Q.hash_nodes + threadIdx.x));
+    }
+    __syncthreads();
+    // (2) keys
+    if (threadIdx.x < Q.L) {
+        uint32_t key = 0;
+        for (uint32_t j = 0; j < Q.K; ++j)
+            if (zh[threadIdx.x * Q.K + j] > 0.0f) key |= (1u << j);
+        keys[threadIdx.x] = key;
+        if (Q.codes) Q.codes[((uint64_t)q * P.n_act + P.a) * Q.L + threadIdx.x] = (uint16_t)key;
+    }
+    __syncthreads();
+    // (3) + (4) bucket lists, first B distinct ids, ascending, into the layer's list
+    if (!block_select<IDT>(Q.tables, Q.cap, Q.K, Q.L, P.N, B, keys, idmap, const_cast<uint32_t *>(P.ids) + off, scan_ws,
+                           &scan_total, Q.hash_nodes, Q.pre) &&
+        threadIdx.x == 0)
+        slonn_report(Q.status, SLONN_ERR_ARG, q, Q.layer);
+    __syncthreads();
+    // (5) the selected nodes
+    cols_order_and_gather<BF16, R, false>(P, S, smem4, q, off, B, 0u, B, scan_ws, &scan_total);
 }
 
 // ---------------------------------------------------------------------------
