@@ -88,6 +88,8 @@ def gathered_bytes(wl, budget_bp, force_rows=False, force_cols=False, cols_max_b
                 use_cols[:] = bp.size * int(b_out.max()) > 148 * 64
             elif big:
                 use_cols = bp <= cols_max_bp
+            elif bp.size * int(b_out.max()) > 148 * 64 and D >= 2048 and int(bp.max()) <= 1500:
+                use_cols = bp <= 1500
         b_in = budget_nodes(bp, D) if list_input else np.full(bp.size, D, np.int64)
         if wl.has_act[l] and wl.K * wl.L <= 32:
             layer += int(((b_out[use_cols] + wl.K * wl.L) * b_in[use_cols]).sum()) * esz

@@ -213,8 +213,9 @@ typedef struct {
  * ways with identical results: row kernels read each selected weight row whole; input-stationary
  * kernels walk the query's nonzero inputs and read single weights from a transposed copy the model
  * keeps of such layers.  By default the library picks per query by budget: up to SLONN_COLS_MAX_BP
- * the input list is sparse enough for the input-stationary kernels to win (batches too small to fill
- * the GPU with their 64-node warp passes keep the row kernels).  These two flags force one kind for the whole batch, for testing and
+ * the input list is sparse enough for the input-stationary kernels to win (batches of tens of queries
+ * only when no budget exceeds 1500 bp and only for layers at least 2048 inputs wide; a handful of queries keep
+ * the row kernels).  These two flags force one kind for the whole batch, for testing and
  * tuning; setting both is an error.  They apply to the per-stage kernels and to the
  * one-warp-per-query kernel; the one-cluster-per-query kernel has row form only.
  */

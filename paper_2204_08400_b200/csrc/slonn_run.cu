@@ -203,12 +203,12 @@ int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint
 #ifndef SLONN_COLS_R
 #define SLONN_COLS_R 2
 #endif
-template <bool BF16, int R>
+template <bool BF16, int R, bool SPLIT>
 int launch_gather_cols_t(const slonn_gather_params &P, uint64_t grid, uint32_t threads, size_t smem, cudaStream_t st)
 {
-    const int rc = set_smem(gather_cols_kernel<BF16, R>, smem);
+    const int rc = set_smem(gather_cols_kernel<BF16, R, SPLIT>, smem);
     if (rc) return rc;
-    gather_cols_kernel<BF16, R><<<(uint32_t)grid, threads, smem, st>>>(P);
+    gather_cols_kernel<BF16, R, SPLIT><<<(uint32_t)grid, threads, smem, st>>>(P);
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
@@ -217,10 +217,12 @@ int launch_gather_cols(const slonn_model *m, slonn_gather_params &P, uint32_t n,
     const uint32_t R = SLONN_COLS_R;
     const uint32_t passes = (max_rows + 32u * R - 1u) / (32u * R);
     const uint64_t want_ctas = 148ull * 8;
+    // too few warp passes to fill the GPU: one block per pass, its warps sharing the walk over the input list
+    const bool split = (uint64_t)n * passes < want_ctas;
     uint64_t ppc = ((uint64_t)n * passes + want_ctas - 1) / want_ctas; // passes per block
     ppc = std::min<uint64_t>(std::max<uint64_t>(ppc, 1), passes);
     const uint32_t rounds = (uint32_t)((ppc + 7) / 8);
-    const uint32_t warps = std::max(4u, (uint32_t)((ppc + rounds - 1) / rounds));
+    const uint32_t warps = split ? 8u : std::max(4u, (uint32_t)((ppc + rounds - 1) / rounds));
     P.rows_per_cta = (uint32_t)ppc * 32u * R;
     P.ctas_per_query = (max_rows + P.rows_per_cta - 1) / P.rows_per_cta;
     const bool bf = m->dtype == SLONN_BF16;
@@ -229,12 +231,15 @@ int launch_gather_cols(const slonn_model *m, slonn_gather_params &P, uint32_t n,
     if (P.use_list && P.colpos) scratch = std::max(scratch, ((size_t)2 * ((P.N + 31u) / 32u) + (size_t)3 * max_rows) * 4);
     scratch = (scratch + 15) & ~(size_t)15;
     P.scratch_bytes = (uint32_t)scratch;
-    const size_t smem = scratch + (size_t)cols_ent_cap(P.D, P.in_cap) * 8;
+    const size_t smem = scratch + (size_t)cols_ent_cap(P.D, P.in_cap) * 8 + (split ? (size_t)32 * R * 32 * 4 : 0);
     if (smem > 200 * 1024) return SLONN_ERR_DIM; // caller falls back to the row kernel
     const uint64_t grid = (uint64_t)n * P.ctas_per_query;
     if (grid == 0 || grid > 0x7fffffffull) return SLONN_ERR_DIM;
-    return bf ? launch_gather_cols_t<true, SLONN_COLS_R>(P, grid, warps * 32u, smem, st)
-              : launch_gather_cols_t<false, SLONN_COLS_R>(P, grid, warps * 32u, smem, st);
+    if (split)
+        return bf ? launch_gather_cols_t<true, SLONN_COLS_R, true>(P, grid, warps * 32u, smem, st)
+                  : launch_gather_cols_t<false, SLONN_COLS_R, true>(P, grid, warps * 32u, smem, st);
+    return bf ? launch_gather_cols_t<true, SLONN_COLS_R, false>(P, grid, warps * 32u, smem, st)
+              : launch_gather_cols_t<false, SLONN_COLS_R, false>(P, grid, warps * 32u, smem, st);
 }
 
 template <bool BF16, typename IDT>
@@ -277,12 +282,16 @@ int launch_layer_cols(const slonn_model *m, const slonn_layer &ly, uint32_t laye
 }
 
 // Budgets 1..limit take the input-stationary kernels in this layer (0: none do).
-uint32_t cols_budget_limit(const slonn_layer &ly, const slonn_gather_params &P, const slonn_batch *b, uint32_t n, uint32_t max_rows)
+uint32_t cols_budget_limit(const slonn_layer &ly, const slonn_gather_params &P, const slonn_batch *b, uint32_t n, uint32_t max_rows,
+                           uint32_t max_bp)
 {
     if (!ly.WT || P.in.kind != SLONN_IN_LIST || (b->flags & SLONN_FLAG_ROW_KERNELS)) return 0;
-    // small batches cannot fill the GPU with 64-node warp passes: they keep the row kernels unless told otherwise
     if (b->flags & SLONN_FLAG_COLUMN_KERNELS) return (uint64_t)n * max_rows > 148ull * 64 ? 10000u : 0u;
-    return (uint64_t)n * max_rows >= 148ull * 1024 ? SLONN_COLS_MAX_BP : 0u;
+    if ((uint64_t)n * max_rows >= 148ull * 1024) return SLONN_COLS_MAX_BP;
+    // tens of queries: the one-block-per-64-nodes variant pays only for long weight rows and very sparse lists
+    // (c4, 64 queries: 0.36 -> 0.30 ms per step at 10 %, but 0.57 -> 0.92 ms at 25 %)
+    // and only when no query of the batch needs the row kernels (a second launch of idle blocks costs such a batch 6 %)
+    return ((uint64_t)n * max_rows > 148ull * 64 && ly.D >= 2048u && max_bp <= 1500u) ? 1500u : 0u;
 }
 
 // Rows of one layer for a batch whose layer input is `P.in`: the input-stationary kernel for the queries
@@ -290,7 +299,7 @@ uint32_t cols_budget_limit(const slonn_layer &ly, const slonn_gather_params &P, 
 int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_params &P, const slonn_batch *b,
                       uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st, stage_timer *tm)
 {
-    const uint32_t cols_bp = cols_budget_limit(ly, P, b, n, max_rows);
+    const uint32_t cols_bp = cols_budget_limit(ly, P, b, n, max_rows, max_bp);
     int rc;
     if (cols_bp) {
         const bool both = max_bp > cols_bp;
@@ -324,7 +333,7 @@ int launch_act_layer(const slonn_model *m, const slonn_layer &ly, uint32_t l, sl
                      stage_timer *tm)
 {
     int rc;
-    const uint32_t cols_bp = cols_budget_limit(ly, gp, b, n, max_rows);
+    const uint32_t cols_bp = cols_budget_limit(ly, gp, b, n, max_rows, max_bp);
     if (cols_bp && ly.WH) {
         const bool both = max_bp > cols_bp;
         const uint32_t pre = slonn_model_pre(m);

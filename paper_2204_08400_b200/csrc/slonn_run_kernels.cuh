@@ -548,7 +548,7 @@ __global__ void __launch_bounds__(SLONN_THREADS, 2) gather_short_kernel(slonn_ga
 // query's selected nodes in column order and evaluates nodes [r0, r1) of that order against the staged
 // input list S.  `order_mem` is block scratch of P.scratch_bytes (the staging image, dead by now).  NC: the
 // id list was written by an earlier launch and may be read through the read-only path.
-template <bool BF16, int R, bool NC>
+template <bool BF16, int R, bool NC, bool SPLIT = false>
 __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params &P, const cols_stage &S, void *order_mem,
                                                       uint32_t q, uint64_t off, uint32_t B, uint32_t r0, uint32_t r1,
                                                       uint32_t *scan_ws, uint32_t *scan_total_p)
@@ -589,6 +589,72 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
     }
 
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    if constexpr (SPLIT) {
+        // Few queries: the block owns the 32 * R nodes [r0, r1) and its warps share the 32 segments, so that a
+        // node's walk over the input list is 32 / nwarps segments long instead of 32; the partial sums meet in
+        // shared memory and one thread per node adds them in the fixed tree.
+        float *zpart = reinterpret_cast<float *>(S.ent + cols_ent_cap(P.D, P.in_cap)); // [32][R][32]
+        uint32_t e[R], nd[R], col[R];
+#pragma unroll
+        for (int k = 0; k < R; ++k) {
+            const uint32_t rr = min(r0 + k * 32u + lane, r1 - 1);
+            e[k] = rr; nd[k] = rr; col[k] = rr;
+            if (ordered) { e[k] = sidx[rr]; col[k] = spos[rr]; }
+            if (P.use_list) {
+                nd[k] = list_id(e[k]);
+                if (!ordered) col[k] = nd[k];
+            }
+        }
+        for (uint32_t p = warp; p < 32; p += nwarps) {
+            float a[R];
+#pragma unroll
+            for (int k = 0; k < R; ++k) a[k] = 0.0f;
+            const uint32_t end = S.segstart[p + 1];
+            for (uint32_t i = S.segstart[p]; i < end; i += 4) {
+                const uint4 e0 = *reinterpret_cast<const uint4 *>(S.ent + i), e1 = *reinterpret_cast<const uint4 *>(S.ent + i + 2);
+                float w[R][4];
+#pragma unroll
+                for (int k = 0; k < R; ++k) {
+                    w[k][0] = cols_weight<BF16>(P.WT, e0.x * P.N + col[k]);
+                    w[k][1] = cols_weight<BF16>(P.WT, e0.z * P.N + col[k]);
+                    w[k][2] = cols_weight<BF16>(P.WT, e1.x * P.N + col[k]);
+                    w[k][3] = cols_weight<BF16>(P.WT, e1.z * P.N + col[k]);
+                }
+#pragma unroll
+                for (int k = 0; k < R; ++k) {
+                    a[k] = fmaf(w[k][0], __uint_as_float(e0.y), a[k]);
+                    a[k] = fmaf(w[k][1], __uint_as_float(e0.w), a[k]);
+                    a[k] = fmaf(w[k][2], __uint_as_float(e1.y), a[k]);
+                    a[k] = fmaf(w[k][3], __uint_as_float(e1.w), a[k]);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < R; ++k) zpart[(p * R + k) * 32u + lane] = a[k];
+        }
+        __syncthreads();
+        if (warp < (uint32_t)R) { // warp k finishes the nodes r0 + 32 k + lane
+            uint32_t me = e[0], mnd = nd[0];
+#pragma unroll
+            for (int k = 1; k < R; ++k)
+                if (warp == (uint32_t)k) { me = e[k]; mnd = nd[k]; }
+            float acc[32];
+#pragma unroll
+            for (int p = 0; p < 32; ++p) acc[p] = zpart[(p * R + warp) * 32u + lane];
+            float z = cols_tree(acc) + __ldg(P.bias + mnd);
+            if (P.relu) z = z > 0.0f ? z : 0.0f;
+            if (r0 + warp * 32u + lane < r1) {
+                if (P.use_list) {
+                    if (P.out_vals) P.out_vals[off + me] = z;
+                    if (P.out_dense) {
+                        P.out_dense[(uint64_t)q * P.out_stride + me] = z;
+                        if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q * P.out_stride + me] = mnd;
+                    }
+                } else {
+                    P.out_dense[(uint64_t)q * P.out_stride + mnd] = z;
+                }
+            }
+        }
+    } else
     for (uint32_t r = r0 + warp * (32u * R); r < r1; r += nwarps * (32u * R)) {
         uint32_t e[R], nd[R], col[R]; // place in the list, node id, column of WT
 #pragma unroll
@@ -629,7 +695,9 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
 // query's columns), so that the 32 lanes of a pass read neighbouring columns.  Same sums, same
 // order, same results as gather_dot_kernel; results are written at the node's place in the
 // id-ascending list.
-template <bool BF16, int R>
+// SPLIT: the variant for batches of tens of queries -- one block per (query, 32 * R nodes), the segments
+// of the input list spread over the block's warps (see cols_order_and_gather).
+template <bool BF16, int R, bool SPLIT>
 __global__ void __launch_bounds__(SLONN_THREADS) gather_cols_kernel(slonn_gather_params P)
 {
     extern __shared__ float4 smem4[];
@@ -662,7 +730,7 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_cols_kernel(slonn_gather
     const uint32_t len = min((uint32_t)(P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add + 1] - s0), P.in_cap);
     cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D);
 
-    cols_order_and_gather<BF16, R, true>(P, S, smem4, q, off, B, r0, r1, scan_ws, &scan_total);
+    cols_order_and_gather<BF16, R, true, SPLIT>(P, S, smem4, q, off, B, r0, r1, scan_ws, &scan_total);
 }
 
 // A whole list-fed activator layer for one query per block, input-stationary: the input list is grouped

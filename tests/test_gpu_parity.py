@@ -463,6 +463,16 @@ def test_input_stationary_kernel_on_a_wide_list_fed_layer():
     check(wl)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_input_stationary_kernel_for_a_few_dozen_queries(dtype):
+    # too few 64-node warp passes to fill the GPU: one block per (query, 64 nodes) whose warps share the
+    # walk over the input list and add their partial sums through shared memory; widths that are no
+    # multiple of 64 nodes or 32 chunks, budgets from one node to the whole layer
+    wl = custom_workload(76, [40, 296, 200, 12], [1, 1, 0], dtype, n=60, n_cal=200, K=3, L=2,
+                         budgets=(30, 500, 2500, 10000))
+    check(wl)
+
+
 def test_input_stationary_kernels_with_an_all_zero_list():
     # biases far below zero: every selected node of the first layer outputs exactly 0, so the next
     # layer's grouped input list is empty and its pre-activations are the biases
