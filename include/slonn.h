@@ -30,9 +30,11 @@
  *     multiply-add in ascending j, V = 16 bytes / weight element size; a fixed
  *     pairwise tree with strides 16, 8, 4, 2, 1; bias added last).  For a
  *     first layer fed by CSR input, j is the position in the row's id-ascending
- *     nonzero list and V = 1.  Hash bits are signs of such sums, so the order is
- *     part of the interface: it does not depend on batch size, budget or launch
- *     shape.  bf16 weights are widened exactly; activations and biases are fp32.
+ *     nonzero list and V = 1.  An input that is exactly 0 leaves its partial
+ *     sum unchanged and may be skipped (weights must be finite).  Hash bits are
+ *     signs of such sums, so the order is part of the interface: it does not
+ *     depend on batch size, budget or launch shape.  bf16 weights are widened
+ *     exactly; activations and biases are fp32.
  */
 #ifndef SLONN_H
 #define SLONN_H
