@@ -203,6 +203,9 @@ int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint
 #ifndef SLONN_COLS_R
 #define SLONN_COLS_R 2
 #endif
+// few-queries variants: warps per block, four segments of the input list each (4, 16 and 32 warps measured
+// slower on c4 with 64 queries: 0.237 / 0.248 / 0.372 ms against 0.195 ms for the seven hidden layers)
+#define SLONN_SPLIT_WARPS 8u
 template <bool BF16, int R, bool SPLIT>
 int launch_gather_cols_t(const slonn_gather_params &P, uint64_t grid, uint32_t threads, size_t smem, cudaStream_t st)
 {
@@ -222,7 +225,7 @@ int launch_gather_cols(const slonn_model *m, slonn_gather_params &P, uint32_t n,
     uint64_t ppc = ((uint64_t)n * passes + want_ctas - 1) / want_ctas; // passes per block
     ppc = std::min<uint64_t>(std::max<uint64_t>(ppc, 1), passes);
     const uint32_t rounds = (uint32_t)((ppc + 7) / 8);
-    const uint32_t warps = split ? 8u : std::max(4u, (uint32_t)((ppc + rounds - 1) / rounds));
+    const uint32_t warps = split ? SLONN_SPLIT_WARPS : std::max(4u, (uint32_t)((ppc + rounds - 1) / rounds));
     P.rows_per_cta = (uint32_t)ppc * 32u * R;
     P.ctas_per_query = (max_rows + P.rows_per_cta - 1) / P.rows_per_cta;
     const bool bf = m->dtype == SLONN_BF16;
@@ -242,43 +245,54 @@ int launch_gather_cols(const slonn_model *m, slonn_gather_params &P, uint32_t n,
               : launch_gather_cols_t<false, SLONN_COLS_R, false>(P, grid, warps * 32u, smem, st);
 }
 
-template <bool BF16, typename IDT>
-int launch_layer_cols_t(const slonn_layer_cols_params &Q, uint32_t n, uint32_t threads, size_t smem, cudaStream_t st)
+template <bool BF16, typename IDT, bool SPLIT>
+int launch_layer_cols_t(const slonn_layer_cols_params &Q, uint64_t grid, uint32_t threads, size_t smem, cudaStream_t st)
 {
-    const int rc = set_smem(layer_cols_kernel<BF16, IDT>, smem);
+    const int rc = set_smem(layer_cols_kernel<BF16, IDT, SPLIT>, smem);
     if (rc) return rc;
-    layer_cols_kernel<BF16, IDT><<<n, threads, smem, st>>>(Q);
+    layer_cols_kernel<BF16, IDT, SPLIT><<<(uint32_t)grid, threads, smem, st>>>(Q);
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
-// Hash, selection and input-stationary gather of a list-fed activator layer in one launch, one block per
-// query.  SLONN_ERR_DIM: not applicable here (no side-by-side hash rows, a batch so small that a query's
-// nodes should be spread over several blocks, or the staging does not fit) -- the caller takes the
-// separate kernels.
+template <bool BF16, typename IDT>
+int launch_layer_cols_s(const slonn_layer_cols_params &Q, bool split, uint64_t grid, uint32_t threads, size_t smem, cudaStream_t st)
+{
+    return split ? launch_layer_cols_t<BF16, IDT, true>(Q, grid, threads, smem, st)
+                 : launch_layer_cols_t<BF16, IDT, false>(Q, grid, threads, smem, st);
+}
+
+// Hash, selection and input-stationary gather of a list-fed activator layer in one launch: one block per
+// query, or, for batches of tens of queries, one block per (query, 64 nodes) with the selection repeated in
+// every block of a query.  SLONN_ERR_DIM: not applicable here (no side-by-side hash rows, or the staging
+// does not fit) -- the caller takes the separate kernels.
 int launch_layer_cols(const slonn_model *m, const slonn_layer &ly, uint32_t layer, slonn_gather_params G,
                       const slonn_batch *b, uint32_t n, uint32_t max_rows, cudaStream_t st)
 {
     if (!ly.WH || !ly.WT || !ly.colpos || !G.use_list) return SLONN_ERR_DIM;
     const uint32_t passes = (max_rows + 63u) / 64u;
-    if ((uint64_t)n * passes < 148ull * 8) return SLONN_ERR_DIM; // whole queries per block would leave SMs idle
+    const bool split = (uint64_t)n * passes < 148ull * 8; // whole queries per block would leave SMs idle
     const uint32_t rounds = (passes + 7) / 8;
-    const uint32_t warps = std::max(4u, (passes + rounds - 1) / rounds);
+    const uint32_t warps = split ? SLONN_SPLIT_WARPS : std::max(4u, (passes + rounds - 1) / rounds);
     const bool bf = m->dtype == SLONN_BF16;
     G.rows_cap = max_rows;
-    G.rows_per_cta = passes * 64u; G.ctas_per_query = 1;
+    G.rows_per_cta = split ? 64u : passes * 64u;
+    G.ctas_per_query = split ? passes : 1u;
     size_t scratch = cols_image_bytes(G.D, bf ? 8u : 4u);
     scratch = std::max(scratch, ((size_t)2 * ((G.N + 31u) / 32u) + (size_t)3 * max_rows) * 4);
     scratch = (scratch + 15) & ~(size_t)15;
     G.scratch_bytes = (uint32_t)scratch;
-    const size_t smem = scratch + (size_t)cols_ent_cap(G.D, G.in_cap) * 8 + (size_t)((G.N + 31u) / 32u) * 4 + 32 * 32 * 4;
+    const size_t smem = scratch + (size_t)cols_ent_cap(G.D, G.in_cap) * 8 + (size_t)((G.N + 31u) / 32u) * 4 + 32 * 2 * 32 * 4 +
+                        (split ? (size_t)max_rows * 4 : 0);
     if (smem > 200 * 1024) return SLONN_ERR_DIM;
+    const uint64_t grid = (uint64_t)n * G.ctas_per_query;
+    if (grid == 0 || grid > 0x7fffffffull) return SLONN_ERR_DIM;
     slonn_layer_cols_params Q;
     memset(&Q, 0, sizeof(Q));
     Q.G = G; Q.WH = ly.WH; Q.hash_nodes = ly.hash_nodes; Q.tables = ly.tables; Q.cap = ly.cap;
     Q.K = m->K; Q.L = m->L; Q.pre = slonn_model_pre(m); Q.layer = layer; Q.codes = b->codes; Q.status = b->status;
     const bool id16 = ly.id_bytes == 2;
-    if (bf) return id16 ? launch_layer_cols_t<true, uint16_t>(Q, n, warps * 32u, smem, st) : launch_layer_cols_t<true, uint32_t>(Q, n, warps * 32u, smem, st);
-    return id16 ? launch_layer_cols_t<false, uint16_t>(Q, n, warps * 32u, smem, st) : launch_layer_cols_t<false, uint32_t>(Q, n, warps * 32u, smem, st);
+    if (bf) return id16 ? launch_layer_cols_s<true, uint16_t>(Q, split, grid, warps * 32u, smem, st) : launch_layer_cols_s<true, uint32_t>(Q, split, grid, warps * 32u, smem, st);
+    return id16 ? launch_layer_cols_s<false, uint16_t>(Q, split, grid, warps * 32u, smem, st) : launch_layer_cols_s<false, uint32_t>(Q, split, grid, warps * 32u, smem, st);
 }
 
 // Budgets 1..limit take the input-stationary kernels in this layer (0: none do).

@@ -550,11 +550,13 @@ __global__ void __launch_bounds__(SLONN_THREADS, 2) gather_short_kernel(slonn_ga
 // id list was written by an earlier launch and may be read through the read-only path.
 template <bool BF16, int R, bool NC, bool SPLIT = false>
 __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params &P, const cols_stage &S, void *order_mem,
-                                                      uint32_t q, uint64_t off, uint32_t B, uint32_t r0, uint32_t r1,
-                                                      uint32_t *scan_ws, uint32_t *scan_total_p)
+                                                      const uint32_t *idlist, float *zpart, uint32_t q, uint64_t off,
+                                                      uint32_t B, uint32_t r0, uint32_t r1, uint32_t *scan_ws,
+                                                      uint32_t *scan_total_p)
 {
+    // idlist: the query's id-ascending node list (global or shared memory; unused when every node is computed)
     auto list_id = [&](uint32_t e) -> uint32_t {
-        const uint32_t v = NC ? __ldg(P.ids + off + e) : P.ids[off + e];
+        const uint32_t v = NC ? __ldg(idlist + e) : idlist[e];
         return min(v, P.N - 1u);
     };
     // the query's nodes in column order: spos[slot] = column, sidx[slot] = place in the id-ascending list
@@ -593,7 +595,7 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
         // Few queries: the block owns the 32 * R nodes [r0, r1) and its warps share the 32 segments, so that a
         // node's walk over the input list is 32 / nwarps segments long instead of 32; the partial sums meet in
         // shared memory and one thread per node adds them in the fixed tree.
-        float *zpart = reinterpret_cast<float *>(S.ent + cols_ent_cap(P.D, P.in_cap)); // [32][R][32]
+        // zpart: [32][R][32] floats of block scratch
         uint32_t e[R], nd[R], col[R];
 #pragma unroll
         for (int k = 0; k < R; ++k) {
@@ -730,7 +732,8 @@ __global__ void __launch_bounds__(SLONN_THREADS) gather_cols_kernel(slonn_gather
     const uint32_t len = min((uint32_t)(P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add + 1] - s0), P.in_cap);
     cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D);
 
-    cols_order_and_gather<BF16, R, true, SPLIT>(P, S, smem4, q, off, B, r0, r1, scan_ws, &scan_total);
+    cols_order_and_gather<BF16, R, true, SPLIT>(P, S, smem4, P.ids + off, reinterpret_cast<float *>(S.ent + cols_ent_cap(P.D, P.in_cap)),
+                                                 q, off, B, r0, r1, scan_ws, &scan_total);
 }
 
 // A whole list-fed activator layer for one query per block, input-stationary: the input list is grouped
@@ -748,7 +751,11 @@ struct slonn_layer_cols_params {
     uint32_t *status;
 };
 
-template <bool BF16, typename IDT>
+// SPLIT: the variant for batches of tens of queries -- one block per (query, 64 nodes).  Every block of a
+// query groups the input list, computes the hash functions and runs the selection itself (the same result
+// in each; only the first block writes keys and list to global memory), then evaluates its 64 nodes with
+// the segments of the input list spread over its warps.
+template <bool BF16, typename IDT, bool SPLIT>
 __global__ void __launch_bounds__(SLONN_THREADS) layer_cols_kernel(slonn_layer_cols_params Q)
 {
     extern __shared__ float4 smem4[];
@@ -761,23 +768,30 @@ __global__ void __launch_bounds__(SLONN_THREADS) layer_cols_kernel(slonn_layer_c
     __shared__ uint32_t scan_total;
     __shared__ uint32_t keys[8];
     __shared__ float zh[32];
-    const uint32_t q = blockIdx.x;
+    const uint32_t q = SPLIT ? blockIdx.x / P.ctas_per_query : blockIdx.x;
+    const uint32_t chunk = SPLIT ? blockIdx.x - q * P.ctas_per_query : 0u;
     if (P.skip_bp && P.skip_bp[q] == 10000u) return;
     if (!bp_in_range(P.range_bp, P.bp_lo, P.bp_hi, q)) return;
     const uint64_t off = P.indptr[(uint64_t)q * P.n_act + P.a];
     const uint32_t B = min((uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - off), P.rows_cap);
+    const uint32_t r0 = SPLIT ? chunk * P.rows_per_cta : 0u;
+    if (r0 >= B) return;
+    const uint32_t r1 = SPLIT ? min(B, r0 + P.rows_per_cta) : B;
+    const bool writer = chunk == 0u; // the block that publishes the query's keys and list
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t H = Q.K * Q.L;
     const uint32_t nwords = (P.N + 31u) >> 5;
 
-    // shared memory: [scratch: input image, then node order][entries][selection bitmap][hash partial sums]
+    // shared memory: [scratch: input image, then node order][entries][selection bitmap][partial sums]
+    // [SPLIT: the query's node list]
     cols_stage S;
     S.xs = reinterpret_cast<float *>(smem4);
     S.ent = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(smem4) + P.scratch_bytes);
     S.segcnt = segcnt;
     S.segstart = segstart;
     uint32_t *idmap = reinterpret_cast<uint32_t *>(S.ent + cols_ent_cap(P.D, P.in_cap));
-    float *zpart = reinterpret_cast<float *>(idmap + nwords);
+    float *zpart = reinterpret_cast<float *>(idmap + nwords);           // [32][R][32]
+    uint32_t *own_list = reinterpret_cast<uint32_t *>(zpart + 32 * R * 32); // [rows_cap], SPLIT only
     const uint64_t s0 = P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add];
     const uint32_t len = min((uint32_t)(P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add + 1] - s0), P.in_cap);
     cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D);
@@ -812,17 +826,21 @@ __global__ void __launch_bounds__(SLONN_THREADS) layer_cols_kernel(slonn_layer_c
         for (uint32_t j = 0; j < Q.K; ++j)
             if (zh[threadIdx.x * Q.K + j] > 0.0f) key |= (1u << j);
         keys[threadIdx.x] = key;
-        if (Q.codes) Q.codes[((uint64_t)q * P.n_act + P.a) * Q.L + threadIdx.x] = (uint16_t)key;
+        if (Q.codes && writer) Q.codes[((uint64_t)q * P.n_act + P.a) * Q.L + threadIdx.x] = (uint16_t)key;
     }
     __syncthreads();
-    // (3) + (4) bucket lists, first B distinct ids, ascending, into the layer's list
-    if (!block_select<IDT>(Q.tables, Q.cap, Q.K, Q.L, P.N, B, keys, idmap, const_cast<uint32_t *>(P.ids) + off, scan_ws,
-                           &scan_total, Q.hash_nodes, Q.pre) &&
-        threadIdx.x == 0)
+    // (3) + (4) bucket lists, first B distinct ids, ascending: into the layer's list, or, when several blocks
+    // work on the query, into this block's own copy, which the first block then publishes
+    uint32_t *global_list = const_cast<uint32_t *>(P.ids) + off;
+    uint32_t *list = SPLIT ? own_list : global_list;
+    if (!block_select<IDT>(Q.tables, Q.cap, Q.K, Q.L, P.N, B, keys, idmap, list, scan_ws, &scan_total, Q.hash_nodes, Q.pre) &&
+        threadIdx.x == 0 && writer)
         slonn_report(Q.status, SLONN_ERR_ARG, q, Q.layer);
     __syncthreads();
+    if (SPLIT && writer)
+        for (uint32_t i = threadIdx.x; i < B; i += blockDim.x) global_list[i] = own_list[i];
     // (5) the selected nodes
-    cols_order_and_gather<BF16, R, false>(P, S, smem4, q, off, B, 0u, B, scan_ws, &scan_total);
+    cols_order_and_gather<BF16, R, false, SPLIT>(P, S, smem4, list, zpart, q, off, B, r0, r1, scan_ws, &scan_total);
 }
 
 // ---------------------------------------------------------------------------
