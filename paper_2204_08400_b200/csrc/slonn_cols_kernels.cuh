@@ -117,6 +117,21 @@ __device__ __forceinline__ float cols_weight(const void *WT, uint32_t idx)
     return __ldg(reinterpret_cast<const float *>(WT) + idx);
 }
 
+// Two neighbouring weights WT[idx], WT[idx + 1] with one load; idx even.
+template <bool BF16>
+__device__ __forceinline__ void cols_weight2(const void *WT, uint32_t idx, float &w0, float &w1)
+{
+    if (BF16) {
+        const uint32_t u = __ldg(reinterpret_cast<const uint32_t *>(reinterpret_cast<const uint16_t *>(WT) + idx));
+        w0 = __uint_as_float(u << 16);
+        w1 = __uint_as_float(u & 0xffff0000u);
+    } else {
+        const float2 v = __ldg(reinterpret_cast<const float2 *>(reinterpret_cast<const float *>(WT) + idx));
+        w0 = v.x;
+        w1 = v.y;
+    }
+}
+
 // a[0] + ... + a[31] in the fixed tree: strides 16, 8, 4, 2, 1
 __device__ __forceinline__ float cols_tree(float (&acc)[32])
 {
@@ -136,7 +151,9 @@ __device__ __forceinline__ float cols_tree(float (&acc)[32])
 // with at most five pending partial results per node instead of 32 registers.
 // A segment holds a multiple of 4 entries; 4 entries x R loads are in flight at a time.
 // Row j of WT starts at element j * ld.
-template <bool BF16, int R>
+// PAIR (R = 2): the two nodes are the neighbouring columns col[0] (even) and col[0] + 1 of a WT with even ld,
+// fetched with one load per input.
+template <bool BF16, int R, bool PAIR = false>
 __device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, uint32_t ld, const uint32_t (&col)[R],
                                           float (&sum)[R])
 {
@@ -160,12 +177,19 @@ __device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, u
         for (; k < e; k += 4) {
             const uint4 e0 = *reinterpret_cast<const uint4 *>(S.ent + k), e1 = *reinterpret_cast<const uint4 *>(S.ent + k + 2);
             float w[R][4];
+            if constexpr (PAIR) {
+                cols_weight2<BF16>(WT, e0.x * ld + col[0], w[0][0], w[R - 1][0]);
+                cols_weight2<BF16>(WT, e0.z * ld + col[0], w[0][1], w[R - 1][1]);
+                cols_weight2<BF16>(WT, e1.x * ld + col[0], w[0][2], w[R - 1][2]);
+                cols_weight2<BF16>(WT, e1.z * ld + col[0], w[0][3], w[R - 1][3]);
+            } else {
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                w[r][0] = cols_weight<BF16>(WT, e0.x * ld + col[r]);
-                w[r][1] = cols_weight<BF16>(WT, e0.z * ld + col[r]);
-                w[r][2] = cols_weight<BF16>(WT, e1.x * ld + col[r]);
-                w[r][3] = cols_weight<BF16>(WT, e1.z * ld + col[r]);
+                for (int r = 0; r < R; ++r) {
+                    w[r][0] = cols_weight<BF16>(WT, e0.x * ld + col[r]);
+                    w[r][1] = cols_weight<BF16>(WT, e0.z * ld + col[r]);
+                    w[r][2] = cols_weight<BF16>(WT, e1.x * ld + col[r]);
+                    w[r][3] = cols_weight<BF16>(WT, e1.z * ld + col[r]);
+                }
             }
 #pragma unroll
             for (int r = 0; r < R; ++r) a[r] = fmaf(w[r][0], __uint_as_float(e0.y), a[r]);

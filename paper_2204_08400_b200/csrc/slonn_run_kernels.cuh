@@ -656,6 +656,25 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
                 }
             }
         }
+    } else if (R == 2 && !P.use_list && (P.N & 1u) == 0u && (r0 & 1u) == 0u) {
+        // every node of the layer (a layer without activator): a lane takes two neighbouring columns and
+        // fetches both weights of an input with one load
+        for (uint32_t r = r0 + warp * 64u; r < r1; r += nwarps * 64u) {
+            const uint32_t c0 = min(r + 2u * lane, (r1 - 1u) & ~1u); // even; c0 + 1 < N because N is even
+            const uint32_t col[R] = {c0, c0 + 1u};
+            float sum[R];
+            cols_walk<BF16, R, true>(S, P.WT, P.N, col, sum);
+            if (r + 2u * lane < r1) {
+#pragma unroll
+                for (int k = 0; k < R; ++k) {
+                    if (col[k] < r1) {
+                        float z = sum[k] + __ldg(P.bias + col[k]);
+                        if (P.relu) z = z > 0.0f ? z : 0.0f;
+                        P.out_dense[(uint64_t)q * P.out_stride + col[k]] = z;
+                    }
+                }
+            }
+        }
     } else
     for (uint32_t r = r0 + warp * (32u * R); r < r1; r += nwarps * (32u * R)) {
         uint32_t e[R], nd[R], col[R]; // place in the list, node id, column of WT
