@@ -76,6 +76,12 @@ bool tc_route(const slonn_model *m, uint32_t max_bp, uint32_t flags)
            !m->layer[m->n_layers - 1].has_act;
 }
 
+// whether a batch with this largest budget may hold 100 % queries that the grouped full-network kernel can take
+bool full_route_possible(const slonn_model *m, uint32_t max_bp)
+{
+    return max_bp == 10000u && !m->first_sparse;
+}
+
 ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp, uint32_t flags)
 {
     ws_layout w;
@@ -90,9 +96,11 @@ ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp, uint32_t flag
     w.dense0 = o; o += db;
     w.dense1 = o; o += db;
     w.tc_list = w.tc_count = w.tc_a0 = w.tc_a1 = 0;
-    if (tc_route(m, max_bp, flags)) {
+    if (tc_route(m, max_bp, flags) || full_route_possible(m, max_bp)) { // the batch's 100 % queries, compacted
         w.tc_list = o; o = align_up(o + (uint64_t)n * sizeof(uint32_t), 256);
         w.tc_count = o; o += 256;
+    }
+    if (tc_route(m, max_bp, flags)) {
         const uint64_t ab = align_up((uint64_t)n * tc_width(m) * sizeof(uint16_t), 256);
         w.tc_a0 = o; o += ab;
         w.tc_a1 = o; o += ab;
@@ -379,6 +387,37 @@ int launch_act_layer(const slonn_model *m, const slonn_layer &ly, uint32_t l, sl
     TOC();
     if (rc) return rc;
     return launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st, tm);
+}
+
+// ---- 100 % queries, four per block ---------------------------------------------
+
+template <bool BF16>
+int launch_full_rows_t(const slonn_full_params &P, uint64_t grid, size_t smem, cudaStream_t st)
+{
+    const int rc = set_smem(full_rows_kernel<BF16>, smem);
+    if (rc) return rc;
+    full_rows_kernel<BF16><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(P);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+// SLONN_ERR_DIM: four staged inputs do not fit shared memory (the caller leaves these queries to the other kernels,
+// which it can only decide before the first layer: see full_route_fits)
+int launch_full_rows(const slonn_model *m, slonn_full_params &P, uint32_t n, cudaStream_t st)
+{
+    const uint32_t groups = (n + SLONN_FULL_GROUP - 1) / SLONN_FULL_GROUP;
+    P.rows_per_cta = std::min((P.N + 31u) / 32u * 32u, 1024u);
+    P.ctas_per_group = (P.N + P.rows_per_cta - 1) / P.rows_per_cta;
+    const size_t smem = (size_t)SLONN_FULL_GROUP * P.D * 4;
+    const uint64_t grid = (uint64_t)groups * P.ctas_per_group;
+    if (grid == 0 || grid > 0x7fffffffull || smem > 200 * 1024) return SLONN_ERR_DIM;
+    return m->dtype == SLONN_BF16 ? launch_full_rows_t<true>(P, grid, smem, st) : launch_full_rows_t<false>(P, grid, smem, st);
+}
+
+bool full_route_fits(const slonn_model *m)
+{
+    for (uint32_t l = 0; l < m->n_layers; ++l)
+        if ((size_t)SLONN_FULL_GROUP * m->layer[l].D * 4 > 200 * 1024) return false;
+    return true;
 }
 
 // ---- whole-network kernel for narrow layers -----------------------------------
@@ -743,6 +782,19 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
     }
 
+    // Queries at a 100 % budget all compute the same rows (every node of every layer): they are taken out of the
+    // per-query kernels, compacted, and evaluated four per block by full_rows_kernel, layer by layer beside the
+    // others.  Same fixed-order sums, so nothing about their results changes.
+    uint32_t *full_list = nullptr, *full_count = nullptr;
+    if (!skip_bp && full_route_possible(m, max_bp) && full_route_fits(m) && n >= 256) {
+        full_list = (uint32_t *)(ws + wl.tc_list);
+        full_count = (uint32_t *)(ws + wl.tc_count);
+        if (cudaMemsetAsync(full_count, 0, sizeof(uint32_t), st) != cudaSuccess) return SLONN_ERR_CUDA;
+        dense_compact_kernel<<<(n + 255) / 256, 256, 0, st>>>(b->budget_bp, n, full_list, full_count);
+        if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+        skip_bp = b->budget_bp;
+    }
+
     // input := x
     slonn_input in;
     memset(&in, 0, sizeof(in));
@@ -775,6 +827,30 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         gp.n_act = m->n_act; gp.indptr = indptr; gp.ids = ids;
         gp.relu = is_last ? 0u : 1u;
         uint32_t max_rows = ly.N;
+        if (full_list) { // this layer for the batch's 100 % queries
+            slonn_full_params fp;
+            memset(&fp, 0, sizeof(fp));
+            fp.list = full_list; fp.count = full_count; fp.in = in;
+            fp.W = ly.W; fp.bias = ly.bias; fp.D = ly.D; fp.N = ly.N; fp.nchunks = nchunks;
+            fp.has_act = ly.has_act; fp.n_act = m->n_act; fp.a = m->act_index[l]; fp.indptr = indptr;
+            fp.out_ids = ids; fp.out_vals = vals; fp.relu = is_last ? 0u : 1u;
+            if (ly.has_act) {
+                if (is_last) { fp.out_dense = b->logits; fp.out_dense_ids = b->logit_ids; fp.out_stride = stride; }
+            } else {
+                fp.out_dense = is_last ? b->logits : dense[dense_cur];
+                fp.out_stride = ly.N;
+            }
+            TIC(SLONN_STAGE_GATHER_DOT);
+            rc = launch_full_rows(m, fp, n, st);
+            TOC();
+            if (rc) return rc;
+            if (ly.has_act && b->codes) { // keys from the signs of the hash nodes' activations (all nodes were computed)
+                const uint32_t t = n * m->L;
+                dense_codes_kernel<<<(t + 127) / 128, 128, 0, st>>>(full_list, full_count, vals, indptr, m->n_act, m->act_index[l],
+                                                                   ly.hash_nodes, m->K, m->L, b->codes);
+                if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+            }
+        }
         if (ly.has_act) {
             const uint32_t a = m->act_index[l];
             slonn_select_params sp;
