@@ -337,9 +337,21 @@ def main():
         ms, cnt = sl.slonn_run_timed(dm.model, batch.batch, batch.ws, batch.ws_bytes, stream)
         for s in sl.STAGES:
             stage_ms[s] += ms[s]; stage_cnt[s] += cnt[s]
+    def full_route_active(bps):
+        """The library's rule for taking the 100 % queries out of the per-query kernels (four per block)."""
+        weights = sum(wl.dims[l] * wl.dims[l + 1] for l in range(len(wl.dims) - 1))
+        return (not (flags & sl.FLAG_DENSE_TC) and not wl.first_sparse and bps.size >= 256 and int(bps.max()) == 10000
+                and bps.size * weights >= 2 ** 32 and 16 * max(wl.dims[:-1]) <= 200 * 1024)
+
     def stage_roofline(ms_by_stage, cnt_by_stage, bps, steps):
         """Dominant kernel of the step and its achieved rate on the weight bytes it must touch."""
-        if flags & sl.FLAG_DENSE_TC:     # queries at 100 % leave the row kernels
+        esz = 2 if wl.dtype == "bf16" else 4
+        n_full = int((bps == 10000).sum()) if bps.size and full_route_active(bps) else 0
+        full_b = n_full * sum(wl.dims[l] * wl.dims[l + 1] for l in range(len(wl.dims) - 1)) * esz
+        if n_full and ms_by_stage["full_rows"] >= max(ms_by_stage.values()):
+            ms, launches = ms_by_stage["full_rows"] / steps, cnt_by_stage["full_rows"] // steps
+            return "full_rows_kernel", ms, launches, full_b, full_b / (ms / 1e3) / 1e9
+        if (flags & sl.FLAG_DENSE_TC) or n_full:     # queries at 100 % leave the per-query kernels
             bps = bps[bps != 10000]
         row_b, col_b, layer_b = gathered_bytes(wl, bps, args.row_kernels, args.column_kernels, sl.COLS_MAX_BP)
         cols_ms = ms_by_stage["gather_cols"] + ms_by_stage["layer_cols"]

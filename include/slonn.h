@@ -387,7 +387,8 @@ int slonn_run_static(const slonn_model *m, const slonn_batch *batch, void *strea
 #define SLONN_STAGE_CLUSTER 7       /* all of 1, 2, 4 in the one-cluster-per-query kernel */
 #define SLONN_STAGE_GATHER_COLS 8   /* selected nodes' dot products, input-stationary kernel */
 #define SLONN_STAGE_LAYER_COLS 9    /* all of 1 and 8 for a list-fed activator layer in one launch */
-#define SLONN_N_STAGES 10
+#define SLONN_STAGE_FULL_ROWS 10    /* every layer of the 100 % budget queries, four queries per block */
+#define SLONN_N_STAGES 11
 int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *workspace,
                     uint64_t workspace_bytes, void *stream, float *stage_ms,
                     uint32_t *stage_launches);

@@ -424,7 +424,7 @@ def slonn_run_static(model: Model, batch: _Batch, stream=None) -> None:
         raise SlonnError(rc, "slonn_run_static")
 
 
-STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused", "dense_tc", "cluster", "gather_cols", "layer_cols")
+STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused", "dense_tc", "cluster", "gather_cols", "layer_cols", "full_rows")
 COLS_MAX_BP = 3500   # SLONN_COLS_MAX_BP
 FLAG_DENSE_TC = 1
 FLAG_ROW_KERNELS = 2

@@ -652,6 +652,64 @@ extern "C" int slonn_workspace_bytes(const slonn_model *m, uint32_t n, uint32_t 
     return SLONN_OK;
 }
 
+// Every layer for the batch's 100 % queries (compacted in `list` / `count`), four queries per block.  They share
+// nothing with the other queries but the output arrays (disjoint entries), so this runs as a pass of its own.
+static int run_full_route(const slonn_model *m, const slonn_batch *b, uint32_t n, const uint32_t *list, const uint32_t *count,
+                          const uint64_t *indptr, uint32_t *ids, float *vals, float *const dense[2], uint32_t stride,
+                          cudaStream_t st, stage_timer *tm)
+{
+    slonn_input in;
+    memset(&in, 0, sizeof(in));
+    in.kind = SLONN_IN_DENSE;
+    in.dense = b->x_dense;
+    int dense_cur = 0;
+    const uint32_t esz = m->dtype == SLONN_BF16 ? 2u : 4u;
+    for (uint32_t l = 0; l < m->n_layers; ++l) {
+        const slonn_layer &ly = m->layer[l];
+        const bool is_last = (l + 1 == m->n_layers);
+        slonn_full_params fp;
+        memset(&fp, 0, sizeof(fp));
+        fp.list = list; fp.count = count; fp.in = in;
+        fp.W = ly.W; fp.bias = ly.bias; fp.D = ly.D; fp.N = ly.N; fp.nchunks = ly.D * esz / 16u;
+        fp.has_act = ly.has_act; fp.n_act = m->n_act; fp.a = m->act_index[l]; fp.indptr = indptr;
+        fp.out_ids = ids; fp.out_vals = vals; fp.relu = is_last ? 0u : 1u;
+        if (ly.has_act) {
+            if (is_last) { fp.out_dense = b->logits; fp.out_dense_ids = b->logit_ids; fp.out_stride = stride; }
+        } else {
+            fp.out_dense = is_last ? b->logits : dense[dense_cur];
+            fp.out_stride = ly.N;
+        }
+        TIC(SLONN_STAGE_FULL_ROWS);
+        const int rc = launch_full_rows(m, fp, n, st);
+        TOC();
+        if (rc) return rc;
+        if (ly.has_act) {
+            if (b->codes) { // keys from the signs of the hash nodes' values (every node was computed)
+                const uint32_t t = n * m->L;
+                dense_codes_kernel<<<(t + 127) / 128, 128, 0, st>>>(list, count, vals, indptr, m->n_act, m->act_index[l],
+                                                                   ly.hash_nodes, m->K, m->L, b->codes);
+                if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+            }
+            in.kind = SLONN_IN_LIST; in.indptr = indptr; in.ids = ids; in.vals = vals;
+            in.ip_mul = m->n_act; in.ip_add = m->act_index[l];
+        } else {
+            in.kind = SLONN_IN_DENSE; in.dense = fp.out_dense;
+            dense_cur ^= 1;
+        }
+    }
+    return SLONN_OK;
+}
+
+// whether the batch's 100 % queries are taken out of the per-query kernels and run four per block: the batch must be
+// able to hold some (largest budget 100 %), and be large enough for the extra launches to vanish in the work
+static bool full_route_wanted(const slonn_model *m, uint32_t n, uint32_t max_bp)
+{
+    if (!full_route_possible(m, max_bp) || !full_route_fits(m) || n < 256) return false;
+    uint64_t weights = 0;
+    for (uint32_t l = 0; l < m->n_layers; ++l) weights += (uint64_t)m->layer[l].N * m->layer[l].D;
+    return (uint64_t)n * weights >= (1ull << 32);
+}
+
 static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes,
                     void *stream, stage_timer *tm)
 {
@@ -698,7 +756,9 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     // counts from the budget), which saves the two planning launches
     if (b->kernel_path == SLONN_PATH_FUSED && !fused_eligible(m)) return SLONN_ERR_DIM;
     const bool use_fused = b->kernel_path == SLONN_PATH_FUSED || (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n >= 512);
-    const bool no_plan = use_fused && !tc_route(m, max_bp, b->flags) && !b->active_indptr && !b->active_ids && !b->active_vals;
+    const bool full_route = !tc_route(m, max_bp, b->flags) && full_route_wanted(m, n, max_bp);
+    const bool no_plan = use_fused && !tc_route(m, max_bp, b->flags) && !full_route && !b->active_indptr && !b->active_ids &&
+                         !b->active_vals;
 
     // offsets of every (query, activator layer) list
     if (m->n_act && !no_plan) {
@@ -766,6 +826,19 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     }
 
     // narrow networks with enough queries to fill the GPU: one warp per query, every layer in one launch
+    // Queries at a 100 % budget all compute the same rows (every node of every layer): they are taken out of the
+    // per-query kernels, compacted, and evaluated four per block by full_rows_kernel.  Same fixed-order sums, so
+    // nothing about their results changes.
+    if (full_route) {
+        uint32_t *full_list = (uint32_t *)(ws + wl.tc_list), *full_count = (uint32_t *)(ws + wl.tc_count);
+        if (cudaMemsetAsync(full_count, 0, sizeof(uint32_t), st) != cudaSuccess) return SLONN_ERR_CUDA;
+        dense_compact_kernel<<<(n + 255) / 256, 256, 0, st>>>(b->budget_bp, n, full_list, full_count);
+        if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+        const int rc = run_full_route(m, b, n, full_list, full_count, indptr, ids, vals, dense, stride, st, tm);
+        if (rc) return rc;
+        skip_bp = b->budget_bp;
+    }
+
     if (use_fused) {
         TIC(SLONN_STAGE_FUSED);
         const int rc = launch_fused(m, b, no_plan ? nullptr : indptr, stride, skip_bp, max_bp, st);
@@ -780,19 +853,6 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         else argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
         TOC();
         return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
-    }
-
-    // Queries at a 100 % budget all compute the same rows (every node of every layer): they are taken out of the
-    // per-query kernels, compacted, and evaluated four per block by full_rows_kernel, layer by layer beside the
-    // others.  Same fixed-order sums, so nothing about their results changes.
-    uint32_t *full_list = nullptr, *full_count = nullptr;
-    if (!skip_bp && full_route_possible(m, max_bp) && full_route_fits(m) && n >= 256) {
-        full_list = (uint32_t *)(ws + wl.tc_list);
-        full_count = (uint32_t *)(ws + wl.tc_count);
-        if (cudaMemsetAsync(full_count, 0, sizeof(uint32_t), st) != cudaSuccess) return SLONN_ERR_CUDA;
-        dense_compact_kernel<<<(n + 255) / 256, 256, 0, st>>>(b->budget_bp, n, full_list, full_count);
-        if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
-        skip_bp = b->budget_bp;
     }
 
     // input := x
@@ -827,30 +887,6 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         gp.n_act = m->n_act; gp.indptr = indptr; gp.ids = ids;
         gp.relu = is_last ? 0u : 1u;
         uint32_t max_rows = ly.N;
-        if (full_list) { // this layer for the batch's 100 % queries
-            slonn_full_params fp;
-            memset(&fp, 0, sizeof(fp));
-            fp.list = full_list; fp.count = full_count; fp.in = in;
-            fp.W = ly.W; fp.bias = ly.bias; fp.D = ly.D; fp.N = ly.N; fp.nchunks = nchunks;
-            fp.has_act = ly.has_act; fp.n_act = m->n_act; fp.a = m->act_index[l]; fp.indptr = indptr;
-            fp.out_ids = ids; fp.out_vals = vals; fp.relu = is_last ? 0u : 1u;
-            if (ly.has_act) {
-                if (is_last) { fp.out_dense = b->logits; fp.out_dense_ids = b->logit_ids; fp.out_stride = stride; }
-            } else {
-                fp.out_dense = is_last ? b->logits : dense[dense_cur];
-                fp.out_stride = ly.N;
-            }
-            TIC(SLONN_STAGE_GATHER_DOT);
-            rc = launch_full_rows(m, fp, n, st);
-            TOC();
-            if (rc) return rc;
-            if (ly.has_act && b->codes) { // keys from the signs of the hash nodes' activations (all nodes were computed)
-                const uint32_t t = n * m->L;
-                dense_codes_kernel<<<(t + 127) / 128, 128, 0, st>>>(full_list, full_count, vals, indptr, m->n_act, m->act_index[l],
-                                                                   ly.hash_nodes, m->K, m->L, b->codes);
-                if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
-            }
-        }
         if (ly.has_act) {
             const uint32_t a = m->act_index[l];
             slonn_select_params sp;
