@@ -64,7 +64,7 @@ def budget_nodes(bp, N):
 
 def gathered_bytes(wl, budget_bp, force_rows=False, force_cols=False, cols_max_bp=3500):
     """Algorithmic weight bytes of one step's gather launches, all queries, split by kernel kind:
-    (row kernels, gather_cols_kernel, layer_cols_kernel).
+    (row kernels, gather_cols_kernel, layer_cols_kernel, full_rows_kernel on layers without activator).
     Row kernels (dense input, or a list input that is not sparse enough): every selected weight row
     once per query, whole (row-granular).  Input-stationary kernels (a layer fed by the list of the
     activator layer below, budgets up to cols_max_bp): selected nodes x input list entries
@@ -72,9 +72,9 @@ def gathered_bytes(wl, budget_bp, force_rows=False, force_cols=False, cols_max_b
     activator layer also reads its K*L hash rows at the list entries."""
     esz = 2 if wl.dtype == "bf16" else 4
     bp = np.asarray(budget_bp)
-    rows = cols = layer = 0
+    rows = cols = layer = grouped = 0
     if bp.size == 0:
-        return 0, 0, 0
+        return 0, 0, 0, 0
     for l in range(len(wl.dims) - 1):
         if l == 0 and wl.first_sparse:
             continue
@@ -95,8 +95,14 @@ def gathered_bytes(wl, budget_bp, force_rows=False, force_cols=False, cols_max_b
             layer += int(((b_out[use_cols] + wl.K * wl.L) * b_in[use_cols]).sum()) * esz
         else:
             cols += int((b_out[use_cols] * b_in[use_cols]).sum()) * esz
-        rows += int(b_out[~use_cols].sum()) * D * esz
-    return rows, cols, layer
+        row_bytes = int(b_out[~use_cols].sum()) * D * esz
+        # a layer without activator: the row-kernel queries share every row and run four per block
+        if (not wl.has_act[l] and bp.size >= 256 and bp.size * N * D >= 2 ** 30 and 16 * D <= 200 * 1024
+                and not use_cols.all()):
+            grouped += row_bytes
+        else:
+            rows += row_bytes
+    return rows, cols, layer, grouped
 
 
 class ClockSampler:
@@ -348,18 +354,19 @@ def main():
         esz = 2 if wl.dtype == "bf16" else 4
         n_full = int((bps == 10000).sum()) if bps.size and full_route_active(bps) else 0
         full_b = n_full * sum(wl.dims[l] * wl.dims[l + 1] for l in range(len(wl.dims) - 1)) * esz
-        if n_full and ms_by_stage["full_rows"] >= max(ms_by_stage.values()):
-            ms, launches = ms_by_stage["full_rows"] / steps, cnt_by_stage["full_rows"] // steps
-            return "full_rows_kernel", ms, launches, full_b, full_b / (ms / 1e3) / 1e9
         if (flags & sl.FLAG_DENSE_TC) or n_full:     # queries at 100 % leave the per-query kernels
             bps = bps[bps != 10000]
-        row_b, col_b, layer_b = gathered_bytes(wl, bps, args.row_kernels, args.column_kernels, sl.COLS_MAX_BP)
+        row_b, col_b, layer_b, grouped_b = gathered_bytes(wl, bps, args.row_kernels, args.column_kernels, sl.COLS_MAX_BP)
+        if ms_by_stage["full_rows"] > 0 and ms_by_stage["full_rows"] >= max(ms_by_stage.values()):
+            ms, launches = ms_by_stage["full_rows"] / steps, cnt_by_stage["full_rows"] // steps
+            nbytes = full_b + (grouped_b if ms_by_stage["fused"] == 0 and ms_by_stage["cluster"] == 0 else 0)
+            return "full_rows_kernel", ms, launches, nbytes, nbytes / (ms / 1e3) / 1e9
         cols_ms = ms_by_stage["gather_cols"] + ms_by_stage["layer_cols"]
         if ms_by_stage["fused"] > 0:     # one launch does hash + select + gather for every layer
-            row_b = gathered_bytes(wl, bps, force_rows=True)[0]
+            row_b = sum(gathered_bytes(wl, bps, force_rows=True)[i] for i in (0, 3))
             kernel, ms, launches, nbytes = "fused_network_kernel", ms_by_stage["fused"], cnt_by_stage["fused"], row_b + hash_bytes(wl, bps.size)
         elif ms_by_stage["cluster"] > 0:
-            row_b = gathered_bytes(wl, bps, force_rows=True)[0]
+            row_b = sum(gathered_bytes(wl, bps, force_rows=True)[i] for i in (0, 3))
             kernel, ms, launches, nbytes = "cluster_network_kernel", ms_by_stage["cluster"], cnt_by_stage["cluster"], row_b + hash_bytes(wl, bps.size)
         elif cols_ms > ms_by_stage["gather_dot"]:
             # the input-stationary kernels: the whole-layer kernel of the activator layers (hash + selection +

@@ -96,10 +96,9 @@ ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp, uint32_t flag
     w.dense0 = o; o += db;
     w.dense1 = o; o += db;
     w.tc_list = w.tc_count = w.tc_a0 = w.tc_a1 = 0;
-    if (tc_route(m, max_bp, flags) || full_route_possible(m, max_bp)) { // the batch's 100 % queries, compacted
-        w.tc_list = o; o = align_up(o + (uint64_t)n * sizeof(uint32_t), 256);
-        w.tc_count = o; o += 256;
-    }
+    // a compacted list of queries: the batch's 100 % queries, or the queries a grouped launch serves
+    w.tc_list = o; o = align_up(o + (uint64_t)n * sizeof(uint32_t), 256);
+    w.tc_count = o; o += 256;
     if (tc_route(m, max_bp, flags)) {
         const uint64_t ab = align_up((uint64_t)n * tc_width(m) * sizeof(uint16_t), 256);
         w.tc_a0 = o; o += ab;
@@ -318,11 +317,14 @@ uint32_t cols_budget_limit(const slonn_layer &ly, const slonn_gather_params &P, 
 
 // Rows of one layer for a batch whose layer input is `P.in`: the input-stationary kernel for the queries
 // whose input list is sparse (by budget), the row kernel for the others.  Results do not depend on the split.
+// rows_done: the queries above the input-stationary limit were served by another launch already.
 int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_params &P, const slonn_batch *b,
-                      uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st, stage_timer *tm)
+                      uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st, stage_timer *tm,
+                      bool rows_done = false)
 {
     const uint32_t cols_bp = cols_budget_limit(ly, P, b, n, max_rows, max_bp);
     int rc;
+    if (!cols_bp && rows_done) return SLONN_OK;
     if (cols_bp) {
         const bool both = max_bp > cols_bp;
         slonn_gather_params C = P;
@@ -336,8 +338,10 @@ int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_
         rc = launch_gather_cols(m, C, n, cols_rows, st);
         TOC();
         if (rc != SLONN_ERR_DIM) { // SLONN_ERR_DIM: the staging does not fit shared memory, rows for everyone
-            if (rc || !both) return rc;
+            if (rc || !both || rows_done) return rc;
             P.range_bp = b->budget_bp; P.bp_lo = cols_bp + 1; P.bp_hi = 0xffffu;
+        } else if (rows_done) { // only the low budgets are still open
+            P.range_bp = b->budget_bp; P.bp_lo = 0; P.bp_hi = cols_bp;
         }
     }
     TIC(SLONN_STAGE_GATHER_DOT);
@@ -909,7 +913,30 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             gp.use_list = 0;
             gp.out_dense = is_last ? b->logits : dense[dense_cur];
             gp.out_stride = ly.N;
-            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st, tm);
+            // A layer without activator computes every node for every query: the queries the row kernel would
+            // serve (budgets above the input-stationary limit) share all their weight rows, so they are
+            // compacted and taken four per block.
+            bool rows_done = false;
+            const uint32_t cols_bp = cols_budget_limit(ly, gp, b, n, max_rows, max_bp);
+            if (n >= 256 && (uint64_t)n * ly.N * ly.D >= (1ull << 30) && (size_t)SLONN_FULL_GROUP * ly.D * 4 <= 200 * 1024 &&
+                cols_bp < max_bp) {
+                uint32_t *glist = (uint32_t *)(ws + wl.tc_list), *gcount = (uint32_t *)(ws + wl.tc_count);
+                if (cudaMemsetAsync(gcount, 0, sizeof(uint32_t), st) != cudaSuccess) return SLONN_ERR_CUDA;
+                range_compact_kernel<<<(n + 255) / 256, 256, 0, st>>>(b->budget_bp, skip_bp, n, cols_bp ? cols_bp + 1 : 0u, 0xffffu,
+                                                                     glist, gcount);
+                if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+                slonn_full_params fp;
+                memset(&fp, 0, sizeof(fp));
+                fp.list = glist; fp.count = gcount; fp.in = in;
+                fp.W = ly.W; fp.bias = ly.bias; fp.D = ly.D; fp.N = ly.N; fp.nchunks = nchunks;
+                fp.has_act = 0; fp.out_dense = gp.out_dense; fp.out_stride = ly.N; fp.relu = gp.relu;
+                TIC(SLONN_STAGE_FULL_ROWS);
+                rc = launch_full_rows(m, fp, n, st);
+                TOC();
+                if (rc) return rc;
+                rows_done = true;
+            }
+            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st, tm, rows_done);
             if (rc) return rc;
             in.kind = SLONN_IN_DENSE; in.dense = gp.out_dense;
             dense_cur ^= 1;

@@ -1125,6 +1125,25 @@ __global__ void __launch_bounds__(256) argmax_block_kernel(slonn_argmax_params P
 // ---------------------------------------------------------------------------
 // tensor-core route for 100 % budgets: which queries, their inputs as bf16 rows, their codes
 // ---------------------------------------------------------------------------
+// list[0 .. *count) = the queries whose budget lies in [lo, hi] and is not skipped (any order)
+__global__ void range_compact_kernel(const uint16_t *bp, const uint16_t *skip_bp, uint32_t n, uint32_t lo, uint32_t hi,
+                                     uint32_t *list, uint32_t *count)
+{
+    const uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t lane = threadIdx.x & 31u;
+    bool take = false;
+    if (q < n) {
+        const uint32_t v = bp[q];
+        take = v >= lo && v <= hi && !(skip_bp && v == 10000u);
+    }
+    const uint32_t mask = __ballot_sync(SLONN_FULL_MASK, take);
+    if (mask == 0u) return;
+    uint32_t base = 0;
+    if (lane == (uint32_t)(__ffs(mask) - 1)) base = atomicAdd(count, (uint32_t)__popc(mask));
+    base = __shfl_sync(SLONN_FULL_MASK, base, __ffs(mask) - 1);
+    if (take) list[base + __popc(mask & ((1u << lane) - 1u))] = q;
+}
+
 __global__ void dense_compact_kernel(const uint16_t *bp, uint32_t n, uint32_t *list, uint32_t *count)
 {
     const uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;

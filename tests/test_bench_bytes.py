@@ -26,7 +26,7 @@ def test_budget_nodes_rounds_half_up_with_a_floor_of_one():
 def test_row_and_input_stationary_bytes_of_a_toy_network():
     wl, bp = toy()
     n, esz, H = bp.size, 2, 20
-    rows, cols, layer = bench.gathered_bytes(wl, bp)
+    rows, cols, layer, grouped = bench.gathered_bytes(wl, bp)
     # layer 0: dense input, 20 selected rows of 64 weights
     assert rows == n * 20 * 64 * esz
     # layer 1: fed by layer 0's 20-entry list, own activator: (20 selected + 20 hash nodes) x 20 entries
@@ -38,7 +38,7 @@ def test_row_and_input_stationary_bytes_of_a_toy_network():
 def test_forced_rows_count_whole_rows_everywhere():
     wl, bp = toy("f32")
     n, esz = bp.size, 4
-    rows, cols, layer = bench.gathered_bytes(wl, bp, force_rows=True)
+    rows, cols, layer, grouped = bench.gathered_bytes(wl, bp, force_rows=True)
     assert (cols, layer) == (0, 0)
     assert rows == n * (20 * 64 + 20 * 200 + 10 * 200) * esz
 
@@ -46,7 +46,7 @@ def test_forced_rows_count_whole_rows_everywhere():
 def test_budgets_above_the_split_take_the_row_kernels():
     wl, _ = toy()
     bp = np.array([1000] * 12000 + [5000] * 4000, np.uint16)
-    rows, cols, layer = bench.gathered_bytes(wl, bp)
+    rows, cols, layer, grouped = bench.gathered_bytes(wl, bp)
     esz, H = 2, 20
     low, high = 12000, 4000
     assert layer == low * (20 + H) * 20 * esz
@@ -56,11 +56,20 @@ def test_budgets_above_the_split_take_the_row_kernels():
 
 def test_small_batches_keep_the_row_kernels():
     wl, bp = toy(n=40)      # 40 queries x 20 nodes: far too few warp passes, and the layers are narrow
-    rows, cols, layer = bench.gathered_bytes(wl, bp)
+    rows, cols, layer, grouped = bench.gathered_bytes(wl, bp)
     assert (cols, layer) == (0, 0)
     assert rows == 40 * (20 * 64 + 20 * 200 + 10 * 200) * 2
 
 
 def test_empty_batch_has_no_bytes():
     wl, _ = toy()
-    assert bench.gathered_bytes(wl, np.zeros(0, np.uint16)) == (0, 0, 0)
+    assert bench.gathered_bytes(wl, np.zeros(0, np.uint16)) == (0, 0, 0, 0)
+
+
+def test_row_queries_of_a_layer_without_activator_are_counted_as_grouped():
+    wl = types.SimpleNamespace(dims=[64, 2048, 1024], has_act=[1, 0], dtype="bf16", first_sparse=False, K=10, L=2)
+    bp = np.full(16000, 5000, np.uint16)        # above the split: row kernels; the second layer computes every node
+    rows, cols, layer, grouped = bench.gathered_bytes(wl, bp)
+    assert (cols, layer) == (0, 0)
+    assert rows == 16000 * 1024 * 64 * 2        # first layer: 1024 selected rows of 64 weights
+    assert grouped == 16000 * 1024 * 2048 * 2   # second layer: every row, whole, per query
