@@ -211,7 +211,8 @@ int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint
 #define SLONN_COLS_R 2
 #endif
 // few-queries variants: warps per block, four segments of the input list each (4, 16 and 32 warps measured
-// slower on c4 with 64 queries: 0.237 / 0.248 / 0.372 ms against 0.195 ms for the seven hidden layers)
+// slower on a 4096-wide nine-layer network with 64 queries: 0.237 / 0.248 / 0.372 ms against 0.195 ms for its
+// seven hidden layers)
 #define SLONN_SPLIT_WARPS 8u
 template <bool BF16, int R, bool SPLIT>
 int launch_gather_cols_t(const slonn_gather_params &P, uint64_t grid, uint32_t threads, size_t smem, cudaStream_t st)
@@ -310,7 +311,7 @@ uint32_t cols_budget_limit(const slonn_layer &ly, const slonn_gather_params &P, 
     if (b->flags & SLONN_FLAG_COLUMN_KERNELS) return (uint64_t)n * max_rows > 148ull * 64 ? 10000u : 0u;
     if ((uint64_t)n * max_rows >= 148ull * 1024) return SLONN_COLS_MAX_BP;
     // tens of queries: the one-block-per-64-nodes variant pays only for long weight rows and very sparse lists
-    // (c4, 64 queries: 0.36 -> 0.30 ms per step at 10 %, but 0.57 -> 0.92 ms at 25 %)
+    // (4096-wide nine-layer network, 64 queries: 0.36 -> 0.30 ms per step at 10 %, but 0.57 -> 0.92 ms at 25 %)
     // and only when no query of the batch needs the row kernels (a second launch of idle blocks costs such a batch 6 %)
     return ((uint64_t)n * max_rows > 148ull * 64 && ly.D >= 2048u && max_bp <= 1500u) ? 1500u : 0u;
 }
