@@ -1179,12 +1179,15 @@ extern "C" int slonn_run_host(const slonn_model *m, const slonn_batch *hb, void 
     // Large dense batches go through in pieces on two internal streams, so that the copy of one
     // piece overlaps the kernels of the other.  The per-(query, layer) lists are indexed from the
     // start of the batch, so a caller that wants them back gets the batch in one piece.
-    const uint32_t pieces = 8;
+#ifndef SLONN_PIECE_QUERIES
+#define SLONN_PIECE_QUERIES 2048u // fewest queries per piece
+#endif
+    const uint32_t pieces = std::min(8u, std::max(1u, n / SLONN_PIECE_QUERIES));
     const bool wants_lists = hb->active_indptr || hb->active_ids || hb->active_vals;
     uint32_t piece = (n + pieces - 1) / pieces;
     piece = (piece + 255u) / 256u * 256u;
     const uint64_t half = ((ws_bytes - 256) / 2) & ~(uint64_t)255; // two piece areas, then the pieces' status words
-    bool piecewise = !m->first_sparse && !wants_lists && n >= 8192 && !(hb->flags & SLONN_FLAG_DENSE_TC);
+    bool piecewise = !m->first_sparse && !wants_lists && pieces >= 2 && !(hb->flags & SLONN_FLAG_DENSE_TC);
     if (piecewise && carve_host(m, piece, max_bp, hb->flags, 0).total > half) piecewise = false;
 
     if (!piecewise) {
@@ -1194,7 +1197,7 @@ extern "C" int slonn_run_host(const slonn_model *m, const slonn_batch *hb, void 
     } else {
         cudaStream_t s2[2] = {nullptr, nullptr};
         cudaEvent_t ev_start = nullptr, ev_done[2] = {nullptr, nullptr};
-        uint32_t status[pieces + 1][4];
+        uint32_t status[9][4]; // at most 8 pieces
         memset(status, 0, sizeof(status));
         int rc = SLONN_OK;
         bool ok = cudaStreamCreateWithFlags(&s2[0], cudaStreamNonBlocking) == cudaSuccess &&
