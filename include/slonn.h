@@ -336,6 +336,17 @@ int slonn_dense_layer(const void *x_bf16, const void *w_bf16, const float *bias,
                       uint32_t *status, void *stream);
 
 /*
+ * Testing aid for the give-up path of the tensor-core kernel (no passage of the paper: the library's own
+ * failure reporting).  Every on-chip wait of that kernel is bounded; when one runs out the block stops issuing
+ * work, lets copies in flight land, frees its tensor memory and writes -SLONN_ERR_TIMEOUT to status[0].  With
+ * polls != 0 every later slonn_dense_layer / SLONN_FLAG_DENSE_TC launch of this process makes its loader wait,
+ * for at most `polls` polls, on a barrier that nothing signals -- before it has issued any copy or product -- so
+ * the launch ends through that path and computes nothing.  0 restores normal operation.  Process-wide; not for
+ * production use.
+ */
+int slonn_test_tc_wait_limit(uint32_t polls);
+
+/*
  * slonn_run without a caller-provided workspace.  (The paper has no counterpart;
  * this exists for deployment.)
  *
@@ -392,6 +403,29 @@ int slonn_run_static(const slonn_model *m, const slonn_batch *batch, void *strea
 int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *workspace,
                     uint64_t workspace_bytes, void *stream, float *stage_ms,
                     uint32_t *stage_launches);
+
+/*
+ * The same measurement launch by launch: which stage, which layer, which queries (by budget range) and, for
+ * the whole-network kernels, which form the list-fed layers took -- enough for a caller that knows the
+ * budgets to count the weight bytes each launch had to touch (Sec. 3.3: hashed rows, bucket lists, selected
+ * nodes times input entries) without repeating the library's kernel choice.  `records` is a HOST array of
+ * `capacity` entries (SLONN_MAX_RECORDS always suffices); *n_records (host) receives how many were written,
+ * in launch order.  Synchronises `stream`; creates and destroys events.
+ */
+#define SLONN_ALL_LAYERS 0xffffffffu
+#define SLONN_MAX_RECORDS (10 * SLONN_MAX_LAYERS)
+typedef struct {
+    uint32_t stage;      /* SLONN_STAGE_*                                                             */
+    uint32_t layer;      /* the layer the launch works on, or SLONN_ALL_LAYERS                        */
+    uint32_t bp_lo, bp_hi; /* it serves the queries whose budget lies in [bp_lo, bp_hi] ...           */
+    uint32_t skips_full; /* ... 1: except those at 10000 bp, which another launch serves              */
+    uint32_t cols_bp;    /* whole-network launches: queries with budgets up to this evaluated their   */
+                         /* list-fed activator layers input-stationary (0 = every layer row-wise)     */
+    float ms;            /* device time between the event pair around the launch                      */
+} slonn_launch_record;
+int slonn_run_traced(const slonn_model *m, const slonn_batch *batch, void *workspace,
+                     uint64_t workspace_bytes, void *stream, slonn_launch_record *records,
+                     uint32_t capacity, uint32_t *n_records);
 
 /*
  * Same computation for callers that keep queries and results in HOST memory:

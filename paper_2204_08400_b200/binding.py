@@ -23,7 +23,7 @@ EXPORTS = [
     "slonn_run_timed", "slonn_run_static", "slonn_dense_layer", "slonn_serialized_bytes", "slonn_serialize",
     "slonn_deserialize", "slonn_lcao_budgets", "slonn_confidence_build", "slonn_confidence_to_host",
     "slonn_confidence_free", "slonn_aclo_budgets",
-    "slonn_host_workspace_bytes", "slonn_run_host",
+    "slonn_host_workspace_bytes", "slonn_run_host", "slonn_test_tc_wait_limit", "slonn_run_traced",
 ]
 
 
@@ -43,6 +43,11 @@ class _BuildDesc(C.Structure):
 class _Rows(C.Structure):
     _fields_ = [("n_rows", C.c_uint32), ("dense", C.c_void_p), ("indptr", C.c_void_p),
                 ("ids", C.c_void_p), ("vals", C.c_void_p)]
+
+
+class _LaunchRecord(C.Structure):
+    _fields_ = [("stage", C.c_uint32), ("layer", C.c_uint32), ("bp_lo", C.c_uint32), ("bp_hi", C.c_uint32),
+                ("skips_full", C.c_uint32), ("cols_bp", C.c_uint32), ("ms", C.c_float)]
 
 
 class _Batch(C.Structure):
@@ -110,9 +115,14 @@ def lib():
         L.slonn_dense_layer.restype = C.c_int
         L.slonn_dense_layer.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32,
                                         C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.slonn_test_tc_wait_limit.restype = C.c_int
+        L.slonn_test_tc_wait_limit.argtypes = [C.c_uint32]
         L.slonn_run_timed.restype = C.c_int
         L.slonn_run_timed.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p,
                                       C.c_void_p, C.c_void_p]
+        L.slonn_run_traced.restype = C.c_int
+        L.slonn_run_traced.argtypes = [C.c_void_p, C.POINTER(_Batch), C.c_void_p, C.c_uint64, C.c_void_p,
+                                       C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
         L.slonn_host_workspace_bytes.restype = C.c_int
         L.slonn_host_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64,
                                                  C.POINTER(C.c_uint64)]
@@ -410,6 +420,14 @@ def slonn_dense_layer(x_bf16, w_bf16, bias, M: int, N: int, D: int, relu: bool, 
         raise SlonnError(rc, "slonn_dense_layer")
 
 
+def slonn_test_tc_wait_limit(polls: int) -> None:
+    """Testing aid: polls != 0 makes later tensor-core launches give up on their first wait after that many
+    polls (status[0] = 8, nothing computed); 0 restores normal operation."""
+    rc = lib().slonn_test_tc_wait_limit(int(polls))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_test_tc_wait_limit")
+
+
 STATIC_WORKSPACE_BYTES = 16 << 20
 
 
@@ -441,6 +459,24 @@ def slonn_run_timed(model: Model, batch: _Batch, workspace, workspace_bytes: int
     if rc != SLONN_OK:
         raise SlonnError(rc, "slonn_run_timed")
     return dict(zip(STAGES, ms.tolist())), dict(zip(STAGES, cnt.tolist()))
+
+
+ALL_LAYERS = 0xFFFFFFFF
+MAX_RECORDS = 160
+
+
+def slonn_run_traced(model: Model, batch: _Batch, workspace, workspace_bytes: int, stream=None) -> List[dict]:
+    """One run with an event pair around every launch; returns the launch records in order, each a dict
+    with stage (name), layer (None = every layer), bp_lo, bp_hi, skips_full, cols_bp, ms."""
+    rec = (_LaunchRecord * MAX_RECORDS)()
+    n = C.c_uint32()
+    rc = lib().slonn_run_traced(model.handle, C.byref(batch), _ptr(workspace), workspace_bytes,
+                                _stream_ptr(stream), C.addressof(rec), MAX_RECORDS, C.byref(n))
+    if rc != SLONN_OK:
+        raise SlonnError(rc, "slonn_run_traced")
+    return [dict(stage=STAGES[r.stage], layer=None if r.layer == ALL_LAYERS else int(r.layer), bp_lo=int(r.bp_lo),
+                 bp_hi=int(r.bp_hi), skips_full=bool(r.skips_full), cols_bp=int(r.cols_bp), ms=float(r.ms))
+            for r in rec[: n.value]]
 
 
 def slonn_run_host(model: Model, host_batch: _Batch, workspace, workspace_bytes: int, stream=None):

@@ -15,6 +15,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <numeric>
 #include <vector>
 
 #include "slonn_common.cuh"
@@ -371,60 +372,51 @@ __global__ void fill_tables_kernel(const uint32_t *sorted /* [segs][N] */, const
 }
 
 // ---------------------------------------------------------------------------
-// host: hash-node sampling.  SplitMix64 stream; each draw takes one node from the
-// not-yet-drawn ones with probability proportional to its variance (inverse CDF in id
-// order); once no positive variance is left the draw is uniform over what remains.
+// host: hash-node sampling (Sec. 3.4: probability proportional to activation variance).
+// The not-yet-drawn nodes are kept as a dense array in id order together with the running
+// sums of their variances; a draw is a search in those running sums and removes its node.
+// The running sums are rebuilt front to back after every removal, so a draw sees exactly
+// the left-to-right fp64 sums of the remaining variances.  Uniform numbers come from a
+// SplitMix64 stream (53 bits each).  When the remaining variances sum to zero the draw is
+// uniform over the remaining nodes.
 // ---------------------------------------------------------------------------
-struct sm64 {
-    uint64_t s;
-    uint64_t next()
+class splitmix_stream {
+public:
+    explicit splitmix_stream(uint64_t seed) : state_(seed) {}
+    double uniform53()
     {
-        s += 0x9E3779B97F4A7C15ull;
-        uint64_t z = s;
-        z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
-        z ^= z >> 27; z *= 0x94D049BB133111EBull;
-        z ^= z >> 31;
-        return z;
+        uint64_t z = (state_ += 0x9E3779B97F4A7C15ull);
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+        return (double)((z ^ (z >> 31)) >> 11) * 0x1.0p-53;
     }
-    double unit() { return (double)(next() >> 11) * 0x1.0p-53; }
+private:
+    uint64_t state_;
 };
 
 void sample_hash_nodes(const std::vector<double> &var, uint32_t H, uint64_t seed, uint32_t layer, uint32_t *out)
 {
-    const uint32_t N = (uint32_t)var.size();
-    std::vector<char> used(N, 0);
-    sm64 rng{seed ^ (0xD6E8FEB86659FD93ull * (uint64_t)(layer + 1))};
+    std::vector<uint32_t> pool(var.size()); // ids still available, ascending
+    std::iota(pool.begin(), pool.end(), 0u);
+    std::vector<double> running(var.size()); // running[k] = var[pool[0]] + ... + var[pool[k]]
+    splitmix_stream rng(seed ^ (0xD6E8FEB86659FD93ull * (uint64_t)(layer + 1)));
     for (uint32_t d = 0; d < H; ++d) {
-        const double u = rng.unit();
-        double mass = 0.0;
-        uint32_t left = 0;
-        for (uint32_t i = 0; i < N; ++i) {
-            if (used[i]) continue;
-            mass += var[i];
-            ++left;
-        }
-        uint32_t chosen = N;
-        if (mass > 0.0) {
-            const double target = u * mass;
-            double cum = 0.0;
-            uint32_t last_positive = N;
-            for (uint32_t i = 0; i < N && chosen == N; ++i) {
-                if (used[i] || !(var[i] > 0.0)) continue;
-                cum += var[i];
-                last_positive = i;
-                if (cum > target) chosen = i;
-            }
-            if (chosen == N) chosen = last_positive;
+        const double u = rng.uniform53();
+        double s = 0.0;
+        for (size_t k = 0; k < pool.size(); ++k) running[k] = (s += var[pool[k]]);
+        const auto first = running.begin(), last = running.begin() + pool.size();
+        size_t k;
+        if (s > 0.0) {
+            // first node whose running sum exceeds u * total (its own variance is then positive); if rounding
+            // leaves none, the last node with a positive variance
+            k = (size_t)(std::upper_bound(first, last, u * s) - first);
+            if (k == pool.size())
+                do { --k; } while (k > 0 && !(var[pool[k]] > 0.0));
         } else {
-            uint32_t skip = (uint32_t)(u * (double)left);
-            if (skip >= left) skip = left - 1;
-            for (uint32_t i = 0; i < N; ++i) {
-                if (used[i]) continue;
-                if (skip-- == 0) { chosen = i; break; }
-            }
+            k = std::min((size_t)(u * (double)pool.size()), pool.size() - 1);
         }
-        used[chosen] = 1;
-        out[d] = chosen;
+        out[d] = pool[k];
+        pool.erase(pool.begin() + (std::ptrdiff_t)k);
     }
 }
 

@@ -128,7 +128,9 @@ cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
             else dst[i] = v;
         }
     }
-    __syncthreads();
+    // every block of the cluster must be running before a peer's shared memory is written (the hash sums of
+    // the first layer are the first such stores); this also orders the staging above within the block
+    cluster.sync();
 
     for (uint32_t l = 0; l < P.n_layers; ++l) {
         const slonn_cluster_layer &ly = P.layer[l];

@@ -21,6 +21,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstring>
 #include <mutex>
 
@@ -76,9 +77,10 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 // Bounded wait; false when it gave up or another role already raised the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          uint32_t limit = WAIT_LIMIT)
 {
-    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
@@ -161,8 +163,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 __global__ void __launch_bounds__(THREADS, 1)
 dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_out, uint32_t tma_out, const slonn_dense_epilogue E, uint32_t N,
-                uint32_t K, uint32_t bn)
+                uint32_t K, uint32_t bn, uint32_t probe_limit)
 {
+    // probe_limit: 0 in normal use.  Otherwise (a test of the give-up path) the producer first waits, for at most
+    // that many polls, on a barrier nobody arrives at -- before any copy or MMA has been issued.
     // map_out / tma_out: the bf16 output matrix as a tensor of 64-column x 32-row boxes (128-byte swizzle),
     // valid when tma_out != 0
     // bn: columns per tile, a multiple of 16 up to BN (narrow layers take a narrower MMA and B tile)
@@ -180,6 +184,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const uint32_t full0 = bars, empty0 = bars + 8 * STAGES;
     const uint32_t tfull0 = bars + 16 * STAGES, tempty0 = tfull0 + 16;
     const uint32_t tmem_slot_addr = tempty0 + 16;
+    const uint32_t probe_bar = tempty0 + 32;
     const uint32_t epi_addr = bars + 256;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot_addr - smem_u32(smem_raw)));
     volatile uint32_t *abort_flag = tmem_slot + 1;
@@ -187,6 +192,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, EPI_WARPS); }
+        mbar_init(probe_bar, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -205,6 +211,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
+            if (probe_limit) ok = mbar_wait(probe_bar, 0u, abort_flag, probe_limit); // never completes: runs out
             for (uint32_t t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
                 const uint32_t m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * bn;
                 for (uint32_t kb = 0; kb < num_kb; ++kb, ++it) {
@@ -449,7 +456,19 @@ int make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols, ui
     return r == CUDA_SUCCESS ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
+constexpr int MAX_DEVICES = 64;
+std::mutex g_dev_mu;
+bool g_attr_set[MAX_DEVICES];
+int g_sm_count[MAX_DEVICES];
+std::atomic<uint32_t> g_probe_limit{0}; // slonn_test_tc_wait_limit
+
 } // namespace
+
+extern "C" int slonn_test_tc_wait_limit(uint32_t polls)
+{
+    g_probe_limit.store(polls);
+    return SLONN_OK;
+}
 
 int slonn_dense_tc_launch(const void *A, const void *W, uint32_t N, uint32_t K, const slonn_dense_epilogue &E,
                           cudaStream_t st)
@@ -460,18 +479,23 @@ int slonn_dense_tc_launch(const void *A, const void *W, uint32_t N, uint32_t K, 
     if ((rc = make_map(&ma, A, E.M, K, BM))) return rc;
     const uint32_t bn = std::min<uint32_t>((uint32_t)BN, (N + 15u) / 16u * 16u);
     if ((rc = make_map(&mb, W, N, K, bn))) return rc;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(dense_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
-            return SLONN_ERR_CUDA;
-        attr_set = true;
-    }
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 1)
-            return SLONN_ERR_CUDA;
+    // the shared-memory opt-in and the SM count belong to a device: looked up once per device ordinal
+    int dev = 0, sm_count = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SLONN_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> lock(g_dev_mu);
+        const bool cached = dev >= 0 && dev < MAX_DEVICES;
+        if (!cached || !g_attr_set[dev]) {
+            if (cudaFuncSetAttribute(dense_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
+                return SLONN_ERR_CUDA;
+            if (cached) g_attr_set[dev] = true;
+        }
+        sm_count = cached ? g_sm_count[dev] : 0;
+        if (sm_count == 0) {
+            if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 1)
+                return SLONN_ERR_CUDA;
+            if (cached) g_sm_count[dev] = sm_count;
+        }
     }
     // bf16 outputs leave through a TMA store when nothing needs per-row list addressing
     CUtensorMap mo;
@@ -484,7 +508,7 @@ int slonn_dense_tc_launch(const void *A, const void *W, uint32_t N, uint32_t K, 
     }
     const uint64_t tiles = (uint64_t)((N + bn - 1) / bn) * ((E.M + BM - 1) / BM);
     const uint32_t grid = (uint32_t)std::min<uint64_t>(tiles, (uint64_t)sm_count); // one persistent block per SM
-    dense_tc_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, mo, tma_out, E, N, K, bn);
+    dense_tc_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, mo, tma_out, E, N, K, bn, g_probe_limit.load());
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 

@@ -12,26 +12,31 @@
 
 namespace {
 
-// Optional per-stage timing: an event pair around every launch of a stage.
+// Optional per-launch timing: an event pair around every launch, with what the launch covers.
 struct stage_timer {
-    struct span { int stage; cudaEvent_t a, b; };
-    span spans[8 * SLONN_MAX_LAYERS];
+    struct span { int stage; uint32_t layer, bp_lo, bp_hi, skips_full, cols_bp; cudaEvent_t a, b; };
+    span spans[10 * SLONN_MAX_LAYERS];
     int n = 0;
     bool failed = false;
     cudaStream_t st = nullptr;
-    void tic(int stage)
+    uint32_t layer = SLONN_ALL_LAYERS; // layer the next launches work on
+    void tic(int stage, const uint16_t *range_bp = nullptr, uint32_t lo = 0, uint32_t hi = 0xffffu, const uint16_t *skip_bp = nullptr,
+             uint32_t cols_bp = 0)
     {
         if (n >= (int)(sizeof(spans) / sizeof(spans[0]))) { failed = true; return; }
         span &s = spans[n];
-        s.stage = stage;
+        s.stage = stage; s.layer = layer;
+        s.bp_lo = range_bp ? lo : 0u; s.bp_hi = range_bp ? std::min(hi, 10000u) : 10000u;
+        s.skips_full = skip_bp ? 1u : 0u; s.cols_bp = cols_bp;
         if (cudaEventCreate(&s.a) != cudaSuccess || cudaEventCreate(&s.b) != cudaSuccess) { failed = true; return; }
         cudaEventRecord(s.a, st);
         ++n;
     }
     void toc() { if (n > 0 && !failed) cudaEventRecord(spans[n - 1].b, st); }
 };
-#define TIC(stage) do { if (tm) tm->tic(stage); } while (0)
+#define TIC(...) do { if (tm) tm->tic(__VA_ARGS__); } while (0)
 #define TOC() do { if (tm) tm->toc(); } while (0)
+#define AT_LAYER(l) do { if (tm) tm->layer = (l); } while (0)
 
 inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
@@ -335,7 +340,7 @@ int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_
         const uint32_t pre = slonn_model_pre(m);
         const uint32_t cols_rows = (both && P.use_list) ? std::min(max_rows, slonn_layer_nodes(cols_bp, ly.N, pre)) : max_rows;
         C.in_cap = both ? std::min(in_cap, slonn_layer_nodes(cols_bp, ly.D, pre)) : in_cap;
-        TIC(SLONN_STAGE_GATHER_COLS);
+        TIC(SLONN_STAGE_GATHER_COLS, C.range_bp, C.bp_lo, C.bp_hi, C.skip_bp);
         rc = launch_gather_cols(m, C, n, cols_rows, st);
         TOC();
         if (rc != SLONN_ERR_DIM) { // SLONN_ERR_DIM: the staging does not fit shared memory, rows for everyone
@@ -345,7 +350,7 @@ int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_
             P.range_bp = b->budget_bp; P.bp_lo = 0; P.bp_hi = cols_bp;
         }
     }
-    TIC(SLONN_STAGE_GATHER_DOT);
+    TIC(SLONN_STAGE_GATHER_DOT, P.range_bp, P.bp_lo, P.bp_hi, P.skip_bp);
     rc = launch_gather(m, P, n, max_rows, st);
     TOC();
     return rc;
@@ -369,25 +374,25 @@ int launch_act_layer(const slonn_model *m, const slonn_layer &ly, uint32_t l, sl
         if (both) { C.range_bp = b->budget_bp; C.bp_lo = 0; C.bp_hi = cols_bp; }
         const uint32_t cols_rows = both ? std::min(max_rows, slonn_layer_nodes(cols_bp, ly.N, pre)) : max_rows;
         C.in_cap = both ? std::min(in_cap, slonn_layer_nodes(cols_bp, ly.D, pre)) : in_cap;
-        TIC(SLONN_STAGE_LAYER_COLS);
+        TIC(SLONN_STAGE_LAYER_COLS, C.range_bp, C.bp_lo, C.bp_hi, C.skip_bp);
         rc = launch_layer_cols(m, ly, l, C, b, n, cols_rows, st);
         TOC();
         if (rc == SLONN_OK) {
             if (!both) return SLONN_OK;
             sp.range_bp = b->budget_bp; sp.bp_lo = cols_bp + 1; sp.bp_hi = 0xffffu;
-            TIC(SLONN_STAGE_HASH_SELECT);
+            TIC(SLONN_STAGE_HASH_SELECT, sp.range_bp, sp.bp_lo, sp.bp_hi, sp.skip_bp);
             rc = launch_select(m, sp, n, max_rows, st);
             TOC();
             if (rc) return rc;
             gp.range_bp = b->budget_bp; gp.bp_lo = cols_bp + 1; gp.bp_hi = 0xffffu;
-            TIC(SLONN_STAGE_GATHER_DOT);
+            TIC(SLONN_STAGE_GATHER_DOT, gp.range_bp, gp.bp_lo, gp.bp_hi, gp.skip_bp);
             rc = launch_gather(m, gp, n, max_rows, st);
             TOC();
             return rc;
         }
         if (rc != SLONN_ERR_DIM) return rc;
     }
-    TIC(SLONN_STAGE_HASH_SELECT);
+    TIC(SLONN_STAGE_HASH_SELECT, sp.range_bp, sp.bp_lo, sp.bp_hi, sp.skip_bp);
     rc = launch_select(m, sp, n, max_rows, st);
     TOC();
     if (rc) return rc;
@@ -464,7 +469,7 @@ int launch_fused_t(const slonn_fused_params &P, cudaStream_t st)
 }
 
 int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *indptr, uint32_t stride,
-                 const uint16_t *skip_bp, uint32_t max_bp, cudaStream_t st)
+                 const uint16_t *skip_bp, uint32_t max_bp, cudaStream_t st, uint32_t *cols_bp_out)
 {
     slonn_fused_params P;
     memset(&P, 0, sizeof(P));
@@ -500,6 +505,7 @@ int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *ind
     P.status = b->status;
     P.xbuf_floats = xbuf; P.ids_cap = ids_cap; P.bitmap_words = words;
     P.cols_bp = ent_cap ? cols_bp : 0u; P.ent_cap = ent_cap; P.budget_bp = b->budget_bp;
+    *cols_bp_out = P.cols_bp;
     P.warp_bytes = (uint32_t)align_up(align_up((uint64_t)xbuf * 4 + (uint64_t)ids_cap * 2 + (uint64_t)words * 4, 16) +
                                           (ent_cap ? (uint64_t)ent_cap * 8 + 66 * 4 : 0), 16);
     const bool bf = m->dtype == SLONN_BF16;
@@ -684,7 +690,8 @@ static int run_full_route(const slonn_model *m, const slonn_batch *b, uint32_t n
             fp.out_dense = is_last ? b->logits : dense[dense_cur];
             fp.out_stride = ly.N;
         }
-        TIC(SLONN_STAGE_FULL_ROWS);
+        AT_LAYER(l);
+        TIC(SLONN_STAGE_FULL_ROWS, b->budget_bp, 10000u, 10000u);
         const int rc = launch_full_rows(m, fp, n, st);
         TOC();
         if (rc) return rc;
@@ -749,6 +756,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     if (b->kernel_path == SLONN_PATH_CLUSTER && (!cluster_eligible(m) || tc_route(m, max_bp, b->flags))) return SLONN_ERR_DIM;
     if (b->kernel_path == SLONN_PATH_CLUSTER || (b->kernel_path == SLONN_PATH_AUTO && cluster_eligible(m) && n <= 4 && !tc_route(m, max_bp, b->flags) &&
          cluster_max_rows(m, max_bp) <= 1024)) {
+        AT_LAYER(SLONN_ALL_LAYERS);
         TIC(SLONN_STAGE_CLUSTER);
         const int rc = launch_cluster(m, b, max_bp, stride, st);
         TOC();
@@ -779,6 +787,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         pp.indptr = indptr; pp.status = b->status;
         const uint64_t tiles = ((uint64_t)n * m->n_act + SLONN_PLAN_TILE - 1) / SLONN_PLAN_TILE;
         uint64_t *tile_sums = (uint64_t *)(ws + wl.plan_sums);
+        AT_LAYER(SLONN_ALL_LAYERS);
         TIC(SLONN_STAGE_PLAN);
         plan_partial_kernel<<<(uint32_t)tiles, SLONN_PLAN_THREADS, 0, st>>>(pp, tile_sums);
         plan_final_kernel<<<(uint32_t)tiles, SLONN_PLAN_THREADS, 0, st>>>(pp, tile_sums);
@@ -792,7 +801,8 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     if (tc_route(m, max_bp, b->flags)) {
         uint32_t *tc_list = (uint32_t *)(ws + wl.tc_list), *tc_count = (uint32_t *)(ws + wl.tc_count);
         uint16_t *A[2] = {(uint16_t *)(ws + wl.tc_a0), (uint16_t *)(ws + wl.tc_a1)};
-        TIC(SLONN_STAGE_DENSE_TC);
+        AT_LAYER(SLONN_ALL_LAYERS);
+        TIC(SLONN_STAGE_DENSE_TC, b->budget_bp, 10000u, 10000u);
         int rc = SLONN_OK;
         if (cudaMemsetAsync(tc_count, 0, sizeof(uint32_t), st) != cudaSuccess) rc = SLONN_ERR_CUDA;
         if (!rc) {
@@ -845,15 +855,25 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     }
 
     if (use_fused) {
-        TIC(SLONN_STAGE_FUSED);
-        const int rc = launch_fused(m, b, no_plan ? nullptr : indptr, stride, skip_bp, max_bp, st);
+        AT_LAYER(SLONN_ALL_LAYERS);
+        uint32_t fused_cols_bp = 0;
+        TIC(SLONN_STAGE_FUSED, nullptr, 0u, 0xffffu, skip_bp);
+        const int rc = launch_fused(m, b, no_plan ? nullptr : indptr, stride, skip_bp, max_bp, st, &fused_cols_bp);
+        if (tm && tm->n > 0) tm->spans[tm->n - 1].cols_bp = fused_cols_bp;
         TOC();
         if (rc || !skip_bp || !b->pred) return rc;
-        // predictions of the tensor-core queries (the fused kernel wrote the others; same rule)
+        // predictions of the 100 % queries that another route served (the fused kernel wrote the others and
+        // theirs must stay; same rule)
         slonn_argmax_params ap;
         memset(&ap, 0, sizeof(ap));
-        ap.logits = b->logits; ap.stride = stride; ap.n = n; ap.pred = b->pred; ap.fixed_len = last.N;
-        TIC(SLONN_STAGE_ARGMAX);
+        ap.logits = b->logits; ap.stride = stride; ap.n = n; ap.pred = b->pred; ap.only_full = skip_bp;
+        if (last.has_act) {
+            ap.logit_ids = b->logit_ids; ap.indptr = indptr; ap.n_act = m->n_act;
+            ap.a = m->act_index[m->n_layers - 1];
+        } else {
+            ap.fixed_len = last.N;
+        }
+        TIC(SLONN_STAGE_ARGMAX, b->budget_bp, 10000u, 10000u);
         if (stride >= 2048) argmax_block_kernel<<<n, 256, 0, st>>>(ap);
         else argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
         TOC();
@@ -874,6 +894,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         const uint32_t esz = m->dtype == SLONN_BF16 ? 2u : 4u;
         const uint32_t nchunks = ly.D * esz / 16u;
         int rc;
+        AT_LAYER(l);
         if (l == 0 && m->first_sparse) {
             float *o = is_last ? b->logits : dense[dense_cur];
             TIC(SLONN_STAGE_SPARSE_FIRST);
@@ -931,7 +952,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
                 fp.list = glist; fp.count = gcount; fp.in = in;
                 fp.W = ly.W; fp.bias = ly.bias; fp.D = ly.D; fp.N = ly.N; fp.nchunks = nchunks;
                 fp.has_act = 0; fp.out_dense = gp.out_dense; fp.out_stride = ly.N; fp.relu = gp.relu;
-                TIC(SLONN_STAGE_FULL_ROWS);
+                TIC(SLONN_STAGE_FULL_ROWS, b->budget_bp, cols_bp ? cols_bp + 1 : 0u, 0xffffu, skip_bp);
                 rc = launch_full_rows(m, fp, n, st);
                 TOC();
                 if (rc) return rc;
@@ -954,6 +975,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         } else {
             ap.fixed_len = last.N;
         }
+        AT_LAYER(SLONN_ALL_LAYERS);
         TIC(SLONN_STAGE_ARGMAX);
         if (stride >= 2048) argmax_block_kernel<<<n, 256, 0, st>>>(ap);
         else argmax_kernel<<<(n + 7) / 8, 256, 0, st>>>(ap);
@@ -969,26 +991,57 @@ extern "C" int slonn_run(const slonn_model *m, const slonn_batch *b, void *works
     return run_impl(m, b, workspace, ws_bytes, stream, nullptr);
 }
 
-extern "C" int slonn_run_timed(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes,
-                               void *stream, float *stage_ms, uint32_t *stage_launches)
+static int run_with_timer(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes, void *stream,
+                          stage_timer &tm, float *span_ms)
 {
-    if (!stage_ms || !stage_launches) return SLONN_ERR_ARG;
-    stage_timer tm;
     tm.st = (cudaStream_t)stream;
     int rc = run_impl(m, b, workspace, ws_bytes, stream, &tm);
     if (cudaStreamSynchronize(tm.st) != cudaSuccess && rc == SLONN_OK) rc = SLONN_ERR_CUDA;
-    for (int s = 0; s < SLONN_N_STAGES; ++s) { stage_ms[s] = 0.0f; stage_launches[s] = 0; }
     for (int i = 0; i < tm.n; ++i) {
         float ms = 0.0f;
-        if (rc == SLONN_OK && !tm.failed && cudaEventElapsedTime(&ms, tm.spans[i].a, tm.spans[i].b) == cudaSuccess) {
-            stage_ms[tm.spans[i].stage] += ms;
-            stage_launches[tm.spans[i].stage] += 1;
-        }
+        if (rc == SLONN_OK && !tm.failed && cudaEventElapsedTime(&ms, tm.spans[i].a, tm.spans[i].b) != cudaSuccess) rc = SLONN_ERR_CUDA;
+        span_ms[i] = ms;
         cudaEventDestroy(tm.spans[i].a);
         cudaEventDestroy(tm.spans[i].b);
     }
     if (tm.failed && rc == SLONN_OK) rc = SLONN_ERR_CUDA;
     return rc;
+}
+
+extern "C" int slonn_run_timed(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes,
+                               void *stream, float *stage_ms, uint32_t *stage_launches)
+{
+    if (!stage_ms || !stage_launches) return SLONN_ERR_ARG;
+    stage_timer tm;
+    float ms[sizeof(tm.spans) / sizeof(tm.spans[0])];
+    const int rc = run_with_timer(m, b, workspace, ws_bytes, stream, tm, ms);
+    for (int s = 0; s < SLONN_N_STAGES; ++s) { stage_ms[s] = 0.0f; stage_launches[s] = 0; }
+    if (rc == SLONN_OK)
+        for (int i = 0; i < tm.n; ++i) {
+            stage_ms[tm.spans[i].stage] += ms[i];
+            stage_launches[tm.spans[i].stage] += 1;
+        }
+    return rc;
+}
+
+extern "C" int slonn_run_traced(const slonn_model *m, const slonn_batch *b, void *workspace, uint64_t ws_bytes,
+                                void *stream, slonn_launch_record *records, uint32_t capacity, uint32_t *n_records)
+{
+    if (!records || !n_records) return SLONN_ERR_ARG;
+    stage_timer tm;
+    float ms[sizeof(tm.spans) / sizeof(tm.spans[0])];
+    const int rc = run_with_timer(m, b, workspace, ws_bytes, stream, tm, ms);
+    *n_records = 0;
+    if (rc != SLONN_OK) return rc;
+    if ((uint32_t)tm.n > capacity) return SLONN_ERR_ARG;
+    for (int i = 0; i < tm.n; ++i) {
+        const stage_timer::span &s = tm.spans[i];
+        slonn_launch_record &r = records[i];
+        r.stage = (uint32_t)s.stage; r.layer = s.layer; r.bp_lo = s.bp_lo; r.bp_hi = s.bp_hi;
+        r.skips_full = s.skips_full; r.cols_bp = s.cols_bp; r.ms = ms[i];
+    }
+    *n_records = (uint32_t)tm.n;
+    return SLONN_OK;
 }
 
 // ---- run on the library's own fixed scratch area --------------------------------

@@ -1048,6 +1048,7 @@ struct slonn_argmax_params {
     const uint64_t *indptr;    // budgeted last layer: length of (q, a)
     uint32_t n_act, a;
     uint32_t *pred;
+    const uint16_t *only_full; // nullable: only queries whose budget is 10000 bp (the others were served elsewhere)
 };
 
 __global__ void __launch_bounds__(256) argmax_kernel(slonn_argmax_params P)
@@ -1055,6 +1056,7 @@ __global__ void __launch_bounds__(256) argmax_kernel(slonn_argmax_params P)
     const uint32_t q = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const uint32_t lane = threadIdx.x & 31u;
     if (q >= P.n) return;
+    if (P.only_full && P.only_full[q] != 10000u) return;
     uint32_t len = P.fixed_len;
     if (P.indptr)
         len = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - P.indptr[(uint64_t)q * P.n_act + P.a]);
@@ -1086,6 +1088,7 @@ __global__ void __launch_bounds__(256) argmax_block_kernel(slonn_argmax_params P
     __shared__ uint32_t wbi[8];
     const uint32_t q = blockIdx.x;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    if (P.only_full && P.only_full[q] != 10000u) return; // uniform for the block
     uint32_t len = P.fixed_len;
     if (P.indptr)
         len = (uint32_t)(P.indptr[(uint64_t)q * P.n_act + P.a + 1] - P.indptr[(uint64_t)q * P.n_act + P.a]);

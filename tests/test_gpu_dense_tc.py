@@ -103,3 +103,33 @@ def test_full_budget_queries_on_tensor_cores_narrow(kernel_path):
 def test_full_budget_queries_on_tensor_cores_wide():
     wl = wl_mod.load("c5", n_queries=300, n_cal=256, dims=[2048, 4096, 4096, 1000])
     check_tc_route(wl, 0)
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    # one-tile problem; the loader's first wait is on a barrier nothing signals and gives up after a few hundred
+    # polls, before any copy or product was issued: the launch must end by itself, report SLONN_ERR_TIMEOUT in
+    # status[0], leave the output untouched, and the next launch (hook cleared) must compute as usual
+    import torch
+    from paper_2204_08400_b200 import binding as sl, harness
+    dev = torch.device("cuda:0")
+    M = N = 128
+    D = 64
+    rng = np.random.default_rng(7)
+    xb = wl_mod.f32_to_bf16_bits(rng.standard_normal((M, D), dtype=np.float32))
+    wb = wl_mod.f32_to_bf16_bits(rng.standard_normal((N, D), dtype=np.float32))
+    dx, dw = harness._dev(xb, dev), harness._dev(wb, dev)
+    out = torch.full((M, N), -7.0, dtype=torch.float32, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    sl.slonn_test_tc_wait_limit(300)
+    try:
+        sl.slonn_dense_layer(dx, dw, None, M, N, D, False, out_f32=out, status=status)
+        torch.cuda.synchronize()
+    finally:
+        sl.slonn_test_tc_wait_limit(0)
+    assert int(status[0]) == -sl.ERR["TIMEOUT"]
+    assert bool((out == -7.0).all())
+    sl.slonn_dense_layer(dx, dw, None, M, N, D, False, out_f32=out, status=status)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    want = wl_mod.bf16_bits_to_f32(xb).astype(np.float64) @ wl_mod.bf16_bits_to_f32(wb).astype(np.float64).T
+    assert np.max(np.abs(out.cpu().numpy() - want)) < 1e-4 * np.max(np.abs(want))

@@ -31,12 +31,17 @@ def kernel_paths(wl):
     return (1,) + ((2,) if fused_ok else ()) + ((3,) if cluster_ok else ())
 
 
-def check(wl, n_cal=None, sample=None, expect_build=True):
+def check(wl, n_cal=None, sample=None, expect_build=True, models=None):
+    """models: a (device model, oracle model) pair built earlier from the same weights and calibration rows
+    (the tables do not depend on the budgets); it is then neither compared again nor freed here."""
     from paper_2204_08400_b200 import binding as sl, harness
-    dm = harness.DeviceModel(wl, n_cal=n_cal)
-    om = oracle_model(wl, n_cal=n_cal)
-    if expect_build:
-        assert_build_parity(dm, om, wl)
+    if models is None:
+        dm = harness.DeviceModel(wl, n_cal=n_cal)
+        om = oracle_model(wl, n_cal=n_cal)
+        if expect_build:
+            assert_build_parity(dm, om, wl)
+    else:
+        dm, om = models
     n_act = sum(wl.has_act)
     if sample is None:
         x, bp = wl.x, wl.budget_bp
@@ -71,8 +76,18 @@ def check(wl, n_cal=None, sample=None, expect_build=True):
     if sample is not None:
         g = slice_results(g, sample, n_act)
     assert_run_parity(g, o32, o64, wl, n_act, bool(wl.has_act[-1]))
-    dm.free()
+    if models is None:
+        dm.free()
     return info
+
+
+def build_both(wl, n_cal=None):
+    """Device model and oracle model of a workload, bucket contents compared."""
+    from paper_2204_08400_b200 import harness
+    dm = harness.DeviceModel(wl, n_cal=n_cal)
+    om = oracle_model(wl, n_cal=n_cal)
+    assert_build_parity(dm, om, wl)
+    return dm, om
 
 
 def slice_results(g, idx, n_act):
@@ -162,11 +177,19 @@ def test_c5_mixed_budgets_reduced():
 
 # ---- full sizes, in the launch configuration the benchmark times, on sampled queries ----
 
-def test_c2_full_size_sampled():
+def with_budget(wl, bp):
+    import dataclasses
+    return dataclasses.replace(wl, budget_bp=np.full(wl.n_queries, bp, np.uint16))
+
+
+def test_c2_full_size_every_named_budget_sampled():
     wl = wl_mod.load("c2", budget_bp=1000)                      # 65,536 queries, 16,384 calibration rows
     sample = np.unique(np.linspace(0, wl.n_queries - 1, 192).astype(np.int64))
-    info = check(wl, sample=sample)
-    assert info["decision_disagreements"] <= 2
+    models = build_both(wl)
+    for bp in (1000, 500, 2500, 5000, 10000):
+        info = check(with_budget(wl, bp), sample=sample, models=models)
+        assert info["decision_disagreements"] <= 2
+    models[0].free()
 
 
 def test_c5_full_widths_mixed_budgets_sampled():
@@ -175,21 +198,47 @@ def test_c5_full_widths_mixed_budgets_sampled():
     check(wl, n_cal=512, sample=sample)
 
 
-def test_c4_full_widths_batch_sizes_sampled():
+def test_c5_full_widths_single_budgets_sampled():
+    # the budget sweep of the benchmark: 8192 queries at one budget each
+    wl = wl_mod.load("c5", n_queries=8192, n_cal=512, budget_bp=500)
+    sample = np.unique(np.linspace(0, wl.n_queries - 1, 16).astype(np.int64))
+    models = build_both(wl, n_cal=512)
+    for bp in (500, 1000, 2500, 5000, 10000):
+        check(with_budget(wl, bp), sample=sample, models=models)
+    models[0].free()
+
+
+def test_c4_full_widths_batch_sizes_and_budgets_sampled():
     import dataclasses
-    full = wl_mod.load("c4", n_queries=64, n_cal=192, budget_bp=1000)
     big = wl_mod.load("c4", n_queries=4096, n_cal=192, budget_bp=1000)   # the batch size the benchmark times
-    for n, k in ((1, 1), (64, 8), (4096, 24)):
-        src = big if n > 64 else full
-        wl = dataclasses.replace(src, x=src.x[:n], budget_bp=src.budget_bp[:n])
+    models = build_both(big, n_cal=192)
+    for n, k, budgets in ((1, 1, (1000, 2500, 5000)), (64, 8, (1000, 2500, 5000)), (4096, 16, (1000, 2500, 5000))):
+        wl = dataclasses.replace(big, x=big.x[:n], budget_bp=big.budget_bp[:n])
         sample = np.unique(np.linspace(0, n - 1, k).astype(np.int64))
-        check(wl, n_cal=192, sample=sample, expect_build=(n == 1))
+        for bp in budgets:
+            check(with_budget(wl, bp), sample=sample, models=models)
+    models[0].free()
 
 
 def test_c3_full_width_output_layer_sampled():
+    # 200,000 output nodes; lists cut at the largest budget the workload names (10 %)
     wl = wl_mod.load("c3", n_queries=256, n_cal=256, budget_bp=1000, list_cap=20000)
     sample = np.arange(0, 256, 32)
-    check(wl, n_cal=256, sample=sample)
+    models = build_both(wl, n_cal=256)
+    for bp in (1000, 500, 100):
+        check(with_budget(wl, bp), sample=sample, models=models)
+    models[0].free()
+
+
+def test_c3_full_width_complete_rankings_sampled():
+    # the tables the benchmark builds: every bucket list a complete ranking of the 200,000 nodes (1.6 GB)
+    wl = wl_mod.load("c3", n_queries=256, n_cal=256, budget_bp=1000)
+    assert wl.list_cap == 0
+    sample = np.arange(5, 256, 50)
+    models = build_both(wl, n_cal=256)
+    for bp in (100, 1000):
+        check(with_budget(wl, bp), sample=sample, models=models)
+    models[0].free()
 
 
 # ---- edge cases -----------------------------------------------------------------
@@ -255,6 +304,18 @@ def test_one_warp_per_query_kernel_without_active_lists(last_budgeted):
     st = b.results()["status"]
     assert st[0] == 5 and st[1] == 11     # SLONN_ERR_BUDGET at query 11
     dm.free()
+
+
+def test_full_budget_queries_beside_the_one_warp_per_query_kernel_with_a_budgeted_last_layer():
+    # large enough (queries x weights >= 2^32) for the 100 % queries to leave the one-warp-per-query kernel and
+    # run four per block; the last layer carries an activator, so the prediction of every other query is an
+    # argmax over its own computed logits and must survive the pass that predicts the 100 % ones
+    wl = custom_workload(77, [64, 1024, 1024], [1, 1], "bf16", n=4200, n_cal=512, K=4, L=2,
+                         budgets=(500, 2500, 10000))
+    assert wl.n_queries * (64 * 1024 + 1024 * 1024) >= 2 ** 32
+    sample = np.unique(np.linspace(0, wl.n_queries - 1, 160).astype(np.int64))
+    assert len(set(wl.budget_bp[sample].tolist())) == 3
+    check(wl, sample=sample)
 
 
 def test_runs_are_deterministic():

@@ -46,6 +46,13 @@ def test_static_scratch_run_matches_the_workspace_run_twice_in_a_row():
         assert got["status"][0] == 0
         for k in KEYS:
             assert np.array_equal(got[k], expect[k]), k
+    # the point of the entry point: a call obtains no device memory.  The driver's free-byte count (which
+    # sees every allocation of the process, torch's cache or not) must not move across a call.
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    sl.slonn_run_static(dm.model, b1.batch)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
     dm.free()
 
 
