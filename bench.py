@@ -1,15 +1,18 @@
 """Benchmark of the SLO-NN inference path on B200.
 
-One step = one pass of the whole hot path (plan, hash+select, gather-dot per
-layer, argmax) over one batch of synthetic queries.  Default workload: the
-784-1024-1024-10 bf16 MLP with 65,536 queries ("c2"), headline budget 10 %,
-plus a sweep over the other budgets.  Prints ONE JSON line on rank 0.
+One step = one pass of the whole hot path (FreeHash, bucket lookup, top-k% cut, selected nodes layer by
+layer, prediction) over one batch of synthetic queries.  Headline workload: the nine-layer 4096-wide bf16
+MLP ("c4") with 4096 queries at a 10 % budget -- the only named network whose weights (276 MB) exceed the
+L2 cache.  The same line carries a `configs` block with every named network at every named budget.
+Prints ONE JSON line on rank 0.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--budget-bp 1000]
-  python bench.py --impl reference ...     # the CPU oracle on a bounded sample
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--queries 4096] [--budget-bp 1000]
+  python bench.py --impl reference ...     # the CPU oracle on a bounded sample of the same workload
 
-Multi-GPU: queries are independent, so ranks are replicas that each process
-their own batch (weak scaling); there is no data-path collective.
+Timing: the L2 is flushed (a 256 MB buffer is overwritten) before every timed step, each step has its own
+CUDA event pair on the launching stream, `ms_per_step` is the median of the K steps (max over ranks).
+Multi-GPU: queries are independent, so ranks are replicas that each process their own batch (weak
+scaling); there is no data-path collective.
 """
 import argparse
 import json
@@ -24,15 +27,20 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2204_08400_b200 import workloads  # noqa: E402
+from paper_2204_08400_b200 import accounting, workloads  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
+FLUSH_BYTES = 256 * 1024 * 1024
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu captures
-# summarised under profiles/ (same workload, same launch shape).  Keyed by (kernel, workload, queries, budget);
-# anything else reports null.  Set an entry to None when its kernel changes until the capture is redone.
+# calibration rows used when --n-cal is not given: the named count where the CPU oracle can train the same
+# tables within a minute (it is timed beside the GPU on the headline workload), fewer rows for the wide networks
+DEFAULT_N_CAL = {"c1": 16384, "c2": 16384, "c3": 2048, "c3xl": 2048, "c4": 1024, "c5": 2048}
+DEFAULT_QUERIES = {"c1": 1024, "c2": 65536, "c3": 256, "c3xl": 256, "c4": 4096, "c5": 8192}
+
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu captures
+# summarised under profiles/ (same kernel, same workload and launch shape).  Keyed by (kernel, workload,
+# queries, budget); anything else reports null.  An entry is set to None when its kernel has changed since.
 NCU_TRAFFIC = {
-    ("fused_network_kernel", "c2", 65536, 1000): 217.0e6,   # profiles/fused_network_c2_65536q_10pct.md
 }
 
 
@@ -40,69 +48,8 @@ def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return float(d["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
-
-
-def measured_tensor_peak():
-    """Dense bf16 TFLOP/s of a kernel timed alone (the burst figure)."""
-    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(p):
-        return float(json.load(open(p))["bf16_tflops"]), "measured"
-    return 1590.0, "fallback"
-
-
-def hash_bytes(wl, n):
-    """Weight bytes of the FreeHash rows of one step: K*L rows per query and activator layer."""
-    esz = 2 if wl.dtype == "bf16" else 4
-    return sum(wl.K * wl.L * wl.dims[l] * esz * n for l in range(len(wl.dims) - 1) if wl.has_act[l])
-
-
-def budget_nodes(bp, N):
-    return np.minimum(np.maximum((bp.astype(np.int64) * N + 5000) // 10000, 1), N)
-
-
-def gathered_bytes(wl, budget_bp, force_rows=False, force_cols=False, cols_max_bp=3500):
-    """Algorithmic weight bytes of one step's gather launches, all queries, split by kernel kind:
-    (row kernels, gather_cols_kernel, layer_cols_kernel, full_rows_kernel on layers without activator).
-    Row kernels (dense input, or a list input that is not sparse enough): every selected weight row
-    once per query, whole (row-granular).  Input-stationary kernels (a layer fed by the list of the
-    activator layer below, budgets up to cols_max_bp): selected nodes x input list entries
-    (B_out * B_in weights), the weights such a query needs at all; the whole-layer kernel of an
-    activator layer also reads its K*L hash rows at the list entries."""
-    esz = 2 if wl.dtype == "bf16" else 4
-    bp = np.asarray(budget_bp)
-    rows = cols = layer = grouped = 0
-    if bp.size == 0:
-        return 0, 0, 0, 0
-    for l in range(len(wl.dims) - 1):
-        if l == 0 and wl.first_sparse:
-            continue
-        D, N = wl.dims[l], wl.dims[l + 1]
-        b_out = budget_nodes(bp, N) if wl.has_act[l] else np.full(bp.size, N, np.int64)
-        list_input = l > 0 and wl.has_act[l - 1]
-        use_cols = np.zeros(bp.size, bool)
-        if list_input and not force_rows:
-            big = bp.size * int(b_out.max()) >= 148 * 1024
-            if force_cols:
-                use_cols[:] = bp.size * int(b_out.max()) > 148 * 64
-            elif big:
-                use_cols = bp <= cols_max_bp
-            elif bp.size * int(b_out.max()) > 148 * 64 and D >= 2048 and int(bp.max()) <= 1500:
-                use_cols = bp <= 1500
-        b_in = budget_nodes(bp, D) if list_input else np.full(bp.size, D, np.int64)
-        if wl.has_act[l] and wl.K * wl.L <= 32:
-            layer += int(((b_out[use_cols] + wl.K * wl.L) * b_in[use_cols]).sum()) * esz
-        else:
-            cols += int((b_out[use_cols] * b_in[use_cols]).sum()) * esz
-        row_bytes = int(b_out[~use_cols].sum()) * D * esz
-        # a layer without activator: the row-kernel queries share every row and run four per block
-        if (not wl.has_act[l] and bp.size >= 256 and bp.size * N * D >= 2 ** 30 and 16 * D <= 200 * 1024
-                and not use_cols.all()):
-            grouped += row_bytes
-        else:
-            rows += row_bytes
-    return rows, cols, layer, grouped
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
+    return 6650.0, 1590.0, "fallback"
 
 
 class ClockSampler:
@@ -151,59 +98,68 @@ class ClockSampler:
         return out
 
 
-def oracle_queries_per_sec(wl, budget_bp, target_seconds=12.0):
-    """The CPU oracle as it stands, timed on a bounded prefix of the workload's queries."""
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
+def resolve(args):
+    """Query count, calibration rows and budget of the headline workload (identical in both arms)."""
+    n = args.queries if args.queries is not None else DEFAULT_QUERIES[args.workload]
+    n_cal = args.n_cal if args.n_cal is not None else DEFAULT_N_CAL[args.workload]
+    return n, n_cal
+
+
+def load_workload(args):
+    n, n_cal = resolve(args)
+    return workloads.load(args.workload, n_queries=n, n_cal=n_cal, budget_bp=args.budget_bp if args.budget_bp else None,
+                          free_hash_nodes=args.free_hash_nodes)
+
+
+def config_block(args, wl, world):
+    """`config` of the JSON line; both arms print the same dict."""
+    n, n_cal = resolve(args)
+    label = (f"{args.workload}: " + "-".join(map(str, wl.dims)) + f" {wl.dtype} weights, {n} queries/GPU, budget " +
+             (f"{args.budget_bp} bp" if args.budget_bp else "mixed 5/10/25/50/100 %") + f", K={wl.K} L={wl.L}, " +
+             f"tables trained on {n_cal} calibration rows" + (", hash nodes always active" if wl.free_hash_nodes else ""))
+    return {"workload": label, "queries_per_step_per_gpu": n, "budget_bp": args.budget_bp, "n_cal": n_cal,
+            "l2": "flushed_between_steps", "parallelism": f"replicas x{world}"}
+
+
+# ---- the CPU oracle (reference arm and cpu_baseline leg) ---------------------------------------
+
+def oracle_sample(wl, target_seconds):
+    """The oracle as it stands on a prefix of the workload's queries sized for about target_seconds.
+    Returns (queries, seconds, threads, closure that repeats the timed call)."""
     from oracle import oracle as orc
-    from parity_util import oracle_model, oracle_run, take_queries
+    from oracle.run_workload import oracle_model, oracle_run, take_queries
     om = oracle_model(wl)
-    n0 = min(wl.n_queries, 256)
-    idx = np.arange(n0)
-    bp = wl.budget_bp[:n0] if budget_bp is None else np.full(n0, budget_bp, np.uint16)
-    t0 = time.perf_counter()
-    oracle_run(om, wl, take_queries(wl, idx), bp, orc.CANON32)
-    dt = max(time.perf_counter() - t0, 1e-4)
+    n0 = min(wl.n_queries, 128)
+    for _ in range(2):      # the second pass of the pilot sample is the one that sizes the timed sample
+        t0 = time.perf_counter()
+        oracle_run(om, wl, take_queries(wl, np.arange(n0)), wl.budget_bp[:n0], orc.CANON32)
+        dt = max(time.perf_counter() - t0, 1e-4)
     n1 = int(min(wl.n_queries, max(n0, n0 * target_seconds / dt)))
-    idx = np.arange(n1)
-    bp = wl.budget_bp[:n1] if budget_bp is None else np.full(n1, budget_bp, np.uint16)
-    xs = take_queries(wl, idx)
-    t0 = time.perf_counter()
-    oracle_run(om, wl, xs, bp, orc.CANON32)
-    dt = time.perf_counter() - t0
-    return n1 / dt, orc.threads(), n1, dt, (om, xs, bp)
+    xs, bp = take_queries(wl, np.arange(n1)), wl.budget_bp[:n1]
 
-
-def workload_label(args, wl):
-    return (f"{args.workload}: " + "-".join(map(str, wl.dims)) + f" {wl.dtype} weights, {wl.n_queries} queries/GPU, budget " +
-            (f"{args.budget_bp} bp" if args.budget_bp else "mixed 5/10/25/50/100 %") + f", K={wl.K} L={wl.L}" +
-            (", hash nodes always active" if wl.free_hash_nodes else ""))
+    def again():
+        t = time.perf_counter()
+        oracle_run(om, wl, xs, bp, orc.CANON32)
+        return time.perf_counter() - t
+    return n1, again, orc.threads()
 
 
 def run_reference(args, rank, world):
     if rank != 0:
         return
-    wl = workloads.load(args.workload, n_queries=args.queries, n_cal=args.n_cal,
-                        budget_bp=args.budget_bp if args.budget_bp else None, free_hash_nodes=args.free_hash_nodes)
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from oracle import oracle as orc
-    from parity_util import oracle_run
-    qps, cores, n1, dt, (om, xs, bp) = oracle_queries_per_sec(wl, args.budget_bp if args.budget_bp else None,
-                                                              target_seconds=6.0)
-    for _ in range(args.warmup):
-        pass  # the sizing pass above already warmed caches; warm-up steps would only repeat it
-    times = []
-    for _ in range(args.steps):
-        t0 = time.perf_counter()
-        oracle_run(om, wl, xs, bp, orc.CANON32)
-        times.append(time.perf_counter() - t0)
-    ms = 1e3 * float(np.sum(times)) / max(args.steps, 1)
+    wl = load_workload(args)
+    steps = max(args.steps, 1)
+    n1, again, cores = oracle_sample(wl, target_seconds=min(6.0, 90.0 / steps))
+    for _ in range(min(args.warmup, 1)):
+        again()
+    times = [again() for _ in range(steps)]
+    ms = 1e3 * float(np.median(times))
     value = n1 / (ms / 1e3)
     line = {
         "impl": "reference", "metric": "queries_per_sec_at_budget", "value": value, "unit": "queries/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": workload_label(args, wl), "queries_per_step_per_gpu": wl.n_queries,
-                   "budget_bp": args.budget_bp, "queries_timed_per_step": n1},
+        "config": config_block(args, wl, world),
         "cpu_baseline": {"value": value, "unit": "queries/s", "cores": cores, "kind": "oracle",
                          "sample": f"first {n1} of {wl.n_queries} queries per step"},
         "e2e": {"value": value, "unit": "queries/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -212,17 +168,190 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+# ---- GPU arm -------------------------------------------------------------------------------------
+
+class Rig:
+    """One device model with the plumbing to time batches on it."""
+
+    def __init__(self, wl, dev, world, n_cal=None):
+        import torch
+        from paper_2204_08400_b200 import harness
+        self.torch, self.wl, self.dev, self.world = torch, wl, dev, world
+        self.dm = harness.DeviceModel(wl, device=dev, n_cal=n_cal)
+        self.stream = torch.cuda.current_stream(dev)
+        self.shape = accounting.NetShape.of(wl)
+        self.x_nnz = (wl.x[0][1:] - wl.x[0][:-1]).astype(np.int64) if wl.first_sparse else None
+
+    def barrier(self):
+        import torch.distributed as dist
+        self.torch.cuda.synchronize(self.dev)
+        if self.world > 1:
+            dist.barrier()
+        self.torch.cuda.synchronize(self.dev)
+
+    def take(self, n):
+        """Inputs of the first n queries."""
+        wl = self.wl
+        if wl.first_sparse:
+            ip = wl.x[0][: n + 1]
+            return (ip, wl.x[1][: int(ip[-1])], wl.x[2][: int(ip[-1])])
+        return wl.x[:n]
+
+    def batch(self, bps, flags=0, kernel_path=0):
+        from paper_2204_08400_b200 import harness
+        return harness.DeviceBatch(self.dm, self.take(bps.size), bps, max_budget_bp=int(bps.max()), full_outputs=False,
+                                   flags=flags, kernel_path=kernel_path)
+
+    def time_steps(self, batch, steps, warmup, flush):
+        """Per-step device times (ms): L2 flushed before every step, an event pair around each."""
+        torch = self.torch
+        for _ in range(warmup):
+            batch.run(self.stream)
+        self.barrier()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in ev:
+            flush.zero_()
+            a.record(self.stream)
+            batch.run(self.stream)
+            b.record(self.stream)
+        self.barrier()
+        st = batch.status.cpu().numpy()
+        assert st[0] == 0, f"device status {st}"
+        return np.array([a.elapsed_time(b) for a, b in ev])
+
+    def trace(self, batch, reps=3):
+        """Launch records of one step, times averaged over `reps` traced runs."""
+        from paper_2204_08400_b200 import binding as sl
+        runs = [sl.slonn_run_traced(self.dm.model, batch.batch, batch.ws, batch.ws_bytes, self.stream) for _ in range(reps + 1)][1:]
+        recs = [dict(r) for r in runs[0]]
+        for i, r in enumerate(recs):
+            r["ms"] = float(np.mean([run[i]["ms"] for run in runs]))
+        return recs
+
+    def kernels(self, batch, bps):
+        """Per-kernel launches, time and byte counts of one step, plus the dominant kernel's roofline entry."""
+        recs = self.trace(batch)
+        table = accounting.per_kernel(self.shape, recs, bps, self.x_nnz[: bps.size] if self.x_nnz is not None else None)
+        return recs, table
+
+
+def roofline_of(table, workload, n, budget_bp, dense_tc):
+    """Roofline entry of the kernel with the largest share of the step's device time."""
+    hbm, tflops, kind = measured_peaks()
+    name = max(table, key=lambda k: table[k]["ms"])
+    k = table[name]
+    total_ms = sum(v["ms"] for v in table.values())
+    common = {"kernel": name, "launches_per_step": k["launches"], "avg_launch_ms": k["ms"] / max(k["launches"], 1),
+              "share_of_step": k["ms"] / total_ms if total_ms else 0.0, "peak_kind": kind}
+    if name == "dense_tc_kernel":
+        ach = k["flops"] / (k["ms"] / 1e3) / 1e12
+        return dict(common, bound="tensor", achieved=ach, peak=tflops, unit="TFLOP/s", frac=ach / tflops, traffic=None,
+                    flops_per_step=k["flops"])
+    sec = k["ms"] / 1e3
+    ach = k["algorithmic"] / sec / 1e9 if sec > 0 else 0.0
+    traffic = None if dense_tc else NCU_TRAFFIC.get((name, workload, n, budget_bp))
+    return dict(common, bound="hbm", achieved=ach, peak=hbm, unit="GB/s", frac=ach / hbm, traffic=traffic,
+                frac_of_nominal_8TBps=ach / 8000.0, bytes_per_step=int(k["algorithmic"]),
+                bytes_as_run=int(k["as_run"]), frac_as_run=k["as_run"] / sec / 1e9 / hbm if sec > 0 else 0.0,
+                bytes_row_granular=int(k["row_granular"]),
+                frac_row_granular=k["row_granular"] / sec / 1e9 / hbm if sec > 0 else 0.0,
+                dram_frac=(traffic * k["launches"] / sec / 1e9 / hbm) if traffic else None,
+                note="bytes_per_step: hash rows, bucket lists and selected nodes x input entries (the least any form must "
+                     "load); bytes_as_run: whole rows where a layer ran row-wise.  A fraction above 1, or a traffic far "
+                     "below bytes_per_step, means the rows were served from L2/L1, not HBM")
+
+
+def measure(rig, bps, flags, steps, warmup, flush, workload, want_table=True):
+    """One (batch size, budgets, flags) point: median step time, dominant kernel, byte counts."""
+    batch = rig.batch(bps, flags=flags)
+    t = rig.time_steps(batch, steps, warmup, flush)
+    out = {"ms": float(np.median(t)), "ms_mean": float(np.mean(t)), "queries_per_s": bps.size / (float(np.median(t)) / 1e3)}
+    if want_table:
+        recs, table = rig.kernels(batch, bps)
+        bp_key = int(bps[0]) if np.all(bps == bps[0]) else 0
+        roof = roofline_of(table, workload, int(bps.size), bp_key, bool(flags & 1))
+        out.update(kernel=roof["kernel"], frac=roof["frac"], share_of_step=roof["share_of_step"], bound=roof["bound"],
+                   frac_as_run=roof.get("frac_as_run"), launches=len(recs))
+        sb = accounting.step_bytes(rig.shape, bps, rig.x_nnz[: bps.size] if rig.x_nnz is not None else None)
+        out["step_GBps_algorithmic"] = sb["algorithmic"] / (out["ms"] / 1e3) / 1e9
+        out["step_frac_of_hbm_peak"] = out["step_GBps_algorithmic"] / measured_peaks()[0]
+    del batch
+    return out
+
+
+def latency_block(rig, bps, reps, flags=0):
+    """p50/p90/p99 of single steps answered one at a time, also as a CUDA-graph replay."""
+    torch, dev, stream = rig.torch, rig.dev, rig.stream
+    batch = rig.batch(bps, flags=flags)
+    for _ in range(5):
+        batch.run(stream)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b_ in evs:
+        a.record(stream)
+        batch.run(stream)
+        b_.record(stream)
+        torch.cuda.synchronize(dev)      # a server answers one request before it takes the next
+    t = np.array([a.elapsed_time(b_) for a, b_ in evs]) * 1e3
+    out = {"unit": "us per batch", "launches": reps, "p50": float(np.percentile(t, 50)),
+           "p90": float(np.percentile(t, 90)), "p99": float(np.percentile(t, 99)), "min": float(t.min())}
+    gs = torch.cuda.Stream(dev)
+    with torch.cuda.stream(gs):
+        batch.run(gs)
+        gs.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=gs):
+            batch.run(torch.cuda.current_stream(dev))
+        tg = []
+        for _ in range(reps):
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); graph.replay(); b_.record()
+            torch.cuda.synchronize(dev)
+            tg.append(a.elapsed_time(b_) * 1e3)
+    out["graph_replay_p50"] = float(np.percentile(tg, 50))
+    out["graph_replay_p99"] = float(np.percentile(tg, 99))
+    return out
+
+
+def sweep(rig, n, budgets, steps, flush, workload, mixed=None, small=False):
+    """Every named budget at n queries, the 100 % budget on the fixed-order kernels and (where the library
+    offers it) on the tensor cores, and each budget's speed-up over both -- the paper's own measure
+    (Sec. 5.2: speed-up over the full network)."""
+    from paper_2204_08400_b200 import binding as sl
+    wl = rig.wl
+    out = {}
+    full = measure(rig, np.full(n, 10000, np.uint16), 0, steps, 3, flush, workload)
+    tc_ok = wl.dtype == "bf16" and not wl.first_sparse and not wl.has_act[-1]
+    full_tc = measure(rig, np.full(n, 10000, np.uint16), sl.FLAG_DENSE_TC, steps, 3, flush, workload) if tc_ok else None
+    points = [(str(bp), np.full(n, bp, np.uint16)) for bp in budgets]
+    if mixed is not None:
+        points.insert(0, ("mixed", mixed[:n]))
+    for key, bps in points:
+        if key == "10000":
+            m = dict(full)
+        else:
+            m = measure(rig, bps, 0, steps, 3, flush, workload)
+        m["speedup_vs_full"] = full["ms"] / m["ms"]
+        m["speedup_vs_full_on_tensor_cores"] = full_tc["ms"] / m["ms"] if full_tc else None
+        if small:
+            m["latency"] = latency_block(rig, bps, 200)
+        out[key] = m
+    out["full_budget_ms"] = {"fixed_order_kernels": full["ms"], "tensor_cores": full_tc["ms"] if full_tc else None}
+    if small:
+        out["full_budget_latency"] = latency_block(rig, np.full(n, 10000, np.uint16), 200)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--workload", default="c4")
     ap.add_argument("--budget-bp", type=int, default=1000,
                     help="budget of every query in basis points; 0 = the workload's mixed per-query budgets (c5)")
     ap.add_argument("--queries", type=int, default=None, help="override the workload's query count")
-    ap.add_argument("--n-cal", type=int, default=None)
+    ap.add_argument("--n-cal", type=int, default=None, help="calibration rows the tables are trained on")
     ap.add_argument("--dense-tc", action="store_true",
                     help="route 100 %% budget queries to the tensor-core dense path (not bit-exact for them)")
     ap.add_argument("--free-hash-nodes", action="store_true",
@@ -230,10 +359,11 @@ def main():
     ap.add_argument("--row-kernels", action="store_true", help="sparse-input layers: force the row kernels")
     ap.add_argument("--column-kernels", action="store_true", help="sparse-input layers: force the input-stationary kernels")
     ap.add_argument("--kernel-path", type=int, default=0, help="0 auto, 1 per-stage kernels, 2 one warp per query, 3 cluster")
-    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="headline workload only (e.g. under a profiler)")
+    ap.add_argument("--configs", default="c1,c2,c3,c4,c5", help="networks of the configs block")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-baseline", action="store_true", help="time the oracle also for workloads other than c1/c2")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-policy", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -257,32 +387,15 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
 
-    # every rank is a replica with its own batch (same law, rank-specific seed is not needed:
-    # throughput does not depend on the draw; parity tests cover the values)
-    wl = workloads.load(args.workload, n_queries=args.queries, n_cal=args.n_cal,
-                        budget_bp=args.budget_bp if args.budget_bp else None, free_hash_nodes=args.free_hash_nodes)
-    max_bp = int(wl.budget_bp.max())
+    # every rank is a replica with its own batch (same law; throughput does not depend on the draw and the
+    # parity tests cover the values)
+    wl = load_workload(args)
     n = wl.n_queries
-    dm = harness.DeviceModel(wl, device=dev)
-    stream = torch.cuda.current_stream(dev)
-
-    def barrier():
-        torch.cuda.synchronize(dev)
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize(dev)
-
-    def timed(batch, steps, warmup):
-        for _ in range(warmup):
-            batch.run(stream)
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(steps):
-            batch.run(stream)
-        e1.record(stream)
-        barrier()
-        return replicas.slowest_rank_ms(e0.elapsed_time(e1), dev) / steps
+    max_bp = int(wl.budget_bp.max())
+    rig = Rig(wl, dev, world)
+    dm, stream = rig.dm, rig.stream
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    hbm_peak, _, _ = measured_peaks()
 
     # ---- headline: device-resident inputs ----
     flags = sl.FLAG_DENSE_TC if args.dense_tc else 0
@@ -297,130 +410,25 @@ def main():
             batch.run(stream)
         torch.cuda.synchronize(dev)
         time.sleep(0.3)
-    ms_step = timed(batch, args.steps, args.warmup)
+    step_ms = rig.time_steps(batch, args.steps, args.warmup, flush)
     clocks = sampler.stop() if rank == 0 else None
-    status = batch.status.cpu().numpy()
-    assert status[0] == 0, f"device status {status}"
+    ms_step = replicas.slowest_rank_ms(float(np.median(step_ms)), dev)
     n_all = replicas.total_units(n, dev)          # queries all ranks processed in one step
     value = n_all / (ms_step / 1e3)
-    launches_per_step = None  # counted below from the per-stage launch counters
 
-    # ---- per-query latency for small batches (the paper serves at batch size 1): one event pair per step ----
-    latency = None
-    if n <= 64:
-        reps = max(args.steps, 1000)
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
-        for a, b_ in evs:
-            a.record(stream)
-            batch.run(stream)
-            b_.record(stream)
-            torch.cuda.synchronize(dev)      # a server answers one request before it takes the next
-        t = np.array([a.elapsed_time(b_) for a, b_ in evs]) * 1e3
-        latency = {"unit": "us per batch", "launches": reps, "p50": float(np.percentile(t, 50)),
-                   "p90": float(np.percentile(t, 90)), "p99": float(np.percentile(t, 99)), "min": float(t.min())}
-        # the same step captured once in a CUDA graph and replayed per request
-        gs = torch.cuda.Stream(dev)
-        with torch.cuda.stream(gs):
-            batch.run(gs)
-            gs.synchronize()
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=gs):
-                batch.run(torch.cuda.current_stream(dev))
-            tg = []
-            for _ in range(reps):
-                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(); graph.replay(); b_.record()
-                torch.cuda.synchronize(dev)
-                tg.append(a.elapsed_time(b_) * 1e3)
-        latency["graph_replay_p50"] = float(np.percentile(tg, 50))
-        latency["graph_replay_p99"] = float(np.percentile(tg, 99))
+    # ---- per-launch device time of the same step, byte counts per kernel ----
+    recs, table = rig.kernels(batch, wl.budget_bp)
+    roofline = roofline_of(table, args.workload, n, args.budget_bp, args.dense_tc)
+    roofline["kernels"] = {k: {"launches": v["launches"], "ms": v["ms"], "GBps_algorithmic": (v["algorithmic"] / (v["ms"] / 1e3) / 1e9) if v["ms"] else 0.0,
+                               "frac": (v["algorithmic"] / (v["ms"] / 1e3) / 1e9 / hbm_peak) if v["ms"] else 0.0}
+                           for k, v in table.items()}
+    sb = accounting.step_bytes(rig.shape, wl.budget_bp, rig.x_nnz)
+    roofline["step"] = {"bytes_algorithmic": int(sb["algorithmic"]), "bytes_row_granular": int(sb["row_granular"]),
+                        "GBps_algorithmic": sb["algorithmic"] / (ms_step / 1e3) / 1e9,
+                        "frac": sb["algorithmic"] / (ms_step / 1e3) / 1e9 / hbm_peak}
+    launches_per_step = len(recs) + sum(1 for r in recs if r["stage"] == "plan")   # the plan record covers two launches
 
-    # ---- per-stage device time of the same step (event pair around every launch) ----
-    stage_ms = {s: 0.0 for s in sl.STAGES}
-    stage_cnt = {s: 0 for s in sl.STAGES}
-    prof_steps = max(3, min(args.steps, 10))
-    for _ in range(prof_steps):
-        ms, cnt = sl.slonn_run_timed(dm.model, batch.batch, batch.ws, batch.ws_bytes, stream)
-        for s in sl.STAGES:
-            stage_ms[s] += ms[s]; stage_cnt[s] += cnt[s]
-    def full_route_active(bps):
-        """The library's rule for taking the 100 % queries out of the per-query kernels (four per block)."""
-        weights = sum(wl.dims[l] * wl.dims[l + 1] for l in range(len(wl.dims) - 1))
-        return (not (flags & sl.FLAG_DENSE_TC) and not wl.first_sparse and bps.size >= 256 and int(bps.max()) == 10000
-                and bps.size * weights >= 2 ** 32 and 16 * max(wl.dims[:-1]) <= 200 * 1024)
-
-    def stage_roofline(ms_by_stage, cnt_by_stage, bps, steps):
-        """Dominant kernel of the step and its achieved rate on the weight bytes it must touch."""
-        esz = 2 if wl.dtype == "bf16" else 4
-        n_full = int((bps == 10000).sum()) if bps.size and full_route_active(bps) else 0
-        full_b = n_full * sum(wl.dims[l] * wl.dims[l + 1] for l in range(len(wl.dims) - 1)) * esz
-        if (flags & sl.FLAG_DENSE_TC) or n_full:     # queries at 100 % leave the per-query kernels
-            bps = bps[bps != 10000]
-        row_b, col_b, layer_b, grouped_b = gathered_bytes(wl, bps, args.row_kernels, args.column_kernels, sl.COLS_MAX_BP)
-        if ms_by_stage["full_rows"] > 0 and ms_by_stage["full_rows"] >= max(ms_by_stage.values()):
-            ms, launches = ms_by_stage["full_rows"] / steps, cnt_by_stage["full_rows"] // steps
-            nbytes = full_b + (grouped_b if ms_by_stage["fused"] == 0 and ms_by_stage["cluster"] == 0 else 0)
-            return "full_rows_kernel", ms, launches, nbytes, nbytes / (ms / 1e3) / 1e9
-        cols_ms = ms_by_stage["gather_cols"] + ms_by_stage["layer_cols"]
-        if ms_by_stage["fused"] > 0:     # one launch does hash + select + gather for every layer
-            row_b = sum(gathered_bytes(wl, bps, force_rows=True)[i] for i in (0, 3))
-            kernel, ms, launches, nbytes = "fused_network_kernel", ms_by_stage["fused"], cnt_by_stage["fused"], row_b + hash_bytes(wl, bps.size)
-        elif ms_by_stage["cluster"] > 0:
-            row_b = sum(gathered_bytes(wl, bps, force_rows=True)[i] for i in (0, 3))
-            kernel, ms, launches, nbytes = "cluster_network_kernel", ms_by_stage["cluster"], cnt_by_stage["cluster"], row_b + hash_bytes(wl, bps.size)
-        elif cols_ms > ms_by_stage["gather_dot"]:
-            # the input-stationary kernels: the whole-layer kernel of the activator layers (hash + selection +
-            # nodes) or, if larger, the plain gather of the layers without activator
-            if ms_by_stage["layer_cols"] >= ms_by_stage["gather_cols"]:
-                kernel, ms, launches, nbytes = "layer_cols_kernel", ms_by_stage["layer_cols"], cnt_by_stage["layer_cols"], layer_b
-            else:
-                kernel, ms, launches, nbytes = "gather_cols_kernel", ms_by_stage["gather_cols"], cnt_by_stage["gather_cols"], col_b
-        else:
-            esz = 2 if wl.dtype == "bf16" else 4
-            gather_layers = [l for l in range(len(wl.dims) - 1) if not (l == 0 and wl.first_sparse)]
-            short = all(wl.dims[l] * esz <= 512 for l in gather_layers)   # rows of one 512-byte round
-            kernel = "gather_short_kernel" if short else "gather_dot_kernel"
-            ms, launches, nbytes = ms_by_stage["gather_dot"], cnt_by_stage["gather_dot"], row_b
-        ms /= steps
-        launches //= steps
-        ach = nbytes / (ms / 1e3) / 1e9 if ms > 0 else 0.0
-        return kernel, ms, launches, nbytes, ach
-
-    peak, peak_kind = measured_peaks()
-    kernel, k_ms, k_launches, k_bytes, achieved = stage_roofline(stage_ms, stage_cnt, wl.budget_bp, prof_steps)
-    roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": peak_kind,
-                "traffic": NCU_TRAFFIC.get((kernel, args.workload, n, args.budget_bp)) if not args.dense_tc else None,
-                "frac_of_nominal_8TBps": achieved / 8000.0,
-                "bytes_per_step": int(k_bytes), "launches_per_step": k_launches,
-                "avg_launch_ms": k_ms / max(k_launches, 1),
-                "stage_ms_per_step": {s: stage_ms[s] / prof_steps for s in sl.STAGES}}
-    if stage_ms["dense_tc"] >= max(stage_ms.values()):
-        # the step is dominated by the tensor-core route: its roofline is the tensor pipe.  The stage time
-        # covers the compaction of the routed queries and the bf16 copy of their inputs as well.
-        n_tc = int((wl.budget_bp == 10000).sum())
-        flops = sum(2.0 * n_tc * wl.dims[l] * wl.dims[l + 1] for l in range(len(wl.dims) - 1))
-        tc_ms = stage_ms["dense_tc"] / prof_steps
-        tpeak, tkind = measured_tensor_peak()
-        ach = flops / (tc_ms / 1e3) / 1e12
-        roofline = {"bound": "tensor", "kernel": "dense_tc_kernel", "achieved": ach, "peak": tpeak, "unit": "TFLOP/s",
-                    "frac": ach / tpeak, "peak_kind": tkind, "traffic": None, "flops_per_step": flops,
-                    "launches_per_step": len(wl.dims) - 1, "avg_launch_ms": tc_ms / (len(wl.dims) - 1),
-                    "stage_ms_per_step": {s: stage_ms[s] / prof_steps for s in sl.STAGES}}
-
-    # ---- budget sweep (the latency profile T(k, isolated) of the paper) ----
-    sweep = {}
-    if not args.no_sweep and world == 1:
-        for bp in wl.budgets_named:
-            bps = np.full(n, bp, np.uint16)
-            b2 = harness.DeviceBatch(dm, wl.x, bps, max_budget_bp=bp, full_outputs=False, flags=flags,
-                                     kernel_path=args.kernel_path)
-            ms2 = timed(b2, max(3, args.steps // 4), 3)
-            st_ms, st_cnt = sl.slonn_run_timed(dm.model, b2.batch, b2.ws, b2.ws_bytes, stream)
-            k2, _, _, _, ach2 = stage_roofline(st_ms, st_cnt, bps, 1)
-            sweep[str(bp)] = {"queries_per_s": n / (ms2 / 1e3), "ms_per_step": ms2, "kernel": k2,
-                              "weight_GBps": ach2, "frac_of_peak": ach2 / peak}
-            del b2
+    latency = latency_block(rig, wl.budget_bp, max(args.steps, 1000), flags) if n <= 64 else None
 
     # ---- end to end through the host-buffer entry point ----
     e2e = None
@@ -445,26 +453,55 @@ def main():
                                logit_ids=h_lids, pred=h_pred, flags=flags)
         nb = sl.slonn_host_workspace_bytes(dm.model, n, max_bp, x_nnz, flags)
         hws = torch.empty(nb, dtype=torch.uint8, device=dev)
-        e_steps = max(3, min(args.steps, 10))
+        e_steps = max(3, min(args.steps, 20))
         for _ in range(3):
             up, down = sl.slonn_run_host(dm.model, hb, hws, nb, stream)
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(e_steps):
+        rig.barrier()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(e_steps)]
+        for a, b_ in ev:
+            a.record(stream)
             up, down = sl.slonn_run_host(dm.model, hb, hws, nb, stream)
-        e1.record(stream)
-        barrier()
-        ms_e = replicas.slowest_rank_ms(e0.elapsed_time(e1), dev) / e_steps
+            b_.record(stream)
+        rig.barrier()
+        ms_e = replicas.slowest_rank_ms(float(np.median([a.elapsed_time(b_) for a, b_ in ev])), dev)
         assert int(h_status[0]) == 0
         e2e = {"value": n_all / (ms_e / 1e3), "unit": "queries/s", "h2d_bytes_per_step": int(up),
                "d2h_bytes_per_step": int(down), "ms_per_step": ms_e}
+        del hws
+
+    # ---- every named network at every named budget (rank 0 of a single-GPU run) ----
+    configs = None
+    if rank == 0 and world == 1 and not args.no_configs:
+        configs = {}
+        cfg_steps = max(5, min(args.steps, 10))
+        for name in [c for c in args.configs.split(",") if c]:
+            same = (name == args.workload and not args.free_hash_nodes and resolve(args)[1] == DEFAULT_N_CAL[name]
+                    and n >= DEFAULT_QUERIES[name])
+            if same:
+                r2 = rig
+            else:
+                w2 = workloads.load(name, n_queries=DEFAULT_QUERIES[name], n_cal=DEFAULT_N_CAL[name])
+                r2 = Rig(w2, dev, world)
+            budgets = list(r2.wl.budgets_named)
+            mixed = workloads.draw_mixed_budgets(DEFAULT_QUERIES[name], 4) if name == "c5" else None
+            entry = {"network": "-".join(map(str, r2.wl.dims)) + " " + r2.wl.dtype, "n_cal": r2.dm.n_cal,
+                     "table_bytes": r2.dm.table_bytes(),
+                     "table_build_ms": r2.dm.build_ms}
+            entry[f"{DEFAULT_QUERIES[name]}_queries"] = sweep(r2, DEFAULT_QUERIES[name], budgets, cfg_steps, flush, name, mixed)
+            if name == "c4":      # the paper serves at batch size 1: per-batch latency of small batches
+                for small_n in (64, 1):
+                    entry[f"{small_n}_queries"] = sweep(r2, small_n, budgets, cfg_steps, flush, name, small=True)
+            configs[name] = entry
+            if r2 is not rig:
+                r2.dm.free()
+                del r2
+                torch.cuda.empty_cache()
 
     # ---- budget policies on the device (outside the timed region): Confidence tables + ACLO lookup ----
     policy = None
-    if rank == 0 and world == 1 and not args.no_sweep and wl.has_act[0] and not wl.first_sparse and not wl.has_act[-1]:
+    if (rank == 0 and world == 1 and not args.no_policy and wl.has_act[0] and not wl.first_sparse and not wl.has_act[-1]):
         prof = np.array(sorted(set(wl.budgets_named) | {10000}), np.uint16)
-        rows = harness._dev(wl.calib[: min(dm.n_cal, 4096)], dev)
+        rows = harness._dev(wl.calib[: min(dm.n_cal, 1024)], dev)
         torch.cuda.synchronize(dev)
         t0 = time.perf_counter()
         conf = sl.slonn_confidence_build(dm.model, rows, prof, stream)
@@ -488,32 +525,31 @@ def main():
 
     # ---- the CPU oracle beside it (rank 0, single-GPU runs only) ----
     cpu = None
-    # the oracle builds its own tables from the same calibration rows: seconds for c1/c2, many minutes for
-    # the wide networks, so those need --cpu-baseline (and usually --n-cal) to be asked for explicitly
-    want_cpu = args.cpu_baseline or (args.workload in ("c1", "c2") and not args.no_cpu_baseline)
-    if rank == 0 and world == 1 and want_cpu:
-        qps, cores, n1, dt, _ = oracle_queries_per_sec(wl, None if not args.budget_bp else args.budget_bp)
-        cpu = {"value": qps, "unit": "queries/s", "cores": cores, "kind": "oracle",
-               "sample": f"first {n1} of {n} queries, {dt:.1f} s"}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n1, again, cores = oracle_sample(wl, target_seconds=15.0)
+        dt = again()
+        cpu = {"value": n1 / dt, "unit": "queries/s", "cores": cores, "kind": "oracle",
+               "sample": f"first {n1} of {n} queries, {dt:.1f} s, tables trained by the oracle on the same {dm.n_cal} calibration rows"}
 
     if rank == 0:
-        esz_name = "f32"  # every sum is accumulated in fp32 (bf16 weights are widened)
         line = {
             "metric": "queries_per_sec_at_budget", "value": value, "unit": "queries/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": esz_name, "data": "synthetic",
-            "config": {"workload": workload_label(args, wl),
-                       "queries_per_step_per_gpu": n, "budget_bp": args.budget_bp,
-                       "l2": "inputs_larger_than_l2" if (wl.x.nbytes if not wl.first_sparse else 0) > L2_BYTES
-                             else "weights_and_inputs_l2_resident",
-                       "table_bytes": dm.table_bytes(), "parallelism": f"replicas x{world}",
-                       "full_budget_route": "tensor cores (bf16 activations)" if args.dense_tc else "fixed-order fp32 kernels"},
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32",   # every sum is accumulated in fp32 (bf16 weights are widened)
+            "data": "synthetic",
+            "config": config_block(args, wl, world),
+            "timing": {"statistic": "median of the timed steps", "ms_per_step_mean": float(np.mean(step_ms)),
+                       "ms_per_step_min": float(np.min(step_ms)), "l2_flush_bytes": FLUSH_BYTES},
+            "full_budget_route": "tensor cores (bf16 activations)" if args.dense_tc else "fixed-order fp32 kernels",
             "clocks": clocks, "e2e": e2e,
-            "gpu_launches": (sum(stage_cnt.values()) // prof_steps + (1 if stage_cnt["plan"] else 0)) * args.steps,
-            "roofline": roofline, "cpu_baseline": cpu, "budget_sweep": sweep, "latency": latency,
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "configs": configs, "latency": latency,
             "policy": policy,
-            "table_build": {"ms": dm.build_ms, "calibration_rows": dm.n_cal,
+            "table_build": {"ms": dm.build_ms, "calibration_rows": dm.n_cal, "table_bytes": dm.table_bytes(),
                             "rows_per_s": dm.n_cal / (dm.build_ms / 1e3), "timing": "host wall clock around slonn_build"},
+            "paper_context": "the paper reports only speed-ups over the full network (1.3-56.7x, CPU, NumPy+Numba, batch size 1); "
+                             "speedup_vs_full in `configs` is that measure on this GPU",
         }
         print(json.dumps(line), flush=True)
     if world > 1:
