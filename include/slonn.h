@@ -224,7 +224,13 @@ typedef struct {
 #define SLONN_COLS_MAX_BP 3500u /* default split: budgets up to this take the input-stationary kernels */
 #define SLONN_FLAG_ROW_KERNELS 2u
 #define SLONN_FLAG_COLUMN_KERNELS 4u
-#define SLONN_FLAG_ALL 7u
+/*
+ * The row kernels take the queries of a large batch four per block, so that a weight row most of the four
+ * selected is loaded once for all of them (the batch formulation of Sec. 7).  This flag keeps every query in
+ * a block of its own (results are identical; for testing and tuning).
+ */
+#define SLONN_FLAG_UNGROUPED_ROWS 8u
+#define SLONN_FLAG_ALL 15u
 
 #define SLONN_PATH_AUTO 0    /* library chooses                                               */
 #define SLONN_PATH_STAGED 1  /* one block per query and stage: any width, any batch size      */
@@ -399,7 +405,8 @@ int slonn_run_static(const slonn_model *m, const slonn_batch *batch, void *strea
 #define SLONN_STAGE_GATHER_COLS 8   /* selected nodes' dot products, input-stationary kernel */
 #define SLONN_STAGE_LAYER_COLS 9    /* all of 1 and 8 for a list-fed activator layer in one launch */
 #define SLONN_STAGE_FULL_ROWS 10    /* every layer of the 100 % budget queries, four queries per block */
-#define SLONN_N_STAGES 11
+#define SLONN_STAGE_GROUP_ROWS 11   /* selected rows' dot products, four queries per block   */
+#define SLONN_N_STAGES 12
 int slonn_run_timed(const slonn_model *m, const slonn_batch *batch, void *workspace,
                     uint64_t workspace_bytes, void *stream, float *stage_ms,
                     uint32_t *stage_launches);

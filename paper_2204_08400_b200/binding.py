@@ -442,11 +442,13 @@ def slonn_run_static(model: Model, batch: _Batch, stream=None) -> None:
         raise SlonnError(rc, "slonn_run_static")
 
 
-STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused", "dense_tc", "cluster", "gather_cols", "layer_cols", "full_rows")
+STAGES = ("plan", "hash_select", "gather_dot", "sparse_first", "argmax", "fused", "dense_tc", "cluster", "gather_cols", "layer_cols", "full_rows",
+          "group_rows")
 COLS_MAX_BP = 3500   # SLONN_COLS_MAX_BP
 FLAG_DENSE_TC = 1
 FLAG_ROW_KERNELS = 2
 FLAG_COLUMN_KERNELS = 4
+FLAG_UNGROUPED_ROWS = 8
 PATH_AUTO, PATH_STAGED, PATH_FUSED, PATH_CLUSTER = 0, 1, 2, 3
 
 

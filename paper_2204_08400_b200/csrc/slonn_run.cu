@@ -188,6 +188,9 @@ int launch_gather_short_t(const slonn_gather_params &P, uint64_t grid, size_t sm
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
+#ifndef SLONN_GATHER_R
+#define SLONN_GATHER_R 4 // rows per warp pass of the row kernel for rows longer than one 512-byte round (4 or 8)
+#endif
 int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint32_t max_rows, cudaStream_t st)
 {
     // so few rows that the GPU cannot be filled: latency variant, 4 warps per block, one row per warp
@@ -199,7 +202,7 @@ int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint
         P.rows_per_cta = 4;
         P.ctas_per_query = (max_rows + 3) / 4;
     } else {
-        gather_shape(n, max_rows, short_rows ? 32u : 4u, &P.rows_per_cta, &P.ctas_per_query);
+        gather_shape(n, max_rows, short_rows ? 32u : (uint32_t)SLONN_GATHER_R, &P.rows_per_cta, &P.ctas_per_query);
     }
     const size_t smem = (size_t)P.D * 4;
     const uint64_t grid = (uint64_t)n * P.ctas_per_query;
@@ -207,7 +210,84 @@ int launch_gather(const slonn_model *m, slonn_gather_params &P, uint32_t n, uint
     const bool bf = m->dtype == SLONN_BF16;
     if (lat) return bf ? launch_gather_t<true, true, 4>(P, grid, threads, smem, st) : launch_gather_t<false, true, 4>(P, grid, threads, smem, st);
     if (short_rows) return bf ? launch_gather_short_t<true>(P, grid, smem, st) : launch_gather_short_t<false>(P, grid, smem, st);
-    return bf ? launch_gather_t<true, false, 4>(P, grid, threads, smem, st) : launch_gather_t<false, false, 4>(P, grid, threads, smem, st);
+    return bf ? launch_gather_t<true, false, SLONN_GATHER_R>(P, grid, threads, smem, st)
+              : launch_gather_t<false, false, SLONN_GATHER_R>(P, grid, threads, smem, st);
+}
+
+// ---- selected rows, four queries per block --------------------------------------
+
+struct group_ws { uint32_t *list, *count; }; // workspace for the compacted list of the queries a launch serves
+
+template <bool BF16>
+int launch_group_rows_t(const slonn_group_params &Q, uint64_t grid, size_t smem, cudaStream_t st)
+{
+    const int rc = set_smem(group_rows_kernel<BF16>, smem);
+    if (rc) return rc;
+    group_rows_kernel<BF16><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(Q);
+    return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+}
+
+size_t group_rows_smem(const slonn_gather_params &P, uint32_t max_rows, uint32_t *shared_cap)
+{
+    const uint32_t nwords = (P.N + 31u) / 32u;
+    *shared_cap = std::min<uint64_t>(P.N, (uint64_t)4 * max_rows / 3 + 1);
+    return (size_t)SLONN_GROUP * P.D * 4 + (size_t)(2 * SLONN_GROUP + 1) * nwords * 4 + (size_t)((*shared_cap + 7u) & ~7u) * 2 +
+           (size_t)SLONN_GROUP * ((max_rows + 7u) & ~7u) * 2;
+}
+
+// The selected rows of a list-selecting layer for the queries in P's budget range.  In a large batch the queries
+// whose budget exceeds SLONN_GROUP_MIN_BP are taken four per block (rows that most of the four selected are loaded
+// once for all of them): at such budgets any four queries share most of their rows.  Below that, and for small
+// batches, layers of more than 65,535 nodes, rows of a single 512-byte round and shapes whose staging does not
+// fit two blocks per SM, every query has a block (or several) of its own.  Same values either way.
+// Measured on a 4096-wide layer with 4096 queries: 50 % budget 3.5 -> 2.8 ms per layer, 25 % 1.77 -> 1.68 ms,
+// 10 % 0.72 -> 0.79 ms (hence the limit).
+#ifndef SLONN_GROUP_MIN_BP
+#define SLONN_GROUP_MIN_BP 2000u
+#endif
+int launch_rows(const slonn_model *m, slonn_gather_params &P, const slonn_batch *b, uint32_t n, uint32_t max_bp,
+                uint32_t max_rows, const group_ws &gw, cudaStream_t st, stage_timer *tm)
+{
+    uint32_t shared_cap = 0;
+    const size_t smem = group_rows_smem(P, max_rows, &shared_cap);
+    const uint32_t lo = P.range_bp ? P.bp_lo : 0u, hi = std::min(P.range_bp ? P.bp_hi : 0xffffu, max_bp);
+    const uint32_t split = std::max(lo, SLONN_GROUP_MIN_BP + 1u); // budgets from here on are grouped
+    const bool grouped = P.use_list && n >= 256 && P.N <= 65535u && P.nchunks > 32 && gw.list && smem <= 110 * 1024 &&
+                         !(b->flags & SLONN_FLAG_UNGROUPED_ROWS) && hi >= split;
+    int rc;
+    if (!grouped) {
+        TIC(SLONN_STAGE_GATHER_DOT, P.range_bp, P.bp_lo, P.bp_hi, P.skip_bp);
+        rc = launch_gather(m, P, n, max_rows, st);
+        TOC();
+        return rc;
+    }
+    if (lo < split) { // the low budgets of this launch: one query per block
+        slonn_gather_params A = P;
+        A.range_bp = b->budget_bp; A.bp_lo = lo; A.bp_hi = split - 1u;
+        TIC(SLONN_STAGE_GATHER_DOT, A.range_bp, A.bp_lo, A.bp_hi, A.skip_bp);
+        rc = launch_gather(m, A, n, std::min(max_rows, slonn_layer_nodes(split - 1u, P.N, slonn_model_pre(m))), st);
+        TOC();
+        if (rc) return rc;
+    }
+    // the others, compacted in two budget classes so that the queries of a group select about as many rows
+    if (cudaMemsetAsync(gw.count, 0, sizeof(uint32_t), st) != cudaSuccess) return SLONN_ERR_CUDA;
+    const uint32_t mid = 3750u;
+    if (split <= mid)
+        range_compact_kernel<<<(n + 255) / 256, 256, 0, st>>>(b->budget_bp, P.skip_bp, n, split, std::min(mid, hi), gw.list, gw.count);
+    if (hi > mid)
+        range_compact_kernel<<<(n + 255) / 256, 256, 0, st>>>(b->budget_bp, P.skip_bp, n, std::max(split, mid + 1u), hi, gw.list, gw.count);
+    if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+    slonn_group_params Q;
+    memset(&Q, 0, sizeof(Q));
+    Q.G = P; Q.list = gw.list; Q.count = gw.count; Q.rows_cap = max_rows; Q.shared_cap = shared_cap;
+    const uint32_t groups = (n + SLONN_GROUP - 1) / SLONN_GROUP;
+    // enough blocks for a few waves of two per SM, but no block with fewer than 32 rows of each kind
+    Q.ctas_per_group = std::max(1u, std::min(std::min(8u, (148u * 8u + groups - 1) / groups), max_rows / 32u));
+    TIC(SLONN_STAGE_GROUP_ROWS, b->budget_bp, split, hi, P.skip_bp);
+    rc = m->dtype == SLONN_BF16 ? launch_group_rows_t<true>(Q, (uint64_t)groups * Q.ctas_per_group, smem, st)
+                                : launch_group_rows_t<false>(Q, (uint64_t)groups * Q.ctas_per_group, smem, st);
+    TOC();
+    return rc;
 }
 
 // Input-stationary gather for a layer fed by (id, value) lists: 32 * R nodes per warp pass, the passes of
@@ -325,8 +405,8 @@ uint32_t cols_budget_limit(const slonn_layer &ly, const slonn_gather_params &P, 
 // whose input list is sparse (by budget), the row kernel for the others.  Results do not depend on the split.
 // rows_done: the queries above the input-stationary limit were served by another launch already.
 int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_params &P, const slonn_batch *b,
-                      uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st, stage_timer *tm,
-                      bool rows_done = false)
+                      uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, const group_ws &gw, cudaStream_t st,
+                      stage_timer *tm, bool rows_done = false)
 {
     const uint32_t cols_bp = cols_budget_limit(ly, P, b, n, max_rows, max_bp);
     int rc;
@@ -350,10 +430,7 @@ int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_
             P.range_bp = b->budget_bp; P.bp_lo = 0; P.bp_hi = cols_bp;
         }
     }
-    TIC(SLONN_STAGE_GATHER_DOT, P.range_bp, P.bp_lo, P.bp_hi, P.skip_bp);
-    rc = launch_gather(m, P, n, max_rows, st);
-    TOC();
-    return rc;
+    return launch_rows(m, P, b, n, max_bp, max_rows, gw, st, tm);
 }
 
 // An activator layer: FreeHash, selection and the selected nodes.  A list-fed layer with the copies for it
@@ -361,8 +438,8 @@ int launch_layer_rows(const slonn_model *m, const slonn_layer &ly, slonn_gather_
 // every query where that launch does not apply) take the selection kernel followed by the row or
 // input-stationary gather.
 int launch_act_layer(const slonn_model *m, const slonn_layer &ly, uint32_t l, slonn_select_params &sp, slonn_gather_params &gp,
-                     const slonn_batch *b, uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, cudaStream_t st,
-                     stage_timer *tm)
+                     const slonn_batch *b, uint32_t n, uint32_t max_bp, uint32_t max_rows, uint32_t in_cap, const group_ws &gw,
+                     cudaStream_t st, stage_timer *tm)
 {
     int rc;
     const uint32_t cols_bp = cols_budget_limit(ly, gp, b, n, max_rows, max_bp);
@@ -385,10 +462,7 @@ int launch_act_layer(const slonn_model *m, const slonn_layer &ly, uint32_t l, sl
             TOC();
             if (rc) return rc;
             gp.range_bp = b->budget_bp; gp.bp_lo = cols_bp + 1; gp.bp_hi = 0xffffu;
-            TIC(SLONN_STAGE_GATHER_DOT, gp.range_bp, gp.bp_lo, gp.bp_hi, gp.skip_bp);
-            rc = launch_gather(m, gp, n, max_rows, st);
-            TOC();
-            return rc;
+            return launch_rows(m, gp, b, n, max_bp, max_rows, gw, st, tm);
         }
         if (rc != SLONN_ERR_DIM) return rc;
     }
@@ -396,7 +470,7 @@ int launch_act_layer(const slonn_model *m, const slonn_layer &ly, uint32_t l, sl
     rc = launch_select(m, sp, n, max_rows, st);
     TOC();
     if (rc) return rc;
-    return launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st, tm);
+    return launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, gw, st, tm);
 }
 
 // ---- 100 % queries, four per block ---------------------------------------------
@@ -887,6 +961,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     in.dense = b->x_dense;
     int dense_cur = 0;
     uint32_t in_cap = 0; // most entries the current input list holds (list inputs only)
+    const group_ws gw = {(uint32_t *)(ws + wl.tc_list), (uint32_t *)(ws + wl.tc_count)};
 
     for (uint32_t l = 0; l < m->n_layers; ++l) {
         const slonn_layer &ly = m->layer[l];
@@ -926,7 +1001,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
             max_rows = slonn_layer_nodes(max_bp, ly.N, slonn_model_pre(m));
             gp.use_list = 1; gp.a = a; gp.out_vals = vals;
             if (is_last) { gp.out_dense = b->logits; gp.out_dense_ids = b->logit_ids; gp.out_stride = stride; }
-            rc = launch_act_layer(m, ly, l, sp, gp, b, n, max_bp, max_rows, in_cap, st, tm);
+            rc = launch_act_layer(m, ly, l, sp, gp, b, n, max_bp, max_rows, in_cap, gw, st, tm);
             if (rc) return rc;
             in.kind = SLONN_IN_LIST; in.indptr = indptr; in.ids = ids; in.vals = vals;
             in.ip_mul = m->n_act; in.ip_add = a;
@@ -958,7 +1033,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
                 if (rc) return rc;
                 rows_done = true;
             }
-            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, st, tm, rows_done);
+            rc = launch_layer_rows(m, ly, gp, b, n, max_bp, max_rows, in_cap, gw, st, tm, rows_done);
             if (rc) return rc;
             in.kind = SLONN_IN_DENSE; in.dense = gp.out_dense;
             dense_cur ^= 1;

@@ -572,6 +572,201 @@ __global__ void __launch_bounds__(SLONN_THREADS, SLONN_FULL_MIN_BLOCKS) full_row
     }
 }
 
+// Selected rows of a layer for queries taken FOUR AT A TIME (the batch formulation the paper leaves open in
+// Sec. 7): the importance rankings of all buckets start with much the same nodes, so the active sets of any four
+// queries overlap heavily.  A block stages four inputs, marks each query's active set in a bitmap and splits the
+// union of the four sets in two:
+//   rows that at least three of the four queries selected -- evaluated once for all four, every 16-byte weight
+//     chunk a lane loads feeding four queries' partial sums (the result of a query that did not select the row is
+//     dropped);
+//   the other rows -- evaluated for the queries that selected them, one query at a time.
+// Each (query, row) sum is formed in the library's fixed order either way, so the values are those of
+// gather_dot_kernel bit for bit; they are written to the row's place in the query's id-ascending list, which is
+// the popcount of the query's bitmap below the row.
+// `list` / `count`: the queries this launch serves (range_compact_kernel); group g = entries 4g .. 4g + 3.
+struct slonn_group_params {
+    slonn_gather_params G;    // in, W, bias, D, N, nchunks, n_act, a, indptr, ids, out_vals, out_dense(_ids), out_stride, relu
+    const uint32_t *list;
+    const uint32_t *count;
+    uint32_t ctas_per_group;  // blocks that share a group's rows
+    uint32_t rows_cap;        // most rows a query of this launch selects
+    uint32_t shared_cap;      // entries of the shared-row list: min(N, 4 * rows_cap / 3 + 1)
+};
+
+#define SLONN_GROUP 4
+#ifndef SLONN_GROUP_MIN_BLOCKS
+#define SLONN_GROUP_MIN_BLOCKS 2
+#endif
+
+template <bool BF16>
+__global__ void __launch_bounds__(SLONN_THREADS, SLONN_GROUP_MIN_BLOCKS) group_rows_kernel(slonn_group_params Q)
+{
+    extern __shared__ float4 smem4[];
+    constexpr int VPC = BF16 ? 8 : 4;
+    constexpr int G = SLONN_GROUP, R = 4;
+    const slonn_gather_params &P = Q.G;
+    __shared__ uint64_t scan_ws[32];
+    __shared__ uint64_t scan_total;
+    const uint32_t g = blockIdx.x / Q.ctas_per_group;
+    const uint32_t chunk = blockIdx.x - g * Q.ctas_per_group;
+    const uint32_t cnt = *Q.count;
+    if (g * G >= cnt) return;
+    const uint32_t nq = min((uint32_t)G, cnt - g * G);
+    const uint32_t per_q = (BF16 ? 2u : 1u) * P.nchunks; // float4 per staged input
+    const uint32_t nwords = (P.N + 31u) >> 5;
+
+    // shared memory: four staged inputs | four bitmaps | shared-row bitmap | four position prefixes |
+    // shared-row list | four lists of a query's other rows
+    uint32_t *bm = reinterpret_cast<uint32_t *>(smem4 + G * per_q);
+    uint32_t *shbits = bm + G * nwords;
+    uint32_t *pre = shbits + nwords;
+    uint16_t *shlist = reinterpret_cast<uint16_t *>(pre + G * nwords);
+    uint16_t *rem = shlist + ((Q.shared_cap + 7u) & ~7u);
+    const uint32_t rem_stride = (Q.rows_cap + 7u) & ~7u;
+
+    uint32_t q[G], B[G];
+    uint64_t off[G];
+#pragma unroll
+    for (int k = 0; k < G; ++k) {
+        q[k] = __ldg(Q.list + g * G + min((uint32_t)k, nq - 1)); // a short last group repeats its last query
+        off[k] = P.indptr[(uint64_t)q[k] * P.n_act + P.a];
+        B[k] = min((uint32_t)(P.indptr[(uint64_t)q[k] * P.n_act + P.a + 1] - off[k]), Q.rows_cap);
+        stage_input<BF16>(P.in, q[k], P.D, P.nchunks, smem4 + k * per_q);
+    }
+    for (uint32_t i = threadIdx.x; i < G * nwords; i += blockDim.x) bm[i] = 0u;
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < G; ++k)
+        if ((uint32_t)k < nq)
+            for (uint32_t i = threadIdx.x; i < B[k]; i += blockDim.x) {
+                const uint32_t id = min(__ldg(P.ids + off[k] + i), P.N - 1u);
+                atomicOr(&bm[k * nwords + (id >> 5)], 1u << (id & 31u));
+            }
+    __syncthreads();
+
+    // per bitmap word: the rows at least three queries want, each query's other rows; counts -> offsets
+    const uint32_t wpt = (nwords + blockDim.x - 1) / blockDim.x;
+    const uint32_t w0 = threadIdx.x * wpt, w1 = min(w0 + wpt, nwords);
+    uint64_t c_all = 0, c_rem = 0; // four 16-bit counts each (N <= 65535)
+    uint32_t c_sh = 0;
+    for (uint32_t w = w0; w < w1; ++w) {
+        const uint32_t b0 = bm[w], b1 = bm[nwords + w], b2 = bm[2 * nwords + w], b3 = bm[3 * nwords + w];
+        const uint32_t s = (b0 & b1 & (b2 | b3)) | (b2 & b3 & (b0 | b1));
+        shbits[w] = s;
+        c_sh += __popc(s);
+        c_all += (uint64_t)__popc(b0) | ((uint64_t)__popc(b1) << 16) | ((uint64_t)__popc(b2) << 32) | ((uint64_t)__popc(b3) << 48);
+        c_rem += (uint64_t)__popc(b0 & ~s) | ((uint64_t)__popc(b1 & ~s) << 16) | ((uint64_t)__popc(b2 & ~s) << 32) |
+                 ((uint64_t)__popc(b3 & ~s) << 48);
+    }
+    uint64_t o_all = block_exclusive_scan<uint64_t>(c_all, scan_ws, &scan_total);
+    uint64_t o_rem = block_exclusive_scan<uint64_t>(c_rem, scan_ws, &scan_total);
+    const uint64_t rem_total = scan_total;
+    uint64_t o_sh = block_exclusive_scan<uint64_t>((uint64_t)c_sh, scan_ws, &scan_total);
+    const uint32_t n_sh = (uint32_t)scan_total;
+    for (uint32_t w = w0; w < w1; ++w) {
+        const uint32_t s = shbits[w];
+        uint32_t bits = s;
+        while (bits) {
+            const uint32_t t = __ffs(bits) - 1;
+            bits &= bits - 1;
+            if (o_sh < Q.shared_cap) shlist[o_sh] = (uint16_t)((w << 5) + t);
+            ++o_sh;
+        }
+#pragma unroll
+        for (int k = 0; k < G; ++k) {
+            const uint32_t b = bm[k * nwords + w];
+            pre[k * nwords + w] = (uint32_t)(o_all >> (16 * k)) & 0xffffu;
+            uint32_t o = (uint32_t)(o_rem >> (16 * k)) & 0xffffu;
+            bits = b & ~s;
+            while (bits) {
+                const uint32_t t = __ffs(bits) - 1;
+                bits &= bits - 1;
+                if (o < Q.rows_cap) rem[k * rem_stride + o] = (uint16_t)((w << 5) + t);
+                ++o;
+            }
+            o_all += (uint64_t)__popc(b) << (16 * k);
+            o_rem += (uint64_t)__popc(b & ~s) << (16 * k);
+        }
+    }
+    __syncthreads();
+
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    auto emit = [&](int k, uint32_t n, float sum) { // row n of query k, if the query selected it
+        const uint32_t word = bm[k * nwords + (n >> 5)], bit = 1u << (n & 31u);
+        if (!(word & bit)) return;
+        const uint32_t pos = pre[k * nwords + (n >> 5)] + __popc(word & (bit - 1u));
+        float z = sum + __ldg(P.bias + n);
+        if (P.relu) z = z > 0.0f ? z : 0.0f;
+        if (P.out_vals) P.out_vals[off[k] + pos] = z;
+        if (P.out_dense) {
+            P.out_dense[(uint64_t)q[k] * P.out_stride + pos] = z;
+            if (P.out_dense_ids) P.out_dense_ids[(uint64_t)q[k] * P.out_stride + pos] = n;
+        }
+    };
+
+    // (A) the rows at least three of the four queries selected: one weight load feeds four sums
+    {
+        const uint32_t per = (n_sh + Q.ctas_per_group - 1) / Q.ctas_per_group;
+        const uint32_t a0 = min(chunk * per, n_sh), a1 = min(a0 + per, n_sh);
+        for (uint32_t r = a0 + warp * R; r < a1; r += nwarps * R) {
+            const uint4 *rows[R];
+#pragma unroll
+            for (int j = 0; j < R; ++j)
+                rows[j] = reinterpret_cast<const uint4 *>(P.W) + (uint64_t)shlist[min(r + j, a1 - 1)] * P.nchunks;
+            float acc[G][R];
+#pragma unroll
+            for (int k = 0; k < G; ++k)
+#pragma unroll
+                for (int j = 0; j < R; ++j) acc[k][j] = 0.0f;
+            for (uint32_t c = lane; c < P.nchunks; c += 32) {
+                uint4 w[R];
+#pragma unroll
+                for (int j = 0; j < R; ++j) w[j] = __ldg(rows[j] + c);
+#pragma unroll
+                for (int k = 0; k < G; ++k) {
+                    const float4 *xs4 = smem4 + k * per_q;
+                    float x[VPC];
+                    const float4 xa = xs4[c];
+                    x[0] = xa.x; x[1] = xa.y; x[2] = xa.z; x[3] = xa.w;
+                    if (BF16) {
+                        const float4 xb = xs4[P.nchunks + c];
+                        x[VPC - 4] = xb.x; x[VPC - 3] = xb.y; x[VPC - 2] = xb.z; x[VPC - 1] = xb.w;
+                    }
+                    chunk_fma<BF16, R, 0, VPC>::run(w, x, acc[k]);
+                }
+            }
+            const uint32_t mr = r + (lane >> 3);
+            const uint32_t n = shlist[min(mr, a1 - 1)];
+#pragma unroll
+            for (int k = 0; k < G; ++k) {
+                const float sum = reduce_rows4(acc[k], lane); // row r + (lane >> 3)
+                if ((lane & 7u) == 0u && mr < a1 && (uint32_t)k < nq) emit(k, n, sum);
+            }
+        }
+    }
+    // (B) every query's other rows, one query at a time
+#pragma unroll
+    for (int k = 0; k < G; ++k) {
+        if ((uint32_t)k >= nq) break;
+        const uint32_t n_rem = min((uint32_t)(rem_total >> (16 * k)) & 0xffffu, Q.rows_cap);
+        const uint32_t per = (n_rem + Q.ctas_per_group - 1) / Q.ctas_per_group;
+        const uint32_t a0 = min(chunk * per, n_rem), a1 = min(a0 + per, n_rem);
+        const uint16_t *mine = rem + k * rem_stride;
+        const float4 *xs4 = smem4 + k * per_q;
+        for (uint32_t r = a0 + warp * R; r < a1; r += nwarps * R) {
+            const uint4 *rows[R];
+#pragma unroll
+            for (int j = 0; j < R; ++j)
+                rows[j] = reinterpret_cast<const uint4 *>(P.W) + (uint64_t)mine[min(r + j, a1 - 1)] * P.nchunks;
+            float acc[R];
+            warp_dot_rows<BF16, R>(rows, xs4, P.nchunks, lane, acc);
+            const float sum = reduce_rows4(acc, lane); // row r + (lane >> 3)
+            const uint32_t mr = r + (lane >> 3);
+            if ((lane & 7u) == 0u && mr < a1) emit(k, mine[mr], sum);
+        }
+    }
+}
+
 // Rows of at most one 512-byte round (one 16-byte chunk per lane): the lane's piece of the input is
 // loaded once and kept in registers, a warp fetches 32 row ids with one coalesced load and works
 // through them 8 rows at a time, so that the only loads inside the loop are the weight chunks

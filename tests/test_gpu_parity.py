@@ -53,7 +53,9 @@ def check(wl, n_cal=None, sample=None, expect_build=True, models=None):
     for path in kernel_paths(wl):
         # the per-stage and one-warp-per-query kernels evaluate a sparse-input layer row-wise or
         # input-wise: library's choice, then each kind forced for the whole batch
-        for flags in ((0, sl.FLAG_ROW_KERNELS, sl.FLAG_COLUMN_KERNELS) if path in (1, 2) else (0,)):
+        # (and, for the per-stage row kernels, every query in a block of its own instead of four per block)
+        for flags in ((0, sl.FLAG_ROW_KERNELS, sl.FLAG_COLUMN_KERNELS) + ((sl.FLAG_ROW_KERNELS | sl.FLAG_UNGROUPED_ROWS,) if path == 1 else ())
+                      if path in (1, 2) else (0,)):
             g = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=path, flags=flags)
             if sample is not None:
                 g = slice_results(g, sample, n_act)
