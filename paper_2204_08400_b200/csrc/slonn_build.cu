@@ -118,14 +118,14 @@ __global__ void popularity_kernel(const IDT *tables, uint64_t n_lists, uint32_t 
 //   WH      [D][32] the layer's hash rows side by side (activator layers with K*L <= 32)
 // and the plain transposed copy of a first layer fed by CSR rows.  phase 0: the CSR first layer (needed
 // by the calibration pass); phase 1: the rest (needs the finished tables).
-// Copies whose element index would not fit 32 bits are left out (such layers keep the row kernels).
+// Copies of 4 GiB or more are left out: the kernels address them with 32-bit byte offsets (such layers keep the row kernels).
 int make_transposed_copies(slonn_model *m, cudaStream_t st, int phase)
 {
     const uint32_t esz = m->dtype == SLONN_BF16 ? 2u : 4u;
     for (uint32_t l = 0; l < m->n_layers; ++l) {
         slonn_layer &ly = m->layer[l];
         const bool csr_first = (l == 0 && m->first_sparse);
-        const bool list_input = (l > 0 && m->layer[l - 1].has_act && (uint64_t)ly.N * ly.D < (1ull << 32));
+        const bool list_input = (l > 0 && m->layer[l - 1].has_act && (uint64_t)ly.N * ly.D * esz < (1ull << 32));
         if (phase == 0 ? !csr_first : !list_input) continue;
         if (cudaMalloc(&ly.WT, (uint64_t)ly.N * ly.D * esz) != cudaSuccess) return SLONN_ERR_NOMEM;
         const dim3 grid((ly.D + 31) / 32, (ly.N + 31) / 32), block(32, 8);

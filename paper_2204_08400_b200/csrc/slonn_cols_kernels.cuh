@@ -117,6 +117,32 @@ __device__ __forceinline__ float cols_weight(const void *WT, uint32_t idx)
     return __ldg(reinterpret_cast<const float *>(WT) + idx);
 }
 
+// The weight `off` BYTES into WT.  Offsets are 32-bit (a transposed copy is kept only for layers of less
+// than 4 GiB), so an address is the matrix base plus one 32-bit sum per load.
+template <bool BF16>
+__device__ __forceinline__ float cols_weight_at(const void *WT, uint32_t off)
+{
+    const char *p = reinterpret_cast<const char *>(WT) + off;
+    if (BF16) return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p)) << 16);
+    return __ldg(reinterpret_cast<const float *>(p));
+}
+
+// Two neighbouring weights with one load, the first `off` bytes into WT (a multiple of two element sizes).
+template <bool BF16>
+__device__ __forceinline__ void cols_weight2_at(const void *WT, uint32_t off, float &w0, float &w1)
+{
+    const char *p = reinterpret_cast<const char *>(WT) + off;
+    if (BF16) {
+        const uint32_t u = __ldg(reinterpret_cast<const uint32_t *>(p));
+        w0 = __uint_as_float(u << 16);
+        w1 = __uint_as_float(u & 0xffff0000u);
+    } else {
+        const float2 v = __ldg(reinterpret_cast<const float2 *>(p));
+        w0 = v.x;
+        w1 = v.y;
+    }
+}
+
 // Two neighbouring weights WT[idx], WT[idx + 1] with one load; idx even.
 template <bool BF16>
 __device__ __forceinline__ void cols_weight2(const void *WT, uint32_t idx, float &w0, float &w1)
@@ -158,6 +184,11 @@ __device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, u
                                           float (&sum)[R])
 {
     float p0[R], p1[R], p2[R], p3[R], p4[R];
+    constexpr uint32_t ESZ = BF16 ? 2u : 4u;
+    const uint32_t ldb = ld * ESZ; // bytes per row of WT
+    uint32_t cb[R];                // byte offset of each node's column
+#pragma unroll
+    for (int r = 0; r < R; ++r) cb[r] = col[r] * ESZ;
 #ifndef SLONN_COLS_UNROLL
 #define SLONN_COLS_UNROLL 32 // measured: full unrolling of the segment loop beats 1, 4 and 8
 #endif
@@ -177,18 +208,19 @@ __device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, u
         for (; k < e; k += 4) {
             const uint4 e0 = *reinterpret_cast<const uint4 *>(S.ent + k), e1 = *reinterpret_cast<const uint4 *>(S.ent + k + 2);
             float w[R][4];
+            const uint32_t t0 = e0.x * ldb, t1 = e0.z * ldb, t2 = e1.x * ldb, t3 = e1.z * ldb; // row offsets
             if constexpr (PAIR) {
-                cols_weight2<BF16>(WT, e0.x * ld + col[0], w[0][0], w[R - 1][0]);
-                cols_weight2<BF16>(WT, e0.z * ld + col[0], w[0][1], w[R - 1][1]);
-                cols_weight2<BF16>(WT, e1.x * ld + col[0], w[0][2], w[R - 1][2]);
-                cols_weight2<BF16>(WT, e1.z * ld + col[0], w[0][3], w[R - 1][3]);
+                cols_weight2_at<BF16>(WT, t0 + cb[0], w[0][0], w[R - 1][0]);
+                cols_weight2_at<BF16>(WT, t1 + cb[0], w[0][1], w[R - 1][1]);
+                cols_weight2_at<BF16>(WT, t2 + cb[0], w[0][2], w[R - 1][2]);
+                cols_weight2_at<BF16>(WT, t3 + cb[0], w[0][3], w[R - 1][3]);
             } else {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    w[r][0] = cols_weight<BF16>(WT, e0.x * ld + col[r]);
-                    w[r][1] = cols_weight<BF16>(WT, e0.z * ld + col[r]);
-                    w[r][2] = cols_weight<BF16>(WT, e1.x * ld + col[r]);
-                    w[r][3] = cols_weight<BF16>(WT, e1.z * ld + col[r]);
+                    w[r][0] = cols_weight_at<BF16>(WT, t0 + cb[r]);
+                    w[r][1] = cols_weight_at<BF16>(WT, t1 + cb[r]);
+                    w[r][2] = cols_weight_at<BF16>(WT, t2 + cb[r]);
+                    w[r][3] = cols_weight_at<BF16>(WT, t3 + cb[r]);
                 }
             }
 #pragma unroll
