@@ -478,9 +478,9 @@ int launch_act_layer(const slonn_model *m, const slonn_layer &ly, uint32_t l, sl
 template <bool BF16>
 int launch_full_rows_t(const slonn_full_params &P, uint64_t grid, size_t smem, cudaStream_t st)
 {
-    const int rc = set_smem(full_rows_kernel<BF16>, smem);
+    const int rc = set_smem(full_rows_kernel<BF16, SLONN_FULL_R>, smem);
     if (rc) return rc;
-    full_rows_kernel<BF16><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(P);
+    full_rows_kernel<BF16, SLONN_FULL_R><<<(uint32_t)grid, SLONN_THREADS, smem, st>>>(P);
     return cudaGetLastError() == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 

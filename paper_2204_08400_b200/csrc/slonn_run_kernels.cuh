@@ -493,15 +493,18 @@ struct slonn_full_params {
 
 #define SLONN_FULL_GROUP 4
 #ifndef SLONN_FULL_MIN_BLOCKS
-#define SLONN_FULL_MIN_BLOCKS 3 // 80 registers; measured 10 % faster than 2 blocks at 115
+#define SLONN_FULL_MIN_BLOCKS 2 // with 8 rows per pass (123 registers); 4 rows: 3 blocks at 80 registers beat 2 at 115
 #endif
 
-template <bool BF16>
+#ifndef SLONN_FULL_R
+#define SLONN_FULL_R 8 // rows per warp pass (4 or 8); measured on 2048-4096-4096-1000 at 100 %: 15.2 ms with 4, 14.7 with 8
+#endif
+template <bool BF16, int R>
 __global__ void __launch_bounds__(SLONN_THREADS, SLONN_FULL_MIN_BLOCKS) full_rows_kernel(slonn_full_params P)
 {
     extern __shared__ float4 smem4[];
     constexpr int VPC = BF16 ? 8 : 4;
-    constexpr int G = SLONN_FULL_GROUP, R = 4;
+    constexpr int G = SLONN_FULL_GROUP;
     const uint32_t g = blockIdx.x / P.ctas_per_group;
     const uint32_t chunk = blockIdx.x - g * P.ctas_per_group;
     const uint32_t cnt = *P.count;
@@ -549,12 +552,15 @@ __global__ void __launch_bounds__(SLONN_THREADS, SLONN_FULL_MIN_BLOCKS) full_row
                 chunk_fma<BF16, R, 0, VPC>::run(w, x, acc[k]);
             }
         }
-        const uint32_t mr = r + (lane >> 3);
+        const uint32_t mr = r + (R == 8 ? (lane >> 2) : (lane >> 3));
+        const bool writer = R == 8 ? (lane & 3u) == 0u : (lane & 7u) == 0u;
         const float b = __ldg(P.bias + min(mr, P.N - 1u));
 #pragma unroll
         for (int k = 0; k < G; ++k) {
-            const float sum = reduce_rows4(acc[k], lane); // row r + (lane >> 3)
-            if ((lane & 7u) == 0u && mr < r1 && (uint32_t)k < nq) {
+            float sum;
+            if constexpr (R == 8) sum = reduce_rows8(acc[k], lane); // row r + (lane >> 2)
+            else sum = reduce_rows4(acc[k], lane);                  // row r + (lane >> 3)
+            if (writer && mr < r1 && (uint32_t)k < nq) {
                 float z = sum + b;
                 if (P.relu) z = z > 0.0f ? z : 0.0f;
                 if (P.has_act) {
