@@ -158,6 +158,57 @@ __device__ __forceinline__ void cols_weight2(const void *WT, uint32_t idx, float
     }
 }
 
+// Entries [k, e) of one segment of the staged list (a multiple of four) for R nodes per lane:
+// a[r] = fmaf(weight(row of the entry, column byte offset cb[r]), value of the entry, a[r]), entries in order.
+// ldb: bytes per row of WT.  DEEP: eight entries at a time while the segment has that many left (8 * R loads
+// in flight instead of 4 * R) -- for launches in which a block's chain of dependent loads, not the number of
+// resident warps, sets the pace.
+template <bool BF16, int R, bool DEEP>
+__device__ __forceinline__ void cols_segment(const uint2 *ent, uint32_t k, uint32_t e, const void *WT, uint32_t ldb,
+                                             const uint32_t (&cb)[R], float (&a)[R])
+{
+    if (DEEP) {
+        for (; k + 8 <= e; k += 8) {
+            uint4 q[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) q[i] = *reinterpret_cast<const uint4 *>(ent + k + 2 * i);
+            float w[R][8];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    w[r][2 * i] = cols_weight_at<BF16>(WT, q[i].x * ldb + cb[r]);
+                    w[r][2 * i + 1] = cols_weight_at<BF16>(WT, q[i].z * ldb + cb[r]);
+                }
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    a[r] = fmaf(w[r][2 * i], __uint_as_float(q[i].y), a[r]);
+                    a[r] = fmaf(w[r][2 * i + 1], __uint_as_float(q[i].w), a[r]);
+                }
+        }
+    }
+    for (; k < e; k += 4) {
+        const uint4 e0 = *reinterpret_cast<const uint4 *>(ent + k), e1 = *reinterpret_cast<const uint4 *>(ent + k + 2);
+        float w[R][4];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            w[r][0] = cols_weight_at<BF16>(WT, e0.x * ldb + cb[r]);
+            w[r][1] = cols_weight_at<BF16>(WT, e0.z * ldb + cb[r]);
+            w[r][2] = cols_weight_at<BF16>(WT, e1.x * ldb + cb[r]);
+            w[r][3] = cols_weight_at<BF16>(WT, e1.z * ldb + cb[r]);
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            a[r] = fmaf(w[r][0], __uint_as_float(e0.y), a[r]);
+            a[r] = fmaf(w[r][1], __uint_as_float(e0.w), a[r]);
+            a[r] = fmaf(w[r][2], __uint_as_float(e1.y), a[r]);
+            a[r] = fmaf(w[r][3], __uint_as_float(e1.w), a[r]);
+        }
+    }
+}
+
 // a[0] + ... + a[31] in the fixed tree: strides 16, 8, 4, 2, 1
 __device__ __forceinline__ float cols_tree(float (&acc)[32])
 {

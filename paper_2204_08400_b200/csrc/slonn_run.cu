@@ -116,6 +116,9 @@ ws_layout carve(const slonn_model *m, uint32_t n, uint32_t max_bp, uint32_t flag
 template <typename K>
 int set_smem(K kernel, size_t bytes)
 {
+#ifdef SLONN_CARVEOUT
+    cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, SLONN_CARVEOUT);
+#endif
     if (bytes > 48 * 1024) {
         if (bytes > 227 * 1024) return SLONN_ERR_DIM;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)

@@ -387,7 +387,12 @@ struct slonn_gather_params {
 // R: rows per warp pass, 4 (6-shuffle reduction) or 8 (9 shuffles; pays off for rows of one
 // 512-byte round, where the reduction is most of the work).
 template <bool BF16, bool LAT, int R>
-__global__ void __launch_bounds__(SLONN_THREADS) gather_dot_kernel(slonn_gather_params P)
+#ifdef SLONN_GATHER_MIN_BLOCKS
+__launch_bounds__(SLONN_THREADS, SLONN_GATHER_MIN_BLOCKS)
+#else
+__launch_bounds__(SLONN_THREADS)
+#endif
+__global__ void gather_dot_kernel(slonn_gather_params P)
 {
     extern __shared__ float4 smem4[];
     const uint32_t q = blockIdx.x / P.ctas_per_query;
@@ -914,29 +919,15 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
                 if (!ordered) col[k] = nd[k];
             }
         }
+        constexpr uint32_t ESZ = BF16 ? 2u : 4u;
+        uint32_t cb[R];
+#pragma unroll
+        for (int k = 0; k < R; ++k) cb[k] = col[k] * ESZ;
         for (uint32_t p = warp; p < 32; p += nwarps) {
             float a[R];
 #pragma unroll
             for (int k = 0; k < R; ++k) a[k] = 0.0f;
-            const uint32_t end = S.segstart[p + 1];
-            for (uint32_t i = S.segstart[p]; i < end; i += 4) {
-                const uint4 e0 = *reinterpret_cast<const uint4 *>(S.ent + i), e1 = *reinterpret_cast<const uint4 *>(S.ent + i + 2);
-                float w[R][4];
-#pragma unroll
-                for (int k = 0; k < R; ++k) {
-                    w[k][0] = cols_weight<BF16>(P.WT, e0.x * P.N + col[k]);
-                    w[k][1] = cols_weight<BF16>(P.WT, e0.z * P.N + col[k]);
-                    w[k][2] = cols_weight<BF16>(P.WT, e1.x * P.N + col[k]);
-                    w[k][3] = cols_weight<BF16>(P.WT, e1.z * P.N + col[k]);
-                }
-#pragma unroll
-                for (int k = 0; k < R; ++k) {
-                    a[k] = fmaf(w[k][0], __uint_as_float(e0.y), a[k]);
-                    a[k] = fmaf(w[k][1], __uint_as_float(e0.w), a[k]);
-                    a[k] = fmaf(w[k][2], __uint_as_float(e1.y), a[k]);
-                    a[k] = fmaf(w[k][3], __uint_as_float(e1.w), a[k]);
-                }
-            }
+            cols_segment<BF16, R, true>(S.ent, S.segstart[p], S.segstart[p + 1], P.WT, P.N * ESZ, cb, a);
 #pragma unroll
             for (int k = 0; k < R; ++k) zpart[(p * R + k) * 32u + lane] = a[k];
         }
@@ -1026,7 +1017,12 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
 // SPLIT: the variant for batches of tens of queries -- one block per (query, 32 * R nodes), the segments
 // of the input list spread over the block's warps (see cols_order_and_gather).
 template <bool BF16, int R, bool SPLIT>
-__global__ void __launch_bounds__(SLONN_THREADS) gather_cols_kernel(slonn_gather_params P)
+#ifdef SLONN_GATHER_COLS_MIN_BLOCKS
+__launch_bounds__(SLONN_THREADS, SLONN_GATHER_COLS_MIN_BLOCKS)
+#else
+__launch_bounds__(SLONN_THREADS)
+#endif
+__global__ void gather_cols_kernel(slonn_gather_params P)
 {
     extern __shared__ float4 smem4[];
     constexpr int V = BF16 ? 8 : 4;
@@ -1082,7 +1078,10 @@ struct slonn_layer_cols_params {
 // in each; only the first block writes keys and list to global memory), then evaluates its 64 nodes with
 // the segments of the input list spread over its warps.
 template <bool BF16, typename IDT, bool SPLIT>
-__global__ void __launch_bounds__(SLONN_THREADS) layer_cols_kernel(slonn_layer_cols_params Q)
+#ifndef SLONN_LAYER_COLS_MIN_BLOCKS
+#define SLONN_LAYER_COLS_MIN_BLOCKS 6 // 40 registers: seven blocks of seven warps per SM (48 registers, five blocks: 2 % slower)
+#endif
+__global__ void __launch_bounds__(SLONN_THREADS, SLONN_LAYER_COLS_MIN_BLOCKS) layer_cols_kernel(slonn_layer_cols_params Q)
 {
     extern __shared__ float4 smem4[];
     constexpr int V = BF16 ? 8 : 4;
@@ -1123,19 +1122,14 @@ __global__ void __launch_bounds__(SLONN_THREADS) layer_cols_kernel(slonn_layer_c
     cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D);
 
     // (1) FreeHash: partial sum p of hash function `lane`, segments spread over the warps
-    for (uint32_t p = warp; p < 32; p += nwarps) {
-        float a = 0.0f;
-        const uint32_t e = segstart[p + 1];
-        for (uint32_t k = segstart[p]; k < e; k += 4) {
-            const uint4 e0 = *reinterpret_cast<const uint4 *>(S.ent + k), e1 = *reinterpret_cast<const uint4 *>(S.ent + k + 2);
-            const float w0 = cols_weight<BF16>(Q.WH, e0.x * 32u + lane), w1 = cols_weight<BF16>(Q.WH, e0.z * 32u + lane);
-            const float w2 = cols_weight<BF16>(Q.WH, e1.x * 32u + lane), w3 = cols_weight<BF16>(Q.WH, e1.z * 32u + lane);
-            a = fmaf(w0, __uint_as_float(e0.y), a);
-            a = fmaf(w1, __uint_as_float(e0.w), a);
-            a = fmaf(w2, __uint_as_float(e1.y), a);
-            a = fmaf(w3, __uint_as_float(e1.w), a);
+    {
+        constexpr uint32_t ESZ = BF16 ? 2u : 4u;
+        const uint32_t cb[1] = {lane * ESZ};
+        for (uint32_t p = warp; p < 32; p += nwarps) {
+            float a[1] = {0.0f};
+            cols_segment<BF16, 1, true>(S.ent, segstart[p], segstart[p + 1], Q.WH, 32u * ESZ, cb, a);
+            zpart[p * 32u + lane] = a[0];
         }
-        zpart[p * 32u + lane] = a;
     }
     for (uint32_t i = threadIdx.x; i < nwords; i += blockDim.x) idmap[i] = 0u;
     __syncthreads();
