@@ -209,6 +209,19 @@ __device__ __forceinline__ void cols_segment(const uint2 *ent, uint32_t k, uint3
     }
 }
 
+// The 16 / element size neighbouring weights that start `off` bytes into WT (a multiple of 16), with one load.
+template <bool BF16>
+__device__ __forceinline__ void cols_weights16_at(const void *WT, uint32_t off, float (&f)[BF16 ? 8 : 4])
+{
+    const uint4 q = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const char *>(WT) + off));
+    if constexpr (BF16) {
+        f[0] = bf16_lo(q.x); f[1] = bf16_hi(q.x); f[2] = bf16_lo(q.y); f[3] = bf16_hi(q.y);
+        f[4] = bf16_lo(q.z); f[5] = bf16_hi(q.z); f[6] = bf16_lo(q.w); f[7] = bf16_hi(q.w);
+    } else {
+        f[0] = __uint_as_float(q.x); f[1] = __uint_as_float(q.y); f[2] = __uint_as_float(q.z); f[3] = __uint_as_float(q.w);
+    }
+}
+
 // a[0] + ... + a[31] in the fixed tree: strides 16, 8, 4, 2, 1
 __device__ __forceinline__ float cols_tree(float (&acc)[32])
 {
@@ -228,9 +241,11 @@ __device__ __forceinline__ float cols_tree(float (&acc)[32])
 // with at most five pending partial results per node instead of 32 registers.
 // A segment holds a multiple of 4 entries; 4 entries x R loads are in flight at a time.
 // Row j of WT starts at element j * ld.
-// PAIR (R = 2): the two nodes are the neighbouring columns col[0] (even) and col[0] + 1 of a WT with even ld,
-// fetched with one load per input.
-template <bool BF16, int R, bool PAIR = false>
+// LOAD = COLS_LOAD_PAIR (R = 2): the two nodes are the neighbouring columns col[0] (even) and col[0] + 1 of a WT
+// with even ld, fetched with one load per input.  LOAD = COLS_LOAD_VEC (R = 16 / element size): the nodes are the
+// R neighbouring columns from col[0] (a multiple of R) of a WT whose ld is a multiple of R, one 16-byte load per input.
+enum { COLS_LOAD_ONE = 0, COLS_LOAD_PAIR = 1, COLS_LOAD_VEC = 2 };
+template <bool BF16, int R, int LOAD = COLS_LOAD_ONE>
 __device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, uint32_t ld, const uint32_t (&col)[R],
                                           float (&sum)[R])
 {
@@ -260,7 +275,16 @@ __device__ __forceinline__ void cols_walk(const cols_stage &S, const void *WT, u
             const uint4 e0 = *reinterpret_cast<const uint4 *>(S.ent + k), e1 = *reinterpret_cast<const uint4 *>(S.ent + k + 2);
             float w[R][4];
             const uint32_t t0 = e0.x * ldb, t1 = e0.z * ldb, t2 = e1.x * ldb, t3 = e1.z * ldb; // row offsets
-            if constexpr (PAIR) {
+            if constexpr (LOAD == COLS_LOAD_VEC) {
+                static_assert(LOAD != COLS_LOAD_VEC || R == (BF16 ? 8 : 4), "one 16-byte load holds R weights");
+                float f0[BF16 ? 8 : 4], f1[BF16 ? 8 : 4], f2[BF16 ? 8 : 4], f3[BF16 ? 8 : 4];
+                cols_weights16_at<BF16>(WT, t0 + cb[0], f0);
+                cols_weights16_at<BF16>(WT, t1 + cb[0], f1);
+                cols_weights16_at<BF16>(WT, t2 + cb[0], f2);
+                cols_weights16_at<BF16>(WT, t3 + cb[0], f3);
+#pragma unroll
+                for (int r = 0; r < R; ++r) { w[r][0] = f0[r]; w[r][1] = f1[r]; w[r][2] = f2[r]; w[r][3] = f3[r]; }
+            } else if constexpr (LOAD == COLS_LOAD_PAIR) {
                 cols_weight2_at<BF16>(WT, t0 + cb[0], w[0][0], w[R - 1][0]);
                 cols_weight2_at<BF16>(WT, t1 + cb[0], w[0][1], w[R - 1][1]);
                 cols_weight2_at<BF16>(WT, t2 + cb[0], w[0][2], w[R - 1][2]);

@@ -10,6 +10,9 @@
 #include "slonn_cols_kernels.cuh"
 
 #define SLONN_THREADS 256
+#ifndef SLONN_DEEP_WALK
+#define SLONN_DEEP_WALK true // eight list entries per step in the walks whose warps share the segments
+#endif
 
 // whether query q's budget lies in [lo, hi] (range_bp == NULL: every query)
 __device__ __forceinline__ bool bp_in_range(const uint16_t *range_bp, uint32_t lo, uint32_t hi, uint32_t q)
@@ -860,7 +863,9 @@ __global__ void __launch_bounds__(SLONN_THREADS, 2) gather_short_kernel(slonn_ga
 // query's selected nodes in column order and evaluates nodes [r0, r1) of that order against the staged
 // input list S.  `order_mem` is block scratch of P.scratch_bytes (the staging image, dead by now).  NC: the
 // id list was written by an earlier launch and may be read through the read-only path.
-template <bool BF16, int R, bool NC, bool SPLIT = false>
+// VEC: compiled with the path for a layer that computes every node and whose width is a multiple of the
+// 16 / element size nodes one load holds: a lane takes that many neighbouring columns.
+template <bool BF16, int R, bool NC, bool SPLIT = false, bool VEC = false>
 __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params &P, const cols_stage &S, void *order_mem,
                                                       const uint32_t *idlist, float *zpart, uint32_t q, uint64_t off,
                                                       uint32_t B, uint32_t r0, uint32_t r1, uint32_t *scan_ws,
@@ -927,7 +932,7 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
             float a[R];
 #pragma unroll
             for (int k = 0; k < R; ++k) a[k] = 0.0f;
-            cols_segment<BF16, R, true>(S.ent, S.segstart[p], S.segstart[p + 1], P.WT, P.N * ESZ, cb, a);
+            cols_segment<BF16, R, SLONN_DEEP_WALK>(S.ent, S.segstart[p], S.segstart[p + 1], P.WT, P.N * ESZ, cb, a);
 #pragma unroll
             for (int k = 0; k < R; ++k) zpart[(p * R + k) * 32u + lane] = a[k];
         }
@@ -954,6 +959,26 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
                 }
             }
         }
+    } else if (VEC && !P.use_list && (P.N % (BF16 ? 8u : 4u)) == 0u && (r0 % (BF16 ? 8u : 4u)) == 0u) {
+        // every node of the layer, its width a multiple of the nodes a 16-byte load holds: a lane takes that many
+        // neighbouring columns and fetches their weights of an input with one load (r1 is such a multiple too)
+        constexpr int NV = BF16 ? 8 : 4;
+        for (uint32_t r = r0 + warp * (32u * NV); r < r1; r += nwarps * (32u * NV)) {
+            const uint32_t c0 = min(r + NV * lane, r1 - NV);
+            uint32_t col[NV];
+#pragma unroll
+            for (int k = 0; k < NV; ++k) col[k] = c0 + k;
+            float sum[NV];
+            cols_walk<BF16, NV, COLS_LOAD_VEC>(S, P.WT, P.N, col, sum);
+            if (r + NV * lane < r1) {
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    float z = sum[k] + __ldg(P.bias + col[k]);
+                    if (P.relu) z = z > 0.0f ? z : 0.0f;
+                    P.out_dense[(uint64_t)q * P.out_stride + col[k]] = z;
+                }
+            }
+        }
     } else if (R == 2 && !P.use_list && (P.N & 1u) == 0u && (r0 & 1u) == 0u) {
         // every node of the layer (a layer without activator): a lane takes two neighbouring columns and
         // fetches both weights of an input with one load
@@ -961,7 +986,7 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
             const uint32_t c0 = min(r + 2u * lane, (r1 - 1u) & ~1u); // even; c0 + 1 < N because N is even
             const uint32_t col[R] = {c0, c0 + 1u};
             float sum[R];
-            cols_walk<BF16, R, true>(S, P.WT, P.N, col, sum);
+            cols_walk<BF16, R, COLS_LOAD_PAIR>(S, P.WT, P.N, col, sum);
             if (r + 2u * lane < r1) {
 #pragma unroll
                 for (int k = 0; k < R; ++k) {
@@ -1016,7 +1041,7 @@ __device__ __forceinline__ void cols_order_and_gather(const slonn_gather_params 
 // id-ascending list.
 // SPLIT: the variant for batches of tens of queries -- one block per (query, 32 * R nodes), the segments
 // of the input list spread over the block's warps (see cols_order_and_gather).
-template <bool BF16, int R, bool SPLIT>
+template <bool BF16, int R, bool SPLIT, bool VEC = false>
 #ifdef SLONN_GATHER_COLS_MIN_BLOCKS
 __launch_bounds__(SLONN_THREADS, SLONN_GATHER_COLS_MIN_BLOCKS)
 #else
@@ -1054,7 +1079,7 @@ __global__ void gather_cols_kernel(slonn_gather_params P)
     const uint32_t len = min((uint32_t)(P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add + 1] - s0), P.in_cap);
     cols_stage_list<V>(S, P.in.ids, P.in.vals, s0, len, P.D);
 
-    cols_order_and_gather<BF16, R, true, SPLIT>(P, S, smem4, P.ids + off, reinterpret_cast<float *>(S.ent + cols_ent_cap(P.D, P.in_cap)),
+    cols_order_and_gather<BF16, R, true, SPLIT, VEC>(P, S, smem4, P.ids + off, reinterpret_cast<float *>(S.ent + cols_ent_cap(P.D, P.in_cap)),
                                                  q, off, B, r0, r1, scan_ws, &scan_total);
 }
 
@@ -1077,11 +1102,12 @@ struct slonn_layer_cols_params {
 // query groups the input list, computes the hash functions and runs the selection itself (the same result
 // in each; only the first block writes keys and list to global memory), then evaluates its 64 nodes with
 // the segments of the input list spread over its warps.
-template <bool BF16, typename IDT, bool SPLIT>
-#ifndef SLONN_LAYER_COLS_MIN_BLOCKS
-#define SLONN_LAYER_COLS_MIN_BLOCKS 6 // 40 registers: seven blocks of seven warps per SM (48 registers, five blocks: 2 % slower)
-#endif
-__global__ void __launch_bounds__(SLONN_THREADS, SLONN_LAYER_COLS_MIN_BLOCKS) layer_cols_kernel(slonn_layer_cols_params Q)
+// TIGHT: compiled for 40 registers, so that seven blocks of up to seven warps fit an SM (measured on a 4096-wide
+// layer with 4096 queries: +3 % at a 10 % budget, where a block has seven warps; with eight warps per block, at
+// 25 %, the tighter allocation costs 9-15 %, so those launches take the other instantiation).
+template <bool BF16, typename IDT, bool SPLIT, bool TIGHT>
+__launch_bounds__(SLONN_THREADS, (SPLIT || TIGHT) ? 6 : 5) // 40 or 48 registers
+__global__ void layer_cols_kernel(slonn_layer_cols_params Q)
 {
     extern __shared__ float4 smem4[];
     constexpr int V = BF16 ? 8 : 4;
@@ -1127,7 +1153,7 @@ __global__ void __launch_bounds__(SLONN_THREADS, SLONN_LAYER_COLS_MIN_BLOCKS) la
         const uint32_t cb[1] = {lane * ESZ};
         for (uint32_t p = warp; p < 32; p += nwarps) {
             float a[1] = {0.0f};
-            cols_segment<BF16, 1, true>(S.ent, segstart[p], segstart[p + 1], Q.WH, 32u * ESZ, cb, a);
+            cols_segment<BF16, 1, SLONN_DEEP_WALK>(S.ent, segstart[p], segstart[p + 1], Q.WH, 32u * ESZ, cb, a);
             zpart[p * 32u + lane] = a[0];
         }
     }
