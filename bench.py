@@ -41,6 +41,9 @@ DEFAULT_QUERIES = {"c1": 1024, "c2": 65536, "c3": 256, "c3xl": 256, "c4": 4096, 
 # summarised under profiles/ (same kernel, same workload and launch shape).  Keyed by (kernel, workload,
 # queries, budget); anything else reports null.  An entry is set to None when its kernel has changed since.
 NCU_TRAFFIC = {
+    # profiles/layer_cols_c4_4096q_10pct.md: a launch that starts with cold caches (the profiler's default cache
+    # control); with the caches as the previous layer leaves them the same launch moves 1.3 MB
+    ("layer_cols_kernel", "c4", 4096, 1000): 21.1e6,
 }
 
 
