@@ -308,6 +308,40 @@ def test_one_warp_per_query_kernel_without_active_lists(last_budgeted):
     dm.free()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_four_queries_per_block_row_kernel_on_a_budgeted_last_layer(dtype):
+    # rows longer than one 512-byte round, 300 queries (75 groups of four, budgets in both grouping classes and
+    # below the grouping limit), the last layer budgeted: the grouped row kernel writes logits and their ids by
+    # position; a 100 % budget inside a group selects every row
+    wl = custom_workload(78, [512, 640, 520], [1, 1], dtype, n=302, n_cal=400, K=4, L=2,
+                         budgets=(700, 2500, 3000, 5000, 10000))
+    check(wl)
+
+
+def test_launch_records_cover_the_step_and_name_what_each_launch_serves():
+    from paper_2204_08400_b200 import binding as sl, harness
+    wl = custom_workload(79, [512, 640, 520, 24], [1, 1, 0], "bf16", n=600, n_cal=300, K=4, L=2,
+                         budgets=(700, 3000, 5000, 10000))
+    dm = harness.DeviceModel(wl)
+    b = harness.DeviceBatch(dm, wl.x, wl.budget_bp, full_outputs=False, kernel_path=sl.PATH_STAGED)
+    recs = sl.slonn_run_traced(dm.model, b.batch, b.ws, b.ws_bytes)
+    ms, cnt = sl.slonn_run_timed(dm.model, b.batch, b.ws, b.ws_bytes)
+    assert b.results()["status"][0] == 0
+    assert len(recs) == sum(cnt.values()) and all(r["ms"] > 0 for r in recs)
+    for stage in sl.STAGES:
+        assert sum(1 for r in recs if r["stage"] == stage) == cnt[stage], stage
+    assert [r["stage"] for r in recs][0] == "plan" and recs[-1]["stage"] == "argmax"
+    layers = [r["layer"] for r in recs if r["layer"] is not None]
+    assert layers == sorted(layers) and set(layers) == {0, 1, 2}
+    # every budget of the batch is served exactly once by the node launches of each layer
+    for l in (0, 1, 2):
+        for bp in (700, 3000, 5000, 10000):
+            served = [r for r in recs if r["layer"] == l and r["stage"] in ("gather_dot", "group_rows", "gather_cols", "layer_cols", "full_rows")
+                      and r["bp_lo"] <= bp <= r["bp_hi"] and not (r["skips_full"] and bp == 10000)]
+            assert len(served) == 1, (l, bp, served)
+    dm.free()
+
+
 def test_full_budget_queries_beside_the_one_warp_per_query_kernel_with_a_budgeted_last_layer():
     # large enough (queries x weights >= 2^32) for the 100 % queries to leave the one-warp-per-query kernel and
     # run four per block; the last layer carries an activator, so the prediction of every other query is an
