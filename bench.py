@@ -253,7 +253,15 @@ def roofline_of(table, workload, n, budget_bp, dense_tc):
     sec = k["ms"] / 1e3
     ach = k["algorithmic"] / sec / 1e9 if sec > 0 else 0.0
     traffic = None if dense_tc else NCU_TRAFFIC.get((name, workload, n, budget_bp))
-    return dict(common, bound="hbm", achieved=ach, peak=hbm, unit="GB/s", frac=ach / hbm, traffic=traffic,
+    # what actually limits the kernel when DRAM is nearly idle: the rows come from L2 / L1 and the issue slots fill up
+    dram_share = traffic * k["launches"] / k["algorithmic"] if traffic and k["algorithmic"] else None
+    limiter = None
+    if dram_share is not None:
+        limiter = ("instruction issue with L2-resident data (DRAM moves %.1f %% of the algorithmic bytes)" % (100 * dram_share)
+                   if dram_share < 0.25 else "HBM")
+    elif ach > hbm:
+        limiter = "L2 / L1 / instruction issue (faster than an HBM stream could deliver the bytes)"
+    return dict(common, bound="hbm", limiter=limiter, achieved=ach, peak=hbm, unit="GB/s", frac=ach / hbm, traffic=traffic,
                 frac_of_nominal_8TBps=ach / 8000.0, bytes_per_step=int(k["algorithmic"]),
                 bytes_as_run=int(k["as_run"]), frac_as_run=k["as_run"] / sec / 1e9 / hbm if sec > 0 else 0.0,
                 bytes_row_granular=int(k["row_granular"]),

@@ -239,6 +239,10 @@ typedef struct {
                              /* first layer, no SLONN_FLAG_DENSE_TC                             */
 #define SLONN_PATH_FUSED 2   /* one warp per query through all layers: widths <= 1024 inputs, */
                              /* <= 4096 nodes per layer, dense first layer                    */
+#define SLONN_PATH_BLOCK 4   /* one block of four warps per query through all layers: the same */
+                             /* networks as _FUSED; chosen by itself for batches of at most 512 */
+                             /* queries whose layers compute at most 64 rows per query; no      */
+                             /* SLONN_FLAG_DENSE_TC                                             */
 
 /*
  * Latency-Constrained Accuracy-Optimized budgets (Sec. 2.3, Eq. 3): for each query the largest

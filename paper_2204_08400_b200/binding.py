@@ -449,7 +449,7 @@ FLAG_DENSE_TC = 1
 FLAG_ROW_KERNELS = 2
 FLAG_COLUMN_KERNELS = 4
 FLAG_UNGROUPED_ROWS = 8
-PATH_AUTO, PATH_STAGED, PATH_FUSED, PATH_CLUSTER = 0, 1, 2, 3
+PATH_AUTO, PATH_STAGED, PATH_FUSED, PATH_CLUSTER, PATH_BLOCK = 0, 1, 2, 3, 4
 
 
 def slonn_run_timed(model: Model, batch: _Batch, workspace, workspace_bytes: int, stream=None):

@@ -1,5 +1,9 @@
 // Latency path for a handful of queries (the paper's setting: batch size 1, Sec. 4): one
-// thread-block CLUSTER carries one query through every layer in a single launch.
+// thread-block CLUSTER carries one query through every layer in a single launch.  The same kernel
+// with a cluster of ONE block of four warps serves narrow networks at batches of tens to a few
+// thousand queries, where one warp per query leaves most of the GPU waiting on a long chain of
+// dependent loads: four warps share a query's rows, the cluster barriers become block barriers and
+// the remote stores local ones.
 //
 // Each block of the cluster keeps a full copy of the current layer input in its shared memory.
 // Per layer:
@@ -47,6 +51,7 @@ struct slonn_cluster_params {
     const uint16_t *budget_bp; // [n]
     uint32_t max_bp;
     uint64_t *indptr_out;    // [n * n_act + 1], nullable: written for the caller (the kernel derives its own offsets)
+    const uint64_t *indptr_in; // [n * n_act + 1], nullable: offsets planned by an earlier launch (many queries)
     uint32_t *out_ids;       // CSR payload, nullable
     float *out_vals;         // CSR payload, nullable
     uint16_t *codes;         // nullable
@@ -72,8 +77,8 @@ __device__ __forceinline__ uint32_t cluster_count(const slonn_cluster_params &P,
     return B;
 }
 
-template <bool BF16>
-__global__ void __launch_bounds__(SLONN_CLUSTER_THREADS, 1)
+template <bool BF16, int THREADS, int MIN_BLOCKS>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS)
 cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
 {
     namespace cg = cooperative_groups;
@@ -98,7 +103,17 @@ cluster_network_kernel(const __grid_constant__ slonn_cluster_params P)
     // layer) entries before its own instead of waiting for a separate planning launch.
     __shared__ uint64_t s_off[SLONN_MAX_LAYERS];
     __shared__ uint32_t s_cnt[SLONN_MAX_LAYERS];
-    if (threadIdx.x == 0) {
+    const bool need_offsets = P.out_ids || P.out_vals || P.indptr_out;
+    if (threadIdx.x == 0 && (P.indptr_in || !need_offsets)) {
+        // offsets planned by an earlier launch, or not needed at all (no list is written)
+        bool bad;
+        for (uint32_t l = 0; l < P.n_layers; ++l) {
+            if (!P.layer[l].has_act) continue;
+            s_cnt[l] = cluster_count(P, q, l, &bad);
+            s_off[l] = P.indptr_in ? P.indptr_in[(uint64_t)q * P.n_act + P.layer[l].a] : 0;
+            if (bad && rank == 0) slonn_report(P.status, SLONN_ERR_BUDGET, q, l);
+        }
+    } else if (threadIdx.x == 0) {
         uint64_t run = 0;
         bool bad;
         for (uint32_t qq = 0; qq <= q; ++qq)

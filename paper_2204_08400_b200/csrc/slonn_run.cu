@@ -611,6 +611,18 @@ int launch_fused(const slonn_model *m, const slonn_batch *b, const uint64_t *ind
 
 // ---- one cluster per query: latency path for a handful of queries ---------------
 
+// One block of four warps per query (the cluster kernel with a cluster of one): chosen for narrow networks when the
+// batch has at most 512 queries (four resident blocks of 128 registers per SM: 592 at a time) and no layer computes
+// more than 64 rows per query.  Measured on 784-112-112-10 fp32, 256 queries: 37 us at a 10 % budget against 59 us
+// with the per-stage kernels and 43 us with one warp per query; with 102 rows per layer (784-1024-1024-10) the
+// per-stage kernels win, and beyond one wave of blocks one warp per query does.  Six or eight resident blocks spill.
+#ifndef SLONN_BLOCK_MINB
+#define SLONN_BLOCK_MINB 4
+#endif
+#ifndef SLONN_BLOCK_PATH_MAX_QUERIES
+#define SLONN_BLOCK_PATH_MAX_QUERIES 512u
+#endif
+#define SLONN_BLOCK_PATH_MAX_ROWS 64u
 bool cluster_eligible(const slonn_model *m)
 {
     if (m->first_sparse) return false;
@@ -628,19 +640,17 @@ uint32_t cluster_max_rows(const slonn_model *m, uint32_t max_bp)
     return r;
 }
 
-template <bool BF16>
+template <bool BF16, int THREADS, int MIN_BLOCKS>
 int launch_cluster_t(const slonn_cluster_params &P, size_t smem, cudaStream_t st)
 {
-    if (cudaFuncSetAttribute(cluster_network_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
-        return SLONN_ERR_CUDA;
-    if (P.cluster > 8 && cudaFuncSetAttribute(cluster_network_kernel<BF16>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) !=
-                             cudaSuccess)
+    auto kernel = cluster_network_kernel<BF16, THREADS, MIN_BLOCKS>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SLONN_ERR_CUDA;
+    if (P.cluster > 8 && cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
         return SLONN_ERR_CUDA;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(P.n * P.cluster, 1, 1);
-    cfg.blockDim = dim3(SLONN_CLUSTER_THREADS, 1, 1);
+    cfg.blockDim = dim3(THREADS, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -651,14 +661,17 @@ int launch_cluster_t(const slonn_cluster_params &P, size_t smem, cudaStream_t st
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int clusters = 0; // the device must be able to co-schedule at least one such cluster
-    if (cudaOccupancyMaxActiveClusters(&clusters, cluster_network_kernel<BF16>, &cfg) != cudaSuccess || clusters < 1) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) != cudaSuccess || clusters < 1) {
         cudaGetLastError();
         return SLONN_ERR_DIM;
     }
-    return cudaLaunchKernelEx(&cfg, cluster_network_kernel<BF16>, P) == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, kernel, P) == cudaSuccess ? SLONN_OK : SLONN_ERR_CUDA;
 }
 
-int launch_cluster(const slonn_model *m, const slonn_batch *b, uint32_t max_bp, uint32_t stride, cudaStream_t st)
+// cluster_size 16: a handful of queries, 512 threads per block.  cluster_size 1: one block of four warps per query
+// (narrow networks, batches up to a few thousand queries); indptr_in: the planned offsets when lists are written.
+int launch_cluster(const slonn_model *m, const slonn_batch *b, uint32_t max_bp, uint32_t stride, cudaStream_t st,
+                   uint32_t cluster_size = SLONN_CLUSTER_SIZE, const uint64_t *indptr_in = nullptr)
 {
     slonn_cluster_params P;
     memset(&P, 0, sizeof(P));
@@ -677,16 +690,20 @@ int launch_cluster(const slonn_model *m, const slonn_batch *b, uint32_t max_bp, 
             words = std::max(words, (ly.N + 31u) / 32u);
         }
     }
-    P.n_layers = m->n_layers; P.n = b->n_queries; P.n_act = m->n_act; P.K = m->K; P.L = m->L; P.cluster = SLONN_CLUSTER_SIZE;
+    P.n_layers = m->n_layers; P.n = b->n_queries; P.n_act = m->n_act; P.K = m->K; P.L = m->L; P.cluster = cluster_size;
     P.pre = slonn_model_pre(m);
-    P.x = b->x_dense; P.budget_bp = b->budget_bp; P.max_bp = max_bp; P.indptr_out = b->active_indptr;
+    P.x = b->x_dense; P.budget_bp = b->budget_bp; P.max_bp = max_bp;
+    P.indptr_in = indptr_in; P.indptr_out = indptr_in ? nullptr : b->active_indptr;
     P.out_ids = b->active_ids; P.out_vals = b->active_vals; P.codes = b->codes;
     P.logits = b->logits; P.logit_stride = stride; P.logit_ids = b->logit_ids; P.pred = b->pred;
     P.status = b->status;
     P.xbuf_floats = xbuf; P.ids_cap = ids_cap; P.bitmap_words = words;
     const size_t smem = (size_t)xbuf * 8 + (size_t)ids_cap * 4 + (size_t)words * 4;
     if (smem > 200 * 1024) return SLONN_ERR_DIM;
-    return m->dtype == SLONN_BF16 ? launch_cluster_t<true>(P, smem, st) : launch_cluster_t<false>(P, smem, st);
+    if (cluster_size == 1)
+        return m->dtype == SLONN_BF16 ? launch_cluster_t<true, 128, SLONN_BLOCK_MINB>(P, smem, st) : launch_cluster_t<false, 128, SLONN_BLOCK_MINB>(P, smem, st);
+    return m->dtype == SLONN_BF16 ? launch_cluster_t<true, SLONN_CLUSTER_THREADS, 1>(P, smem, st)
+                                  : launch_cluster_t<false, SLONN_CLUSTER_THREADS, 1>(P, smem, st);
 }
 
 } // namespace
@@ -839,7 +856,7 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     // list offsets itself, so no planning launch either)
     if (b->flags & ~SLONN_FLAG_ALL) return SLONN_ERR_ARG;
     if ((b->flags & SLONN_FLAG_ROW_KERNELS) && (b->flags & SLONN_FLAG_COLUMN_KERNELS)) return SLONN_ERR_ARG;
-    if (b->kernel_path > SLONN_PATH_CLUSTER) return SLONN_ERR_ARG;
+    if (b->kernel_path > SLONN_PATH_BLOCK) return SLONN_ERR_ARG;
     if (b->kernel_path == SLONN_PATH_CLUSTER && (!cluster_eligible(m) || tc_route(m, max_bp, b->flags))) return SLONN_ERR_DIM;
     if (b->kernel_path == SLONN_PATH_CLUSTER || (b->kernel_path == SLONN_PATH_AUTO && cluster_eligible(m) && n <= 4 && !tc_route(m, max_bp, b->flags) &&
          cluster_max_rows(m, max_bp) <= 1024)) {
@@ -855,9 +872,14 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
     // caller wants no active lists back it needs no list offsets either (each warp derives its node
     // counts from the budget), which saves the two planning launches
     if (b->kernel_path == SLONN_PATH_FUSED && !fused_eligible(m)) return SLONN_ERR_DIM;
-    const bool use_fused = b->kernel_path == SLONN_PATH_FUSED || (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n >= 512);
+    if (b->kernel_path == SLONN_PATH_BLOCK && (!fused_eligible(m) || tc_route(m, max_bp, b->flags))) return SLONN_ERR_DIM;
     const bool full_route = !tc_route(m, max_bp, b->flags) && full_route_wanted(m, n, max_bp);
-    const bool no_plan = use_fused && !tc_route(m, max_bp, b->flags) && !full_route && !b->active_indptr && !b->active_ids &&
+    // narrow networks at batches too small to fill the GPU with one warp per query: one block of four warps per query
+    const bool use_block = b->kernel_path == SLONN_PATH_BLOCK ||
+                           (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n <= SLONN_BLOCK_PATH_MAX_QUERIES &&
+                            cluster_max_rows(m, max_bp) <= SLONN_BLOCK_PATH_MAX_ROWS && !tc_route(m, max_bp, b->flags) && !full_route);
+    const bool use_fused = !use_block && (b->kernel_path == SLONN_PATH_FUSED || (b->kernel_path == SLONN_PATH_AUTO && fused_eligible(m) && n >= 512));
+    const bool no_plan = (use_fused || use_block) && !tc_route(m, max_bp, b->flags) && !full_route && !b->active_indptr && !b->active_ids &&
                          !b->active_vals;
 
     // offsets of every (query, activator layer) list
@@ -880,6 +902,15 @@ static int run_impl(const slonn_model *m, const slonn_batch *b, void *workspace,
         plan_final_kernel<<<(uint32_t)tiles, SLONN_PLAN_THREADS, 0, st>>>(pp, tile_sums);
         TOC();
         if (cudaGetLastError() != cudaSuccess) return SLONN_ERR_CUDA;
+    }
+
+    if (use_block) {
+        AT_LAYER(SLONN_ALL_LAYERS);
+        TIC(SLONN_STAGE_CLUSTER);
+        const int rc = launch_cluster(m, b, max_bp, stride, st, 1u, no_plan ? nullptr : indptr);
+        TOC();
+        if (rc != SLONN_ERR_DIM || b->kernel_path == SLONN_PATH_BLOCK) return rc;
+        // the staging does not fit: fall through to the other kernels (the offsets are planned already)
     }
 
     // queries at a 100 % budget on the tensor cores (on request): they compute every node of every

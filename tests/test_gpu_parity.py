@@ -28,7 +28,7 @@ def kernel_paths(wl):
     """Both kernel families where the network fits the one-warp-per-query kernel, else the staged one."""
     fused_ok = (not wl.first_sparse) and max(wl.dims[:-1]) <= 1024 and max(wl.dims[1:]) <= 4096
     cluster_ok = (not wl.first_sparse) and max(wl.dims) <= 8192 and wl.n_queries <= 600
-    return (1,) + ((2,) if fused_ok else ()) + ((3,) if cluster_ok else ())
+    return (1,) + ((2, 4) if fused_ok else ()) + ((3,) if cluster_ok else ())   # 4: one block of four warps per query
 
 
 def check(wl, n_cal=None, sample=None, expect_build=True, models=None):
@@ -264,7 +264,7 @@ def test_invalid_budget_is_reported_not_fatal():
     from paper_2204_08400_b200 import harness
     wl = custom_workload(57, [32, 64, 8], [1, 0], "f32", n=16, n_cal=80, K=2, L=2, budgets=(2500,))
     dm = harness.DeviceModel(wl)
-    for path in (1, 2, 3):
+    for path in (1, 2, 3, 4):
         bp = wl.budget_bp.copy()
         bp[5] = 0
         g = harness.run_once(dm, wl.x, bp, max_budget_bp=5000, kernel_path=path)
@@ -358,7 +358,7 @@ def test_runs_are_deterministic():
     from paper_2204_08400_b200 import harness
     wl = custom_workload(58, [136, 200, 96, 24], [1, 1, 0], "bf16", n=256, n_cal=300, K=4, L=2)
     dm = harness.DeviceModel(wl)
-    runs = [harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=p) for p in (1, 1, 2, 2, 3, 3, 0)]
+    runs = [harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=p) for p in (1, 1, 2, 2, 3, 3, 4, 4, 0)]
     for b in runs[1:]:
         for k in ("logits", "pred", "codes", "active_ids", "active_vals"):
             assert np.array_equal(runs[0][k], b[k])
@@ -447,7 +447,7 @@ def test_slonn_run_replays_from_a_cuda_graph():
     from paper_2204_08400_b200 import harness
     wl = custom_workload(63, [136, 200, 96, 24], [1, 1, 0], "bf16", n=3, n_cal=300, K=4, L=2)
     dm = harness.DeviceModel(wl)
-    for path in (1, 2, 3):
+    for path in (1, 2, 3, 4):
         want = harness.run_once(dm, wl.x, wl.budget_bp, kernel_path=path)
         b = harness.DeviceBatch(dm, wl.x, wl.budget_bp, kernel_path=path)
         s = torch.cuda.Stream()
