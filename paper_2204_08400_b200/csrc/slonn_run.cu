@@ -1351,10 +1351,18 @@ extern "C" int slonn_run_host(const slonn_model *m, const slonn_batch *hb, void 
     // Large dense batches go through in pieces on two internal streams, so that the copy of one
     // piece overlaps the kernels of the other.  The per-(query, layer) lists are indexed from the
     // start of the batch, so a caller that wants them back gets the batch in one piece.
+    // The first piece's copy overlaps nothing, which argues for small pieces where a query's input is
+    // large; kernels on few queries fill the SMs worse, which argues for large ones.  A piece carries
+    // about 16 MiB of input, between 1024 and 2048 queries (4096 fp32 inputs per query: four pieces of
+    // 1024 queries took 4.5 ms end to end where two of 2048 took 4.9 ms; 1024 inputs per query at
+    // mixed budgets: 2048-query pieces 9.6 ms, 1024-query pieces 11.0 ms).
 #ifndef SLONN_PIECE_QUERIES
-#define SLONN_PIECE_QUERIES 2048u // fewest queries per piece
+    const uint64_t row_bytes = (uint64_t)m->layer[0].D * sizeof(float);
+    const uint32_t piece_min = (uint32_t)std::min<uint64_t>(2048u, std::max<uint64_t>(1024u, (16ull << 20) / std::max<uint64_t>(row_bytes, 1)));
+#else
+    const uint32_t piece_min = SLONN_PIECE_QUERIES;
 #endif
-    const uint32_t pieces = std::min(8u, std::max(1u, n / SLONN_PIECE_QUERIES));
+    const uint32_t pieces = std::min(8u, std::max(1u, n / piece_min));
     const bool wants_lists = hb->active_indptr || hb->active_ids || hb->active_vals;
     uint32_t piece = (n + pieces - 1) / pieces;
     piece = (piece + 255u) / 256u * 256u;
