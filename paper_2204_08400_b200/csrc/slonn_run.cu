@@ -1331,6 +1331,68 @@ static int run_host_range(const slonn_model *m, const slonn_batch *hb, uint32_t 
     return SLONN_OK;
 }
 
+namespace {
+// The two internal streams and three events of a piecewise host call, kept per device between calls.  A call
+// that finds its device's set taken (two host calls at once) makes a set of its own and destroys it afterwards.
+struct piece_streams {
+    cudaStream_t s[2] = {nullptr, nullptr};
+    cudaEvent_t start = nullptr, done[2] = {nullptr, nullptr};
+    bool create()
+    {
+        return cudaStreamCreateWithFlags(&s[0], cudaStreamNonBlocking) == cudaSuccess &&
+               cudaStreamCreateWithFlags(&s[1], cudaStreamNonBlocking) == cudaSuccess &&
+               cudaEventCreateWithFlags(&start, cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventCreateWithFlags(&done[0], cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventCreateWithFlags(&done[1], cudaEventDisableTiming) == cudaSuccess;
+    }
+    void destroy()
+    {
+        for (int i = 0; i < 2; ++i) {
+            if (s[i]) cudaStreamDestroy(s[i]);
+            if (done[i]) cudaEventDestroy(done[i]);
+            s[i] = nullptr; done[i] = nullptr;
+        }
+        if (start) cudaEventDestroy(start);
+        start = nullptr;
+    }
+};
+std::mutex g_piece_mu;
+piece_streams g_piece_set[64]; // per device ordinal
+bool g_piece_made[64], g_piece_taken[64];
+
+// Takes the device's kept set (made on first use) or, when it is taken or the device ordinal is out of range,
+// makes a new one; *kept tells which.  false: the CUDA calls failed (whatever was created is destroyed).
+bool acquire_piece_streams(int dev, piece_streams *out, bool *kept)
+{
+    *kept = false;
+    if (dev >= 0 && dev < 64) {
+        std::lock_guard<std::mutex> lock(g_piece_mu);
+        if (!g_piece_taken[dev]) {
+            if (!g_piece_made[dev]) {
+                if (!g_piece_set[dev].create()) { g_piece_set[dev].destroy(); return false; }
+                g_piece_made[dev] = true;
+            }
+            g_piece_taken[dev] = true;
+            *out = g_piece_set[dev];
+            *kept = true;
+            return true;
+        }
+    }
+    if (!out->create()) { out->destroy(); return false; }
+    return true;
+}
+
+void release_piece_streams(int dev, piece_streams *ps, bool kept)
+{
+    if (kept) {
+        std::lock_guard<std::mutex> lock(g_piece_mu);
+        g_piece_taken[dev] = false;
+    } else {
+        ps->destroy();
+    }
+}
+} // namespace
+
 extern "C" int slonn_run_host(const slonn_model *m, const slonn_batch *hb, void *workspace, uint64_t ws_bytes,
                               void *stream, uint64_t *h2d_bytes, uint64_t *d2h_bytes)
 {
@@ -1375,20 +1437,16 @@ extern "C" int slonn_run_host(const slonn_model *m, const slonn_batch *hb, void 
         if (rc) return rc;
         if (cudaStreamSynchronize(st) != cudaSuccess) return SLONN_ERR_CUDA;
     } else {
-        cudaStream_t s2[2] = {nullptr, nullptr};
-        cudaEvent_t ev_start = nullptr, ev_done[2] = {nullptr, nullptr};
+        piece_streams ps;
+        bool kept = false;
+        if (!acquire_piece_streams(m->device, &ps, &kept)) return SLONN_ERR_CUDA;
+        cudaStream_t *s2 = ps.s;
         uint32_t status[9][4]; // at most 8 pieces
         memset(status, 0, sizeof(status));
         int rc = SLONN_OK;
-        bool ok = cudaStreamCreateWithFlags(&s2[0], cudaStreamNonBlocking) == cudaSuccess &&
-                  cudaStreamCreateWithFlags(&s2[1], cudaStreamNonBlocking) == cudaSuccess &&
-                  cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming) == cudaSuccess &&
-                  cudaEventCreateWithFlags(&ev_done[0], cudaEventDisableTiming) == cudaSuccess &&
-                  cudaEventCreateWithFlags(&ev_done[1], cudaEventDisableTiming) == cudaSuccess;
-        if (ok) { // the internal streams start after whatever the caller queued on `stream`
-            ok = cudaEventRecord(ev_start, st) == cudaSuccess && cudaStreamWaitEvent(s2[0], ev_start, 0) == cudaSuccess &&
-                 cudaStreamWaitEvent(s2[1], ev_start, 0) == cudaSuccess;
-        }
+        // the internal streams start after whatever the caller queued on `stream`
+        bool ok = cudaEventRecord(ps.start, st) == cudaSuccess && cudaStreamWaitEvent(s2[0], ps.start, 0) == cudaSuccess &&
+                  cudaStreamWaitEvent(s2[1], ps.start, 0) == cudaSuccess;
         uint32_t k = 0;
         for (uint32_t q0 = 0; ok && rc == SLONN_OK && q0 < n; q0 += piece, ++k) {
             const uint32_t cnt = std::min(piece, n - q0);
@@ -1396,19 +1454,15 @@ extern "C" int slonn_run_host(const slonn_model *m, const slonn_batch *hb, void 
                                 (uint32_t *)(ws + 2 * half) + 4 * k, &up, &down);
         }
         if (ok && rc == SLONN_OK) {
-            ok = cudaEventRecord(ev_done[0], s2[0]) == cudaSuccess && cudaEventRecord(ev_done[1], s2[1]) == cudaSuccess &&
-                 cudaStreamWaitEvent(st, ev_done[0], 0) == cudaSuccess && cudaStreamWaitEvent(st, ev_done[1], 0) == cudaSuccess &&
+            ok = cudaEventRecord(ps.done[0], s2[0]) == cudaSuccess && cudaEventRecord(ps.done[1], s2[1]) == cudaSuccess &&
+                 cudaStreamWaitEvent(st, ps.done[0], 0) == cudaSuccess && cudaStreamWaitEvent(st, ps.done[1], 0) == cudaSuccess &&
                  cudaMemcpyAsync(status, ws + 2 * half, (size_t)k * 16, cudaMemcpyDeviceToHost, st) == cudaSuccess;
             down += (uint64_t)k * 16;
         }
-        // nothing below may return before the internal streams are idle and destroyed
+        // nothing below may return before the internal streams are idle and handed back
         const bool synced = cudaStreamSynchronize(s2[0]) == cudaSuccess && cudaStreamSynchronize(s2[1]) == cudaSuccess &&
                             cudaStreamSynchronize(st) == cudaSuccess;
-        if (s2[0]) cudaStreamDestroy(s2[0]);
-        if (s2[1]) cudaStreamDestroy(s2[1]);
-        if (ev_start) cudaEventDestroy(ev_start);
-        if (ev_done[0]) cudaEventDestroy(ev_done[0]);
-        if (ev_done[1]) cudaEventDestroy(ev_done[1]);
+        release_piece_streams(m->device, &ps, kept);
         if (rc) return rc;
         if (!ok || !synced) return SLONN_ERR_CUDA;
         // first error of any piece, query index made batch-relative
