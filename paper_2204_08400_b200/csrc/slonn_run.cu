@@ -385,10 +385,11 @@ int launch_layer_cols(const slonn_model *m, const slonn_layer &ly, uint32_t laye
     G.ctas_per_query = split ? passes : 1u;
     size_t scratch = cols_image_bytes(G.D, bf ? 8u : 4u);
     scratch = std::max(scratch, ((size_t)2 * ((G.N + 31u) / 32u) + (size_t)3 * max_rows) * 4);
+    scratch = std::max(scratch, (size_t)32 * 32 * 4); // the hash functions' partial sums pass through it
     scratch = (scratch + 15) & ~(size_t)15;
     G.scratch_bytes = (uint32_t)scratch;
-    const size_t smem = scratch + (size_t)cols_ent_cap(G.D, G.in_cap) * 8 + (size_t)((G.N + 31u) / 32u) * 4 + 32 * 2 * 32 * 4 +
-                        (split ? (size_t)max_rows * 4 : 0);
+    const size_t smem = scratch + (size_t)cols_ent_cap(G.D, G.in_cap) * 8 + (size_t)((G.N + 31u) / 32u) * 4 +
+                        (split ? (size_t)32 * 2 * 32 * 4 + (size_t)max_rows * 4 : 0);
     if (smem > 200 * 1024) return SLONN_ERR_DIM;
     const uint64_t grid = (uint64_t)n * G.ctas_per_query;
     if (grid == 0 || grid > 0x7fffffffull) return SLONN_ERR_DIM;

@@ -1133,15 +1133,17 @@ __global__ void layer_cols_kernel(slonn_layer_cols_params Q)
     const uint32_t H = Q.K * Q.L;
     const uint32_t nwords = (P.N + 31u) >> 5;
 
-    // shared memory: [scratch: input image, then node order][entries][selection bitmap][partial sums]
-    // [SPLIT: the query's node list]
+    // shared memory: [scratch: input image, then the hash functions' partial sums, then node order][entries]
+    // [selection bitmap][SPLIT: partial sums of hash functions and nodes, the query's node list]
     cols_stage S;
     S.xs = reinterpret_cast<float *>(smem4);
     S.ent = reinterpret_cast<uint2 *>(reinterpret_cast<char *>(smem4) + P.scratch_bytes);
     S.segcnt = segcnt;
     S.segstart = segstart;
     uint32_t *idmap = reinterpret_cast<uint32_t *>(S.ent + cols_ent_cap(P.D, P.in_cap));
-    float *zpart = reinterpret_cast<float *>(idmap + nwords);           // [32][R][32]
+    // [32][R][32] of its own when the node loop needs it too (SPLIT); else [32][32] at the start of the scratch,
+    // which is free between the staging and the node order
+    float *zpart = SPLIT ? reinterpret_cast<float *>(idmap + nwords) : reinterpret_cast<float *>(smem4);
     uint32_t *own_list = reinterpret_cast<uint32_t *>(zpart + 32 * R * 32); // [rows_cap], SPLIT only
     const uint64_t s0 = P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add];
     const uint32_t len = min((uint32_t)(P.in.indptr[(uint64_t)q * P.in.ip_mul + P.in.ip_add + 1] - s0), P.in_cap);
