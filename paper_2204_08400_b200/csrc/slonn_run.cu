@@ -119,8 +119,10 @@ int set_smem(K kernel, size_t bytes)
 #ifdef SLONN_CARVEOUT
     cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, SLONN_CARVEOUT);
 #endif
-    if (bytes > 48 * 1024) {
-        if (bytes > 227 * 1024) return SLONN_ERR_DIM;
+    // The 48 KB a launch gets without opting in and the 227 KB a block can have count the kernel's static shared
+    // memory too (at most 1120 bytes in this library): opt in from 46 KB, refuse above 225 KB.
+    if (bytes > 46 * 1024) {
+        if (bytes > 225 * 1024) return SLONN_ERR_DIM;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return SLONN_ERR_CUDA;
     }

@@ -570,6 +570,19 @@ def test_input_stationary_kernel_for_a_few_dozen_queries(dtype):
     check(wl)
 
 
+@pytest.mark.parametrize("case", [
+    dict(seed=5008, dims=[536, 1872, 1712, 806], has_act=[1, 1, 0], n=700, K=7, L=1, budgets=(500, 1500, 9999)),
+    dict(seed=5479, dims=[2328, 1568, 1656, 595], has_act=[1, 1, 1], n=37, K=2, L=3, budgets=(10000,)),
+])
+def test_dynamic_shared_memory_just_below_the_opt_in_limit(case):
+    """Layer widths at which a kernel asks for a little less than 48 KB of dynamic shared memory: together with
+    its static shared memory that is more than a launch gets without opting in (the four-queries-per-block row
+    kernel in the first case, the one-block-per-query input-stationary kernel in the second)."""
+    wl = custom_workload(case["seed"], case["dims"], case["has_act"], "bf16", n=case["n"], n_cal=900, K=case["K"],
+                         L=case["L"], budgets=case["budgets"])
+    check(wl)
+
+
 def test_input_stationary_kernels_with_an_all_zero_list():
     # biases far below zero: every selected node of the first layer outputs exactly 0, so the next
     # layer's grouped input list is empty and its pre-activations are the biases
