@@ -239,6 +239,29 @@ def test_device_confidence_tables_and_aclo_budgets(dtype):
 
 
 @pytest.mark.gpu
+def test_device_aclo_input_width_just_below_the_shared_memory_opt_in_limit():
+    """11,900 fp32 inputs are 47.6 KB of staged query: with the kernel's static shared memory that is more than a
+    launch gets without opting in."""
+    from test_gpu_parity import custom_workload
+    wl = custom_workload(340, [11900, 64, 10], [1, 0], "f32", n=64, n_cal=200, K=3, L=2)
+    torch, sl, harness, dm, om, conf, s, c = _device_case(wl, 200)
+    thr = np.full((1, PROFILE.size), -1.0, np.float32)
+    want_bp, want_met, want_est = om.aclo_budgets(s, c, PROFILE, wl.x, thr)
+    dev = dm.device
+    bp = torch.zeros(wl.n_queries, dtype=torch.int16, device=dev)
+    estd = torch.zeros((wl.n_queries, PROFILE.size), dtype=torch.float64, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    sl.slonn_aclo_budgets(dm.model, conf, harness._dev(wl.x, dev), harness._dev(thr, dev), bp, estimate=estd, status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().numpy()[0] == 0
+    assert np.allclose(estd.cpu().numpy(), want_est, rtol=1e-11, atol=1e-11)
+    clear = np.min(np.abs(want_est - thr[0].astype(np.float64)), axis=1) > 1e-9
+    assert np.array_equal(bp.cpu().numpy().view(np.uint16)[clear], want_bp[clear])
+    sl.slonn_confidence_free(conf)
+    dm.free()
+
+
+@pytest.mark.gpu
 def test_device_confidence_tables_c2_reduced():
     from paper_2204_08400_b200 import workloads as wl_mod
     wl = wl_mod.load("c2", n_queries=256, n_cal=2048, budget_bp=1000)
