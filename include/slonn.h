@@ -65,6 +65,10 @@ extern "C" {
 #define SLONN_ERR_WORKSPACE (-9) /* workspace missing, misaligned or too small             */
 
 #define SLONN_MAX_LAYERS 16
+/* Widest input of a layer that is not fed by CSR rows: a query's layer input is staged in shared memory as fp32
+ * (225 KB).  On a layer with a Node Activator the bitmap of its nodes shares that space: 4 * D + N / 8 bytes
+ * must fit as well.  slonn_build and slonn_deserialize answer SLONN_ERR_DIM otherwise. */
+#define SLONN_MAX_INPUT_WIDTH 57600u
 
 typedef struct slonn_model slonn_model;
 
@@ -233,7 +237,7 @@ typedef struct {
 #define SLONN_FLAG_ALL 15u
 
 #define SLONN_PATH_AUTO 0    /* library chooses                                               */
-#define SLONN_PATH_STAGED 1  /* one block per query and stage: any width, any batch size      */
+#define SLONN_PATH_STAGED 1  /* one block per query and stage: any model, any batch size      */
 #define SLONN_PATH_CLUSTER 3 /* one thread-block cluster per query through all layers, for a      */
                              /* handful of queries (latency): widths and layers <= 8192, dense  */
                              /* first layer, no SLONN_FLAG_DENSE_TC                             */

@@ -597,6 +597,15 @@ extern "C" int slonn_model_tables_to_host(const slonn_model *m, uint32_t layer, 
                                                                                                 : SLONN_ERR_CUDA;
 }
 
+// The run kernels stage a query's layer input in shared memory as fp32 (and, on an activator layer, a bitmap of
+// the layer's nodes beside it): widths that cannot fit are refused when the model is made.
+static bool widths_fit(uint32_t D, uint32_t N, bool has_act, bool csr_input)
+{
+    if (csr_input) return true;
+    const uint64_t staged = (uint64_t)D * 4 + (has_act ? (uint64_t)((N + 31u) / 32u) * 4 : 0);
+    return D <= SLONN_MAX_INPUT_WIDTH && staged <= (uint64_t)SLONN_MAX_INPUT_WIDTH * 4;
+}
+
 extern "C" int slonn_build(const slonn_build_desc *desc, const void *const *W, const float *const *bias,
                            const slonn_rows *calib, void *stream, slonn_model **out)
 {
@@ -611,6 +620,7 @@ extern "C" int slonn_build(const slonn_build_desc *desc, const void *const *W, c
         if (D == 0 || N == 0) return SLONN_ERR_DIM;
         if (!W[l] || !bias[l]) return SLONN_ERR_ARG;
         const bool sparse0 = (l == 0 && desc->first_layer_sparse);
+        if (!widths_fit(D, N, desc->has_activator[l] != 0, sparse0)) return SLONN_ERR_DIM;
         if (!sparse0 && (((uint64_t)D * esz) & 15u)) return SLONN_ERR_ALIGN;
         if ((uintptr_t)W[l] & 15u) return SLONN_ERR_ALIGN;
         if (desc->has_activator[l]) {
@@ -787,6 +797,7 @@ extern "C" int slonn_deserialize(const void *src_host, uint64_t src_bytes, const
         for (uint32_t l = 0; l < h.n_layers; ++l) {
             const uint32_t D = h.dims[l], N = h.dims[l + 1];
             if (D == 0 || N == 0) return SLONN_ERR_DIM;
+            if (!widths_fit(D, N, h.has_act[l] != 0, l == 0 && h.first_sparse)) return SLONN_ERR_DIM;
             if (!W[l] || !bias[l]) return SLONN_ERR_ARG;
             if ((uintptr_t)W[l] & 15u) return SLONN_ERR_ALIGN;
             if (!(l == 0 && h.first_sparse) && (((uint64_t)D * esz) & 15u)) return SLONN_ERR_ALIGN;

@@ -38,3 +38,16 @@ def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(RuntimeError):
         binding.version()
+
+
+def test_build_refuses_layer_inputs_too_wide_to_stage_before_touching_the_device():
+    """A dense layer input wider than SLONN_MAX_INPUT_WIDTH (or one that leaves no room for an activator layer's
+    node bitmap beside it) is refused with SLONN_ERR_DIM by the argument checks, which run before any device call,
+    so this needs no GPU: the weight pointers are never followed."""
+    from paper_2204_08400_b200 import binding as sl
+    fake = 0x1000                                   # aligned, non-null, never dereferenced
+    for dims, act in (([57604, 8], [0]), ([8, 57604, 8], [0, 0]), ([57000, 400000, 8], [1, 0])):
+        with pytest.raises(sl.SlonnError) as e:
+            sl.slonn_build(dims, act, sl.SLONN_F32, [fake] * (len(dims) - 1), [fake] * (len(dims) - 1),
+                           calib_dense=None, K=2, L=1)
+        assert e.value.code == sl.ERR["DIM"], dims

@@ -583,6 +583,13 @@ def test_dynamic_shared_memory_just_below_the_opt_in_limit(case):
     check(wl)
 
 
+def test_widest_layer_input_the_library_accepts():
+    """57,600 inputs are 225 KB of staged query, the most a block's shared memory takes; one network without and
+    one with an activator on that layer (whose node bitmap sits beside the staged input)."""
+    check(custom_workload(75, [57600, 16, 8], [0, 0], "f32", n=6, n_cal=8, K=2, L=1))
+    check(custom_workload(76, [57536, 512, 8], [1, 0], "bf16", n=6, n_cal=40, K=3, L=2, budgets=(1000, 10000)))
+
+
 def test_input_stationary_kernels_with_an_all_zero_list():
     # biases far below zero: every selected node of the first layer outputs exactly 0, so the next
     # layer's grouped input list is empty and its pre-activations are the biases
