@@ -3,6 +3,8 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <mutex>
+#include <unordered_map>
 
 #include "../../include/slonn.h"
 
@@ -275,6 +277,29 @@ __device__ __forceinline__ void stage_input(const slonn_input &in, uint32_t q, u
 }
 
 // hash nodes that are active whatever the budget (0 unless the model was built that way)
+// Lets `kernel` be launched with `bytes` of dynamic shared memory on the current device.  The 48 KB a launch gets
+// without opting in and the 227 KB a block can have both count the kernel's static shared memory (at most 1120
+// bytes in this library): the opt-in starts at 46 KB and ends at 225 KB (SLONN_ERR_DIM above).  The limit of a
+// kernel is only ever raised, so that two host threads launching the same kernel with different sizes cannot
+// take each other's allowance away between the opt-in and the launch.
+inline int slonn_allow_smem(const void *kernel, size_t bytes)
+{
+    if (bytes <= 46 * 1024) return SLONN_OK;
+    if (bytes > 225 * 1024) return SLONN_ERR_DIM;
+    static std::mutex mu;
+    static std::unordered_map<uint64_t, size_t> allowed; // (kernel, device) -> bytes opted in to so far
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SLONN_ERR_CUDA;
+    const uint64_t key = (uint64_t)reinterpret_cast<uintptr_t>(kernel) * 64u + (uint64_t)(dev & 63);
+    std::lock_guard<std::mutex> lock(mu);
+    size_t &have = allowed[key];
+    if (bytes > have) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return SLONN_ERR_CUDA;
+        have = bytes;
+    }
+    return SLONN_OK;
+}
+
 inline uint32_t slonn_model_pre(const slonn_model *m) { return m->free_hash ? m->H : 0u; }
 
 // ---- internal host entry points shared between translation units ---------------

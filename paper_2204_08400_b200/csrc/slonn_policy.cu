@@ -298,12 +298,10 @@ extern "C" int slonn_aclo_budgets(const slonn_model *m, const slonn_confidence *
     P.budget_bp = budget_bp; P.met = met; P.estimate = estimate; P.status = status;
     const size_t smem = (size_t)l0.D * 4;
     cudaStream_t st = (cudaStream_t)stream;
-    if (smem > 46 * 1024) { // the limits count the kernel's static shared memory too
-        if (smem > 225 * 1024) return SLONN_ERR_DIM;
-        const cudaError_t e = m->dtype == SLONN_BF16
-            ? cudaFuncSetAttribute(aclo_budget_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-            : cudaFuncSetAttribute(aclo_budget_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return SLONN_ERR_CUDA;
+    {
+        const int rc = m->dtype == SLONN_BF16 ? slonn_allow_smem(reinterpret_cast<const void *>(aclo_budget_kernel<true>), smem)
+                                              : slonn_allow_smem(reinterpret_cast<const void *>(aclo_budget_kernel<false>), smem);
+        if (rc) return rc;
     }
     if (m->dtype == SLONN_BF16) aclo_budget_kernel<true><<<n, SLONN_THREADS, smem, st>>>(P);
     else aclo_budget_kernel<false><<<n, SLONN_THREADS, smem, st>>>(P);

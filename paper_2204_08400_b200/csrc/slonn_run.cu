@@ -119,14 +119,7 @@ int set_smem(K kernel, size_t bytes)
 #ifdef SLONN_CARVEOUT
     cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, SLONN_CARVEOUT);
 #endif
-    // The 48 KB a launch gets without opting in and the 227 KB a block can have count the kernel's static shared
-    // memory too (at most 1120 bytes in this library): opt in from 46 KB, refuse above 225 KB.
-    if (bytes > 46 * 1024) {
-        if (bytes > 225 * 1024) return SLONN_ERR_DIM;
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
-            return SLONN_ERR_CUDA;
-    }
-    return SLONN_OK;
+    return slonn_allow_smem(reinterpret_cast<const void *>(kernel), bytes);
 }
 
 template <bool BF16, typename IDT, bool LAT>
@@ -647,7 +640,7 @@ template <bool BF16, int THREADS, int MIN_BLOCKS>
 int launch_cluster_t(const slonn_cluster_params &P, size_t smem, cudaStream_t st)
 {
     auto kernel = cluster_network_kernel<BF16, THREADS, MIN_BLOCKS>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SLONN_ERR_CUDA;
+    { const int rc = slonn_allow_smem(reinterpret_cast<const void *>(kernel), smem); if (rc) return rc; }
     if (P.cluster > 8 && cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
         return SLONN_ERR_CUDA;
     cudaLaunchConfig_t cfg;

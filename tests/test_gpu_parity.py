@@ -590,6 +590,45 @@ def test_widest_layer_input_the_library_accepts():
     check(custom_workload(76, [57536, 512, 8], [1, 0], "bf16", n=6, n_cal=40, K=3, L=2, budgets=(1000, 10000)))
 
 
+def test_two_host_threads_run_different_models_at_once():
+    """slonn_run may be called from several host threads, each with its own workspace and stream.  The two
+    models stage 120 KB and 56 KB of query in the same row kernel, so each thread needs a shared-memory allowance
+    the other must not take back between its opt-in and its launch; results must equal the single-threaded ones."""
+    import threading
+    import torch
+    from paper_2204_08400_b200 import harness
+    wls = [custom_workload(77, [30000, 64, 16], [1, 0], "f32", n=40, n_cal=60, K=3, L=2, budgets=(1000, 10000)),
+           custom_workload(78, [14000, 96, 16], [1, 0], "f32", n=40, n_cal=60, K=3, L=2, budgets=(2500, 10000))]
+    dms = [harness.DeviceModel(wl) for wl in wls]
+    wants = [harness.run_once(dm, wl.x, wl.budget_bp) for dm, wl in zip(dms, wls)]
+    errors = []
+
+    def worker(i):
+        try:
+            s = torch.cuda.Stream()
+            b = harness.DeviceBatch(dms[i], wls[i].x, wls[i].budget_bp)
+            for _ in range(40):
+                b.logits.fill_(-1)
+                with torch.cuda.stream(s):
+                    b.run(s)
+                s.synchronize()
+                got = b.results()
+                assert got["status"][0] == 0
+                for k in ("logits", "pred", "codes", "active_ids", "active_vals"):
+                    assert np.array_equal(got[k], wants[i][k]), k
+        except Exception as e:            # reported by the main thread
+            errors.append((i, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for dm in dms:
+        dm.free()
+
+
 def test_input_stationary_kernels_with_an_all_zero_list():
     # biases far below zero: every selected node of the first layer outputs exactly 0, so the next
     # layer's grouped input list is empty and its pre-activations are the biases
