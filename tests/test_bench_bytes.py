@@ -57,6 +57,10 @@ def test_budget_ranges_and_skipped_full_budget_queries():
     full = acc.launch_bytes(sh, rec("full_rows", 1, 10000, 10000), bp)
     assert full["queries"] == 2 and full["as_run"] == full["algorithmic"] == 2 * 200 * 200 * 2
     assert acc.launch_bytes(sh, rec("gather_dot", 1, 20000, 30000), bp)["queries"] == 0
+    # four queries per block: the same row-wise count as the one-query row kernel for the queries it serves
+    grouped = acc.launch_bytes(sh, rec("group_rows", 1, 2001, 10000, skips_full=True), bp)
+    assert grouped["queries"] == 3 and grouped["as_run"] == high["as_run"] and grouped["algorithmic"] == high["algorithmic"]
+    assert acc.kernel_name(sh, rec("group_rows", 1)) == "group_rows_kernel"
 
 
 def test_whole_network_launch_takes_each_layers_form_from_the_record():
